@@ -1,0 +1,180 @@
+"""ctypes front end of the CPU oracle (``obf_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY.  The oracle is the slow fp64 restatement of the
+paper's Eq. 1-7 / Algorithms 2-3 that the CUDA path is checked against.  Only
+the tests, the smoke check and the benchmark's CPU-baseline leg may import this
+package; the product package never does.
+
+``build()`` compiles the C file with gcc (OpenMP over heads) into
+``oracle/_build/libobf_oracle.so``; the library is rebuilt when the source is
+newer than the binary.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Dict, Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "obf_oracle.c")
+_OUT_DIR = os.path.join(_HERE, "_build")
+_LIB_PATH = os.path.join(_OUT_DIR, "libobf_oracle.so")
+_lib = None
+
+
+class Diag(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_double) for n in (
+        "a_keep", "a_del", "alpha", "vdel_fro2", "r_fro2", "rcr", "rbar_norm",
+        "delta_norm", "kth_score", "next_score", "lam_rho", "lam_next", "lam_1")] + [
+        (n, ctypes.c_int32) for n in ("span_rank", "rho_eff", "n_del", "skipped")]
+
+    def asdict(self) -> Dict[str, float]:
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+def build(force: bool = False) -> str:
+    os.makedirs(_OUT_DIR, exist_ok=True)
+    if (not force and os.path.exists(_LIB_PATH)
+            and os.path.getmtime(_LIB_PATH) >= os.path.getmtime(_SRC)):
+        return _LIB_PATH
+    tmp = _LIB_PATH + ".tmp%d" % os.getpid()
+    cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-Wall", "-Wextra",
+           "-o", tmp, _SRC, "-lm"]
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, _LIB_PATH)
+    return _LIB_PATH
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        fp = ctypes.POINTER(ctypes.c_float)
+        dp = ctypes.POINTER(ctypes.c_double)
+        ip = ctypes.POINTER(ctypes.c_int32)
+        ci = ctypes.c_int
+        _lib.obf_oracle_scores.argtypes = [fp, fp, ci, ci, ci, dp]
+        _lib.obf_oracle_scores.restype = None
+        _lib.obf_oracle_topk.argtypes = [dp, ci, ci, ip, dp, dp]
+        _lib.obf_oracle_topk.restype = ci
+        _lib.obf_oracle_span_basis.argtypes = [dp, ci, ci, dp]
+        _lib.obf_oracle_span_basis.restype = ci
+        _lib.obf_oracle_sym_eig.argtypes = [dp, ci, dp, dp]
+        _lib.obf_oracle_sym_eig.restype = None
+        _lib.obf_oracle_head.argtypes = [fp, fp, fp, ci, ci, ci, ci, ci, ctypes.c_double,
+                                         ip, dp, dp, dp, dp, dp, dp, dp, dp, ctypes.POINTER(Diag)]
+        _lib.obf_oracle_head.restype = ci
+        _lib.obf_oracle_compress.argtypes = [fp, fp, fp, ci, ci, ci, ci, ci, ci, ci, ci,
+                                             ctypes.c_double, ip, dp, dp, dp, ctypes.POINTER(Diag)]
+        _lib.obf_oracle_compress.restype = ci
+        _lib.obf_oracle_num_threads.argtypes = []
+        _lib.obf_oracle_num_threads.restype = ci
+    return _lib
+
+
+def _f32(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.float32)
+
+
+def _f64(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def _p(a: Optional[np.ndarray], ct):
+    return None if a is None else a.ctypes.data_as(ctypes.POINTER(ct))
+
+
+def num_threads() -> int:
+    return int(lib().obf_oracle_num_threads())
+
+
+def scores(K, Q) -> np.ndarray:
+    """Attention mass A[T] of one KV head (Eq. 1); K [T,d], Q [n_q,d]."""
+    K, Q = _f32(K), _f32(Q)
+    T, d = K.shape
+    A = np.empty(T, dtype=np.float64)
+    lib().obf_oracle_scores(_p(K, ctypes.c_float), _p(Q, ctypes.c_float), T, d, Q.shape[0],
+                            _p(A, ctypes.c_double))
+    return A
+
+
+def topk(A, budget: int):
+    """Ascending retained positions, plus the k-th and (k+1)-th largest masses."""
+    A = _f64(A)
+    T = A.shape[0]
+    k = min(budget, T)
+    idx = np.empty(max(k, 1), dtype=np.int32)
+    kth, nxt = ctypes.c_double(), ctypes.c_double()
+    k2 = lib().obf_oracle_topk(_p(A, ctypes.c_double), T, budget, _p(idx, ctypes.c_int32),
+                               ctypes.byref(kth), ctypes.byref(nxt))
+    return idx[:k2].copy(), kth.value, nxt.value
+
+
+def span_basis(X) -> np.ndarray:
+    """Orthonormal rows spanning the row space of X [k,d] (Eq. 2)."""
+    X = _f64(X)
+    k, d = X.shape
+    Qb = np.zeros((max(min(k, d), 1), d), dtype=np.float64)
+    m = lib().obf_oracle_span_basis(_p(X, ctypes.c_double), k, d, _p(Qb, ctypes.c_double))
+    return Qb[:m].copy()
+
+
+def sym_eig(S):
+    """Eigenvalues (descending) and eigenvectors (rows) of a symmetric matrix."""
+    S = _f64(S).copy()
+    n = S.shape[0]
+    lam = np.empty(n, dtype=np.float64)
+    E = np.empty((n, n), dtype=np.float64)
+    lib().obf_oracle_sym_eig(_p(S, ctypes.c_double), n, _p(lam, ctypes.c_double), _p(E, ctypes.c_double))
+    return lam, E
+
+
+def head(K, V, Q, budget: int, rank: int, eps: float = 1e-12) -> Dict[str, object]:
+    """Algorithm 2 (headwise) + Algorithm 3 on one (layer, KV head).
+
+    K, V [T,d]; Q [n_q,d] (float32 values; bf16 inputs up-cast exactly).
+    Returns idx, K_out, V_out (float64), A, delta, rbar, Delta, eigvals, proj, diag.
+    """
+    K, V, Q = _f32(K), _f32(V), _f32(Q)
+    T, d = K.shape
+    k = min(budget, T)
+    idx = np.empty(max(k, 1), dtype=np.int32)
+    K_out = np.zeros((max(k, 1), d), dtype=np.float64)
+    V_out = np.zeros((max(k, 1), d), dtype=np.float64)
+    A = np.empty(T, dtype=np.float64)
+    delta = np.empty(d); rbar = np.empty(d); Delta = np.empty(d); eig = np.empty(d)
+    proj = np.empty((d, d))
+    dg = Diag()
+    cd = ctypes.c_double
+    k2 = lib().obf_oracle_head(
+        _p(K, ctypes.c_float), _p(V, ctypes.c_float), _p(Q, ctypes.c_float),
+        T, d, Q.shape[0], budget, rank, eps,
+        _p(idx, ctypes.c_int32), _p(K_out, cd), _p(V_out, cd), _p(A, cd), _p(delta, cd),
+        _p(rbar, cd), _p(Delta, cd), _p(eig, cd), _p(proj, cd), ctypes.byref(dg))
+    assert k2 == k
+    return {"idx": idx[:k].copy(), "K_out": K_out[:k], "V_out": V_out[:k], "A": A, "delta": delta,
+            "rbar": rbar, "Delta": Delta, "eigvals": eig, "proj": proj, "diag": dg.asdict()}
+
+
+def compress(K, V, Q, q_heads: int, n_obs: int, budget: int, rank: int,
+             eps: float = 1e-12) -> Dict[str, object]:
+    """A whole cache: K, V [layers, kv_heads, T, d]; Q [layers, q_heads, n_obs, d]."""
+    K, V, Q = _f32(K), _f32(V), _f32(Q)
+    layers, kv_heads, T, d = K.shape
+    k = min(budget, T)
+    heads = layers * kv_heads
+    idx = np.empty((layers, kv_heads, k), dtype=np.int32)
+    K_out = np.zeros((layers, kv_heads, k, d), dtype=np.float64)
+    V_out = np.zeros((layers, kv_heads, k, d), dtype=np.float64)
+    delta = np.zeros((layers, kv_heads, d), dtype=np.float64)
+    diags = (Diag * heads)()
+    cd = ctypes.c_double
+    lib().obf_oracle_compress(
+        _p(K, ctypes.c_float), _p(V, ctypes.c_float), _p(Q, ctypes.c_float),
+        layers, kv_heads, q_heads, n_obs, T, d, budget, rank, eps,
+        _p(idx, ctypes.c_int32), _p(K_out, cd), _p(V_out, cd), _p(delta, cd), diags)
+    return {"idx": idx, "K_out": K_out, "V_out": V_out, "delta": delta,
+            "diag": [diags[i].asdict() for i in range(heads)]}

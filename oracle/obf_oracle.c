@@ -1,0 +1,448 @@
+/*
+ * CPU oracle for relay-boundary prompt-KV compression: headwise attention-mass
+ * eviction followed by Orthogonal BackFill (OBF).
+ *
+ * THIS IS TEST INFRASTRUCTURE, NOT THE PRODUCT.  It is a plain, slow, fp64,
+ * step-by-step statement of the paper's definitions (Eq. 1-7, Algorithms 2-3),
+ * used by the tests, by the smoke check and by the benchmark's CPU-baseline
+ * leg.  It shares no code with the CUDA path and the CUDA path never calls it.
+ *
+ * Inputs are float32 (bf16 inputs are up-cast exactly by the caller); every
+ * arithmetic step is carried out in double.  One (layer, KV head) is one
+ * independent problem (Section 4.4 applies every step per layer and KV head).
+ *
+ * Pin status (see tests, all CPU-only):
+ *   scores      pinned: row-sum invariant, equal-key closed form, T=2 sigmoid
+ *               closed form, library softmax, permutation equivariance
+ *   top-k       pinned: brute-force full sort on tiny inputs, library stable
+ *               argsort, planted exact ties
+ *   gather      pinned: bitwise copies
+ *   span basis  pinned: orthonormality, annihilation of V_keep, library
+ *               pseudo-inverse projector, library matrix rank
+ *   eigen/C     pinned: library SVD of the explicit residual, Max-P closed
+ *               form, codimension-1 closed form, hand-worked planted example
+ *   scaling     pinned: single-query identity from the error-bound appendix,
+ *               hand-worked planted example
+ * No function here is "parity unpinned".
+ */
+#include <math.h>
+#include <float.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+typedef struct {
+    double a_keep;       /* sum of attention mass over retained positions (Eq. 6)          */
+    double a_del;        /* sum of attention mass over deleted positions (Eq. 6)           */
+    double alpha;        /* a_del / (a_keep + eps)                                          */
+    double vdel_fro2;    /* ||V_del||_F^2                                                   */
+    double r_fro2;       /* ||R||_F^2                                                       */
+    double rcr;          /* r_fro2 / (vdel_fro2 + eps)   (App. K.2)                         */
+    double rbar_norm;    /* ||r_bar||_2                                                     */
+    double delta_norm;   /* ||delta||_2  (IVN, App. K.2)                                    */
+    double kth_score;    /* k_eff-th largest attention mass                                 */
+    double next_score;   /* (k_eff+1)-th largest attention mass, or -1 if none              */
+    double lam_rho;      /* eigenvalue rho_eff of R^T R (smallest one kept), 0 if none      */
+    double lam_next;     /* eigenvalue rho_eff+1 of R^T R (largest one dropped), 0 if none  */
+    double lam_1;        /* largest eigenvalue of R^T R                                     */
+    int32_t span_rank;   /* numerical rank m of span(V_keep)                                */
+    int32_t rho_eff;     /* min(pca_rank, numerical rank of R)                              */
+    int32_t n_del;       /* number of deleted positions                                     */
+    int32_t skipped;     /* 1 if OBF was skipped for this head (footnote to Eq. 7)          */
+} obf_oracle_diag_t;
+
+/* ------------------------------------------------------------------ */
+/* Step O1 - attention mass, Eq. 1 with the softmax of App. L.1        */
+/* ------------------------------------------------------------------ */
+/*
+ * A_j = sum over the n_q query rows t of softmax_j(q_t . K_j / sqrt(d)).
+ * The n_q rows are all observation queries of all query heads that share this
+ * KV head (Eq. 1's sum extended over the GQA group).  Softmax runs over the T
+ * prompt keys only, natural exponential, maximum subtracted first.
+ */
+void obf_oracle_scores(const float *K, const float *Q, int T, int d, int n_q, double *A)
+{
+    double *s = (double *)malloc((size_t)T * sizeof(double));
+    const double scale = 1.0 / sqrt((double)d);
+    for (int j = 0; j < T; ++j) A[j] = 0.0;
+    for (int t = 0; t < n_q; ++t) {
+        const float *q = Q + (size_t)t * d;
+        double mx = -INFINITY;
+        for (int j = 0; j < T; ++j) {
+            const float *k = K + (size_t)j * d;
+            double acc = 0.0;
+            for (int c = 0; c < d; ++c) acc += (double)q[c] * (double)k[c];
+            s[j] = acc * scale;
+            if (s[j] > mx) mx = s[j];
+        }
+        double Z = 0.0;
+        for (int j = 0; j < T; ++j) { s[j] = exp(s[j] - mx); Z += s[j]; }
+        for (int j = 0; j < T; ++j) A[j] += s[j] / Z;
+    }
+    free(s);
+}
+
+/* ------------------------------------------------------------------ */
+/* Step O2 - TopK_B with deterministic ties                            */
+/* ------------------------------------------------------------------ */
+typedef struct { double a; int32_t j; } score_pos_t;
+
+static int cmp_score_desc_index_asc(const void *x, const void *y)
+{
+    const score_pos_t *p = (const score_pos_t *)x, *q = (const score_pos_t *)y;
+    if (p->a > q->a) return -1;
+    if (p->a < q->a) return 1;
+    return (p->j > q->j) - (p->j < q->j);      /* equal mass: lower position first */
+}
+
+static int cmp_int_asc(const void *x, const void *y)
+{
+    int32_t a = *(const int32_t *)x, b = *(const int32_t *)y;
+    return (a > b) - (a < b);
+}
+
+/*
+ * Order positions by (mass descending, position ascending), keep the first
+ * k_eff = min(budget, T), return them as an ascending index list (Section 3.1:
+ * a retained cache is a subsequence i_1 < ... < i_m).  kth/next receive the
+ * k_eff-th and (k_eff+1)-th largest masses (next = -1 when k_eff == T).
+ */
+int obf_oracle_topk(const double *A, int T, int budget, int32_t *idx, double *kth, double *next)
+{
+    int k = budget < T ? budget : T;
+    if (k < 0) k = 0;
+    score_pos_t *sp = (score_pos_t *)malloc((size_t)T * sizeof(score_pos_t));
+    for (int j = 0; j < T; ++j) { sp[j].a = A[j]; sp[j].j = j; }
+    qsort(sp, (size_t)T, sizeof(score_pos_t), cmp_score_desc_index_asc);
+    for (int r = 0; r < k; ++r) idx[r] = sp[r].j;
+    if (kth)  *kth  = k > 0 ? sp[k - 1].a : -1.0;
+    if (next) *next = k < T ? sp[k].a : -1.0;
+    qsort(idx, (size_t)k, sizeof(int32_t), cmp_int_asc);
+    free(sp);
+    return k;
+}
+
+/* ------------------------------------------------------------------ */
+/* Step O6 - orthonormal basis of span(V_keep), Eq. 2                  */
+/* ------------------------------------------------------------------ */
+/*
+ * X is k x d (rows are retained value states).  Writes an orthonormal basis of
+ * the row space as the rows of Qb (at most min(k,d) rows of length d) and
+ * returns its dimension m.  Gram-Schmidt with largest-remaining-row pivoting
+ * and a second orthogonalisation pass; a direction is accepted while the
+ * largest remaining row norm exceeds max(k,d) * DBL_EPSILON times the largest
+ * original row norm.  Eq. 2 needs any orthonormal basis of that span: only the
+ * span enters the method (through Q Q^T), so the pivot order is free.
+ */
+int obf_oracle_span_basis(const double *X, int k, int d, double *Qb)
+{
+    if (k <= 0) return 0;
+    double *W = (double *)malloc((size_t)k * d * sizeof(double));
+    memcpy(W, X, (size_t)k * d * sizeof(double));
+    int mmax = k < d ? k : d;
+    int m = 0;
+    double ref = 0.0;
+    const double tol = (double)(k > d ? k : d) * DBL_EPSILON;
+    while (m < mmax) {
+        int p = -1; double best = 0.0;
+        for (int i = 0; i < k; ++i) {
+            double n2 = 0.0;
+            for (int c = 0; c < d; ++c) n2 += W[(size_t)i * d + c] * W[(size_t)i * d + c];
+            if (n2 > best) { best = n2; p = i; }
+        }
+        if (p < 0) break;
+        double nrm = sqrt(best);
+        if (m == 0) ref = nrm;
+        if (nrm <= tol * ref) break;
+        double *q = Qb + (size_t)m * d;
+        for (int c = 0; c < d; ++c) q[c] = W[(size_t)p * d + c] / nrm;
+        for (int pass = 0; pass < 2; ++pass) {            /* re-orthogonalise against earlier rows */
+            for (int r = 0; r < m; ++r) {
+                const double *qr = Qb + (size_t)r * d;
+                double dot = 0.0;
+                for (int c = 0; c < d; ++c) dot += q[c] * qr[c];
+                for (int c = 0; c < d; ++c) q[c] -= dot * qr[c];
+            }
+            double n2 = 0.0;
+            for (int c = 0; c < d; ++c) n2 += q[c] * q[c];
+            double inv = 1.0 / sqrt(n2);
+            for (int c = 0; c < d; ++c) q[c] *= inv;
+        }
+        for (int i = 0; i < k; ++i) {                     /* deflate every remaining row */
+            double dot = 0.0;
+            for (int c = 0; c < d; ++c) dot += W[(size_t)i * d + c] * q[c];
+            for (int c = 0; c < d; ++c) W[(size_t)i * d + c] -= dot * q[c];
+        }
+        ++m;
+    }
+    free(W);
+    return m;
+}
+
+/* ------------------------------------------------------------------ */
+/* Step O9 - symmetric eigen-decomposition (cyclic Jacobi)             */
+/* ------------------------------------------------------------------ */
+/*
+ * S is n x n symmetric (destroyed).  On return lam[0] >= lam[1] >= ... and row
+ * i of E is the unit eigenvector of lam[i].  Classical cyclic Jacobi rotations
+ * until every off-diagonal entry is negligible against its diagonal pair.
+ */
+void obf_oracle_sym_eig(double *S, int n, double *lam, double *E)
+{
+    double *U = (double *)calloc((size_t)n * n, sizeof(double));   /* columns = eigenvectors */
+    for (int i = 0; i < n; ++i) U[(size_t)i * n + i] = 1.0;
+    double fro = 0.0;
+    for (int i = 0; i < n * n; ++i) fro += S[i] * S[i];
+    const double floor_abs = DBL_EPSILON * DBL_EPSILON * sqrt(fro);   /* noise floor in null directions */
+    for (int sweep = 0; sweep < 100; ++sweep) {
+        int rotated = 0;
+        for (int p = 0; p < n - 1; ++p) {
+            for (int q = p + 1; q < n; ++q) {
+                double apq = S[(size_t)p * n + q];
+                double app = S[(size_t)p * n + p], aqq = S[(size_t)q * n + q];
+                if (apq == 0.0) continue;
+                if (fabs(apq) <= DBL_EPSILON * 1e-3 * sqrt(fabs(app) * fabs(aqq)) + floor_abs) {
+                    S[(size_t)p * n + q] = S[(size_t)q * n + p] = 0.0;
+                    continue;
+                }
+                rotated = 1;
+                double theta = (aqq - app) / (2.0 * apq);
+                double t = (theta >= 0.0 ? 1.0 : -1.0) / (fabs(theta) + sqrt(theta * theta + 1.0));
+                double c = 1.0 / sqrt(t * t + 1.0), s = t * c;
+                for (int r = 0; r < n; ++r) {             /* columns p, q */
+                    double arp = S[(size_t)r * n + p], arq = S[(size_t)r * n + q];
+                    S[(size_t)r * n + p] = c * arp - s * arq;
+                    S[(size_t)r * n + q] = s * arp + c * arq;
+                }
+                for (int r = 0; r < n; ++r) {             /* rows p, q */
+                    double apr = S[(size_t)p * n + r], aqr = S[(size_t)q * n + r];
+                    S[(size_t)p * n + r] = c * apr - s * aqr;
+                    S[(size_t)q * n + r] = s * apr + c * aqr;
+                }
+                for (int r = 0; r < n; ++r) {
+                    double urp = U[(size_t)r * n + p], urq = U[(size_t)r * n + q];
+                    U[(size_t)r * n + p] = c * urp - s * urq;
+                    U[(size_t)r * n + q] = s * urp + c * urq;
+                }
+            }
+        }
+        if (!rotated) break;
+    }
+    /* selection sort, descending */
+    int *ord = (int *)malloc((size_t)n * sizeof(int));
+    for (int i = 0; i < n; ++i) ord[i] = i;
+    for (int i = 0; i < n; ++i) {
+        int b = i;
+        for (int j = i + 1; j < n; ++j)
+            if (S[(size_t)ord[j] * n + ord[j]] > S[(size_t)ord[b] * n + ord[b]]) b = j;
+        int tmp = ord[i]; ord[i] = ord[b]; ord[b] = tmp;
+    }
+    for (int i = 0; i < n; ++i) {
+        lam[i] = S[(size_t)ord[i] * n + ord[i]];
+        for (int r = 0; r < n; ++r) E[(size_t)i * n + r] = U[(size_t)r * n + ord[i]];
+    }
+    free(ord);
+    free(U);
+}
+
+/* ------------------------------------------------------------------ */
+/* One (layer, KV head): Algorithm 2 (headwise) + Algorithm 3          */
+/* ------------------------------------------------------------------ */
+/*
+ * K, V : [T, d] float32;  Q : [n_q, d] float32.
+ * idx  : [k_eff] ascending retained positions.
+ * K_out, V_out : [k_eff, d] double (K_out rows are exact copies; V_out = V_keep + delta).
+ * Optional (may be NULL): A [T], delta [d] (scaled injection), rbar [d],
+ * Delta [d] (unscaled direction, Eq. 5), eigvals [d] (of R^T R, descending),
+ * proj [d*d] (C^T C, the projector onto the residual principal subspace), diag.
+ * Returns k_eff.
+ */
+int obf_oracle_head(const float *K, const float *V, const float *Q,
+                    int T, int d, int n_q, int budget, int rank, double eps,
+                    int32_t *idx, double *K_out, double *V_out,
+                    double *A_out, double *delta_out, double *rbar_out, double *Delta_out,
+                    double *eigvals_out, double *proj_out, obf_oracle_diag_t *diag)
+{
+    obf_oracle_diag_t dg;
+    memset(&dg, 0, sizeof(dg));
+    dg.next_score = -1.0;
+
+    /* O1: attention mass */
+    double *A = (double *)malloc((size_t)T * sizeof(double));
+    obf_oracle_scores(K, Q, T, d, n_q, A);
+    if (A_out) memcpy(A_out, A, (size_t)T * sizeof(double));
+
+    /* O2: headwise TopK_B, ascending index list */
+    int k = obf_oracle_topk(A, T, budget, idx, &dg.kth_score, &dg.next_score);
+
+    /* O3: gather (Algorithm 2, last step) */
+    for (int r = 0; r < k; ++r)
+        for (int c = 0; c < d; ++c) {
+            K_out[(size_t)r * d + c] = (double)K[(size_t)idx[r] * d + c];
+            V_out[(size_t)r * d + c] = (double)V[(size_t)idx[r] * d + c];
+        }
+
+    if (delta_out)   for (int c = 0; c < d; ++c) delta_out[c] = 0.0;
+    if (rbar_out)    for (int c = 0; c < d; ++c) rbar_out[c] = 0.0;
+    if (Delta_out)   for (int c = 0; c < d; ++c) Delta_out[c] = 0.0;
+    if (eigvals_out) for (int c = 0; c < d; ++c) eigvals_out[c] = 0.0;
+    if (proj_out)    for (int c = 0; c < d * d; ++c) proj_out[c] = 0.0;
+
+    /* deleted positions, ascending (Algorithm 3: P_del = P \ P_keep) */
+    int N = T - k;
+    dg.n_del = N;
+    char *keep = (char *)calloc((size_t)T, 1);
+    for (int r = 0; r < k; ++r) keep[idx[r]] = 1;
+
+    /* O5: demand sums (Eq. 6) - also reported for eviction-only heads */
+    for (int j = 0; j < T; ++j) { if (keep[j]) dg.a_keep += A[j]; else dg.a_del += A[j]; }
+    dg.alpha = dg.a_del / (dg.a_keep + eps);
+
+    /* O4: footnote to Eq. 7 - nothing deleted, or rank 0: plain eviction */
+    if (N == 0 || rank <= 0) {
+        dg.skipped = 1;
+        if (diag) *diag = dg;
+        free(keep); free(A);
+        return k;
+    }
+
+    int *del = (int *)malloc((size_t)N * sizeof(int));
+    { int n = 0; for (int j = 0; j < T; ++j) if (!keep[j]) del[n++] = j; }
+
+    /* O6: Q = orth(V_keep^T), Eq. 2 (rows of Qb span the retained values) */
+    double *Qb = (double *)malloc((size_t)(k < d ? k : d) * d * sizeof(double));
+    int m = obf_oracle_span_basis(V_out, k, d, Qb);
+    dg.span_rank = m;
+
+    /* O7: R = V_del - (V_del Q) Q^T, Eq. 3 */
+    double *R = (double *)malloc((size_t)N * d * sizeof(double));
+    double *coef = (double *)malloc((size_t)(m > 0 ? m : 1) * sizeof(double));
+    for (int n = 0; n < N; ++n) {
+        const float *v = V + (size_t)del[n] * d;
+        double *r = R + (size_t)n * d;
+        for (int c = 0; c < d; ++c) { r[c] = (double)v[c]; dg.vdel_fro2 += r[c] * r[c]; }
+        for (int i = 0; i < m; ++i) {
+            double dot = 0.0;
+            for (int c = 0; c < d; ++c) dot += (double)v[c] * Qb[(size_t)i * d + c];
+            coef[i] = dot;
+        }
+        for (int i = 0; i < m; ++i)
+            for (int c = 0; c < d; ++c) r[c] -= coef[i] * Qb[(size_t)i * d + c];
+        for (int c = 0; c < d; ++c) dg.r_fro2 += r[c] * r[c];
+    }
+    dg.rcr = dg.r_fro2 / (dg.vdel_fro2 + eps);
+
+    /* O8: residual of negligible Frobenius norm -> skip (footnote to Eq. 7) */
+    if (dg.r_fro2 <= 1e-12 * dg.vdel_fro2) {
+        dg.skipped = 1;
+        if (diag) *diag = dg;
+        free(coef); free(R); free(Qb); free(del); free(keep); free(A);
+        return k;
+    }
+
+    /* O9: top right singular vectors of R = top eigenvectors of R^T R (no centring) */
+    double *G = (double *)calloc((size_t)d * d, sizeof(double));
+    for (int n = 0; n < N; ++n) {
+        const double *r = R + (size_t)n * d;
+        for (int a = 0; a < d; ++a) {
+            double ra = r[a];
+            for (int b = 0; b < d; ++b) G[(size_t)a * d + b] += ra * r[b];
+        }
+    }
+    double *lam = (double *)malloc((size_t)d * sizeof(double));
+    double *E = (double *)malloc((size_t)d * d * sizeof(double));
+    obf_oracle_sym_eig(G, d, lam, E);
+    if (eigvals_out) memcpy(eigvals_out, lam, (size_t)d * sizeof(double));
+    int rankR = 0;
+    for (int i = 0; i < d; ++i) if (lam[i] > (double)d * DBL_EPSILON * lam[0]) ++rankR;
+    int rho = rank < rankR ? rank : rankR;          /* k = min(pca_rank, rank(R)) */
+    dg.rho_eff = rho;
+    dg.lam_1 = lam[0];
+    dg.lam_rho = rho > 0 ? lam[rho - 1] : 0.0;
+    dg.lam_next = rho < d ? lam[rho] : 0.0;
+
+    /* O10: attention-weighted residual mean, Eq. 4 */
+    double *rbar = (double *)calloc((size_t)d, sizeof(double));
+    for (int n = 0; n < N; ++n) {
+        double w = A[del[n]] / (dg.a_del + eps);
+        const double *r = R + (size_t)n * d;
+        for (int c = 0; c < d; ++c) rbar[c] += w * r[c];
+    }
+    { double s = 0.0; for (int c = 0; c < d; ++c) s += rbar[c] * rbar[c]; dg.rbar_norm = sqrt(s); }
+    if (rbar_out) memcpy(rbar_out, rbar, (size_t)d * sizeof(double));
+
+    /* O11: Delta = (rbar C^T) C, Eq. 5; delta = alpha * Delta, Eq. 6; V* = V + delta, Eq. 7 */
+    double *Delta = (double *)calloc((size_t)d, sizeof(double));
+    for (int i = 0; i < rho; ++i) {
+        const double *c_i = E + (size_t)i * d;
+        double dot = 0.0;
+        for (int c = 0; c < d; ++c) dot += rbar[c] * c_i[c];
+        for (int c = 0; c < d; ++c) Delta[c] += dot * c_i[c];
+    }
+    if (Delta_out) memcpy(Delta_out, Delta, (size_t)d * sizeof(double));
+    if (proj_out)
+        for (int i = 0; i < rho; ++i)
+            for (int a = 0; a < d; ++a)
+                for (int b = 0; b < d; ++b)
+                    proj_out[(size_t)a * d + b] += E[(size_t)i * d + a] * E[(size_t)i * d + b];
+    double dn = 0.0;
+    for (int c = 0; c < d; ++c) {
+        double dl = dg.alpha * Delta[c];
+        if (delta_out) delta_out[c] = dl;
+        dn += dl * dl;
+        for (int r = 0; r < k; ++r) V_out[(size_t)r * d + c] += dl;     /* keys untouched */
+    }
+    dg.delta_norm = sqrt(dn);
+    if (diag) *diag = dg;
+
+    free(Delta); free(rbar); free(E); free(lam); free(G);
+    free(coef); free(R); free(Qb); free(del); free(keep); free(A);
+    return k;
+}
+
+/* ------------------------------------------------------------------ */
+/* A whole cache: every (layer, KV head) independently                  */
+/* ------------------------------------------------------------------ */
+/*
+ * K, V : [layers, kv_heads, T, d];  Q : [layers, q_heads, n_obs, d] with
+ * q head = kv_head * G + g, so the n_q = G * n_obs rows of one KV head are
+ * contiguous.  Outputs are [layers, kv_heads, k_eff, ...].  delta_out (may be
+ * NULL) is [layers, kv_heads, d].  Heads run in parallel when built with
+ * OpenMP.  Returns k_eff.
+ */
+int obf_oracle_compress(const float *K, const float *V, const float *Q,
+                        int layers, int kv_heads, int q_heads, int n_obs, int T, int d,
+                        int budget, int rank, double eps,
+                        int32_t *idx_out, double *K_out, double *V_out,
+                        double *delta_out, obf_oracle_diag_t *diag_out)
+{
+    const int G = q_heads / kv_heads;
+    const int n_q = G * n_obs;
+    const int k = budget < T ? budget : T;
+    const int heads = layers * kv_heads;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int lh = 0; lh < heads; ++lh) {
+        const float *Kh = K + (size_t)lh * T * d;
+        const float *Vh = V + (size_t)lh * T * d;
+        const float *Qh = Q + (size_t)lh * n_q * d;
+        obf_oracle_head(Kh, Vh, Qh, T, d, n_q, budget, rank, eps,
+                        idx_out + (size_t)lh * k,
+                        K_out + (size_t)lh * k * d, V_out + (size_t)lh * k * d,
+                        NULL, delta_out ? delta_out + (size_t)lh * d : NULL, NULL, NULL, NULL, NULL,
+                        diag_out ? diag_out + lh : NULL);
+    }
+    return k;
+}
+
+int obf_oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
