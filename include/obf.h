@@ -1,0 +1,192 @@
+/*
+ * obf.h - C ABI of the relay-boundary prompt-KV compressor for NVIDIA B200 (sm_100a).
+ *
+ * One call compresses the prompt KV cache of one or more agents at the relay
+ * boundary.  For every (cache, layer, KV head), independently (Section 4.4):
+ *
+ *   a1  score    A_j = sum over the observation queries t mapped to this KV head of
+ *                softmax_j(q_t . K_j / sqrt(head_dim))            (Eq. 1; softmax form of App. L.1)
+ *   a2  select   the k_eff = min(budget, T) positions of largest A_j, equal masses
+ *                resolved towards the lower position, emitted in ascending
+ *                position order                                   (Section 4.3.2; Section 3.1)
+ *   a3  gather   K_keep = K[idx,:], V_keep = V[idx,:]             (Algorithm 2, last step)
+ *   a4  OBF      orthonormal basis of span(V_keep) (Eq. 2); residual of the deleted
+ *                values against that span (Eq. 3); its top-`rank` right singular
+ *                subspace C; attention-weighted residual mean r_bar (Eq. 4);
+ *                Delta = (r_bar C^T) C (Eq. 5); delta = A_del/(A_keep+eps) * Delta
+ *                (Eq. 6); V_out = V_keep + delta on every retained row, keys
+ *                untouched (Eq. 7; Algorithm 3)
+ *
+ * All pointers in obf_cache_t are DEVICE pointers unless a function says
+ * otherwise.  The caller owns every buffer, including the workspace; the
+ * library allocates no device memory, enqueues all work on `stream`, never
+ * synchronises (except obf_last_device_status and the *_host entry point's
+ * final wait, as documented) and does not touch the inputs after the enqueued
+ * work has completed.  Inputs are read-only and must not alias outputs.
+ *
+ * Layout (row-major, contiguous, 16-byte aligned base pointers):
+ *   k, v      [layers, kv_heads, T, head_dim]
+ *   q_obs     [layers, q_heads, n_obs, head_dim]   q head = kv_head * G + g, G = q_heads / kv_heads
+ *   k_out,
+ *   v_out     [layers, kv_heads, k_eff, head_dim]  same dtype as the inputs
+ *   idx_out   [layers, kv_heads, k_eff] int32      ascending positions in [0, T)
+ *
+ * Numerics: bf16 products accumulated in fp32; softmax, pooling, selection
+ * keys and all OBF algebra in fp32; V_out is the fp32 sum rounded once to the
+ * output dtype (bit-exact copy of V_keep wherever delta == 0).  K_out is always
+ * a bit-exact copy.
+ *
+ * Errors: anything detectable on the host (null or misaligned pointer, bad
+ * shape, budget < 1, rank outside [0, head_dim], unsupported head_dim or dtype,
+ * workspace too small) returns a code before anything is enqueued.  Conditions
+ * only the device can see are ORed into a status word in the workspace (and
+ * into obf_diag_t.status of the head concerned); obf_last_device_status reads
+ * it.  A head that hits one keeps its eviction-only result (the skip rule in
+ * the footnote to Eq. 7).
+ */
+#ifndef OBF_H_
+#define OBF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    OBF_OK = 0,
+    OBF_ERR_INVALID_ARG = 1,    /* null/misaligned pointer, bad shape, budget, rank, n_caches    */
+    OBF_ERR_UNSUPPORTED = 2,    /* head_dim not in {64,128}, unknown dtype, too many caches       */
+    OBF_ERR_WORKSPACE = 3,      /* workspace null, misaligned or smaller than obf_workspace_bytes */
+    OBF_ERR_CUDA = 4,           /* a CUDA runtime call failed (launch, attribute, copy)           */
+    OBF_ERR_DEVICE_STATUS = 5   /* the device status word is non-zero (obf_last_device_status)    */
+} obf_status_t;
+
+typedef enum { OBF_F32 = 0, OBF_BF16 = 1 } obf_dtype_t;
+
+/* Bits of the device status word / obf_diag_t.status. */
+#define OBF_DEV_NONFINITE   0x1u   /* a score or softmax normaliser was not finite                 */
+#define OBF_DEV_NO_CONVERGE 0x2u   /* the eigen-iteration hit its sweep limit                      */
+#define OBF_DEV_TIMEOUT     0x4u   /* a bounded on-device wait expired                             */
+#define OBF_DEV_SKIPPED     0x100u /* informational (diag only): OBF skipped, delta = 0            */
+#define OBF_DEV_SPAN_FULL   0x200u /* informational (diag only): span(V_keep) is all of R^d        */
+
+/* obf_params_t.flags */
+#define OBF_FLAG_GENERIC_PATH 0x1u /* run the shape-generic kernels even where the tuned bf16 path applies */
+
+#define OBF_MAX_CACHES 32          /* caches per call                                              */
+#define OBF_MAX_T (1 << 20)        /* prompt positions per cache                                   */
+
+typedef struct {              /* shared by all caches of one call                                   */
+    int32_t layers, kv_heads, q_heads;  /* q_heads % kv_heads == 0                                  */
+    int32_t head_dim;                   /* 64 or 128                                                */
+    int32_t n_obs;                      /* observation queries per query head (>= 1)                */
+    int32_t rank;                       /* pca_rank of Section 4.4; 0 = eviction only               */
+    int32_t dtype;                      /* obf_dtype_t of k, v, q_obs, k_out, v_out                 */
+    float   eps;                        /* the epsilon of Eq. 4 and Eq. 6 (the paper uses 1e-12)    */
+    uint32_t flags;                     /* OBF_FLAG_*                                               */
+} obf_params_t;
+
+typedef struct {              /* per (layer, KV head) diagnostics (App. K.2 names in brackets)      */
+    float a_keep, a_del;      /* attention mass on retained / deleted positions (Eq. 6)             */
+    float alpha;              /* a_del / (a_keep + eps)                              [DR]           */
+    float rcr;                /* ||R||_F^2 / (||V_del||_F^2 + eps)                   [RCR]          */
+    float delta_norm;         /* ||delta||_2                                         [IVN]          */
+    float kth_score;          /* k_eff-th largest A_j                                               */
+    float next_score;         /* (k_eff+1)-th largest A_j, -1 if none                               */
+    float lam_1, lam_rho, lam_next; /* eigenvalues of R^T R: largest, last kept, first dropped      */
+    int32_t span_rank;        /* numerical dimension m of span(V_keep) (-1: not evaluated)          */
+    int32_t rho_eff;          /* number of principal directions actually used                       */
+    uint32_t status;          /* OBF_DEV_* bits                                                     */
+    int32_t reserved;
+} obf_diag_t;
+
+typedef struct {              /* one agent's prompt cache; T and budget may differ between caches   */
+    const void *k, *v;        /* [layers, kv_heads, T, head_dim]                                    */
+    const void *q_obs;        /* [layers, q_heads, n_obs, head_dim]                                 */
+    int32_t T;                /* prompt positions, 1 <= T <= OBF_MAX_T                              */
+    int32_t budget;           /* >= 1; k_eff = min(budget, T)                                       */
+    void *k_out, *v_out;      /* [layers, kv_heads, k_eff, head_dim]                                */
+    int32_t *idx_out;         /* [layers, kv_heads, k_eff]                                          */
+    obf_diag_t *diag_out;     /* optional [layers, kv_heads], or NULL                               */
+    float *scores_out;        /* optional [layers, kv_heads, T] attention mass A (Eq. 1), or NULL   */
+    float *delta_out;         /* optional [layers, kv_heads, head_dim] injected vector (Eq. 6), or NULL */
+} obf_cache_t;
+
+/*
+ * Size in bytes of the scratch workspace obf_compress / evict_only need for
+ * this call shape (Eq. 1's masses, selection flags, the d x d Gram matrices of
+ * Eq. 3 and App. H).  Host-only; enqueues nothing.  Pointers inside `caches`
+ * are not inspected, only T and budget.
+ */
+obf_status_t obf_workspace_bytes(const obf_params_t *params, const obf_cache_t *caches,
+                                 int32_t n_caches, size_t *bytes);
+
+/*
+ * Phi_OBF (Algorithm 3) on every (cache, layer, KV head).  `params`/`caches`
+ * are host structs (copied before return); `workspace` is device memory of at
+ * least obf_workspace_bytes(), 256-byte aligned, private to this call until
+ * the enqueued work completes; `stream` is a cudaStream_t passed as void*.
+ */
+obf_status_t obf_compress(const obf_params_t *params, const obf_cache_t *caches, int32_t n_caches,
+                          void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Phi_Attn with headwise granularity (Algorithm 2): steps a1-a3 only.
+ * Identical to obf_compress with rank = 0 (params->rank is ignored).
+ */
+obf_status_t evict_only(const obf_params_t *params, const obf_cache_t *caches, int32_t n_caches,
+                        void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Size of the device arena obf_compress_host needs (device copies of every
+ * input and output of the call plus the workspace).
+ */
+obf_status_t obf_host_arena_bytes(const obf_params_t *params, const obf_cache_t *caches,
+                                  int32_t n_caches, size_t *bytes);
+
+/*
+ * Same operation for callers whose caches live in HOST memory (Algorithm 1's
+ * relay hand-off when the cache is staged on the host).  Every pointer inside
+ * `caches` is a host pointer (pinned memory makes the copies asynchronous);
+ * `device_arena` is device memory of at least obf_host_arena_bytes(),
+ * 256-byte aligned.  Enqueues host->device copies of k, v, q_obs, the
+ * compression, and device->host copies of k_out, v_out, idx_out (and of
+ * diag_out / delta_out / scores_out when non-NULL) on `stream`, then waits for
+ * the stream.
+ */
+obf_status_t obf_compress_host(const obf_params_t *params, const obf_cache_t *caches, int32_t n_caches,
+                               void *device_arena, size_t arena_bytes, void *stream);
+
+/*
+ * Waits for `stream`, reads the status word the last call left in `workspace`
+ * and stores it in *device_status.  Returns OBF_ERR_DEVICE_STATUS if any of
+ * the error bits (OBF_DEV_NONFINITE, OBF_DEV_NO_CONVERGE, OBF_DEV_TIMEOUT) is set.
+ */
+obf_status_t obf_last_device_status(const void *workspace, void *stream, uint32_t *device_status);
+
+/*
+ * obf_compress with per-kernel device timing, for profiling only.  Enqueues the
+ * same kernels as obf_compress (params->rank == 0 gives evict_only's), with a
+ * CUDA event recorded between consecutive launches, waits for the stream and
+ * writes the elapsed milliseconds of each launch to phase_ms[0 .. *n_phases-1]
+ * (host array with room for OBF_MAX_PHASES floats).  obf_phase_name(i) names
+ * launch i of the last profiled call of this thread.
+ */
+#define OBF_MAX_PHASES 16
+obf_status_t obf_compress_profiled(const obf_params_t *params, const obf_cache_t *caches, int32_t n_caches,
+                                   void *workspace, size_t workspace_bytes, void *stream,
+                                   float *phase_ms, int32_t *n_phases);
+const char *obf_phase_name(int32_t phase);
+
+/* Static, never NULL. */
+const char *obf_status_string(obf_status_t status);
+
+/* Number of kernels the last obf_compress / evict_only call of this thread enqueued. */
+int32_t obf_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OBF_H_ */

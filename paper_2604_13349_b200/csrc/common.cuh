@@ -1,0 +1,158 @@
+// Shared device-side definitions for the relay-compression kernels.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "obf.h"
+
+namespace obf {
+
+// One cache as the kernels see it (device pointers, resolved sizes).
+struct CacheDev {
+    const void *k, *v, *q;
+    void *k_out, *v_out;
+    int32_t *idx_out;
+    obf_diag_t *diag;
+    float *scores_out;
+    float *delta_out;
+    int32_t T, k_eff;
+    int32_t head_base;        // global id of this cache's first (layer, kv head)
+    int32_t pad_;
+    size_t tok_off;           // offset of this cache in the per-token workspace arrays (elements)
+};
+
+// Everything one call needs, passed by value as a __grid_constant__ kernel parameter.
+struct CallDev {
+    CacheDev c[OBF_MAX_CACHES];
+    int32_t n_caches;
+    int32_t heads_per_cache;  // layers * kv_heads
+    int32_t heads_total;
+    int32_t n_q;              // G * n_obs query rows pooled into one KV head
+    int32_t d;
+    int32_t rank;
+    int32_t splits;           // token splits of the Gram pass
+    float eps;
+    // workspace
+    uint32_t *status;
+    float *scores;            // [sum heads*T] attention mass (Eq. 1)
+    uint8_t *keep;            // [sum heads*T] 1 = retained
+    float *stats;             // [heads_total, n_q, 2] softmax row max (log2 domain) and normaliser
+    float *sums;              // [heads_total, 4] a_keep, a_del, kth, next
+    float *gram_d;            // [heads_total, splits, d, d] partial Gram of deleted values
+    float *gram_k;            // [heads_total, splits, d, d] partial Gram of retained values
+    float *uvec;              // [heads_total, splits, d] partial sum_j A_j v_j over deleted j
+    float *delta;             // [heads_total, d]
+    uint32_t *hflag;          // [heads_total] bit0: delta != 0 -> inject
+};
+
+__device__ __forceinline__ void locate(const CallDev &p, int g, int &ci, int &lh)
+{
+    ci = 0;
+#pragma unroll 1
+    for (int i = 1; i < p.n_caches; ++i)
+        if (g >= p.c[i].head_base) ci = i;
+    lh = g - p.c[ci].head_base;
+}
+
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+// Loads `rows_tile` rows of D elements starting at row0 of a [n_rows, D] matrix
+// into shared memory as float with row stride `ld`; rows >= n_rows become zero.
+template <typename TIN, int D, int NT>
+__device__ __forceinline__ void load_rows_f32(float *dst, int ld, const TIN *src, int row0, int n_rows,
+                                              int rows_tile)
+{
+    constexpr int VEC = 16 / sizeof(TIN);        // elements per 16-byte vector
+    constexpr int CH = D / VEC;                  // vectors per row
+    for (int i = threadIdx.x; i < rows_tile * CH; i += NT) {
+        int r = i / CH, ch = i - r * CH;
+        float *o = dst + r * ld + ch * VEC;
+        if (row0 + r < n_rows) {
+            const uint4 raw = *reinterpret_cast<const uint4 *>(src + (size_t)(row0 + r) * D + ch * VEC);
+            if constexpr (sizeof(TIN) == 4) {
+                o[0] = __uint_as_float(raw.x); o[1] = __uint_as_float(raw.y);
+                o[2] = __uint_as_float(raw.z); o[3] = __uint_as_float(raw.w);
+            } else {
+                const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    o[2 * e] = __uint_as_float(w[e] << 16);
+                    o[2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) o[e] = 0.f;
+        }
+    }
+}
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ float warp_max(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// Block-wide sum in a fixed order (deterministic).  `red` holds >= 32 floats.
+template <int NT>
+__device__ __forceinline__ float block_sum(float v, float *red)
+{
+    v = warp_sum(v);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float t = 0.f;
+    if (threadIdx.x < 32) {
+        t = threadIdx.x < NT / 32 ? red[threadIdx.x] : 0.f;
+        t = warp_sum(t);
+        if (threadIdx.x == 0) red[0] = t;
+    }
+    __syncthreads();
+    t = red[0];
+    __syncthreads();
+    return t;
+}
+
+template <int NT>
+__device__ __forceinline__ float block_max(float v, float *red)
+{
+    v = warp_max(v);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float t;
+    if (threadIdx.x < 32) {
+        t = threadIdx.x < NT / 32 ? red[threadIdx.x] : -INFINITY;
+        t = warp_max(t);
+        if (threadIdx.x == 0) red[0] = t;
+    }
+    __syncthreads();
+    t = red[0];
+    __syncthreads();
+    return t;
+}
+
+// Order-preserving map from a float's bits to an unsigned key (larger float -> larger key).
+__device__ __forceinline__ uint32_t score_key(float a)
+{
+    uint32_t u = __float_as_uint(a);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__device__ __forceinline__ float key_score(uint32_t k)
+{
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
+}
+
+}  // namespace obf

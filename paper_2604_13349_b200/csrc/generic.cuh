@@ -1,0 +1,397 @@
+// Shape-generic kernels (any n_q, T; head_dim 64 or 128; fp32 or bf16 inputs).
+// All arithmetic is fp32 on the CUDA cores.  These kernels are the only path for
+// fp32 caches and for shapes the tuned bf16 path does not cover.
+#pragma once
+
+#include "common.cuh"
+
+namespace obf {
+
+constexpr int SC_TILE = 64;           // queries x keys per score tile
+constexpr int SC_NT = 256;
+constexpr float LOG2E = 1.4426950408889634f;
+
+template <int D>
+constexpr size_t score_smem_bytes() { return 2 * SC_TILE * (D + 1) * sizeof(float) + 2 * SC_TILE * sizeof(float)
+                                             + 16 * SC_TILE * sizeof(float); }
+
+// 64x64 tile of Q K^T on a 16x16 thread grid: thread (ty,tx) owns rows ty+16i, cols tx+16j.
+template <int D>
+__device__ __forceinline__ void score_tile(const float *Qs, const float *Ks, int ty, int tx, float (&acc)[4][4])
+{
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+#pragma unroll 4
+    for (int c = 0; c < D; ++c) {
+        float a[4], b[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) a[i] = Qs[(ty + 16 * i) * (D + 1) + c];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) b[j] = Ks[(tx + 16 * j) * (D + 1) + c];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+}
+
+// Step a1, first pass (Eq. 1): for every query row the running maximum of the
+// scaled logits (log2 domain) and the softmax normaliser over all T keys.
+// grid = (ceil(n_q/64), heads_total).
+template <typename TIN, int D>
+__global__ void __launch_bounds__(SC_NT) k_score_stats(const __grid_constant__ CallDev p)
+{
+    extern __shared__ float sm[];
+    float *Qs = sm, *Ks = sm + SC_TILE * (D + 1);
+    int ci, lh;
+    locate(p, blockIdx.y, ci, lh);
+    const CacheDev &c = p.c[ci];
+    const int T = c.T, n_q = p.n_q;
+    const int q0 = blockIdx.x * SC_TILE;
+    const TIN *Kh = reinterpret_cast<const TIN *>(c.k) + (size_t)lh * T * D;
+    const TIN *Qh = reinterpret_cast<const TIN *>(c.q) + (size_t)lh * n_q * D;
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const float sc = LOG2E * rsqrtf((float)D);
+
+    load_rows_f32<TIN, D, SC_NT>(Qs, D + 1, Qh, q0, n_q, SC_TILE);
+    float m[4], Z[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { m[i] = -INFINITY; Z[i] = 0.f; }
+
+    for (int j0 = 0; j0 < T; j0 += SC_TILE) {
+        __syncthreads();
+        load_rows_f32<TIN, D, SC_NT>(Ks, D + 1, Kh, j0, T, SC_TILE);
+        __syncthreads();
+        float acc[4][4];
+        score_tile<D>(Qs, Ks, ty, tx, acc);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float tm = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                acc[i][j] = (j0 + tx + 16 * j < T) ? acc[i][j] * sc : -INFINITY;
+                tm = fmaxf(tm, acc[i][j]);
+            }
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) tm = fmaxf(tm, __shfl_xor_sync(0xffffffffu, tm, o));
+            const float nm = fmaxf(m[i], tm);
+            float s = 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) s += exp2f(acc[i][j] - nm);
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+            Z[i] = Z[i] * exp2f(m[i] - nm) + s;
+            m[i] = nm;
+        }
+    }
+    if (tx == 0) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int row = q0 + ty + 16 * i;
+            if (row < n_q) {
+                float *st = p.stats + ((size_t)blockIdx.y * n_q + row) * 2;
+                st[0] = m[i];
+                st[1] = Z[i];
+            }
+        }
+    }
+}
+
+// Step a1, second pass (Eq. 1): A_j = sum_t exp(s_tj - m_t) / Z_t for a tile of 64 keys.
+// grid = (ceil(T_max/64), heads_total); blocks beyond a cache's T exit.
+template <typename TIN, int D>
+__global__ void __launch_bounds__(SC_NT) k_score_pool(const __grid_constant__ CallDev p)
+{
+    extern __shared__ float sm[];
+    float *Qs = sm, *Ks = sm + SC_TILE * (D + 1);
+    float *rm = Ks + SC_TILE * (D + 1), *rz = rm + SC_TILE, *red = rz + SC_TILE;
+    int ci, lh;
+    locate(p, blockIdx.y, ci, lh);
+    const CacheDev &c = p.c[ci];
+    const int T = c.T, n_q = p.n_q;
+    const int j0 = blockIdx.x * SC_TILE;
+    if (j0 >= T) return;
+    const TIN *Kh = reinterpret_cast<const TIN *>(c.k) + (size_t)lh * T * D;
+    const TIN *Qh = reinterpret_cast<const TIN *>(c.q) + (size_t)lh * n_q * D;
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const float sc = LOG2E * rsqrtf((float)D);
+
+    load_rows_f32<TIN, D, SC_NT>(Ks, D + 1, Kh, j0, T, SC_TILE);
+    float colsum[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int q0 = 0; q0 < n_q; q0 += SC_TILE) {
+        __syncthreads();
+        load_rows_f32<TIN, D, SC_NT>(Qs, D + 1, Qh, q0, n_q, SC_TILE);
+        if (threadIdx.x < SC_TILE) {
+            const int row = q0 + threadIdx.x;
+            const float *st = p.stats + ((size_t)blockIdx.y * n_q + min(row, n_q - 1)) * 2;
+            rm[threadIdx.x] = row < n_q ? st[0] : 0.f;
+            rz[threadIdx.x] = row < n_q ? 1.0f / st[1] : 0.f;
+        }
+        __syncthreads();
+        float acc[4][4];
+        score_tile<D>(Qs, Ks, ty, tx, acc);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float mi = rm[ty + 16 * i], zi = rz[ty + 16 * i];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) colsum[j] += exp2f(acc[i][j] * sc - mi) * zi;
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) red[ty * SC_TILE + tx + 16 * j] = colsum[j];
+    __syncthreads();
+    if (threadIdx.x < SC_TILE && j0 + threadIdx.x < T) {
+        float a = 0.f;
+#pragma unroll
+        for (int r = 0; r < 16; ++r) a += red[r * SC_TILE + threadIdx.x];
+        if (!isfinite(a)) atomicOr(p.status, OBF_DEV_NONFINITE);
+        p.scores[c.tok_off + (size_t)lh * T + j0 + threadIdx.x] = a;
+        if (c.scores_out) c.scores_out[(size_t)lh * T + j0 + threadIdx.x] = a;
+    }
+}
+
+// Step a2: radix select of the k_eff largest masses on their order-preserving
+// 32-bit keys (4 passes of 8 bits), then one ordered pass that emits the
+// retained positions in ascending order; among masses equal to the k_eff-th
+// largest, the lowest positions are taken.  One block per (cache, layer, head).
+constexpr int SEL_NT = 1024;
+
+__global__ void __launch_bounds__(SEL_NT) k_select(const __grid_constant__ CallDev p)
+{
+    __shared__ uint32_t hist[256];
+    __shared__ uint32_t s_prefix, s_want;
+    __shared__ uint32_t wsum[32];
+    __shared__ float red[32];
+    int ci, lh;
+    locate(p, blockIdx.x, ci, lh);
+    const CacheDev &c = p.c[ci];
+    const int T = c.T, k = c.k_eff;
+    const float *A = p.scores + c.tok_off + (size_t)lh * T;
+    uint8_t *keep = p.keep + c.tok_off + (size_t)lh * T;
+    int32_t *idx = c.idx_out + (size_t)lh * k;
+    const int tid = threadIdx.x;
+
+    if (tid == 0) { s_prefix = 0u; s_want = (uint32_t)k; }
+    uint32_t mask = 0u;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        if (tid < 256) hist[tid] = 0u;
+        __syncthreads();
+        const uint32_t prefix = s_prefix;
+        for (int j = tid; j < T; j += SEL_NT) {
+            const uint32_t u = score_key(A[j]);
+            if ((u & mask) == prefix) atomicAdd(&hist[(u >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        if (tid == 0) {
+            uint32_t want = s_want, cum = 0u;
+            int b = 255;
+            for (; b > 0; --b) {
+                if (cum + hist[b] >= want) break;
+                cum += hist[b];
+            }
+            s_want = want - cum;
+            s_prefix = prefix | ((uint32_t)b << shift);
+        }
+        mask |= 255u << shift;
+        __syncthreads();
+    }
+    const uint32_t tau = s_prefix;       // key of the k-th largest mass
+    const uint32_t want = s_want;        // how many positions with key == tau are retained (>= 1)
+
+    uint32_t run_gt = 0u, run_eq = 0u;
+    float sk = 0.f, sd = 0.f, nx = -1.0f;
+    for (int base = 0; base < T; base += SEL_NT) {
+        const int j = base + tid;
+        const bool valid = j < T;
+        const float a = valid ? A[j] : 0.f;
+        const uint32_t u = valid ? score_key(a) : 0u;
+        const bool gt = valid && u > tau, eq = valid && u == tau;
+        uint32_t v = (gt ? 1u : 0u) | (eq ? 0x10000u : 0u);
+        uint32_t inc = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t n = __shfl_up_sync(0xffffffffu, inc, o);
+            if ((tid & 31) >= o) inc += n;
+        }
+        if ((tid & 31) == 31) wsum[tid >> 5] = inc;
+        __syncthreads();
+        if (tid < 32) {
+            uint32_t w = wsum[tid], winc = w;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t n = __shfl_up_sync(0xffffffffu, winc, o);
+                if (tid >= o) winc += n;
+            }
+            wsum[tid] = winc - w;          // exclusive prefix of warp totals
+            if (tid == 31) hist[0] = winc; // block total
+        }
+        __syncthreads();
+        const uint32_t excl = inc - v + wsum[tid >> 5];
+        const uint32_t gt_before = run_gt + (excl & 0xFFFFu), eq_before = run_eq + (excl >> 16);
+        const bool kp = gt || (eq && eq_before < want);
+        if (valid) {
+            keep[j] = kp ? 1 : 0;
+            if (kp) { idx[gt_before + min(eq_before, want)] = j; sk += a; }
+            else { sd += a; nx = fmaxf(nx, a); }
+        }
+        const uint32_t tot = hist[0];
+        run_gt += tot & 0xFFFFu;
+        run_eq += tot >> 16;
+        __syncthreads();
+    }
+    const float a_keep = block_sum<SEL_NT>(sk, red);
+    const float a_del = block_sum<SEL_NT>(sd, red);
+    const float next = block_max<SEL_NT>(nx, red);
+    if (tid == 0) {
+        float *s = p.sums + (size_t)blockIdx.x * 4;
+        s[0] = a_keep; s[1] = a_del; s[2] = key_score(tau); s[3] = next;
+        if (c.diag) {
+            obf_diag_t dg;
+            dg.a_keep = a_keep; dg.a_del = a_del; dg.alpha = a_del / (a_keep + p.eps);
+            dg.rcr = 0.f; dg.delta_norm = 0.f; dg.kth_score = key_score(tau); dg.next_score = next;
+            dg.lam_1 = dg.lam_rho = dg.lam_next = 0.f;
+            dg.span_rank = -1; dg.rho_eff = 0; dg.status = OBF_DEV_SKIPPED; dg.reserved = 0;
+            c.diag[lh] = dg;
+        }
+    }
+}
+
+// Step a3: K_out = K[idx], V_out = V[idx], one warp per retained row, 16-byte vectors.
+// grid = (ceil(k_eff_max/8), heads_total).
+template <int ROW_BYTES>
+__global__ void __launch_bounds__(256) k_gather(const __grid_constant__ CallDev p)
+{
+    int ci, lh;
+    locate(p, blockIdx.y, ci, lh);
+    const CacheDev &c = p.c[ci];
+    const int r = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (r >= c.k_eff) return;
+    const int lane = threadIdx.x & 31;
+    const int j = c.idx_out[(size_t)lh * c.k_eff + r];
+    constexpr int CH = ROW_BYTES / 16;
+    const uint4 *ks = reinterpret_cast<const uint4 *>(reinterpret_cast<const char *>(c.k) + ((size_t)lh * c.T + j) * ROW_BYTES);
+    const uint4 *vs = reinterpret_cast<const uint4 *>(reinterpret_cast<const char *>(c.v) + ((size_t)lh * c.T + j) * ROW_BYTES);
+    uint4 *kd = reinterpret_cast<uint4 *>(reinterpret_cast<char *>(c.k_out) + ((size_t)lh * c.k_eff + r) * ROW_BYTES);
+    uint4 *vd = reinterpret_cast<uint4 *>(reinterpret_cast<char *>(c.v_out) + ((size_t)lh * c.k_eff + r) * ROW_BYTES);
+    for (int ch = lane; ch < CH; ch += 32) {
+        kd[ch] = ks[ch];
+        vd[ch] = vs[ch];
+    }
+}
+
+// Step a4, streaming part: one pass over V accumulating, per head and token
+// split, the Gram matrix of the deleted rows (for R^T R = P G_del P, App. H), the
+// Gram matrix of the retained rows (only when k_eff >= d, for the span test) and
+// u = sum over deleted j of A_j v_j (for r_bar, Eq. 4).
+// grid = (splits, heads_total), 256 threads as a 16x16 grid of (D/16)^2 register tiles.
+constexpr int GR_ROWS = 32;
+
+template <typename TIN, int D>
+__global__ void __launch_bounds__(256) k_gram(const __grid_constant__ CallDev p)
+{
+    constexpr int NV = D / 64;               // float4 groups per thread along each axis
+    constexpr int MT = 4 * NV;
+    __shared__ __align__(16) float Vs[GR_ROWS * D];
+    __shared__ float As[GR_ROWS];
+    __shared__ int Fs[GR_ROWS];
+    int ci, lh;
+    locate(p, blockIdx.y, ci, lh);
+    const CacheDev &c = p.c[ci];
+    const int T = c.T;
+    const bool need_k = c.k_eff >= D;
+    const TIN *Vh = reinterpret_cast<const TIN *>(c.v) + (size_t)lh * T * D;
+    const float *A = p.scores + c.tok_off + (size_t)lh * T;
+    const uint8_t *keep = p.keep + c.tok_off + (size_t)lh * T;
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+
+    const int tiles = (T + GR_ROWS - 1) / GR_ROWS;
+    const int per = (tiles + p.splits - 1) / p.splits;
+    const int t_begin = blockIdx.x * per, t_end = min(tiles, t_begin + per);
+
+    float accD[MT][MT], accK[MT][MT];
+#pragma unroll
+    for (int i = 0; i < MT; ++i)
+#pragma unroll
+        for (int j = 0; j < MT; ++j) { accD[i][j] = 0.f; accK[i][j] = 0.f; }
+    float u = 0.f;
+
+    for (int t = t_begin; t < t_end; ++t) {
+        const int r0 = t * GR_ROWS;
+        __syncthreads();
+        load_rows_f32<TIN, D, 256>(Vs, D, Vh, r0, T, GR_ROWS);
+        if (threadIdx.x < GR_ROWS) {
+            const int j = r0 + threadIdx.x;
+            Fs[threadIdx.x] = j < T ? (int)keep[j] : 2;
+            As[threadIdx.x] = j < T ? A[j] : 0.f;
+        }
+        __syncthreads();
+#pragma unroll 1
+        for (int r = 0; r < GR_ROWS; ++r) {
+            const int f = Fs[r];
+            if (f == 2) break;
+            if (f == 1 && !need_k) continue;
+            float a[MT], b[MT];
+#pragma unroll
+            for (int v = 0; v < NV; ++v) {
+                const float4 fa = *reinterpret_cast<const float4 *>(&Vs[r * D + v * 64 + ty * 4]);
+                const float4 fb = *reinterpret_cast<const float4 *>(&Vs[r * D + v * 64 + tx * 4]);
+                a[4 * v] = fa.x; a[4 * v + 1] = fa.y; a[4 * v + 2] = fa.z; a[4 * v + 3] = fa.w;
+                b[4 * v] = fb.x; b[4 * v + 1] = fb.y; b[4 * v + 2] = fb.z; b[4 * v + 3] = fb.w;
+            }
+            if (f == 0) {
+#pragma unroll
+                for (int i = 0; i < MT; ++i)
+#pragma unroll
+                    for (int j = 0; j < MT; ++j) accD[i][j] = fmaf(a[i], b[j], accD[i][j]);
+                if (threadIdx.x < D) u = fmaf(As[r], Vs[r * D + threadIdx.x], u);
+            } else {
+#pragma unroll
+                for (int i = 0; i < MT; ++i)
+#pragma unroll
+                    for (int j = 0; j < MT; ++j) accK[i][j] = fmaf(a[i], b[j], accK[i][j]);
+            }
+        }
+    }
+    const size_t slot = (size_t)blockIdx.y * p.splits + blockIdx.x;
+    float *gd = p.gram_d + slot * D * D, *gk = p.gram_k + slot * D * D;
+#pragma unroll
+    for (int i = 0; i < MT; ++i) {
+        const int row = (i / 4) * 64 + ty * 4 + (i & 3);
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const int col = v * 64 + tx * 4;
+            *reinterpret_cast<float4 *>(&gd[row * D + col]) =
+                make_float4(accD[i][4 * v], accD[i][4 * v + 1], accD[i][4 * v + 2], accD[i][4 * v + 3]);
+            if (need_k)
+                *reinterpret_cast<float4 *>(&gk[row * D + col]) =
+                    make_float4(accK[i][4 * v], accK[i][4 * v + 1], accK[i][4 * v + 2], accK[i][4 * v + 3]);
+        }
+    }
+    if (threadIdx.x < D) p.uvec[slot * D + threadIdx.x] = u;
+}
+
+// Step a4, Eq. 7: V_out = V_keep + delta on every retained row of heads whose
+// delta is non-zero; the fp32 sum is rounded once to the output type.
+// grid = (ceil(k_eff_max/8), heads_total).
+template <typename TIN, int D>
+__global__ void __launch_bounds__(256) k_inject(const __grid_constant__ CallDev p)
+{
+    if ((p.hflag[blockIdx.y] & 1u) == 0u) return;
+    int ci, lh;
+    locate(p, blockIdx.y, ci, lh);
+    const CacheDev &c = p.c[ci];
+    const int r = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (r >= c.k_eff) return;
+    const int lane = threadIdx.x & 31;
+    const float *dl = p.delta + (size_t)blockIdx.y * D;
+    TIN *row = reinterpret_cast<TIN *>(c.v_out) + ((size_t)lh * c.k_eff + r) * D;
+    for (int e = lane; e < D; e += 32) {
+        const float s = to_f32(row[e]) + dl[e];
+        if constexpr (sizeof(TIN) == 4) row[e] = s;
+        else row[e] = __float2bfloat16_rn(s);
+    }
+}
+
+}  // namespace obf

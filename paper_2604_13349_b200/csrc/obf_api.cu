@@ -1,0 +1,413 @@
+// Host side of the C ABI declared in include/obf.h: argument validation,
+// workspace layout, kernel dispatch.  Allocates no device memory.
+#include <cstdio>
+#include <cstring>
+
+#include "algebra.cuh"
+#include "common.cuh"
+#include "generic.cuh"
+
+namespace obf {
+
+static thread_local int32_t g_last_launches = 0;
+
+// Optional per-launch timing (obf_compress_profiled): an event after every launch.
+struct Profiler {
+    cudaEvent_t ev[OBF_MAX_PHASES + 1];
+    const char *names[OBF_MAX_PHASES];
+    int n = 0;
+    bool active = false;
+};
+static thread_local Profiler g_prof;
+static thread_local const char *g_phase_names[OBF_MAX_PHASES];
+static thread_local int g_phase_count = 0;
+
+static inline void mark(cudaStream_t st, const char *name)
+{
+    ++g_last_launches;
+    if (g_prof.active && g_prof.n < OBF_MAX_PHASES) {
+        g_prof.names[g_prof.n] = name;
+        cudaEventRecord(g_prof.ev[++g_prof.n], st);
+    }
+}
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Layout {
+    size_t off_status, off_scores, off_keep, off_stats, off_sums;
+    size_t off_gram_d, off_gram_k, off_uvec, off_delta, off_hflag;
+    size_t total;
+    int splits;
+    int heads_total;
+    size_t tok_total;
+    size_t tok_off[OBF_MAX_CACHES];
+};
+
+static int choose_splits(int heads_total, int T_max)
+{
+    int s = (2 * 148 + heads_total - 1) / heads_total;
+    const int tiles = (T_max + GR_ROWS - 1) / GR_ROWS;
+    if (s > tiles) s = tiles;
+    if (s > 16) s = 16;
+    if (s < 1) s = 1;
+    return s;
+}
+
+static obf_status_t validate_shapes(const obf_params_t *p, const obf_cache_t *caches, int32_t n, int rank)
+{
+    if (!p || !caches) return OBF_ERR_INVALID_ARG;
+    if (n < 1) return OBF_ERR_INVALID_ARG;
+    if (n > OBF_MAX_CACHES) return OBF_ERR_UNSUPPORTED;
+    if (p->layers < 1 || p->kv_heads < 1 || p->q_heads < 1 || p->n_obs < 1) return OBF_ERR_INVALID_ARG;
+    if (p->q_heads % p->kv_heads != 0) return OBF_ERR_INVALID_ARG;
+    if (p->head_dim != 64 && p->head_dim != 128) return OBF_ERR_UNSUPPORTED;
+    if (p->dtype != OBF_F32 && p->dtype != OBF_BF16) return OBF_ERR_UNSUPPORTED;
+    if (rank < 0 || rank > p->head_dim) return OBF_ERR_INVALID_ARG;
+    if (!(p->eps >= 0.f)) return OBF_ERR_INVALID_ARG;
+    if ((long long)p->layers * p->kv_heads * n > (1 << 24)) return OBF_ERR_UNSUPPORTED;
+    for (int i = 0; i < n; ++i) {
+        if (caches[i].T < 1 || caches[i].T > OBF_MAX_T) return OBF_ERR_INVALID_ARG;
+        if (caches[i].budget < 1) return OBF_ERR_INVALID_ARG;
+    }
+    return OBF_OK;
+}
+
+static void make_layout(const obf_params_t *p, const obf_cache_t *caches, int32_t n, int rank, Layout &L)
+{
+    const int hpc = p->layers * p->kv_heads;
+    const int d = p->head_dim;
+    const int n_q = (p->q_heads / p->kv_heads) * p->n_obs;
+    L.heads_total = hpc * n;
+    size_t tok = 0;
+    int T_max = 1;
+    for (int i = 0; i < n; ++i) {
+        L.tok_off[i] = tok;
+        tok += (size_t)hpc * caches[i].T;
+        if (caches[i].T > T_max) T_max = caches[i].T;
+    }
+    L.tok_total = tok;
+    L.splits = choose_splits(L.heads_total, T_max);
+    size_t o = 0;
+    L.off_status = o; o += 256;
+    L.off_scores = o; o = align_up(o + tok * sizeof(float), 256);
+    L.off_keep = o;   o = align_up(o + tok, 256);
+    L.off_stats = o;  o = align_up(o + (size_t)L.heads_total * n_q * 2 * sizeof(float), 256);
+    L.off_sums = o;   o = align_up(o + (size_t)L.heads_total * 4 * sizeof(float), 256);
+    L.off_gram_d = L.off_gram_k = L.off_uvec = L.off_delta = L.off_hflag = o;
+    if (rank > 0) {
+        const size_t gsz = (size_t)L.heads_total * L.splits * d * d * sizeof(float);
+        L.off_gram_d = o; o = align_up(o + gsz, 256);
+        L.off_gram_k = o; o = align_up(o + gsz, 256);
+        L.off_uvec = o;   o = align_up(o + (size_t)L.heads_total * L.splits * d * sizeof(float), 256);
+        L.off_delta = o;  o = align_up(o + (size_t)L.heads_total * d * sizeof(float), 256);
+        L.off_hflag = o;  o = align_up(o + (size_t)L.heads_total * sizeof(uint32_t), 256);
+    }
+    L.total = o;
+}
+
+static bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+#define OBF_CUDA_TRY(expr)                                                        \
+    do {                                                                          \
+        cudaError_t e_ = (expr);                                                  \
+        if (e_ != cudaSuccess) {                                                  \
+            std::fprintf(stderr, "obf: %s failed: %s\n", #expr, cudaGetErrorString(e_)); \
+            return OBF_ERR_CUDA;                                                  \
+        }                                                                         \
+    } while (0)
+
+template <typename K>
+static obf_status_t set_smem(K kernel, size_t bytes)
+{
+    OBF_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+    return OBF_OK;
+}
+
+template <typename TIN, int D>
+static obf_status_t launch_generic(const CallDev &cd, int T_max, int k_max, cudaStream_t st)
+{
+    const int heads = cd.heads_total;
+    const size_t sm_sc = score_smem_bytes<D>();
+    obf_status_t s;
+    if ((s = set_smem(k_score_stats<TIN, D>, sm_sc)) != OBF_OK) return s;
+    if ((s = set_smem(k_score_pool<TIN, D>, sm_sc)) != OBF_OK) return s;
+    dim3 g1((cd.n_q + SC_TILE - 1) / SC_TILE, heads);
+    k_score_stats<TIN, D><<<g1, SC_NT, sm_sc, st>>>(cd);
+    mark(st, "k_score_stats");
+    dim3 g2((T_max + SC_TILE - 1) / SC_TILE, heads);
+    k_score_pool<TIN, D><<<g2, SC_NT, sm_sc, st>>>(cd);
+    mark(st, "k_score_pool");
+    k_select<<<heads, SEL_NT, 0, st>>>(cd);
+    mark(st, "k_select");
+    dim3 g4((k_max + 7) / 8, heads);
+    k_gather<D * (int)sizeof(TIN)><<<g4, 256, 0, st>>>(cd);
+    mark(st, "k_gather");
+    if (cd.rank > 0) {
+        const size_t sm_alg = algebra_smem_bytes<D>();
+        if ((s = set_smem(k_obf_algebra<TIN, D>, sm_alg)) != OBF_OK) return s;
+        dim3 g5(cd.splits, heads);
+        k_gram<TIN, D><<<g5, 256, 0, st>>>(cd);
+        mark(st, "k_gram");
+        k_obf_algebra<TIN, D><<<heads, ALG_NT, sm_alg, st>>>(cd);
+        mark(st, "k_obf_algebra");
+        k_inject<TIN, D><<<g4, 256, 0, st>>>(cd);
+        mark(st, "k_inject");
+    }
+    OBF_CUDA_TRY(cudaGetLastError());
+    return OBF_OK;
+}
+
+static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_t n, int rank,
+                        void *workspace, size_t workspace_bytes, void *stream)
+{
+    g_last_launches = 0;
+    obf_status_t s = validate_shapes(p, caches, n, rank);
+    if (s != OBF_OK) return s;
+    for (int i = 0; i < n; ++i) {
+        const obf_cache_t &c = caches[i];
+        if (!c.k || !c.v || !c.q_obs || !c.k_out || !c.v_out || !c.idx_out) return OBF_ERR_INVALID_ARG;
+        if (misaligned(c.k) || misaligned(c.v) || misaligned(c.q_obs) || misaligned(c.k_out) ||
+            misaligned(c.v_out) || (reinterpret_cast<uintptr_t>(c.idx_out) & 3u))
+            return OBF_ERR_INVALID_ARG;
+        if (c.diag_out && (reinterpret_cast<uintptr_t>(c.diag_out) & 3u)) return OBF_ERR_INVALID_ARG;
+        if (c.scores_out && (reinterpret_cast<uintptr_t>(c.scores_out) & 3u)) return OBF_ERR_INVALID_ARG;
+        if (c.delta_out && (reinterpret_cast<uintptr_t>(c.delta_out) & 3u)) return OBF_ERR_INVALID_ARG;
+    }
+    Layout L;
+    make_layout(p, caches, n, rank, L);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < L.total)
+        return OBF_ERR_WORKSPACE;
+
+    CallDev cd;
+    std::memset(&cd, 0, sizeof(cd));
+    const int hpc = p->layers * p->kv_heads;
+    int T_max = 1, k_max = 1;
+    for (int i = 0; i < n; ++i) {
+        CacheDev &c = cd.c[i];
+        c.k = caches[i].k; c.v = caches[i].v; c.q = caches[i].q_obs;
+        c.k_out = caches[i].k_out; c.v_out = caches[i].v_out; c.idx_out = caches[i].idx_out;
+        c.diag = caches[i].diag_out; c.scores_out = caches[i].scores_out; c.delta_out = caches[i].delta_out;
+        c.T = caches[i].T;
+        c.k_eff = caches[i].budget < caches[i].T ? caches[i].budget : caches[i].T;
+        c.head_base = i * hpc;
+        c.tok_off = L.tok_off[i];
+        if (c.T > T_max) T_max = c.T;
+        if (c.k_eff > k_max) k_max = c.k_eff;
+    }
+    cd.n_caches = n;
+    cd.heads_per_cache = hpc;
+    cd.heads_total = L.heads_total;
+    cd.n_q = (p->q_heads / p->kv_heads) * p->n_obs;
+    cd.d = p->head_dim;
+    cd.rank = rank;
+    cd.splits = L.splits;
+    cd.eps = p->eps;
+    char *ws = static_cast<char *>(workspace);
+    cd.status = reinterpret_cast<uint32_t *>(ws + L.off_status);
+    cd.scores = reinterpret_cast<float *>(ws + L.off_scores);
+    cd.keep = reinterpret_cast<uint8_t *>(ws + L.off_keep);
+    cd.stats = reinterpret_cast<float *>(ws + L.off_stats);
+    cd.sums = reinterpret_cast<float *>(ws + L.off_sums);
+    cd.gram_d = reinterpret_cast<float *>(ws + L.off_gram_d);
+    cd.gram_k = reinterpret_cast<float *>(ws + L.off_gram_k);
+    cd.uvec = reinterpret_cast<float *>(ws + L.off_uvec);
+    cd.delta = reinterpret_cast<float *>(ws + L.off_delta);
+    cd.hflag = reinterpret_cast<uint32_t *>(ws + L.off_hflag);
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    OBF_CUDA_TRY(cudaMemsetAsync(cd.status, 0, 256, st));
+    if (g_prof.active) cudaEventRecord(g_prof.ev[0], st);
+
+    if (p->dtype == OBF_F32) {
+        return p->head_dim == 64 ? launch_generic<float, 64>(cd, T_max, k_max, st)
+                                 : launch_generic<float, 128>(cd, T_max, k_max, st);
+    }
+    return p->head_dim == 64 ? launch_generic<__nv_bfloat16, 64>(cd, T_max, k_max, st)
+                             : launch_generic<__nv_bfloat16, 128>(cd, T_max, k_max, st);
+}
+
+}  // namespace obf
+
+using namespace obf;
+
+extern "C" {
+
+obf_status_t obf_workspace_bytes(const obf_params_t *params, const obf_cache_t *caches, int32_t n_caches,
+                                 size_t *bytes)
+{
+    if (!bytes) return OBF_ERR_INVALID_ARG;
+    obf_status_t s = validate_shapes(params, caches, n_caches, params ? params->rank : 0);
+    if (s != OBF_OK) return s;
+    Layout L;
+    make_layout(params, caches, n_caches, params->rank, L);
+    *bytes = L.total;
+    return OBF_OK;
+}
+
+obf_status_t obf_compress(const obf_params_t *params, const obf_cache_t *caches, int32_t n_caches,
+                          void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!params) return OBF_ERR_INVALID_ARG;
+    return run(params, caches, n_caches, params->rank, workspace, workspace_bytes, stream);
+}
+
+obf_status_t evict_only(const obf_params_t *params, const obf_cache_t *caches, int32_t n_caches,
+                        void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!params) return OBF_ERR_INVALID_ARG;
+    return run(params, caches, n_caches, 0, workspace, workspace_bytes, stream);
+}
+
+struct HostArena {
+    size_t k[OBF_MAX_CACHES], v[OBF_MAX_CACHES], q[OBF_MAX_CACHES];
+    size_t k_out[OBF_MAX_CACHES], v_out[OBF_MAX_CACHES], idx[OBF_MAX_CACHES];
+    size_t diag[OBF_MAX_CACHES], scores[OBF_MAX_CACHES], delta[OBF_MAX_CACHES];
+    size_t ws, ws_bytes, total;
+};
+
+static void host_arena_layout(const obf_params_t *p, const obf_cache_t *caches, int32_t n, HostArena &H)
+{
+    const size_t e = p->dtype == OBF_F32 ? 4 : 2;
+    const size_t hpc = (size_t)p->layers * p->kv_heads, d = p->head_dim;
+    size_t o = 0;
+    for (int i = 0; i < n; ++i) {
+        const size_t T = caches[i].T, ke = caches[i].budget < caches[i].T ? caches[i].budget : caches[i].T;
+        H.k[i] = o; o = align_up(o + hpc * T * d * e, 256);
+        H.v[i] = o; o = align_up(o + hpc * T * d * e, 256);
+        H.q[i] = o; o = align_up(o + (size_t)p->layers * p->q_heads * p->n_obs * d * e, 256);
+        H.k_out[i] = o; o = align_up(o + hpc * ke * d * e, 256);
+        H.v_out[i] = o; o = align_up(o + hpc * ke * d * e, 256);
+        H.idx[i] = o; o = align_up(o + hpc * ke * 4, 256);
+        H.diag[i] = o; o = align_up(o + hpc * sizeof(obf_diag_t), 256);
+        H.scores[i] = o; if (caches[i].scores_out) o = align_up(o + hpc * T * 4, 256);
+        H.delta[i] = o; o = align_up(o + hpc * d * 4, 256);
+    }
+    Layout L;
+    make_layout(p, caches, n, p->rank, L);
+    H.ws = o; H.ws_bytes = L.total; o += L.total;
+    H.total = o;
+}
+
+obf_status_t obf_host_arena_bytes(const obf_params_t *params, const obf_cache_t *caches, int32_t n_caches,
+                                  size_t *bytes)
+{
+    if (!bytes) return OBF_ERR_INVALID_ARG;
+    obf_status_t s = validate_shapes(params, caches, n_caches, params ? params->rank : 0);
+    if (s != OBF_OK) return s;
+    HostArena H;
+    host_arena_layout(params, caches, n_caches, H);
+    *bytes = H.total;
+    return OBF_OK;
+}
+
+obf_status_t obf_compress_host(const obf_params_t *params, const obf_cache_t *caches, int32_t n_caches,
+                               void *device_arena, size_t arena_bytes, void *stream)
+{
+    obf_status_t s = validate_shapes(params, caches, n_caches, params ? params->rank : 0);
+    if (s != OBF_OK) return s;
+    for (int i = 0; i < n_caches; ++i) {
+        const obf_cache_t &c = caches[i];
+        if (!c.k || !c.v || !c.q_obs || !c.k_out || !c.v_out || !c.idx_out) return OBF_ERR_INVALID_ARG;
+    }
+    HostArena H;
+    host_arena_layout(params, caches, n_caches, H);
+    if (!device_arena || (reinterpret_cast<uintptr_t>(device_arena) & 255u) || arena_bytes < H.total)
+        return OBF_ERR_WORKSPACE;
+    char *base = static_cast<char *>(device_arena);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t e = params->dtype == OBF_F32 ? 4 : 2;
+    const size_t hpc = (size_t)params->layers * params->kv_heads, d = params->head_dim;
+    obf_cache_t dev[OBF_MAX_CACHES];
+    for (int i = 0; i < n_caches; ++i) {
+        const obf_cache_t &c = caches[i];
+        const size_t T = c.T;
+        dev[i] = c;
+        dev[i].k = base + H.k[i]; dev[i].v = base + H.v[i]; dev[i].q_obs = base + H.q[i];
+        dev[i].k_out = base + H.k_out[i]; dev[i].v_out = base + H.v_out[i];
+        dev[i].idx_out = reinterpret_cast<int32_t *>(base + H.idx[i]);
+        dev[i].diag_out = c.diag_out ? reinterpret_cast<obf_diag_t *>(base + H.diag[i]) : nullptr;
+        dev[i].scores_out = c.scores_out ? reinterpret_cast<float *>(base + H.scores[i]) : nullptr;
+        dev[i].delta_out = c.delta_out ? reinterpret_cast<float *>(base + H.delta[i]) : nullptr;
+        OBF_CUDA_TRY(cudaMemcpyAsync(base + H.k[i], c.k, hpc * T * d * e, cudaMemcpyHostToDevice, st));
+        OBF_CUDA_TRY(cudaMemcpyAsync(base + H.v[i], c.v, hpc * T * d * e, cudaMemcpyHostToDevice, st));
+        OBF_CUDA_TRY(cudaMemcpyAsync(base + H.q[i], c.q_obs,
+                                     (size_t)params->layers * params->q_heads * params->n_obs * d * e,
+                                     cudaMemcpyHostToDevice, st));
+    }
+    s = run(params, dev, n_caches, params->rank, base + H.ws, H.ws_bytes, stream);
+    if (s != OBF_OK) return s;
+    for (int i = 0; i < n_caches; ++i) {
+        const obf_cache_t &c = caches[i];
+        const size_t T = c.T, ke = c.budget < c.T ? c.budget : c.T;
+        OBF_CUDA_TRY(cudaMemcpyAsync(c.k_out, base + H.k_out[i], hpc * ke * d * e, cudaMemcpyDeviceToHost, st));
+        OBF_CUDA_TRY(cudaMemcpyAsync(c.v_out, base + H.v_out[i], hpc * ke * d * e, cudaMemcpyDeviceToHost, st));
+        OBF_CUDA_TRY(cudaMemcpyAsync(c.idx_out, base + H.idx[i], hpc * ke * 4, cudaMemcpyDeviceToHost, st));
+        if (c.diag_out)
+            OBF_CUDA_TRY(cudaMemcpyAsync(c.diag_out, base + H.diag[i], hpc * sizeof(obf_diag_t),
+                                         cudaMemcpyDeviceToHost, st));
+        if (c.scores_out)
+            OBF_CUDA_TRY(cudaMemcpyAsync(c.scores_out, base + H.scores[i], hpc * T * 4, cudaMemcpyDeviceToHost, st));
+        if (c.delta_out)
+            OBF_CUDA_TRY(cudaMemcpyAsync(c.delta_out, base + H.delta[i], hpc * d * 4, cudaMemcpyDeviceToHost, st));
+    }
+    OBF_CUDA_TRY(cudaStreamSynchronize(st));
+    return OBF_OK;
+}
+
+obf_status_t obf_last_device_status(const void *workspace, void *stream, uint32_t *device_status)
+{
+    if (!workspace || !device_status) return OBF_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint32_t v = 0;
+    OBF_CUDA_TRY(cudaMemcpyAsync(&v, workspace, sizeof(v), cudaMemcpyDeviceToHost, st));
+    OBF_CUDA_TRY(cudaStreamSynchronize(st));
+    *device_status = v;
+    return (v & (OBF_DEV_NONFINITE | OBF_DEV_NO_CONVERGE | OBF_DEV_TIMEOUT)) ? OBF_ERR_DEVICE_STATUS : OBF_OK;
+}
+
+obf_status_t obf_compress_profiled(const obf_params_t *params, const obf_cache_t *caches, int32_t n_caches,
+                                   void *workspace, size_t workspace_bytes, void *stream,
+                                   float *phase_ms, int32_t *n_phases)
+{
+    if (!params || !phase_ms || !n_phases) return OBF_ERR_INVALID_ARG;
+    for (int i = 0; i <= OBF_MAX_PHASES; ++i) OBF_CUDA_TRY(cudaEventCreate(&g_prof.ev[i]));
+    g_prof.n = 0;
+    g_prof.active = true;
+    obf_status_t s = run(params, caches, n_caches, params->rank, workspace, workspace_bytes, stream);
+    g_prof.active = false;
+    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    *n_phases = 0;
+    if (s == OBF_OK && e == cudaSuccess) {
+        for (int i = 0; i < g_prof.n; ++i) {
+            cudaEventElapsedTime(&phase_ms[i], g_prof.ev[i], g_prof.ev[i + 1]);
+            g_phase_names[i] = g_prof.names[i];
+        }
+        g_phase_count = g_prof.n;
+        *n_phases = g_prof.n;
+    }
+    for (int i = 0; i <= OBF_MAX_PHASES; ++i) cudaEventDestroy(g_prof.ev[i]);
+    if (e != cudaSuccess) return OBF_ERR_CUDA;
+    return s;
+}
+
+const char *obf_phase_name(int32_t phase)
+{
+    return (phase >= 0 && phase < g_phase_count) ? g_phase_names[phase] : "";
+}
+
+const char *obf_status_string(obf_status_t status)
+{
+    switch (status) {
+    case OBF_OK: return "ok";
+    case OBF_ERR_INVALID_ARG: return "invalid argument";
+    case OBF_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+    case OBF_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case OBF_ERR_CUDA: return "CUDA runtime error";
+    case OBF_ERR_DEVICE_STATUS: return "device reported a numerical or timeout condition";
+    }
+    return "unknown status";
+}
+
+int32_t obf_last_launch_count(void) { return g_last_launches; }
+
+}  // extern "C"

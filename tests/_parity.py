@@ -1,0 +1,181 @@
+"""Helpers shared by the GPU parity tests: run the CUDA path through the C ABI and
+compare one (layer, KV head) at a time against the CPU oracle."""
+from __future__ import annotations
+
+import dataclasses
+from typing import Dict, List, Optional, Sequence
+
+import numpy as np
+import torch
+
+import oracle
+import paper_2604_13349_b200 as P
+from paper_2604_13349_b200 import synth
+
+TIE_BAND = 1e-6            # absolute, on masses normalised so that sum_j A_j = n_q
+F32_V_ATOL = 1e-4          # fp32 path: max abs error of compacted values
+BF16_V_RTOL = 2e-2         # bf16 path: relative error of compacted values
+U32 = 2.0 ** -24
+
+
+def to_device(arr: np.ndarray, dtype: str) -> torch.Tensor:
+    if dtype == "bf16":
+        return torch.from_numpy(arr.view(np.int16)).cuda().view(torch.bfloat16)
+    return torch.from_numpy(arr).cuda()
+
+
+def f32_view(arr: np.ndarray, dtype: str) -> np.ndarray:
+    return synth.bf16_bits_to_f32(arr) if dtype == "bf16" else arr
+
+
+def out_to_f32(t: torch.Tensor) -> np.ndarray:
+    return t.float().cpu().numpy()
+
+
+def out_bits(t: torch.Tensor) -> np.ndarray:
+    if t.dtype == torch.bfloat16:
+        return t.view(torch.int16).cpu().numpy()
+    return t.view(torch.int32).cpu().numpy()
+
+
+def params_for(w: synth.Workload, rank: Optional[int] = None, flags: int = 0):
+    return P.make_params(w.layers, w.kv_heads, w.q_heads, w.head.head_dim, w.n_obs,
+                         w.rank if rank is None else rank,
+                         P.OBF_F32 if w.dtype == "f32" else P.OBF_BF16, 1e-12, flags)
+
+
+def run_gpu(w: synth.Workload, arrays: Sequence[Dict[str, np.ndarray]], rank: Optional[int] = None,
+            evict: bool = False, flags: int = 0, want_scores: bool = True):
+    """arrays: per cache the dict from synth.gen_cache.  Returns (outs, device inputs)."""
+    params = params_for(w, rank, flags)
+    dev = []
+    for ci, a in enumerate(arrays):
+        dev.append({"K": to_device(a["K"], w.dtype), "V": to_device(a["V"], w.dtype),
+                    "Q": to_device(a["Q"], w.dtype), "budget": w.caches[ci].budget})
+    outs = P.compress_caches(params, dev, evict=evict, want_scores=want_scores)
+    torch.cuda.synchronize()
+    st = P.obf_last_device_status(outs[0]["workspace"])
+    return outs, dev, st
+
+
+@dataclasses.dataclass
+class HeadReport:
+    in_band: int = 0
+    band_mismatch: bool = False
+    score_err: float = 0.0
+    delta_err: float = 0.0
+    delta_tol: float = 0.0
+    v_err: float = 0.0
+    gap_rel: float = 1.0
+    oracle_skipped: bool = True
+
+
+def check_head(dtype: str, K: np.ndarray, V: np.ndarray, Q: np.ndarray, budget: int, rank: int,
+               g_idx: np.ndarray, g_kbits: np.ndarray, g_vbits: np.ndarray, g_v: np.ndarray,
+               g_scores: Optional[np.ndarray], g_delta: Optional[np.ndarray], g_diag: Optional[dict],
+               in_kbits: np.ndarray, in_vbits: np.ndarray, name: str = "") -> HeadReport:
+    """K, V, Q: float32 values of one head (bf16 already up-cast).  g_*: the CUDA path's outputs."""
+    rep = HeadReport()
+    T, d = K.shape
+    k = min(budget, T)
+    ref = oracle.head(K, V, Q, budget, rank)
+    A = ref["A"]
+    dg = ref["diag"]
+
+    # -- a1: attention mass ------------------------------------------------
+    if g_scores is not None:
+        err = np.abs(g_scores.astype(np.float64) - A)
+        rep.score_err = float((err / (1e-6 + 5e-5 * A)).max())
+        assert rep.score_err <= 1.0, "%s: attention mass off by %.3g x tolerance" % (name, rep.score_err)
+        assert abs(float(g_scores.astype(np.float64).sum()) - Q.shape[0]) <= 1e-3 * Q.shape[0]
+
+    # -- a2: retained positions -----------------------------------------------
+    assert g_idx.shape == (k,)
+    assert np.all(np.diff(g_idx) > 0), "%s: positions not strictly ascending" % name
+    assert g_idx.min() >= 0 and g_idx.max() < T
+    band = np.abs(A - dg["kth_score"]) <= TIE_BAND
+    rep.in_band = int(band.sum())
+    gset, oset = set(g_idx.tolist()), set(ref["idx"].tolist())
+    outside = ~band
+    g_out = {j for j in gset if outside[j]}
+    o_out = {j for j in oset if outside[j]}
+    assert g_out == o_out, "%s: retained sets differ outside the %.0e tie band: %s" % (
+        name, TIE_BAND, sorted(g_out ^ o_out)[:8])
+    rep.band_mismatch = gset != oset
+
+    # -- a3: gather is bit-exact -------------------------------------------------
+    assert np.array_equal(g_kbits, in_kbits[g_idx]), "%s: K_out is not a bit-exact gather" % name
+
+    # -- a4: OBF -------------------------------------------------------------------
+    rep.oracle_skipped = bool(dg["skipped"])
+    if rep.band_mismatch:
+        # another valid retained set: values can only be checked for self-consistency
+        if g_delta is not None and np.linalg.norm(g_delta) == 0:
+            assert np.array_equal(g_vbits, in_vbits[g_idx])
+        return rep
+    if dg["skipped"]:
+        assert np.array_equal(g_vbits, in_vbits[g_idx]), "%s: V_out must equal V_keep bit for bit" % name
+        if g_delta is not None:
+            assert np.all(g_delta == 0)
+        return rep
+
+    lam_rho, lam_next, lam_1 = dg["lam_rho"], dg["lam_next"], dg["lam_1"]
+    gap = (lam_rho - lam_next) / lam_1
+    rep.gap_rel = float(gap)
+    scale = dg["alpha"] * dg["rbar_norm"]
+    # first-order eigenvector perturbation: fp32 Gram error ~ c*u*lam_1 against the eigen-gap
+    rep.delta_tol = max(2e-5 if dtype == "f32" else 2e-4, 200.0 * U32 / max(gap, 1e-12) * scale)
+    if g_delta is not None:
+        rep.delta_err = float(np.linalg.norm(g_delta.astype(np.float64) - ref["delta"]))
+        if gap >= 1e-3:
+            assert rep.delta_err <= rep.delta_tol, "%s: delta off by %.3g (tol %.3g, gap %.3g)" % (
+                name, rep.delta_err, rep.delta_tol, gap)
+        # always: orthogonal to the retained span, inside the residual row space, no longer than alpha*r_bar
+        Vk = V[g_idx].astype(np.float64)
+        gd = g_delta.astype(np.float64)
+        if np.linalg.norm(gd) > 0:
+            assert np.abs(Vk @ gd).max() / (np.linalg.norm(Vk, 2) * np.linalg.norm(gd)) <= 1e-4
+            assert np.linalg.norm(gd) <= scale * (1 + 1e-3)
+    verr = np.abs(g_v.astype(np.float64) - ref["V_out"])
+    rep.v_err = float(verr.max())
+    if gap >= 1e-3:
+        if dtype == "f32":
+            assert rep.v_err <= max(F32_V_ATOL, rep.delta_tol), "%s: V_out max abs err %.3g" % (name, rep.v_err)
+        else:
+            bound = BF16_V_RTOL * np.abs(ref["V_out"]) + rep.delta_tol + 1e-3
+            assert np.all(verr <= bound), "%s: V_out exceeds the bf16 tolerance (max err %.3g)" % (name, rep.v_err)
+    return rep
+
+
+def check_cache(w: synth.Workload, ci: int, arrays: Dict[str, np.ndarray], out: Dict[str, torch.Tensor],
+                heads: Sequence[tuple], rank: Optional[int] = None, name: str = "") -> List[HeadReport]:
+    rank = w.rank if rank is None else rank
+    d, n_q = w.head.head_dim, w.n_q
+    budget = w.caches[ci].budget
+    Qv = arrays["Q"].reshape(w.layers, w.kv_heads, n_q, d)
+    diags = P.parse_diag(out["diag"]) if out.get("diag") is not None else None
+    reps = []
+    for (l, h) in heads:
+        K = f32_view(arrays["K"][l, h], w.dtype)
+        V = f32_view(arrays["V"][l, h], w.dtype)
+        Q = f32_view(Qv[l, h], w.dtype)
+        kb = arrays["K"][l, h].view(np.int16 if w.dtype == "bf16" else np.int32)
+        vb = arrays["V"][l, h].view(np.int16 if w.dtype == "bf16" else np.int32)
+        rep = check_head(
+            w.dtype, K, V, Q, budget, rank,
+            out["idx"][l, h].cpu().numpy(), out_bits(out["K_out"][l, h]), out_bits(out["V_out"][l, h]),
+            out_to_f32(out["V_out"][l, h]),
+            out["scores"][l, h].cpu().numpy() if out.get("scores") is not None else None,
+            out["delta"][l, h].cpu().numpy() if out.get("delta") is not None else None,
+            diags[l * w.kv_heads + h] if diags else None, kb, vb,
+            name="%s cache %d layer %d head %d" % (name or w.name, ci, l, h))
+        reps.append(rep)
+    return reps
+
+
+def summarize(reps: Sequence[HeadReport]) -> str:
+    return ("heads=%d in_band=%d band_mismatch=%d max_score_err=%.3g(xtol) max_delta_err=%.3g max_v_err=%.3g "
+            "min_gap=%.3g obf_active=%d" % (
+                len(reps), sum(r.in_band for r in reps), sum(r.band_mismatch for r in reps),
+                max(r.score_err for r in reps), max(r.delta_err for r in reps), max(r.v_err for r in reps),
+                min(r.gap_rel for r in reps), sum(not r.oracle_skipped for r in reps)))

@@ -1,0 +1,246 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle.
+
+Bar: retained positions bit-exact outside a 1e-6 tie band on the attention
+mass; K_out a bit-exact gather; V_out bit-exact where no injection happens,
+within 1e-4 (fp32) / 2e-2 relative (bf16) otherwise; delta compared with an
+eigen-gap-aware tolerance (the principal subspace is only determined up to the
+gap between the last kept and first dropped eigenvalue).
+"""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2604_13349_b200 as P
+from paper_2604_13349_b200 import synth
+from tests import _parity as par
+
+pytestmark = pytest.mark.gpu
+
+
+def small(name, *, seed=7, layers=1, kv_heads=2, G=2, n_obs=5, d=64, dtype="f32", rank=2,
+          caches=((100, 10),), heavy=3, n_outlier=0, n_sink=0):
+    hs = synth.HeadSpec(head_dim=d, n_q=G * n_obs, n_outlier=n_outlier, heavy_count=heavy, n_sink=n_sink)
+    return synth.Workload(name=name, seed=seed, layers=layers, kv_heads=kv_heads, q_heads=kv_heads * G,
+                          n_obs=n_obs, rank=rank, dtype=dtype, head=hs,
+                          caches=tuple(synth.CacheSpec(T=t, budget=b) for t, b in caches))
+
+
+def all_heads(w):
+    return [(l, h) for l in range(w.layers) for h in range(w.kv_heads)]
+
+
+def run_and_check(w, rank=None, evict=False, heads=None, arrays=None, flags=0):
+    arrays = arrays or [synth.gen_cache(w, ci) for ci in range(len(w.caches))]
+    outs, _, st = par.run_gpu(w, arrays, rank=rank, evict=evict, flags=flags)
+    assert st & 0xFF == 0, "device status %#x" % st
+    eff_rank = 0 if evict else (w.rank if rank is None else rank)
+    reps = []
+    for ci in range(len(w.caches)):
+        reps += par.check_cache(w, ci, arrays[ci], outs[ci], heads or all_heads(w), rank=eff_rank)
+    print("\n[%s] %s" % (w.name, par.summarize(reps)))
+    return outs, reps, arrays
+
+
+# ---------------------------------------------------------------------------
+# BASELINE configurations that the oracle finishes whole
+# ---------------------------------------------------------------------------
+def test_c1_tiny_fp32_whole():
+    outs, reps, _ = run_and_check(synth.workload("c1"))
+    assert all(not r.oracle_skipped for r in reps)          # budget 32 < head_dim 64: OBF is active
+    assert all(not r.band_mismatch for r in reps)
+
+
+def test_c1_rank0_and_evict_only_agree():
+    w = synth.workload("c1")
+    a, _, arrays = run_and_check(w, rank=0)
+    b, _, _ = run_and_check(w, evict=True, arrays=arrays)
+    for x, y in zip(a, b):
+        assert torch.equal(x["idx"], y["idx"]) and torch.equal(x["K_out"], y["K_out"])
+        assert torch.equal(x["V_out"], y["V_out"])
+
+
+def test_c2_bf16_whole():
+    outs, reps, _ = run_and_check(synth.workload("c2"))
+    assert all(r.oracle_skipped for r in reps)              # budget 205 > head_dim: span is full, delta = 0
+    diags = P.parse_diag(outs[0]["diag"])
+    assert all(dg["status"] & P.binding.OBF_DEV_SPAN_FULL for dg in diags)
+    assert all(dg["span_rank"] == 128 for dg in diags)
+
+
+# ---------------------------------------------------------------------------
+# shapes: ragged tiles, tiny T, every dtype / head_dim, multi-layer, ragged batch
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("T,budget", [(1, 1), (2, 1), (63, 9), (65, 64), (129, 17), (1000, 31), (1025, 100)])
+def test_ragged_shapes(dtype, d, T, budget):
+    w = small("ragged", d=d, dtype=dtype, caches=((T, budget),), heavy=min(3, T), seed=T * 3 + d)
+    run_and_check(w)
+
+
+@pytest.mark.parametrize("G,n_obs", [(1, 1), (1, 5), (3, 7), (4, 16), (4, 40), (5, 32)])
+def test_query_counts(G, n_obs):
+    w = small("queries", G=G, n_obs=n_obs, d=128, dtype="bf16", caches=((300, 20),), n_outlier=3, seed=G * 10 + n_obs)
+    run_and_check(w)
+
+
+def test_multi_layer_ragged_batch_in_one_call():
+    w = small("batch", layers=3, kv_heads=2, d=128, dtype="bf16", rank=2, n_sink=4,
+              caches=((130, 13), (64, 64), (777, 100), (40, 3), (1, 1)))
+    outs, reps, _ = run_and_check(w)
+    assert len(reps) == 5 * 6
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_budget_at_least_T_is_the_identity(dtype):
+    w = small("identity", d=64, dtype=dtype, caches=((50, 50), (50, 80)))
+    outs, _, arrays = run_and_check(w)
+    for ci in range(2):
+        assert torch.equal(outs[ci]["idx"][0, 0].cpu(), torch.arange(50, dtype=torch.int32))
+        assert np.array_equal(par.out_bits(outs[ci]["K_out"]), arrays[ci]["K"].view(
+            np.int16 if dtype == "bf16" else np.int32))
+        assert np.array_equal(par.out_bits(outs[ci]["V_out"]), arrays[ci]["V"].view(
+            np.int16 if dtype == "bf16" else np.int32))
+
+
+@pytest.mark.parametrize("rank", [1, 3, 64])
+def test_rank_sweep_including_full_rank_cap(rank):
+    w = small("ranks", d=64, dtype="f32", rank=rank, caches=((200, 12),))
+    outs, reps, _ = run_and_check(w)
+    assert all(not r.oracle_skipped for r in reps)
+
+
+def test_codimension_one():
+    w = small("codim1", d=64, dtype="f32", rank=2, caches=((150, 63),))
+    outs, reps, _ = run_and_check(w)
+    diags = P.parse_diag(outs[0]["diag"])
+    assert all(dg["span_rank"] == 63 and dg["rho_eff"] == 1 for dg in diags)
+
+
+def test_budget_above_head_dim_full_rank_is_bit_exact_eviction():
+    w = small("full", d=64, dtype="bf16", rank=3, caches=((400, 90),))
+    outs, reps, _ = run_and_check(w)
+    assert all(r.oracle_skipped for r in reps)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_rank_deficient_values_with_budget_above_head_dim(dtype):
+    # every value lives in the first 40 channels except a few tokens the keys make unselectable:
+    # budget >= head_dim, span(V_keep) has dimension 40, the residual is not zero.
+    w = small("rd", d=64, dtype=dtype, rank=2, caches=((300, 80),), heavy=0, kv_heads=2, seed=21)
+    arrays = [synth.gen_cache(w, 0)]
+    a = arrays[0]
+    K = par.f32_view(a["K"], dtype).copy(); V = par.f32_view(a["V"], dtype).copy()
+    Qv = par.f32_view(a["Q"], dtype).reshape(1, 2, w.n_q, 64)
+    g = np.random.default_rng(5)
+    V[..., 40:] = 0.0
+    for h in range(2):
+        qm = Qv[0, h].mean(axis=0)
+        odd = g.choice(300, 15, replace=False)
+        K[0, h, odd] = -6.0 * qm / np.linalg.norm(qm) * np.linalg.norm(K[0, h, odd], axis=1, keepdims=True)
+        V[0, h, odd, 40:] = g.standard_normal((15, 24)).astype(np.float32)
+    if dtype == "bf16":
+        a["K"], a["V"] = synth.to_bf16_bits(K), synth.to_bf16_bits(V)
+    else:
+        a["K"], a["V"] = K, V
+    outs, reps, _ = run_and_check(w, arrays=arrays)
+    diags = P.parse_diag(outs[0]["diag"])
+    assert all(dg["span_rank"] == 40 for dg in diags)
+    assert all(not r.oracle_skipped for r in reps)
+    assert torch.all(outs[0]["delta"][..., :40].abs() < 1e-5)
+    assert torch.all(outs[0]["delta"].norm(dim=-1) > 1e-4)
+
+
+def test_exact_ties_go_to_the_lowest_position():
+    # duplicated keys give bit-identical masses on the GPU as well; ties must resolve to lower positions
+    w = small("ties", d=64, dtype="f32", rank=0, caches=((96, 20),), heavy=0, kv_heads=1)
+    arrays = [synth.gen_cache(w, 0)]
+    K = arrays[0]["K"]
+    K[0, 0, 48:] = K[0, 0, :48]                          # position j+48 duplicates position j
+    outs, _, st = par.run_gpu(w, arrays, rank=0)
+    idx = outs[0]["idx"][0, 0].cpu().numpy()
+    sc = outs[0]["scores"][0, 0].cpu().numpy()
+    assert np.array_equal(sc[:48], sc[48:])
+    ref = oracle.topk(sc.astype(np.float64), 20)[0]      # the oracle's rule applied to the GPU's own masses
+    assert np.array_equal(idx, ref)
+    assert all((j - 48) in idx for j in idx if j >= 48)     # a kept duplicate implies its lower twin is kept
+    all_equal = small("alleq", d=64, dtype="bf16", rank=0, caches=((77, 11),), heavy=0, kv_heads=1)
+    arr2 = [synth.gen_cache(all_equal, 0)]
+    arr2[0]["K"][0, 0, :] = arr2[0]["K"][0, 0, 0]
+    o2, _, _ = par.run_gpu(all_equal, arr2, rank=0)
+    assert np.array_equal(o2[0]["idx"][0, 0].cpu().numpy(), np.arange(11))
+
+
+def test_runs_are_deterministic():
+    w = synth.workload("c1")
+    arrays = [synth.gen_cache(w, 0)]
+    a, _, _ = par.run_gpu(w, arrays)
+    b, _, _ = par.run_gpu(w, arrays)
+    for key in ("idx", "K_out", "V_out", "scores", "delta"):
+        assert torch.equal(a[0][key], b[0][key]), key
+
+
+def test_non_finite_inputs_set_the_status_word_and_stay_in_bounds():
+    w = small("nan", d=64, dtype="f32", rank=1, caches=((120, 10),), kv_heads=1)
+    arrays = [synth.gen_cache(w, 0)]
+    arrays[0]["K"][0, 0, 5, 3] = np.nan
+    outs, _, st = par.run_gpu(w, arrays)
+    assert st & P.binding.OBF_DEV_NONFINITE
+    idx = outs[0]["idx"][0, 0].cpu().numpy()
+    assert len(set(idx.tolist())) == 10 and idx.min() >= 0 and idx.max() < 120
+
+
+def test_host_entry_point_matches_the_device_entry_point():
+    w = synth.workload("c1")
+    arrays = [synth.gen_cache(w, 0)]
+    outs, _, _ = par.run_gpu(w, arrays)
+    params = par.params_for(w)
+    k = w.caches[0].budget
+    hK = torch.from_numpy(arrays[0]["K"]).pin_memory(); hV = torch.from_numpy(arrays[0]["V"]).pin_memory()
+    hQ = torch.from_numpy(arrays[0]["Q"]).pin_memory()
+    oK = torch.empty((1, 2, k, 64)).pin_memory(); oV = torch.empty((1, 2, k, 64)).pin_memory()
+    oI = torch.empty((1, 2, k), dtype=torch.int32).pin_memory()
+    oD = torch.empty((1, 2, 64)).pin_memory()
+    c = P.make_cache(hK, hV, hQ, 256, k, oK, oV, oI, None, None, oD)
+    arena = torch.empty(P.obf_host_arena_bytes(params, [c]), dtype=torch.uint8, device="cuda")
+    P.obf_compress_host(params, [c], arena)
+    assert torch.equal(oI, outs[0]["idx"].cpu())
+    assert torch.equal(oK, outs[0]["K_out"].cpu()) and torch.equal(oV, outs[0]["V_out"].cpu())
+    assert torch.equal(oD, outs[0]["delta"].cpu())
+
+
+# ---------------------------------------------------------------------------
+# BASELINE configurations at full size, in the benchmark's launch configuration,
+# checked on sampled heads that the oracle computes one by one
+# ---------------------------------------------------------------------------
+@pytest.fixture(scope="module")
+def c4_arrays():
+    return [synth.gen_cache(synth.workload("c4"), 0)]
+
+
+def test_c3_full_size_sampled_heads():
+    w = synth.workload("c3")
+    run_and_check(w, heads=[(0, 0), (17, 3), (35, 7)])
+
+
+def test_c4_full_size_rank4_sampled_heads(c4_arrays):
+    run_and_check(synth.workload("c4"), heads=[(0, 0), (21, 5), (39, 7)], arrays=c4_arrays)
+
+
+def test_c4_full_size_evict_only_sampled_heads(c4_arrays):
+    run_and_check(synth.workload("c4_evict"), evict=True, heads=[(3, 1), (39, 6)], arrays=c4_arrays)
+
+
+def test_c5_ragged_relay_batch_sampled_heads():
+    w = synth.workload("c5")
+    run_and_check(w, heads=[(0, 0), (35, 7)])
+
+
+def test_paper_regime_budget_32_sampled_heads():
+    # kv_budget = 32 < head_dim with 40 latent steps: OBF's dense algebra runs for every head
+    w = synth.workload("pa")
+    outs, reps, _ = run_and_check(w, heads=[(0, 0), (9, 4), (35, 7)])
+    assert all(not r.oracle_skipped for r in reps)
