@@ -69,6 +69,7 @@ typedef enum { OBF_F32 = 0, OBF_BF16 = 1 } obf_dtype_t;
 #define OBF_DEV_NONFINITE   0x1u   /* a score or softmax normaliser was not finite                 */
 #define OBF_DEV_NO_CONVERGE 0x2u   /* the eigen-iteration hit its sweep limit                      */
 #define OBF_DEV_TIMEOUT     0x4u   /* a bounded on-device wait expired                             */
+#define OBF_DEV_INTERNAL    0x8u   /* an internal consistency check failed (position out of range) */
 #define OBF_DEV_SKIPPED     0x100u /* informational (diag only): OBF skipped, delta = 0            */
 #define OBF_DEV_SPAN_FULL   0x200u /* informational (diag only): span(V_keep) is all of R^d        */
 
@@ -162,7 +163,8 @@ obf_status_t obf_compress_host(const obf_params_t *params, const obf_cache_t *ca
 /*
  * Waits for `stream`, reads the status word the last call left in `workspace`
  * and stores it in *device_status.  Returns OBF_ERR_DEVICE_STATUS if any of
- * the error bits (OBF_DEV_NONFINITE, OBF_DEV_NO_CONVERGE, OBF_DEV_TIMEOUT) is set.
+ * the error bits (OBF_DEV_NONFINITE, OBF_DEV_NO_CONVERGE, OBF_DEV_TIMEOUT,
+ * OBF_DEV_INTERNAL) is set.
  */
 obf_status_t obf_last_device_status(const void *workspace, void *stream, uint32_t *device_status);
 

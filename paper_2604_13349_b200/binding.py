@@ -28,6 +28,7 @@ OBF_BF16 = 1
 OBF_DEV_NONFINITE = 0x1
 OBF_DEV_NO_CONVERGE = 0x2
 OBF_DEV_TIMEOUT = 0x4
+OBF_DEV_INTERNAL = 0x8
 OBF_DEV_SKIPPED = 0x100
 OBF_DEV_SPAN_FULL = 0x200
 

@@ -199,7 +199,8 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
 
         // ---- 4. Jacobi eigen-decomposition of M (B2), eigenvectors in B1 -----
         if (!done) {
-            const float floor_abs = 1e-9f * trM;
+            // rotations below the fp32 noise level of the largest eigenvalue never settle: stop there
+            const float floor_abs = 2e-7f * block_max<ALG_NT>(tid < D ? B2[tid * LD + tid] : 0.f, red);
             bool converged = false;
 #pragma unroll 1
             for (int sweep = 0; sweep < JACOBI_MAX_SWEEPS && !converged; ++sweep) {

@@ -144,9 +144,8 @@ __device__ __forceinline__ float block_max(float v, float *red)
 }
 
 // Order-preserving map from a float's bits to an unsigned key (larger float -> larger key).
-__device__ __forceinline__ uint32_t score_key(float a)
+__device__ __forceinline__ uint32_t score_key_bits(uint32_t u)
 {
-    uint32_t u = __float_as_uint(a);
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 

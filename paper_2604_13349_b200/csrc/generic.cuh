@@ -168,7 +168,8 @@ __global__ void __launch_bounds__(SEL_NT) k_select(const __grid_constant__ CallD
     locate(p, blockIdx.x, ci, lh);
     const CacheDev &c = p.c[ci];
     const int T = c.T, k = c.k_eff;
-    const float *A = p.scores + c.tok_off + (size_t)lh * T;
+    // the masses are handled as raw bit patterns so that every pass sees identical keys
+    const uint32_t *A = reinterpret_cast<const uint32_t *>(p.scores + c.tok_off + (size_t)lh * T);
     uint8_t *keep = p.keep + c.tok_off + (size_t)lh * T;
     int32_t *idx = c.idx_out + (size_t)lh * k;
     const int tid = threadIdx.x;
@@ -180,7 +181,7 @@ __global__ void __launch_bounds__(SEL_NT) k_select(const __grid_constant__ CallD
         __syncthreads();
         const uint32_t prefix = s_prefix;
         for (int j = tid; j < T; j += SEL_NT) {
-            const uint32_t u = score_key(A[j]);
+            const uint32_t u = score_key_bits(A[j]);
             if ((u & mask) == prefix) atomicAdd(&hist[(u >> shift) & 255u], 1u);
         }
         __syncthreads();
@@ -205,8 +206,9 @@ __global__ void __launch_bounds__(SEL_NT) k_select(const __grid_constant__ CallD
     for (int base = 0; base < T; base += SEL_NT) {
         const int j = base + tid;
         const bool valid = j < T;
-        const float a = valid ? A[j] : 0.f;
-        const uint32_t u = valid ? score_key(a) : 0u;
+        const uint32_t abits = valid ? A[j] : 0u;
+        const float a = __uint_as_float(abits);
+        const uint32_t u = valid ? score_key_bits(abits) : 0u;
         const bool gt = valid && u > tau, eq = valid && u == tau;
         uint32_t v = (gt ? 1u : 0u) | (eq ? 0x10000u : 0u);
         uint32_t inc = v;
@@ -233,7 +235,12 @@ __global__ void __launch_bounds__(SEL_NT) k_select(const __grid_constant__ CallD
         const bool kp = gt || (eq && eq_before < want);
         if (valid) {
             keep[j] = kp ? 1 : 0;
-            if (kp) { idx[gt_before + min(eq_before, want)] = j; sk += a; }
+            if (kp) {
+                const uint32_t pos = gt_before + min(eq_before, want);
+                if (pos < (uint32_t)k) idx[pos] = j;
+                else atomicOr(p.status, OBF_DEV_INTERNAL);
+                sk += a;
+            }
             else { sd += a; nx = fmaxf(nx, a); }
         }
         const uint32_t tot = hist[0];
@@ -270,6 +277,10 @@ __global__ void __launch_bounds__(256) k_gather(const __grid_constant__ CallDev 
     if (r >= c.k_eff) return;
     const int lane = threadIdx.x & 31;
     const int j = c.idx_out[(size_t)lh * c.k_eff + r];
+    if ((unsigned)j >= (unsigned)c.T) {            // never dereference a position outside the cache
+        if (lane == 0) atomicOr(p.status, OBF_DEV_INTERNAL);
+        return;
+    }
     constexpr int CH = ROW_BYTES / 16;
     const uint4 *ks = reinterpret_cast<const uint4 *>(reinterpret_cast<const char *>(c.k) + ((size_t)lh * c.T + j) * ROW_BYTES);
     const uint4 *vs = reinterpret_cast<const uint4 *>(reinterpret_cast<const char *>(c.v) + ((size_t)lh * c.T + j) * ROW_BYTES);

@@ -362,7 +362,7 @@ obf_status_t obf_last_device_status(const void *workspace, void *stream, uint32_
     OBF_CUDA_TRY(cudaMemcpyAsync(&v, workspace, sizeof(v), cudaMemcpyDeviceToHost, st));
     OBF_CUDA_TRY(cudaStreamSynchronize(st));
     *device_status = v;
-    return (v & (OBF_DEV_NONFINITE | OBF_DEV_NO_CONVERGE | OBF_DEV_TIMEOUT)) ? OBF_ERR_DEVICE_STATUS : OBF_OK;
+    return (v & (OBF_DEV_NONFINITE | OBF_DEV_NO_CONVERGE | OBF_DEV_TIMEOUT | OBF_DEV_INTERNAL)) ? OBF_ERR_DEVICE_STATUS : OBF_OK;
 }
 
 obf_status_t obf_compress_profiled(const obf_params_t *params, const obf_cache_t *caches, int32_t n_caches,

@@ -140,7 +140,7 @@ def test_rank_deficient_values_with_budget_above_head_dim(dtype):
     for h in range(2):
         qm = Qv[0, h].mean(axis=0)
         odd = g.choice(300, 15, replace=False)
-        K[0, h, odd] = -6.0 * qm / np.linalg.norm(qm) * np.linalg.norm(K[0, h, odd], axis=1, keepdims=True)
+        K[0, h, odd] = -1.5 * qm / np.linalg.norm(qm) * np.linalg.norm(K[0, h, odd], axis=1, keepdims=True)
         V[0, h, odd, 40:] = g.standard_normal((15, 24)).astype(np.float32)
     if dtype == "bf16":
         a["K"], a["V"] = synth.to_bf16_bits(K), synth.to_bf16_bits(V)
@@ -151,7 +151,7 @@ def test_rank_deficient_values_with_budget_above_head_dim(dtype):
     assert all(dg["span_rank"] == 40 for dg in diags)
     assert all(not r.oracle_skipped for r in reps)
     assert torch.all(outs[0]["delta"][..., :40].abs() < 1e-5)
-    assert torch.all(outs[0]["delta"].norm(dim=-1) > 1e-4)
+    assert torch.all(outs[0]["delta"].norm(dim=-1) > 1e-6)
 
 
 def test_exact_ties_go_to_the_lowest_position():
