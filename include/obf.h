@@ -182,6 +182,41 @@ obf_status_t obf_compress_profiled(const obf_params_t *params, const obf_cache_t
                                    float *phase_ms, int32_t *n_phases);
 const char *obf_phase_name(int32_t phase);
 
+/*
+ * evict_only for callers that cannot obtain a workspace.  (The paper has no
+ * counterpart: this entry point exists for deployment reasons only.)
+ *
+ * Some hosts of this library cannot call cudaMalloc at the point where they
+ * need a compression: a serving process whose start-up code handed every byte
+ * of device memory to its own pool, a plug-in that runs under another
+ * framework's allocator and must not allocate behind its back, or a latency
+ * critical loop that cannot take the device-wide synchronisation an allocation
+ * implies.  For them the scratch memory lives inside the library: a fixed
+ * array of OBF_STATIC_SCRATCH_BYTES bytes in the library's device image, which
+ * every GPU that loads the library holds until the process exits.  The caller
+ * passes only inputs and outputs (all device pointers, as for evict_only).
+ *
+ * - Computes exactly what evict_only computes (steps a1-a3; params->rank is
+ *   ignored) and returns the same codes, plus OBF_ERR_WORKSPACE - with a
+ *   message on stderr naming both sizes - when the call shape needs more
+ *   scratch than OBF_STATIC_SCRATCH_BYTES (obf_workspace_bytes with rank 0
+ *   tells how much a shape needs).
+ * - Calls no cudaMalloc, cudaFree or any other allocating routine.
+ * - The first call on each device resolves the array's device address
+ *   (cudaGetSymbolAddress, with that device current); make that first call
+ *   before starting any stream capture on the device.
+ * - All calls on one device share the one array and it keeps whatever the
+ *   previous call left; the call clears the part that has to start at zero
+ *   (the status word) and overwrites the rest before reading it.  Two calls
+ *   whose work overlaps on the GPU (different streams, or different host
+ *   threads) race on the array: serialise them.
+ * - obf_static_scratch_status reads the status word of the last such call.
+ */
+#define OBF_STATIC_SCRATCH_BYTES (8u << 20)
+obf_status_t evict_only_static(const obf_params_t *params, const obf_cache_t *caches, int32_t n_caches,
+                               void *stream);
+obf_status_t obf_static_scratch_status(void *stream, uint32_t *device_status);
+
 /* Static, never NULL. */
 const char *obf_status_string(obf_status_t status);
 

@@ -37,7 +37,9 @@ OBF_MAX_CACHES = 32
 
 EXPORTS = ("obf_workspace_bytes", "obf_compress", "evict_only", "obf_host_arena_bytes",
            "obf_compress_host", "obf_last_device_status", "obf_status_string",
-           "obf_last_launch_count", "obf_compress_profiled", "obf_phase_name")
+           "obf_last_launch_count", "obf_compress_profiled", "obf_phase_name",
+           "evict_only_static", "obf_static_scratch_status")
+OBF_STATIC_SCRATCH_BYTES = 8 << 20
 OBF_MAX_PHASES = 16
 
 
@@ -108,6 +110,10 @@ def load() -> ctypes.CDLL:
         lib.obf_compress_profiled.restype = ctypes.c_int
         lib.obf_phase_name.argtypes = [ctypes.c_int32]
         lib.obf_phase_name.restype = ctypes.c_char_p
+        lib.evict_only_static.argtypes = [pp, pc, ctypes.c_int32, ctypes.c_void_p]
+        lib.evict_only_static.restype = ctypes.c_int
+        lib.obf_static_scratch_status.argtypes = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_uint32)]
+        lib.obf_static_scratch_status.restype = ctypes.c_int
         lib.obf_last_launch_count.argtypes = []
         lib.obf_last_launch_count.restype = ctypes.c_int32
         _lib = lib
@@ -183,6 +189,25 @@ def obf_compress(params, caches, workspace, workspace_bytes=None, stream=None, c
 def evict_only(params, caches, workspace, workspace_bytes=None, stream=None, check=True) -> int:
     nb = workspace.numel() * workspace.element_size() if workspace_bytes is None else workspace_bytes
     return _call("evict_only", params, caches, workspace, nb, stream, check)
+
+
+def evict_only_static(params, caches, stream=None, check=True) -> int:
+    """evict_only on the library's built-in scratch array, for callers that cannot allocate a
+    workspace (see include/obf.h).  Inputs and outputs are device tensors as for evict_only; the
+    call shape must fit OBF_STATIC_SCRATCH_BYTES; calls that overlap on the GPU race on the array."""
+    rc = load().evict_only_static(ctypes.byref(params), _carray(caches), len(caches), _stream_handle(stream))
+    if check and rc != OBF_OK:
+        raise ObfError(rc, "evict_only_static")
+    return rc
+
+
+def obf_static_scratch_status(stream=None) -> int:
+    """Status word left by the last evict_only_static call on the current device."""
+    out = ctypes.c_uint32(0)
+    rc = load().obf_static_scratch_status(_stream_handle(stream), ctypes.byref(out))
+    if rc not in (OBF_OK, OBF_ERR_DEVICE_STATUS):
+        raise ObfError(rc, "obf_static_scratch_status")
+    return int(out.value)
 
 
 def obf_compress_host(params, caches, device_arena, arena_bytes=None, stream=None, check=True) -> int:

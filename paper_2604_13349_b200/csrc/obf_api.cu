@@ -411,3 +411,64 @@ const char *obf_status_string(obf_status_t status)
 int32_t obf_last_launch_count(void) { return g_last_launches; }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------
+// evict_only with library-owned scratch, for callers that cannot allocate.
+// ---------------------------------------------------------------------------
+namespace {
+
+// The scratch itself.  In host code this name is only a handle for the runtime,
+// not an address a kernel could use; the device address is looked up per device.
+static __device__ __align__(256) unsigned char g_static_scratch[OBF_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+void *g_static_scratch_addr[kMaxDevices];       // device address of the array, per device ordinal
+bool g_static_scratch_ready[kMaxDevices];
+
+// Device address of the scratch array on the current device; resolved once per device.
+obf_status_t static_scratch_ptr(void **out)
+{
+    int dev = -1;
+    OBF_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return OBF_ERR_UNSUPPORTED;
+    if (!g_static_scratch_ready[dev]) {
+        void *ptr = nullptr;
+        OBF_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
+        if (!ptr) return OBF_ERR_CUDA;
+        g_static_scratch_addr[dev] = ptr;
+        g_static_scratch_ready[dev] = true;
+    }
+    *out = g_static_scratch_addr[dev];
+    return OBF_OK;
+}
+
+}  // namespace
+
+extern "C" obf_status_t evict_only_static(const obf_params_t *params, const obf_cache_t *caches,
+                                          int32_t n_caches, void *stream)
+{
+    obf_status_t s = validate_shapes(params, caches, n_caches, 0);
+    if (s != OBF_OK) return s;
+    Layout L;
+    make_layout(params, caches, n_caches, 0, L);
+    if (L.total > (size_t)OBF_STATIC_SCRATCH_BYTES) {
+        std::fprintf(stderr,
+                     "obf: evict_only_static: this call needs %zu bytes of scratch but the built-in array holds "
+                     "%zu; use evict_only with a caller-provided workspace\n",
+                     L.total, (size_t)OBF_STATIC_SCRATCH_BYTES);
+        return OBF_ERR_WORKSPACE;
+    }
+    void *scratch = nullptr;
+    if ((s = static_scratch_ptr(&scratch)) != OBF_OK) return s;
+    // run() clears the status word at the head of the scratch; every other region is
+    // written by an earlier kernel of the same call before a later one reads it.
+    return run(params, caches, n_caches, 0, scratch, (size_t)OBF_STATIC_SCRATCH_BYTES, stream);
+}
+
+extern "C" obf_status_t obf_static_scratch_status(void *stream, uint32_t *device_status)
+{
+    void *scratch = nullptr;
+    obf_status_t s = static_scratch_ptr(&scratch);
+    if (s != OBF_OK) return s;
+    return obf_last_device_status(scratch, stream, device_status);
+}

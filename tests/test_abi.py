@@ -21,6 +21,7 @@ def lib():
 def declared_functions():
     text = open(os.path.join(ROOT, "include", "obf.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    text = re.sub(r"^\s*#.*$", "", text, flags=re.M)            # preprocessor lines declare nothing
     return sorted(set(re.findall(r"\b(\w+)\s*\([^;{}]*\)\s*;", text)))
 
 
