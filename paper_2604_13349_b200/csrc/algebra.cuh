@@ -5,9 +5,9 @@
 // retained values G_keep (only when k_eff >= d), u = sum_del A_j v_j, the demand
 // sums, and the retained rows themselves (read back from v_out).
 //
-//   1. k_eff >= d: Cholesky of G_keep.  If every pivot stays above 1e-3 of its
-//      diagonal entry the retained values span R^d, the residual of Eq. 3 is
-//      identically zero and delta = 0.
+//   1. k_eff >= d: k_span_test has factorised G_keep (Cholesky).  If every pivot
+//      stayed above 1e-3 of its diagonal entry the retained values span R^d, the
+//      residual of Eq. 3 is identically zero and delta = 0.
 //   2. Otherwise: orthonormal basis Q of span(V_keep) (Eq. 2) by twice-iterated
 //      Gram-Schmidt over the retained rows; a row adds a direction when what is
 //      left of it exceeds 1e-4 of its own norm.
@@ -20,11 +20,11 @@
 #pragma once
 
 #include "common.cuh"
+#include "span_test.cuh"
 
 namespace obf {
 
 constexpr int ALG_NT = 512;
-constexpr float CHOL_PIVOT_TOL = 1e-3f;
 constexpr float SPAN_ROW_TOL = 1e-4f;
 constexpr float RCR_SKIP_TOL = 1e-6f;
 constexpr float EIG_RANK_TOL = 1e-5f;
@@ -49,7 +49,8 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
     int ci, lh;
     locate(p, g, ci, lh);
     const CacheDev &c = p.c[ci];
-    const int T = c.T, k = c.k_eff, S = p.splits;
+    const int T = c.T, k = c.k_eff, S = p.gram_slots;
+    const int n_del = gram_partial_count(p, c, lh, 0), n_keep = gram_partial_count(p, c, lh, 1);
     const float a_keep = p.sums[(size_t)g * 4], a_del = p.sums[(size_t)g * 4 + 1];
     const float alpha = a_del / (a_keep + p.eps);
 
@@ -57,6 +58,8 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
         p.delta[(size_t)g * D + tid] = 0.f;
         if (c.delta_out) c.delta_out[(size_t)lh * D + tid] = 0.f;
     }
+    const uint32_t hflag_in = p.hflag[g];          // written by k_span_test
+    __syncthreads();
     if (tid == 0) p.hflag[g] = 0u;
     if (T - k == 0 || p.rank <= 0) return;
 
@@ -66,34 +69,8 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
     int rho = 0;
     bool done = false;
 
-    // ---- 1. quick span test when k_eff >= d --------------------------------
-    if (k >= D) {
-        for (int e = tid; e < D * D; e += ALG_NT) {
-            float s = 0.f;
-            for (int sp = 0; sp < S; ++sp) s += p.gram_k[((size_t)g * S + sp) * D * D + e];
-            B0[(e / D) * LD + (e % D)] = s;
-        }
-        __syncthreads();
-        if (tid < D) vl[tid] = B0[tid * LD + tid];
-        __syncthreads();
-        bool ok = true;
-#pragma unroll 1
-        for (int j = 0; j < D; ++j) {
-            const float piv = B0[j * LD + j];
-            if (!(piv > CHOL_PIVOT_TOL * vl[j]) || !(piv > 0.f)) { ok = false; break; }
-            const float inv = rsqrtf(piv);
-            if (tid > j && tid < D) vw[tid] = B0[tid * LD + j] * inv;
-            __syncthreads();
-            const int n = D - 1 - j;
-            for (int e = tid; e < n * n; e += ALG_NT) {
-                const int i = j + 1 + e / n, kk = j + 1 + e % n;
-                if (kk <= i) B0[i * LD + kk] -= vw[i] * vw[kk];
-            }
-            __syncthreads();
-        }
-        if (ok) { m = D; done = true; status |= OBF_DEV_SKIPPED | OBF_DEV_SPAN_FULL; }
-        __syncthreads();
-    }
+    // ---- 1. k_eff >= d: the span test kernel has already factorised G_keep --
+    if (k >= D && (hflag_in & HFLAG_SPAN_FULL)) { m = D; done = true; status |= OBF_DEV_SKIPPED | OBF_DEV_SPAN_FULL; }
 
     // ---- 2. orthonormal basis of span(V_keep), Eq. 2 ------------------------
     if (!done) {
@@ -151,12 +128,12 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
         }
         for (int e = tid; e < D * D; e += ALG_NT) {
             float s = 0.f;
-            for (int sp = 0; sp < S; ++sp) s += p.gram_d[((size_t)g * S + sp) * D * D + e];
+            for (int sp = 0; sp < n_del; ++sp) s += p.gram_d[((size_t)g * S + sp) * D * D + e];
             B2[(e / D) * LD + (e % D)] = s;
         }
         if (tid < D) {
             float s = 0.f;
-            for (int sp = 0; sp < S; ++sp) s += p.uvec[((size_t)g * S + sp) * D + tid];
+            for (int sp = 0; sp < n_del; ++sp) s += p.uvec[((size_t)g * S + sp) * D + tid];
             vu[tid] = s;
         }
         __syncthreads();
@@ -300,7 +277,7 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
                     p.delta[(size_t)g * D + tid] = dl;
                     if (c.delta_out) c.delta_out[(size_t)lh * D + tid] = dl;
                 }
-                if (tid == 0) p.hflag[g] = 1u;
+                if (tid == 0) p.hflag[g] = HFLAG_INJECT;
             }
         }
     }

@@ -1,6 +1,7 @@
 // Shared device-side definitions for the relay-compression kernels.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -19,8 +20,18 @@ struct CacheDev {
     float *delta_out;
     int32_t T, k_eff;
     int32_t head_base;        // global id of this cache's first (layer, kv head)
+    int32_t nsub_del;         // tuned path: 128-token tiles of V per head (ceil(T / 128))
+    int32_t nsub_keep;        // tuned path: 128-row tiles of V_keep per head (0 when the span test is not needed)
     int32_t pad_;
     size_t tok_off;           // offset of this cache in the per-token workspace arrays (elements)
+    long long sub_base;       // tuned path: index of this cache's first tile in the call-wide tile sequence
+};
+
+// Tensor maps of a tuned-path kernel, two per cache, passed as a kernel parameter
+// (score kernel: a = K, b = Q; Gram kernel: a = V, b = compacted V_keep).
+struct TcMaps {
+    CUtensorMap a[OBF_MAX_CACHES];
+    CUtensorMap b[OBF_MAX_CACHES];
 };
 
 // Everything one call needs, passed by value as a __grid_constant__ kernel parameter.
@@ -32,7 +43,11 @@ struct CallDev {
     int32_t n_q;              // G * n_obs query rows pooled into one KV head
     int32_t d;
     int32_t rank;
-    int32_t splits;           // token splits of the Gram pass
+    int32_t splits;           // token splits of the Gram pass (shape-generic path)
+    int32_t gram_slots;       // partial Gram matrices stored per head (stride of gram_d / gram_k / uvec)
+    int32_t tc_per;           // tuned path: tiles per block of the Gram pass (0: shape-generic path)
+    int32_t pad_;
+    long long tc_total_sub;   // tuned path: tiles in the call-wide tile sequence
     float eps;
     // workspace
     uint32_t *status;
@@ -40,9 +55,9 @@ struct CallDev {
     uint8_t *keep;            // [sum heads*T] 1 = retained
     float *stats;             // [heads_total, n_q, 2] softmax row max (log2 domain) and normaliser
     float *sums;              // [heads_total, 4] a_keep, a_del, kth, next
-    float *gram_d;            // [heads_total, splits, d, d] partial Gram of deleted values
-    float *gram_k;            // [heads_total, splits, d, d] partial Gram of retained values
-    float *uvec;              // [heads_total, splits, d] partial sum_j A_j v_j over deleted j
+    float *gram_d;            // [heads_total, gram_slots, d, d] partial Gram of deleted values
+    float *gram_k;            // [heads_total, gram_slots, d, d] partial Gram of retained values
+    float *uvec;              // [heads_total, gram_slots, d] partial sum_j A_j v_j over deleted j
     float *delta;             // [heads_total, d]
     uint32_t *hflag;          // [heads_total] bit0: delta != 0 -> inject
 };
@@ -54,6 +69,20 @@ __device__ __forceinline__ void locate(const CallDev &p, int g, int &ci, int &lh
     for (int i = 1; i < p.n_caches; ++i)
         if (g >= p.c[i].head_base) ci = i;
     lh = g - p.c[ci].head_base;
+}
+
+// How many partial Gram matrices the streaming pass left for one head.
+// kind 0: deleted values (and the u vector), kind 1: retained values.
+// Shape-generic path: one per token split.  Tuned path: the call-wide tile
+// sequence is cut into runs of tc_per tiles, one run per block; a head's tiles
+// of one kind land in consecutive blocks, each of which stores one partial.
+__device__ __forceinline__ int gram_partial_count(const CallDev &p, const CacheDev &c, int lh, int kind)
+{
+    if (p.tc_per == 0) return p.splits;
+    const long long len = kind ? c.nsub_keep : c.nsub_del;
+    if (len == 0) return 0;
+    const long long start = c.sub_base + (long long)lh * (c.nsub_del + c.nsub_keep) + (kind ? c.nsub_del : 0);
+    return (int)((start + len - 1) / p.tc_per - start / p.tc_per) + 1;
 }
 
 __device__ __forceinline__ float to_f32(float x) { return x; }

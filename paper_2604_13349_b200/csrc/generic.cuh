@@ -4,6 +4,7 @@
 #pragma once
 
 #include "common.cuh"
+#include "span_test.cuh"
 
 namespace obf {
 
@@ -389,7 +390,7 @@ __global__ void __launch_bounds__(256) k_gram(const __grid_constant__ CallDev p)
 template <typename TIN, int D>
 __global__ void __launch_bounds__(256) k_inject(const __grid_constant__ CallDev p)
 {
-    if ((p.hflag[blockIdx.y] & 1u) == 0u) return;
+    if ((p.hflag[blockIdx.y] & HFLAG_INJECT) == 0u) return;
     int ci, lh;
     locate(p, blockIdx.y, ci, lh);
     const CacheDev &c = p.c[ci];

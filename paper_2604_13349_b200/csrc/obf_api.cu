@@ -6,6 +6,8 @@
 #include "algebra.cuh"
 #include "common.cuh"
 #include "generic.cuh"
+#include "gram_tc.cuh"
+#include "span_test.cuh"
 
 namespace obf {
 
@@ -41,7 +43,40 @@ struct Layout {
     int heads_total;
     size_t tok_total;
     size_t tok_off[OBF_MAX_CACHES];
+    // tuned bf16 / head_dim 128 path
+    bool tuned;
+    int gram_slots;                 // partial Gram matrices stored per head
+    int tc_per, tc_blocks;          // tiles per block and blocks of the tensor-core Gram pass
+    long long tc_total_sub;
+    int nsub_del[OBF_MAX_CACHES], nsub_keep[OBF_MAX_CACHES];
+    long long sub_base[OBF_MAX_CACHES];
 };
+
+// Streaming multiprocessors of the current device (148 on a B200 when no device can be asked).
+static int sm_count()
+{
+    static int cached[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return 148; }
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) {
+            cudaGetLastError();
+            n = 148;
+        }
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+// The tensor-core kernels cover bf16 caches with head_dim 128 and at least one full 128-token tile.
+static bool tuned_path_applies(const obf_params_t *p, const obf_cache_t *caches, int32_t n)
+{
+    if (p->dtype != OBF_BF16 || p->head_dim != 128 || (p->flags & OBF_FLAG_GENERIC_PATH)) return false;
+    for (int i = 0; i < n; ++i)
+        if (caches[i].T < GT_TILE) return false;
+    return true;
+}
 
 static int choose_splits(int heads_total, int T_max)
 {
@@ -87,6 +122,32 @@ static void make_layout(const obf_params_t *p, const obf_cache_t *caches, int32_
     }
     L.tok_total = tok;
     L.splits = choose_splits(L.heads_total, T_max);
+    L.tuned = tuned_path_applies(p, caches, n);
+    L.gram_slots = L.splits;
+    L.tc_per = 0; L.tc_blocks = 0; L.tc_total_sub = 0;
+    if (L.tuned && rank > 0) {
+        long long total = 0;
+        for (int i = 0; i < n; ++i) {
+            const int T = caches[i].T, ke = caches[i].budget < T ? caches[i].budget : T;
+            L.nsub_del[i] = (T + GT_TILE - 1) / GT_TILE;
+            L.nsub_keep[i] = (ke >= d && T > ke) ? (ke + GT_TILE - 1) / GT_TILE : 0;
+            L.sub_base[i] = total;
+            total += (long long)hpc * (L.nsub_del[i] + L.nsub_keep[i]);
+        }
+        const long long sms = sm_count();
+        const long long blocks = total < sms ? total : sms;
+        L.tc_total_sub = total;
+        L.tc_per = (int)((total + blocks - 1) / blocks);
+        L.tc_blocks = (int)((total + L.tc_per - 1) / L.tc_per);
+        int slots = 1;
+        for (int i = 0; i < n; ++i) {
+            const int a = (L.nsub_del[i] + L.tc_per - 1) / L.tc_per + 1;
+            const int b = L.nsub_keep[i] ? (L.nsub_keep[i] + L.tc_per - 1) / L.tc_per + 1 : 0;
+            if (a > slots) slots = a;
+            if (b > slots) slots = b;
+        }
+        L.gram_slots = slots;
+    }
     size_t o = 0;
     L.off_status = o; o += 256;
     L.off_scores = o; o = align_up(o + tok * sizeof(float), 256);
@@ -95,10 +156,10 @@ static void make_layout(const obf_params_t *p, const obf_cache_t *caches, int32_
     L.off_sums = o;   o = align_up(o + (size_t)L.heads_total * 4 * sizeof(float), 256);
     L.off_gram_d = L.off_gram_k = L.off_uvec = L.off_delta = L.off_hflag = o;
     if (rank > 0) {
-        const size_t gsz = (size_t)L.heads_total * L.splits * d * d * sizeof(float);
+        const size_t gsz = (size_t)L.heads_total * L.gram_slots * d * d * sizeof(float);
         L.off_gram_d = o; o = align_up(o + gsz, 256);
         L.off_gram_k = o; o = align_up(o + gsz, 256);
-        L.off_uvec = o;   o = align_up(o + (size_t)L.heads_total * L.splits * d * sizeof(float), 256);
+        L.off_uvec = o;   o = align_up(o + (size_t)L.heads_total * L.gram_slots * d * sizeof(float), 256);
         L.off_delta = o;  o = align_up(o + (size_t)L.heads_total * d * sizeof(float), 256);
         L.off_hflag = o;  o = align_up(o + (size_t)L.heads_total * sizeof(uint32_t), 256);
     }
@@ -123,8 +184,66 @@ static obf_status_t set_smem(K kernel, size_t bytes)
     return OBF_OK;
 }
 
+// cuTensorMapEncodeTiled, looked up through the runtime so that the library does not link the driver.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn tensor_map_encoder()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) != cudaSuccess || !ptr) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// Tensor map of a bf16 array [heads, rows, 128] for 128-row x 64-column boxes with the
+// 128-byte swizzle; rows past `rows` read as zero.
+static obf_status_t encode_rows_map(CUtensorMap *m, const void *ptr, uint64_t rows, uint64_t heads)
+{
+    EncodeTiledFn enc = tensor_map_encoder();
+    if (!enc) return OBF_ERR_CUDA;
+    cuuint64_t dims[3] = {128, rows, heads};
+    cuuint64_t strides[2] = {128 * 2, rows * 128 * 2};
+    cuuint32_t box[3] = {64, (cuuint32_t)GT_TILE, 1};
+    cuuint32_t es[3] = {1, 1, 1};
+    const CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, es,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        std::fprintf(stderr, "obf: cuTensorMapEncodeTiled failed with %d\n", (int)r);
+        return OBF_ERR_CUDA;
+    }
+    return OBF_OK;
+}
+
+// Streaming pass of OBF on the tensor cores (bf16, head_dim 128).
+static obf_status_t launch_gram_tc(const CallDev &cd, const Layout &L, cudaStream_t st)
+{
+    static thread_local TcMaps maps;
+    const uint64_t hpc = (uint64_t)cd.heads_per_cache;
+    for (int i = 0; i < cd.n_caches; ++i) {
+        obf_status_t s = encode_rows_map(&maps.a[i], cd.c[i].v, (uint64_t)cd.c[i].T, hpc);
+        if (s != OBF_OK) return s;
+        if (L.nsub_keep[i]) {
+            if ((s = encode_rows_map(&maps.b[i], cd.c[i].v_out, (uint64_t)cd.c[i].k_eff, hpc)) != OBF_OK) return s;
+        }
+    }
+    OBF_CUDA_TRY(cudaFuncSetAttribute(k_gram_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GT_SMEM_BYTES));
+    k_gram_tc<<<L.tc_blocks, GT_THREADS, GT_SMEM_BYTES, st>>>(cd, maps);
+    mark(st, "k_gram_tc");
+    return OBF_OK;
+}
+
 template <typename TIN, int D>
-static obf_status_t launch_generic(const CallDev &cd, int T_max, int k_max, cudaStream_t st)
+static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max, int k_max, cudaStream_t st)
 {
     const int heads = cd.heads_total;
     const size_t sm_sc = score_smem_bytes<D>();
@@ -145,9 +264,23 @@ static obf_status_t launch_generic(const CallDev &cd, int T_max, int k_max, cuda
     if (cd.rank > 0) {
         const size_t sm_alg = algebra_smem_bytes<D>();
         if ((s = set_smem(k_obf_algebra<TIN, D>, sm_alg)) != OBF_OK) return s;
-        dim3 g5(cd.splits, heads);
-        k_gram<TIN, D><<<g5, 256, 0, st>>>(cd);
-        mark(st, "k_gram");
+        if constexpr (sizeof(TIN) == 2 && D == 128) {
+            if (L.tuned) {
+                if ((s = launch_gram_tc(cd, L, st)) != OBF_OK) return s;
+            } else {
+                dim3 g5(cd.splits, heads);
+                k_gram<TIN, D><<<g5, 256, 0, st>>>(cd);
+                mark(st, "k_gram");
+            }
+        } else {
+            dim3 g5(cd.splits, heads);
+            k_gram<TIN, D><<<g5, 256, 0, st>>>(cd);
+            mark(st, "k_gram");
+        }
+        const size_t sm_span = span_smem_bytes<D>();
+        if ((s = set_smem(k_span_test<D>, sm_span)) != OBF_OK) return s;
+        k_span_test<D><<<heads, ST_NT, sm_span, st>>>(cd);
+        mark(st, "k_span_test");
         k_obf_algebra<TIN, D><<<heads, ALG_NT, sm_alg, st>>>(cd);
         mark(st, "k_obf_algebra");
         k_inject<TIN, D><<<g4, 256, 0, st>>>(cd);
@@ -191,6 +324,9 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
         c.k_eff = caches[i].budget < caches[i].T ? caches[i].budget : caches[i].T;
         c.head_base = i * hpc;
         c.tok_off = L.tok_off[i];
+        c.nsub_del = L.tc_per ? L.nsub_del[i] : 0;
+        c.nsub_keep = L.tc_per ? L.nsub_keep[i] : 0;
+        c.sub_base = L.tc_per ? L.sub_base[i] : 0;
         if (c.T > T_max) T_max = c.T;
         if (c.k_eff > k_max) k_max = c.k_eff;
     }
@@ -201,6 +337,9 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
     cd.d = p->head_dim;
     cd.rank = rank;
     cd.splits = L.splits;
+    cd.gram_slots = L.gram_slots;
+    cd.tc_per = L.tc_per;
+    cd.tc_total_sub = L.tc_total_sub;
     cd.eps = p->eps;
     char *ws = static_cast<char *>(workspace);
     cd.status = reinterpret_cast<uint32_t *>(ws + L.off_status);
@@ -219,11 +358,11 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
     if (g_prof.active) cudaEventRecord(g_prof.ev[0], st);
 
     if (p->dtype == OBF_F32) {
-        return p->head_dim == 64 ? launch_generic<float, 64>(cd, T_max, k_max, st)
-                                 : launch_generic<float, 128>(cd, T_max, k_max, st);
+        return p->head_dim == 64 ? launch_generic<float, 64>(cd, L, T_max, k_max, st)
+                                 : launch_generic<float, 128>(cd, L, T_max, k_max, st);
     }
-    return p->head_dim == 64 ? launch_generic<__nv_bfloat16, 64>(cd, T_max, k_max, st)
-                             : launch_generic<__nv_bfloat16, 128>(cd, T_max, k_max, st);
+    return p->head_dim == 64 ? launch_generic<__nv_bfloat16, 64>(cd, L, T_max, k_max, st)
+                             : launch_generic<__nv_bfloat16, 128>(cd, L, T_max, k_max, st);
 }
 
 }  // namespace obf
