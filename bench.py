@@ -252,7 +252,8 @@ def main():
     q_bytes = len(w.caches) * hpc * w.n_q * d * e
     out_bytes = sum(hpc * min(c.budget, c.T) * (2 * d * e + 4) for c in w.caches)
     kernel_bytes = {"k_score_stats": kv_bytes + q_bytes, "k_score_pool": kv_bytes + q_bytes,
-                    "k_gram": kv_bytes, "k_gather": 2 * out_bytes, "k_inject": out_bytes,
+                    "k_gram": kv_bytes, "k_gram_tc": kv_bytes, "k_score_tc": kv_bytes + q_bytes, "k_span_test": 0,
+                    "k_gather": 2 * out_bytes, "k_inject": out_bytes,
                     "k_select": sum(hpc * c.T * 4 for c in w.caches),
                     "k_obf_algebra": 0, "k_fused": step_bytes}.get(dom, step_bytes)
     achieved = kernel_bytes / (phase_acc[dom] * 1e-3) / 1e9

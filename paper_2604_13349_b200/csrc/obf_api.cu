@@ -7,6 +7,7 @@
 #include "common.cuh"
 #include "generic.cuh"
 #include "gram_tc.cuh"
+#include "score_tc.cuh"
 #include "span_test.cuh"
 
 namespace obf {
@@ -50,6 +51,12 @@ struct Layout {
     long long tc_total_sub;
     int nsub_del[OBF_MAX_CACHES], nsub_keep[OBF_MAX_CACHES];
     long long sub_base[OBF_MAX_CACHES];
+    // tensor-core score kernel
+    bool sc_on;
+    int sc_nq, sc_subs, sc_blocks, sc_rounds;
+    int sc_team[OBF_MAX_CACHES], sc_hpr[OBF_MAX_CACHES], sc_round_base[OBF_MAX_CACHES];
+    size_t sc_part_off[OBF_MAX_CACHES], sc_part_pairs;
+    size_t off_sc_part, off_sc_head, off_sc_sync;
 };
 
 // Streaming multiprocessors of the current device (148 on a B200 when no device can be asked).
@@ -148,12 +155,53 @@ static void make_layout(const obf_params_t *p, const obf_cache_t *caches, int32_
         }
         L.gram_slots = slots;
     }
+    L.sc_on = false;
+    L.sc_nq = L.sc_subs = L.sc_blocks = L.sc_rounds = 0;
+    L.sc_part_pairs = 0;
+    const int nq_pad = (n_q + 31) / 32 * 32;
+    if (L.tuned && nq_pad <= ST_MAX_NQ) {
+        // chunks of sc_subs 128-key tiles; two slots per block; a head's team must fit in one round
+        L.sc_nq = nq_pad;
+        L.sc_subs = 256 / nq_pad > 4 ? 4 : 256 / nq_pad;
+        const int ch = L.sc_subs * 128;
+        long long slots_wanted = 0;
+        for (int i = 0; i < n; ++i) {
+            L.sc_team[i] = (caches[i].T + ch - 1) / ch;
+            slots_wanted += (long long)hpc * L.sc_team[i];
+        }
+        const long long sms = sm_count();
+        long long blocks = (slots_wanted + 1) / 2;
+        if (blocks > sms) blocks = sms;
+        L.sc_blocks = (int)blocks;
+        const int slots = 2 * L.sc_blocks;
+        bool fits = true;
+        int rounds = 0;
+        size_t pairs = 0;
+        for (int i = 0; i < n; ++i) {
+            if (L.sc_team[i] > slots) { fits = false; break; }
+            L.sc_hpr[i] = slots / L.sc_team[i];
+            if (L.sc_hpr[i] > hpc) L.sc_hpr[i] = hpc;
+            L.sc_round_base[i] = rounds;
+            rounds += (hpc + L.sc_hpr[i] - 1) / L.sc_hpr[i];
+            L.sc_part_off[i] = pairs;
+            pairs += (size_t)hpc * L.sc_team[i] * nq_pad;
+        }
+        L.sc_on = fits;
+        L.sc_rounds = rounds;
+        L.sc_part_pairs = pairs;
+    }
     size_t o = 0;
     L.off_status = o; o += 256;
     L.off_scores = o; o = align_up(o + tok * sizeof(float), 256);
     L.off_keep = o;   o = align_up(o + tok, 256);
     L.off_stats = o;  o = align_up(o + (size_t)L.heads_total * n_q * 2 * sizeof(float), 256);
     L.off_sums = o;   o = align_up(o + (size_t)L.heads_total * 4 * sizeof(float), 256);
+    L.off_sc_part = L.off_sc_head = L.off_sc_sync = o;
+    if (L.sc_on) {
+        L.off_sc_part = o; o = align_up(o + L.sc_part_pairs * 2 * sizeof(float), 256);
+        L.off_sc_head = o; o = align_up(o + (size_t)L.heads_total * L.sc_nq * 2 * sizeof(float), 256);
+        L.off_sc_sync = o; o = align_up(o + (size_t)L.heads_total * 2 * sizeof(uint32_t), 256);
+    }
     L.off_gram_d = L.off_gram_k = L.off_uvec = L.off_delta = L.off_hflag = o;
     if (rank > 0) {
         const size_t gsz = (size_t)L.heads_total * L.gram_slots * d * d * sizeof(float);
@@ -204,15 +252,15 @@ static EncodeTiledFn tensor_map_encoder()
     return fn;
 }
 
-// Tensor map of a bf16 array [heads, rows, 128] for 128-row x 64-column boxes with the
+// Tensor map of a bf16 array [heads, rows, 128] for box_rows x 64-column boxes with the
 // 128-byte swizzle; rows past `rows` read as zero.
-static obf_status_t encode_rows_map(CUtensorMap *m, const void *ptr, uint64_t rows, uint64_t heads)
+static obf_status_t encode_rows_map(CUtensorMap *m, const void *ptr, uint64_t rows, uint64_t heads, uint32_t box_rows = GT_TILE)
 {
     EncodeTiledFn enc = tensor_map_encoder();
     if (!enc) return OBF_ERR_CUDA;
     cuuint64_t dims[3] = {128, rows, heads};
     cuuint64_t strides[2] = {128 * 2, rows * 128 * 2};
-    cuuint32_t box[3] = {64, (cuuint32_t)GT_TILE, 1};
+    cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
     cuuint32_t es[3] = {1, 1, 1};
     const CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, es,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -242,20 +290,42 @@ static obf_status_t launch_gram_tc(const CallDev &cd, const Layout &L, cudaStrea
     return OBF_OK;
 }
 
+// Attention mass on the tensor cores (bf16, head_dim 128): one persistent launch.
+static obf_status_t launch_score_tc(const CallDev &cd, const Layout &L, cudaStream_t st)
+{
+    static thread_local TcMaps maps;
+    const uint64_t hpc = (uint64_t)cd.heads_per_cache;
+    for (int i = 0; i < cd.n_caches; ++i) {
+        obf_status_t s = encode_rows_map(&maps.a[i], cd.c[i].k, (uint64_t)cd.c[i].T, hpc);
+        if (s != OBF_OK) return s;
+        if ((s = encode_rows_map(&maps.b[i], cd.c[i].q, (uint64_t)cd.n_q, hpc, (uint32_t)L.sc_nq)) != OBF_OK) return s;
+    }
+    const size_t smem = score_tc_smem_bytes(L.sc_nq);
+    OBF_CUDA_TRY(cudaFuncSetAttribute(k_score_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    OBF_CUDA_TRY(cudaMemsetAsync(cd.sc_cnt, 0, (size_t)cd.heads_total * 2 * sizeof(uint32_t), st));
+    k_score_tc<<<L.sc_blocks, ST_THREADS, smem, st>>>(cd, maps);
+    mark(st, "k_score_tc");
+    return OBF_OK;
+}
+
 template <typename TIN, int D>
 static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max, int k_max, cudaStream_t st)
 {
     const int heads = cd.heads_total;
     const size_t sm_sc = score_smem_bytes<D>();
     obf_status_t s;
-    if ((s = set_smem(k_score_stats<TIN, D>, sm_sc)) != OBF_OK) return s;
-    if ((s = set_smem(k_score_pool<TIN, D>, sm_sc)) != OBF_OK) return s;
-    dim3 g1((cd.n_q + SC_TILE - 1) / SC_TILE, heads);
-    k_score_stats<TIN, D><<<g1, SC_NT, sm_sc, st>>>(cd);
-    mark(st, "k_score_stats");
-    dim3 g2((T_max + SC_TILE - 1) / SC_TILE, heads);
-    k_score_pool<TIN, D><<<g2, SC_NT, sm_sc, st>>>(cd);
-    mark(st, "k_score_pool");
+    if (L.sc_on) {
+        if ((s = launch_score_tc(cd, L, st)) != OBF_OK) return s;
+    } else {
+        if ((s = set_smem(k_score_stats<TIN, D>, sm_sc)) != OBF_OK) return s;
+        if ((s = set_smem(k_score_pool<TIN, D>, sm_sc)) != OBF_OK) return s;
+        dim3 g1((cd.n_q + SC_TILE - 1) / SC_TILE, heads);
+        k_score_stats<TIN, D><<<g1, SC_NT, sm_sc, st>>>(cd);
+        mark(st, "k_score_stats");
+        dim3 g2((T_max + SC_TILE - 1) / SC_TILE, heads);
+        k_score_pool<TIN, D><<<g2, SC_NT, sm_sc, st>>>(cd);
+        mark(st, "k_score_pool");
+    }
     k_select<<<heads, SEL_NT, 0, st>>>(cd);
     mark(st, "k_select");
     dim3 g4((k_max + 7) / 8, heads);
@@ -327,6 +397,10 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
         c.nsub_del = L.tc_per ? L.nsub_del[i] : 0;
         c.nsub_keep = L.tc_per ? L.nsub_keep[i] : 0;
         c.sub_base = L.tc_per ? L.sub_base[i] : 0;
+        c.sc_team = L.sc_on ? L.sc_team[i] : 0;
+        c.sc_hpr = L.sc_on ? L.sc_hpr[i] : 0;
+        c.sc_round_base = L.sc_on ? L.sc_round_base[i] : 0;
+        c.sc_part_off = L.sc_on ? L.sc_part_off[i] : 0;
         if (c.T > T_max) T_max = c.T;
         if (c.k_eff > k_max) k_max = c.k_eff;
     }
@@ -340,6 +414,9 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
     cd.gram_slots = L.gram_slots;
     cd.tc_per = L.tc_per;
     cd.tc_total_sub = L.tc_total_sub;
+    cd.sc_nq = L.sc_on ? L.sc_nq : 0;
+    cd.sc_subs = L.sc_subs;
+    cd.sc_rounds = L.sc_rounds;
     cd.eps = p->eps;
     char *ws = static_cast<char *>(workspace);
     cd.status = reinterpret_cast<uint32_t *>(ws + L.off_status);
@@ -347,6 +424,10 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
     cd.keep = reinterpret_cast<uint8_t *>(ws + L.off_keep);
     cd.stats = reinterpret_cast<float *>(ws + L.off_stats);
     cd.sums = reinterpret_cast<float *>(ws + L.off_sums);
+    cd.sc_part = reinterpret_cast<float *>(ws + L.off_sc_part);
+    cd.sc_head = reinterpret_cast<float *>(ws + L.off_sc_head);
+    cd.sc_cnt = reinterpret_cast<uint32_t *>(ws + L.off_sc_sync);
+    cd.sc_flag = cd.sc_cnt + L.heads_total;
     cd.gram_d = reinterpret_cast<float *>(ws + L.off_gram_d);
     cd.gram_k = reinterpret_cast<float *>(ws + L.off_gram_k);
     cd.uvec = reinterpret_cast<float *>(ws + L.off_uvec);
