@@ -16,7 +16,8 @@
 //   4. Symmetric eigen-decomposition of M by parallel-order Jacobi rotations run
 //      to convergence; C = eigenvectors of the `rank` largest eigenvalues above
 //      1e-5 of the largest.
-//   5. Delta = C^T C r_bar (Eq. 5), delta = A_del / (A_keep + eps) * Delta (Eq. 6).
+//   5. Delta = C^T C r_bar (Eq. 5), delta = A_del / (A_keep + eps) * Delta (Eq. 6),
+//      V_out = V_keep + delta on the head's retained rows (Eq. 7).
 #pragma once
 
 #include "common.cuh"
@@ -276,8 +277,17 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
                 if (tid < D) {
                     p.delta[(size_t)g * D + tid] = dl;
                     if (c.delta_out) c.delta_out[(size_t)lh * D + tid] = dl;
+                    vw[tid] = dl;
                 }
                 if (tid == 0) p.hflag[g] = HFLAG_INJECT;
+                __syncthreads();
+                // Eq. 7: V_out = V_keep + delta on every retained row; the fp32 sum is rounded once
+                TIN *rows = reinterpret_cast<TIN *>(c.v_out) + (size_t)lh * k * D;
+                for (int e = tid; e < k * D; e += ALG_NT) {
+                    const float sum = to_f32(rows[e]) + vw[e % D];
+                    if constexpr (sizeof(TIN) == 4) rows[e] = sum;
+                    else rows[e] = __float2bfloat16_rn(sum);
+                }
             }
         }
     }

@@ -384,26 +384,4 @@ __global__ void __launch_bounds__(256) k_gram(const __grid_constant__ CallDev p)
     if (threadIdx.x < D) p.uvec[slot * D + threadIdx.x] = u;
 }
 
-// Step a4, Eq. 7: V_out = V_keep + delta on every retained row of heads whose
-// delta is non-zero; the fp32 sum is rounded once to the output type.
-// grid = (ceil(k_eff_max/8), heads_total).
-template <typename TIN, int D>
-__global__ void __launch_bounds__(256) k_inject(const __grid_constant__ CallDev p)
-{
-    if ((p.hflag[blockIdx.y] & HFLAG_INJECT) == 0u) return;
-    int ci, lh;
-    locate(p, blockIdx.y, ci, lh);
-    const CacheDev &c = p.c[ci];
-    const int r = blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (r >= c.k_eff) return;
-    const int lane = threadIdx.x & 31;
-    const float *dl = p.delta + (size_t)blockIdx.y * D;
-    TIN *row = reinterpret_cast<TIN *>(c.v_out) + ((size_t)lh * c.k_eff + r) * D;
-    for (int e = lane; e < D; e += 32) {
-        const float s = to_f32(row[e]) + dl[e];
-        if constexpr (sizeof(TIN) == 4) row[e] = s;
-        else row[e] = __float2bfloat16_rn(s);
-    }
-}
-
 }  // namespace obf

@@ -13,25 +13,27 @@
 // one (head, kind) inside a run is a segment and yields one partial Gram matrix
 // (and one partial u), stored in slot (b - first block touching that head and kind).
 //
-// Block = 10 warps:
-//   warp 0        TMA producer: 128 x 128 bf16 tiles (two 128-byte-swizzled column halves) into a 4-stage ring
+// Block = 14 warps:
+//   warp 0        TMA producer: 128 x 128 bf16 tiles (two 128-byte-swizzled column halves) into a 5-stage ring
 //   warp 1        issues tcgen05.mma: G (+)= tile^T tile, both operands MN-major views of the same tile,
 //                 accumulators (128 lanes x 128 columns fp32) double-buffered in tensor memory
-//   warps 2..5    fix-up: zero the retained rows of a V tile in shared memory and accumulate u on the CUDA cores
-//   warps 6..9    epilogue: tensor memory -> partial Gram matrix in the workspace
+//   warps 2..9    fix-up: zero the retained rows of a V tile in shared memory and accumulate u on the CUDA
+//                 cores; the attention mass and retained flags of the NEXT tile are fetched while the
+//                 current one is processed
+//   warps 10..13  epilogue: tensor memory -> partial Gram matrix in the workspace
 #pragma once
 
 #include "tc_common.cuh"
 
 namespace obf {
 
-constexpr int GT_STAGES = 4;
+constexpr int GT_STAGES = 5;
 constexpr int GT_TILE = 128;                       // tokens per tile
 constexpr int GT_TILE_BYTES = GT_TILE * 128 * 2;   // 32 KiB
-constexpr int GT_THREADS = 320;
-constexpr int GT_FIX_THREADS = 128;
-constexpr size_t GT_SMEM_BYTES = 1024 + (size_t)GT_STAGES * GT_TILE_BYTES + 8 * 128 * sizeof(float) +
-                                 GT_STAGES * 128 * (sizeof(float) + sizeof(int)) + 256;
+constexpr int GT_FIX_THREADS = 256;
+constexpr int GT_THREADS = 64 + GT_FIX_THREADS + 128;
+constexpr size_t GT_SMEM_BYTES = 1024 + (size_t)GT_STAGES * GT_TILE_BYTES + 16 * 128 * sizeof(float) +
+                                 GT_STAGES * 128 * sizeof(float) + 256;
 
 // Walks the segments of one block's run of tiles.
 struct TileRun {
@@ -67,15 +69,39 @@ struct TileRun {
     }
 };
 
+// One tile of a run, with what the fix-up warps need to know about its segment.
+struct TileInfo {
+    int cache, lh, kind, sub, slot;
+    bool first, last;          // first / last tile of its segment within this run
+};
+
+struct TileIter {
+    TileRun run;
+    int cache, lh, kind, sub0, nsub, slot, t;
+    __device__ __forceinline__ void init(const CallDev &p, int block) { run.init(p, block); nsub = 0; t = 0; }
+    __device__ __forceinline__ bool next(const CallDev &p, TileInfo &ti)
+    {
+        if (t >= nsub) {
+            if (!run.next(p, cache, lh, kind, sub0, nsub, slot)) return false;
+            t = 0;
+        }
+        ti.cache = cache; ti.lh = lh; ti.kind = kind; ti.sub = sub0 + t; ti.slot = slot;
+        ti.first = t == 0;
+        ti.last = t == nsub - 1;
+        ++t;
+        return true;
+    }
+};
+
 __global__ void __launch_bounds__(GT_THREADS, 1) k_gram_tc(const __grid_constant__ CallDev p, const __grid_constant__ TcMaps tm)
 {
     constexpr int D = 128;
     extern __shared__ uint8_t gt_smem_raw[];
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(gt_smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *tiles = base;                                                // GT_STAGES x 32 KiB, 1024-byte aligned
-    float *u_red = reinterpret_cast<float *>(tiles + GT_STAGES * GT_TILE_BYTES);   // [8][128]
-    float *s_a = u_red + 8 * 128;                                         // [GT_STAGES][128] attention mass of the tile's tokens
-    int *s_f = reinterpret_cast<int *>(s_a + GT_STAGES * 128);            // [GT_STAGES][128] 0 deleted, 1 retained, 2 beyond T
+    float *u_red = reinterpret_cast<float *>(tiles + GT_STAGES * GT_TILE_BYTES);   // [16][128]
+    // [GT_STAGES][128] per token of the tile: attention mass, -1 for a retained token, 0 beyond T
+    float *s_a = u_red + 16 * 128;
     __shared__ uint64_t bar_full[GT_STAGES], bar_ready[GT_STAGES], bar_empty[GT_STAGES];
     __shared__ uint64_t bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t s_tmem, s_abort;
@@ -155,68 +181,77 @@ __global__ void __launch_bounds__(GT_THREADS, 1) k_gram_tc(const __grid_constant
                 if (s_abort) break;
             }
         }
-    } else if (warp < 6) {
+    } else if (warp < 2 + GT_FIX_THREADS / 32) {
         // ---------------- fix-up: zero retained rows, accumulate u ----------------
-        const int f = tid - 64;                    // 0..127
-        const int cg = f & 15, rg = f >> 4;        // 16-byte column group, row group
+        const int f = tid - 64;                    // 0..255
+        const int cg = f & 15, rg = f >> 4;        // 16-byte column group, row group (16 of them)
         const uint32_t col_off = (uint32_t)(cg >> 3) * (GT_TILE_BYTES / 2);
-        TileRun run;
-        run.init(p, blockIdx.x);
-        int cache, lh, kind, sub0, nsub, slot;
+        // masked attention mass of token f of a tile (threads 0..127 fetch)
+        auto fetch = [&](const TileInfo &ti) -> float {
+            if (ti.kind != 0 || f >= GT_TILE) return 0.f;
+            const CacheDev &c = p.c[ti.cache];
+            const int j = ti.sub * GT_TILE + f;
+            if (j >= c.T) return 0.f;
+            const size_t o = c.tok_off + (size_t)ti.lh * c.T + j;
+            return __ldg(p.keep + o) ? -1.0f : __ldg(p.scores + o);
+        };
+        TileIter iter;
+        iter.init(p, blockIdx.x);
+        TileInfo cur, nxt;
+        bool has_cur = iter.next(p, cur);
+        float a_pre = has_cur ? fetch(cur) : 0.f;
+        float u[8];
         uint32_t it = 0;
-        while (run.next(p, cache, lh, kind, sub0, nsub, slot)) {
-            const CacheDev &c = p.c[cache];
-            const int g = c.head_base + lh;
-            const float *A = p.scores + c.tok_off + (size_t)lh * c.T;
-            const uint8_t *keep = p.keep + c.tok_off + (size_t)lh * c.T;
-            float u[8];
+        while (has_cur) {
+            const bool has_nxt = iter.next(p, nxt);
+            const int s = it % GT_STAGES;
+            if (f < GT_TILE) s_a[s * 128 + f] = a_pre;
+            if (has_nxt) a_pre = fetch(nxt);           // in flight while this tile is processed
+            if (cur.first) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) u[e] = 0.f;
-            for (int t = 0; t < nsub; ++t, ++it) {
-                const int s = it % GT_STAGES;
-                if (kind == 0) {
-                    const int j = (sub0 + t) * GT_TILE + f;
-                    s_f[s * 128 + f] = j < c.T ? (int)keep[j] : 2;
-                    s_a[s * 128 + f] = j < c.T ? A[j] : 0.f;
-                }
-                tc::mbar_wait(&bar_full[s], (it / GT_STAGES) & 1u, wc);
-                if (kind == 0) {
-                    tc::named_barrier(1, GT_FIX_THREADS);
-                    uint8_t *tile = tiles + s * GT_TILE_BYTES + col_off;
-#pragma unroll 4
-                    for (int i = 0; i < 16; ++i) {
-                        const int r = rg + 8 * i;
-                        const int fl = s_f[s * 128 + r];
-                        uint4 *ptr = reinterpret_cast<uint4 *>(tile + r * 128 + (((cg & 7) ^ (r & 7)) << 4));
-                        if (fl == 1) {
-                            *ptr = make_uint4(0u, 0u, 0u, 0u);
-                        } else if (fl == 0) {
-                            const float a = s_a[s * 128 + r];
-                            const uint4 raw = *ptr;
-                            const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                u[2 * e] = fmaf(a, __uint_as_float(w[e] << 16), u[2 * e]);
-                                u[2 * e + 1] = fmaf(a, __uint_as_float(w[e] & 0xFFFF0000u), u[2 * e + 1]);
-                            }
-                        }
-                    }
-                    tc::fence_async_smem();
-                }
-                __syncwarp();
-                if (lane == 0) tc::mbar_arrive(&bar_ready[s]);
+                for (int e = 0; e < 8; ++e) u[e] = 0.f;
             }
-            if (kind == 0) {
-                // u over the 8 row groups, in a fixed order
+            tc::mbar_wait(&bar_full[s], (it / GT_STAGES) & 1u, wc);
+            tc::named_barrier(1, GT_FIX_THREADS);      // s_a[s] is complete; nobody still reads the slot's previous use
+            if (cur.kind == 0) {
+                uint8_t *tile = tiles + s * GT_TILE_BYTES + col_off;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = rg + 16 * i;
+                    const float a = s_a[s * 128 + r];
+                    const bool kept = a < 0.f;
+                    const float am = kept ? 0.f : a;
+                    uint4 *ptr = reinterpret_cast<uint4 *>(tile + r * 128 + (((cg & 7) ^ (r & 7)) << 4));
+                    const uint4 raw = *ptr;
+                    if (kept) *ptr = make_uint4(0u, 0u, 0u, 0u);
+                    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        u[2 * e] = fmaf(am, __uint_as_float(w[e] << 16), u[2 * e]);
+                        u[2 * e + 1] = fmaf(am, __uint_as_float(w[e] & 0xFFFF0000u), u[2 * e + 1]);
+                    }
+                }
+                tc::fence_async_smem();
+            }
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(&bar_ready[s]);
+            if (cur.kind == 0 && cur.last) {
+                // u over the 16 row groups, in a fixed order
+                const int g = p.c[cur.cache].head_base + cur.lh;
                 tc::named_barrier(1, GT_FIX_THREADS);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) u_red[rg * 128 + cg * 8 + e] = u[e];
                 tc::named_barrier(1, GT_FIX_THREADS);
-                float sum = 0.f;
+                if (f < 128) {
+                    float sum = 0.f;
 #pragma unroll
-                for (int r = 0; r < 8; ++r) sum += u_red[r * 128 + f];
-                p.uvec[((size_t)g * p.gram_slots + slot) * D + f] = sum;
+                    for (int r = 0; r < 16; ++r) sum += u_red[r * 128 + f];
+                    p.uvec[((size_t)g * p.gram_slots + cur.slot) * D + f] = sum;
+                }
             }
+            cur = nxt;
+            has_cur = has_nxt;
+            ++it;
         }
     } else {
         // ---------------- epilogue: accumulator -> workspace ----------------

@@ -353,8 +353,6 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
         mark(st, "k_span_test");
         k_obf_algebra<TIN, D><<<heads, ALG_NT, sm_alg, st>>>(cd);
         mark(st, "k_obf_algebra");
-        k_inject<TIN, D><<<g4, 256, 0, st>>>(cd);
-        mark(st, "k_inject");
     }
     OBF_CUDA_TRY(cudaGetLastError());
     return OBF_OK;
