@@ -26,7 +26,7 @@ struct CacheDev {
     size_t tok_off;           // offset of this cache in the per-token workspace arrays (elements)
     long long sub_base;       // tuned path: index of this cache's first tile in the call-wide tile sequence
     // tuned score kernel: a head's chunks are worked on by a team of slots, heads are dealt in rounds
-    int32_t sc_team;          // chunks (= slots) per head
+    int32_t sc_team;          // chunks (= blocks) per head
     int32_t sc_hpr;           // heads per round
     int32_t sc_round_base;    // first round of this cache
     int32_t pad2_;
@@ -54,14 +54,13 @@ struct CallDev {
     int32_t tc_per;           // tuned path: tiles per block of the Gram pass (0: shape-generic path)
     int32_t pad_;
     long long tc_total_sub;   // tuned path: tiles in the call-wide tile sequence
-    int32_t sc_nq;            // tuned score kernel: n_q rounded up to 32 (0: shape-generic score kernels)
+    int32_t sc_nq;            // tuned score kernel: query rows of its tiles (0: shape-generic score kernels)
     int32_t sc_subs;          // 128-key tiles per chunk
     int32_t sc_rounds;        // rounds of the persistent score kernel
     int32_t pad3_;
-    float *sc_part;           // per (head, chunk, query): chunk maximum and normaliser
-    float *sc_head;           // per (head, query): softmax maximum and normaliser over all keys
+    float *sc_part;           // per (head, chunk, query of 128): chunk maximum and normaliser
+    float *sc_head;           // per (head, query of 128): one 64-bit word, low = M + log2(Z) over all keys, high = 1 when valid
     uint32_t *sc_cnt;         // per head: chunks that have published
-    uint32_t *sc_flag;        // per head: sc_head is valid
     float eps;
     // workspace
     uint32_t *status;

@@ -236,6 +236,7 @@ __global__ void __launch_bounds__(SEL_NT) k_select(const __grid_constant__ CallD
         const bool kp = gt || (eq && eq_before < want);
         if (valid) {
             keep[j] = kp ? 1 : 0;
+            if (kp) p.scores[c.tok_off + (size_t)lh * T + j] = -1.0f;   // later passes need the mass of deleted tokens only
             if (kp) {
                 const uint32_t pos = gt_before + min(eq_before, want);
                 if (pos < (uint32_t)k) idx[pos] = j;

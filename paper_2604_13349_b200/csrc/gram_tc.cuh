@@ -18,8 +18,8 @@
 //   warp 1        issues tcgen05.mma: G (+)= tile^T tile, both operands MN-major views of the same tile,
 //                 accumulators (128 lanes x 128 columns fp32) double-buffered in tensor memory
 //   warps 2..9    fix-up: zero the retained rows of a V tile in shared memory and accumulate u on the CUDA
-//                 cores; the attention mass and retained flags of the NEXT tile are fetched while the
-//                 current one is processed
+//                 cores; the attention mass of the tile after next (-1 marks a retained token) is
+//                 fetched while the current one is processed
 //   warps 10..13  epilogue: tensor memory -> partial Gram matrix in the workspace
 #pragma once
 
@@ -186,27 +186,30 @@ __global__ void __launch_bounds__(GT_THREADS, 1) k_gram_tc(const __grid_constant
         const int f = tid - 64;                    // 0..255
         const int cg = f & 15, rg = f >> 4;        // 16-byte column group, row group (16 of them)
         const uint32_t col_off = (uint32_t)(cg >> 3) * (GT_TILE_BYTES / 2);
-        // masked attention mass of token f of a tile (threads 0..127 fetch)
+        // attention mass of token f of a tile as k_select left it: -1 marks a retained token (threads 0..127 fetch)
         auto fetch = [&](const TileInfo &ti) -> float {
             if (ti.kind != 0 || f >= GT_TILE) return 0.f;
             const CacheDev &c = p.c[ti.cache];
             const int j = ti.sub * GT_TILE + f;
             if (j >= c.T) return 0.f;
-            const size_t o = c.tok_off + (size_t)ti.lh * c.T + j;
-            return __ldg(p.keep + o) ? -1.0f : __ldg(p.scores + o);
+            return __ldg(p.scores + c.tok_off + (size_t)ti.lh * c.T + j);
         };
         TileIter iter;
         iter.init(p, blockIdx.x);
-        TileInfo cur, nxt;
+        TileInfo cur, nxt, nxt2;
         bool has_cur = iter.next(p, cur);
-        float a_pre = has_cur ? fetch(cur) : 0.f;
+        bool has_nxt = has_cur && iter.next(p, nxt);
+        float a_cur = has_cur ? fetch(cur) : 0.f;
+        float a_nxt = has_nxt ? fetch(nxt) : 0.f;
         float u[8];
         uint32_t it = 0;
         while (has_cur) {
-            const bool has_nxt = iter.next(p, nxt);
+            // the masses of the tile after next are requested now and used two tiles later
+            const bool has_nxt2 = has_nxt && iter.next(p, nxt2);
             const int s = it % GT_STAGES;
-            if (f < GT_TILE) s_a[s * 128 + f] = a_pre;
-            if (has_nxt) a_pre = fetch(nxt);           // in flight while this tile is processed
+            if (f < GT_TILE) s_a[s * 128 + f] = a_cur;
+            a_cur = a_nxt;
+            a_nxt = has_nxt2 ? fetch(nxt2) : 0.f;
             if (cur.first) {
 #pragma unroll
                 for (int e = 0; e < 8; ++e) u[e] = 0.f;
@@ -250,7 +253,9 @@ __global__ void __launch_bounds__(GT_THREADS, 1) k_gram_tc(const __grid_constant
                 }
             }
             cur = nxt;
+            nxt = nxt2;
             has_cur = has_nxt;
+            has_nxt = has_nxt2;
             ++it;
         }
     } else {

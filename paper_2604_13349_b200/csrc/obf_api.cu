@@ -158,33 +158,28 @@ static void make_layout(const obf_params_t *p, const obf_cache_t *caches, int32_
     L.sc_on = false;
     L.sc_nq = L.sc_subs = L.sc_blocks = L.sc_rounds = 0;
     L.sc_part_pairs = 0;
-    const int nq_pad = (n_q + 31) / 32 * 32;
-    if (L.tuned && nq_pad <= ST_MAX_NQ) {
-        // chunks of sc_subs 128-key tiles; two slots per block; a head's team must fit in one round
-        L.sc_nq = nq_pad;
-        L.sc_subs = 256 / nq_pad > 4 ? 4 : 256 / nq_pad;
-        const int ch = L.sc_subs * 128;
-        long long slots_wanted = 0;
+    if (L.tuned && n_q <= ST_MAX_NQ) {
+        // chunks of ST_TILES 128-key tiles, one per block and round; a head's team must fit in one round
+        L.sc_nq = 128;
+        L.sc_subs = ST_TILES;
+        long long blocks_wanted = 0;
         for (int i = 0; i < n; ++i) {
-            L.sc_team[i] = (caches[i].T + ch - 1) / ch;
-            slots_wanted += (long long)hpc * L.sc_team[i];
+            L.sc_team[i] = (caches[i].T + ST_CHUNK - 1) / ST_CHUNK;
+            blocks_wanted += (long long)hpc * L.sc_team[i];
         }
         const long long sms = sm_count();
-        long long blocks = (slots_wanted + 1) / 2;
-        if (blocks > sms) blocks = sms;
-        L.sc_blocks = (int)blocks;
-        const int slots = 2 * L.sc_blocks;
+        L.sc_blocks = (int)(blocks_wanted < sms ? blocks_wanted : sms);
         bool fits = true;
         int rounds = 0;
         size_t pairs = 0;
         for (int i = 0; i < n; ++i) {
-            if (L.sc_team[i] > slots) { fits = false; break; }
-            L.sc_hpr[i] = slots / L.sc_team[i];
+            if (L.sc_team[i] > L.sc_blocks) { fits = false; break; }
+            L.sc_hpr[i] = L.sc_blocks / L.sc_team[i];
             if (L.sc_hpr[i] > hpc) L.sc_hpr[i] = hpc;
             L.sc_round_base[i] = rounds;
             rounds += (hpc + L.sc_hpr[i] - 1) / L.sc_hpr[i];
             L.sc_part_off[i] = pairs;
-            pairs += (size_t)hpc * L.sc_team[i] * nq_pad;
+            pairs += (size_t)hpc * L.sc_team[i] * 128;
         }
         L.sc_on = fits;
         L.sc_rounds = rounds;
@@ -199,8 +194,9 @@ static void make_layout(const obf_params_t *p, const obf_cache_t *caches, int32_
     L.off_sc_part = L.off_sc_head = L.off_sc_sync = o;
     if (L.sc_on) {
         L.off_sc_part = o; o = align_up(o + L.sc_part_pairs * 2 * sizeof(float), 256);
-        L.off_sc_head = o; o = align_up(o + (size_t)L.heads_total * L.sc_nq * 2 * sizeof(float), 256);
-        L.off_sc_sync = o; o = align_up(o + (size_t)L.heads_total * 2 * sizeof(uint32_t), 256);
+        // sc_head and sc_cnt are cleared together before every launch
+        L.off_sc_head = o; o = align_up(o + (size_t)L.heads_total * 128 * sizeof(unsigned long long), 256);
+        L.off_sc_sync = o; o = align_up(o + (size_t)L.heads_total * sizeof(uint32_t), 256);
     }
     L.off_gram_d = L.off_gram_k = L.off_uvec = L.off_delta = L.off_hflag = o;
     if (rank > 0) {
@@ -298,11 +294,11 @@ static obf_status_t launch_score_tc(const CallDev &cd, const Layout &L, cudaStre
     for (int i = 0; i < cd.n_caches; ++i) {
         obf_status_t s = encode_rows_map(&maps.a[i], cd.c[i].k, (uint64_t)cd.c[i].T, hpc);
         if (s != OBF_OK) return s;
-        if ((s = encode_rows_map(&maps.b[i], cd.c[i].q, (uint64_t)cd.n_q, hpc, (uint32_t)L.sc_nq)) != OBF_OK) return s;
+        if ((s = encode_rows_map(&maps.b[i], cd.c[i].q, (uint64_t)cd.n_q, hpc)) != OBF_OK) return s;
     }
-    const size_t smem = score_tc_smem_bytes(L.sc_nq);
+    const size_t smem = ST_SMEM_BYTES;
     OBF_CUDA_TRY(cudaFuncSetAttribute(k_score_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    OBF_CUDA_TRY(cudaMemsetAsync(cd.sc_cnt, 0, (size_t)cd.heads_total * 2 * sizeof(uint32_t), st));
+    OBF_CUDA_TRY(cudaMemsetAsync(cd.sc_head, 0, (L.off_sc_sync - L.off_sc_head) + (size_t)cd.heads_total * sizeof(uint32_t), st));
     k_score_tc<<<L.sc_blocks, ST_THREADS, smem, st>>>(cd, maps);
     mark(st, "k_score_tc");
     return OBF_OK;
@@ -425,7 +421,6 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
     cd.sc_part = reinterpret_cast<float *>(ws + L.off_sc_part);
     cd.sc_head = reinterpret_cast<float *>(ws + L.off_sc_head);
     cd.sc_cnt = reinterpret_cast<uint32_t *>(ws + L.off_sc_sync);
-    cd.sc_flag = cd.sc_cnt + L.heads_total;
     cd.gram_d = reinterpret_cast<float *>(ws + L.off_gram_d);
     cd.gram_k = reinterpret_cast<float *>(ws + L.off_gram_k);
     cd.uvec = reinterpret_cast<float *>(ws + L.off_uvec);
