@@ -24,10 +24,14 @@
 // one chunk of work after its first, when every block of its team has long published.
 // The wait for M' is bounded like every other wait (tc_common.cuh).
 //
-// Block = 18 warps: warp 0 TMA producer (Q once per chunk, K tiles through a 4-stage
-// ring), warp 1 MMA issuer (accumulators in a 4-deep ring of 128 tensor-memory columns),
+// Block = 19 warps: warp 0 TMA producer (Q once per chunk, one round ahead; K tiles through a
+// 3-stage ring, asked into L2 one round ahead), warp 1 MMA issuer (accumulators in a 4-deep ring of 128 tensor-memory columns),
 // warps 2..17 consumers: warp (quarter, part) reads lanes [32*quarter, +32) and columns
-// [32*part, +32) of every accumulator tile.
+// [32*part, +32) of every accumulator tile, which frees the tile as soon as the 16 warps
+// have it in registers; warp 18 is the messenger: it publishes the
+// chunk statistics the consumers leave in shared memory, folds a head's chunks when it
+// is the last to arrive, and fetches M' for the next pooling pass, so that the
+// consumers never wait for global memory.
 #pragma once
 
 #include "tc_common.cuh"
@@ -36,15 +40,16 @@ namespace obf {
 
 constexpr int ST_TILES = 4;                         // 128-key tiles per chunk
 constexpr int ST_CHUNK = ST_TILES * 128;
-constexpr int ST_STAGES = 4;                        // K tiles in flight in shared memory
+constexpr int ST_STAGES = 3;                        // K tiles in flight in shared memory
+constexpr int ST_QBUF = 3;                          // Q tiles: rounds r, r - 1 (being pooled) and r + 1 (arriving)
 constexpr int ST_TBUF = 4;                          // accumulator tiles in tensor memory
 constexpr int ST_TILE_BYTES = 128 * 128 * 2;
 constexpr int ST_CONSUMERS = 512;
-constexpr int ST_THREADS = 64 + ST_CONSUMERS;
+constexpr int ST_THREADS = 64 + ST_CONSUMERS + 32;
 constexpr int ST_MAX_NQ = 128;
 constexpr float ST_LOG2E = 1.4426950408889634f;
-constexpr size_t ST_SMEM_BYTES = 1024 + 2 * ST_TILE_BYTES + (size_t)ST_STAGES * ST_TILE_BYTES +
-                                 (2 * 4 * 128 + 128 + ST_TILES * 4 * 128) * sizeof(float) + 64;
+constexpr size_t ST_SMEM_BYTES = 1024 + (size_t)ST_QBUF * ST_TILE_BYTES + (size_t)ST_STAGES * ST_TILE_BYTES +
+                                 (2 * 2 * 4 * 128 + 2 * 128 + ST_TBUF * 4 * 128) * sizeof(float) + 64;
 
 struct ScoreItem {
     int cache, lh, chunk, nt;      // nt: tiles of the chunk that hold at least one key
@@ -107,15 +112,18 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
 {
     extern __shared__ uint8_t st_smem_raw[];
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(st_smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t *q_s = base;                                           // 2 x [128 x 128] bf16 (round parity), two 64-column halves each
-    uint8_t *ring = q_s + 2 * ST_TILE_BYTES;                       // ST_STAGES x 32 KiB
-    float *s_m = reinterpret_cast<float *>(ring + ST_STAGES * ST_TILE_BYTES);   // [4 parts][128 queries] running maxima
-    float *s_z = s_m + 4 * 128;                                    // [4 parts][128 queries] running sums
-    float *s_mp = s_z + 4 * 128;                                   // [128] M'_t of the head being pooled
-    float *s_acc = s_mp + 128;                                     // [ST_TILES][4 parts][128 keys] pooled partial masses
-    __shared__ uint64_t bar_q_full[2], bar_q_free[2], bar_full[ST_STAGES], bar_empty[ST_STAGES];
+    uint8_t *q_s = base;                                           // ST_QBUF x [128 x 128] bf16 (round mod ST_QBUF), two 64-column halves each
+    uint8_t *ring = q_s + ST_QBUF * ST_TILE_BYTES;                       // ST_STAGES x 32 KiB
+    float *s_m = reinterpret_cast<float *>(ring + ST_STAGES * ST_TILE_BYTES);   // [2][4 parts][128 queries] chunk maxima
+    float *s_z = s_m + 2 * 4 * 128;                                // [2][4 parts][128 queries] chunk sums
+    float *s_mp = s_z + 2 * 4 * 128;                               // [2][128] M'_t of the head being pooled
+    float *s_acc = s_mp + 2 * 128;                                 // [ST_TBUF][4 parts][128 keys] pooled partial masses
+    __shared__ uint64_t bar_q_full[ST_QBUF], bar_q_free[ST_QBUF], bar_full[ST_STAGES], bar_empty[ST_STAGES];
     __shared__ uint64_t bar_t_full[ST_TBUF], bar_t_empty[ST_TBUF];
-    __shared__ uint32_t s_tmem, s_abort, s_last;
+    // pooled partial masses of an accumulator tile: written by the four column parts, summed by one of them
+    __shared__ uint64_t bar_acc_ready[ST_TBUF], bar_acc_free[ST_TBUF];
+    __shared__ uint64_t bar_st_ready[2], bar_st_free[2], bar_mp_ready[2], bar_mp_free[2];
+    __shared__ uint32_t s_tmem, s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int R = p.sc_rounds;
@@ -123,9 +131,20 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
 
     if (tid == 0) {
         s_abort = 0u;
-        for (int b = 0; b < 2; ++b) { tc::mbar_init(&bar_q_full[b], 1); tc::mbar_init(&bar_q_free[b], 1); }
+        for (int b = 0; b < ST_QBUF; ++b) { tc::mbar_init(&bar_q_full[b], 1); tc::mbar_init(&bar_q_free[b], 1); }
         for (int s = 0; s < ST_STAGES; ++s) { tc::mbar_init(&bar_full[s], 1); tc::mbar_init(&bar_empty[s], 1); }
-        for (int s = 0; s < ST_TBUF; ++s) { tc::mbar_init(&bar_t_full[s], 1); tc::mbar_init(&bar_t_empty[s], ST_CONSUMERS / 32); }
+        for (int s = 0; s < ST_TBUF; ++s) {
+            tc::mbar_init(&bar_t_full[s], 1);
+            tc::mbar_init(&bar_t_empty[s], ST_CONSUMERS / 32);
+            tc::mbar_init(&bar_acc_ready[s], ST_CONSUMERS / 32);
+            tc::mbar_init(&bar_acc_free[s], 4);
+        }
+        for (int b = 0; b < 2; ++b) {
+            tc::mbar_init(&bar_st_ready[b], ST_CONSUMERS / 32);
+            tc::mbar_init(&bar_st_free[b], 1);
+            tc::mbar_init(&bar_mp_ready[b], 1);
+            tc::mbar_init(&bar_mp_free[b], ST_CONSUMERS / 32);
+        }
         tc::mbar_init_fence();
     }
     if (warp == 1) tc::tmem_alloc(&s_tmem, 512);
@@ -137,7 +156,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            uint32_t it = 0, nq[2] = {0u, 0u};
+            uint32_t it = 0, nq[ST_QBUF] = {0u, 0u, 0u};
             bool dead = false;
             for (int i = 0; i <= R && !dead; ++i) {
                 for (int pass = 0; pass < 2 && !dead; ++pass) {
@@ -145,19 +164,27 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                     if (r < 0 || r >= R) continue;
                     ScoreItem item;
                     if (!score_item(p, r, (int)blockIdx.x, item)) continue;
-                    const int qb = r & 1;
+                    const int qb = r % ST_QBUF;
                     if (pass == 0) {
                         // the buffer is free once the pooling MMAs of its previous user are done
-                        if (nq[qb] > 0 && !tc::mbar_wait(&bar_q_free[qb], (nq[qb] - 1) & 1u, wc)) { dead = true; break; }
+                        if (nq[qb] > 0 && !tc::mbar_wait(&bar_q_free[qb], (nq[qb] - 1) & 1u, wc, 32)) { dead = true; break; }
                         const uint32_t qdst = tc::smem_u32(q_s + qb * ST_TILE_BYTES);
                         tc::mbar_expect_tx(&bar_q_full[qb], ST_TILE_BYTES);
                         tc::tma_load_3d(qdst, &tm.b[item.cache], &bar_q_full[qb], 0, 0, item.lh);
                         tc::tma_load_3d(qdst + ST_TILE_BYTES / 2, &tm.b[item.cache], &bar_q_full[qb], 64, 0, item.lh);
                         ++nq[qb];
+                        // the next round's first visit comes from HBM: ask for its tiles now
+                        ScoreItem nx;
+                        if (r + 1 < R && score_item(p, r + 1, (int)blockIdx.x, nx)) {
+                            for (int t = 0; t < nx.nt; ++t) {
+                                tc::tma_prefetch_l2_3d(&tm.a[nx.cache], 0, nx.chunk * ST_CHUNK + t * 128, nx.lh);
+                                tc::tma_prefetch_l2_3d(&tm.a[nx.cache], 64, nx.chunk * ST_CHUNK + t * 128, nx.lh);
+                            }
+                        }
                     }
                     for (int t = 0; t < item.nt; ++t, ++it) {
                         const int s = it % ST_STAGES;
-                        if (!tc::mbar_wait(&bar_empty[s], ((it / ST_STAGES) & 1u) ^ 1u, wc)) { dead = true; break; }
+                        if (!tc::mbar_wait(&bar_empty[s], ((it / ST_STAGES) & 1u) ^ 1u, wc, 32)) { dead = true; break; }
                         tc::mbar_expect_tx(&bar_full[s], ST_TILE_BYTES);
                         const uint32_t dst = tc::smem_u32(ring + s * ST_TILE_BYTES);
                         const int row0 = item.chunk * ST_CHUNK + t * 128;
@@ -168,15 +195,15 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
             }
             // nothing this thread started may still be in flight when the block exits
             for (uint32_t j = it > (uint32_t)ST_STAGES ? it - ST_STAGES : 0u; j < it; ++j)
-                tc::mbar_wait(&bar_full[j % ST_STAGES], (j / ST_STAGES) & 1u, wc);
-            for (int b = 0; b < 2; ++b)
-                if (nq[b] > 0) tc::mbar_wait(&bar_q_full[b], (nq[b] - 1) & 1u, wc);
+                tc::mbar_wait(&bar_full[j % ST_STAGES], (j / ST_STAGES) & 1u, wc, 32);
+            for (int b = 0; b < ST_QBUF; ++b)
+                if (nq[b] > 0) tc::mbar_wait(&bar_q_full[b], (nq[b] - 1) & 1u, wc, 32);
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
             constexpr uint32_t IDESC = tc::idesc_bf16(128, 128, 0, 0);
-            uint32_t it = 0, nq[2] = {0u, 0u};
+            uint32_t it = 0, nq[ST_QBUF] = {0u, 0u, 0u};
             bool dead = false;
             for (int i = 0; i <= R && !dead; ++i) {
                 for (int pass = 0; pass < 2 && !dead; ++pass) {
@@ -184,16 +211,16 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                     if (r < 0 || r >= R) continue;
                     ScoreItem item;
                     if (!score_item(p, r, (int)blockIdx.x, item)) continue;
-                    const int qb = r & 1;
+                    const int qb = r % ST_QBUF;
                     if (pass == 0) {
-                        if (!tc::mbar_wait(&bar_q_full[qb], nq[qb] & 1u, wc)) { dead = true; break; }
+                        if (!tc::mbar_wait(&bar_q_full[qb], nq[qb] & 1u, wc, 32)) { dead = true; break; }
                         ++nq[qb];
                     }
                     const uint32_t qaddr = tc::smem_u32(q_s + qb * ST_TILE_BYTES);
                     for (int t = 0; t < item.nt; ++t, ++it) {
                         const int s = it % ST_STAGES, tb = it % ST_TBUF;
-                        if (!tc::mbar_wait(&bar_t_empty[tb], ((it / ST_TBUF) & 1u) ^ 1u, wc)) { dead = true; break; }
-                        if (!tc::mbar_wait(&bar_full[s], (it / ST_STAGES) & 1u, wc)) { dead = true; break; }
+                        if (!tc::mbar_wait(&bar_t_empty[tb], ((it / ST_TBUF) & 1u) ^ 1u, wc, 32)) { dead = true; break; }
+                        if (!tc::mbar_wait(&bar_full[s], (it / ST_STAGES) & 1u, wc, 32)) { dead = true; break; }
                         tc::tc_fence_after();
                         const uint32_t kaddr = tc::smem_u32(ring + s * ST_TILE_BYTES);
                         const uint32_t acc = tmem + (uint32_t)(tb * 128);
@@ -214,44 +241,51 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                 }
             }
         }
-    } else {
+    } else if (warp < 2 + ST_CONSUMERS / 32) {
         // ---------------- consumers ----------------
-        const int ct = tid - 64;                       // 0..511
         const int q = warp & 3;                        // tensor-memory lane quarter this warp may touch
-        const int part = (warp - 2) >> 2;              // which 32 columns of a tile
+        const int part = (warp - 2) >> 2;              // which tile of a chunk
         const int row = q * 32 + lane;                 // lane of the accumulator tile: a query (pass A) or a key (pass B)
-        const uint32_t tlane = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(part * 32);
+        const uint32_t tlane = tmem + ((uint32_t)(q * 32) << 16);
         const float sc = ST_LOG2E * rsqrtf(128.0f);
-        uint32_t it = 0;
+        uint32_t it = 0, n_a[2] = {0u, 0u}, n_b[2] = {0u, 0u};
+        uint32_t acc_used = 0u, acc_par = 0u;          // per accumulator tile: s_acc slot used before, parity of its uses
 
         for (int i = 0; i <= R; ++i) {
-            // ======== pass A of round i: running maximum and sum per query ========
+            // ======== pass A of round i: maximum and sum per query over columns [32 * part, +32) of the chunk's tiles ========
             ScoreItem item;
             if (i < R && score_item(p, i, (int)blockIdx.x, item)) {
-                const CacheDev &c = p.c[item.cache];
-                const int g = c.head_base + item.lh;
-                const int T = c.T, team = c.sc_team;
+                const int T = p.c[item.cache].T, buf = i & 1;
                 float m = -INFINITY, z = 0.f;
-                for (int t = 0; t < item.nt; ++t, ++it) {
-                    const int tb = it % ST_TBUF;
-                    tc::mbar_wait(&bar_t_full[tb], (it / ST_TBUF) & 1u, wc);
+#pragma unroll 1
+                for (int t = 0; t < item.nt; ++t) {
+                    // columns [32 * part, +32) of every tile of the chunk; the tile is released as soon as they are in registers
+                    const uint32_t ti = it + t;
+                    const int tb = ti % ST_TBUF;
+                    tc::mbar_wait(&bar_t_full[tb], (ti / ST_TBUF) & 1u, wc);
                     tc::tc_fence_after();
                     uint32_t rr[32];
-                    tc::tmem_ld32(tlane + (uint32_t)(tb * 128), rr);
+                    tc::tmem_ld32(tlane + (uint32_t)(tb * 128 + part * 32), rr);
                     tc::tmem_ld_wait();
                     tc::tc_fence_before();
                     __syncwarp();
                     if (lane == 0) tc::mbar_arrive(&bar_t_empty[tb]);
-                    const int key0 = item.chunk * ST_CHUNK + t * 128 + part * 32;      // key of this thread's column 0
+                    const int key0 = item.chunk * ST_CHUNK + t * 128 + part * 32;         // key of column 0 of this block
                     if (key0 + 32 > T) {
 #pragma unroll
                         for (int e = 0; e < 32; ++e)
-                            if (key0 + e >= T) rr[e] = 0xff800000u;                    // -inf: no such key
+                            if (key0 + e >= T) rr[e] = 0xff800000u;                        // -inf: no such key
                     }
-                    float tm_ = -INFINITY;
+                    float t0_ = __uint_as_float(rr[0]), t1_ = __uint_as_float(rr[1]);
+                    float t2_ = __uint_as_float(rr[2]), t3_ = __uint_as_float(rr[3]);
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) tm_ = fmaxf(tm_, __uint_as_float(rr[e]));
-                    const float mn = fmaxf(m, tm_ * sc);
+                    for (int e = 4; e < 32; e += 4) {
+                        t0_ = fmaxf(t0_, __uint_as_float(rr[e]));
+                        t1_ = fmaxf(t1_, __uint_as_float(rr[e + 1]));
+                        t2_ = fmaxf(t2_, __uint_as_float(rr[e + 2]));
+                        t3_ = fmaxf(t3_, __uint_as_float(rr[e + 3]));
+                    }
+                    const float mn = fmaxf(m, fmaxf(fmaxf(t0_, t1_), fmaxf(t2_, t3_)) * sc);
                     if (mn > -INFINITY) {
                         float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
 #pragma unroll
@@ -265,80 +299,35 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                         m = mn;
                     }
                 }
-                // fold the four column parts of every query, publish the chunk's (m, z)
-                s_m[part * 128 + row] = m;
-                s_z[part * 128 + row] = z;
-                tc::named_barrier(1, ST_CONSUMERS);
-                float2 *partials = reinterpret_cast<float2 *>(p.sc_part) + (c.sc_part_off + ((size_t)item.lh * team + item.chunk) * 128);
-                if (ct < p.n_q) {
-                    float M = fmaxf(fmaxf(s_m[ct], s_m[128 + ct]), fmaxf(s_m[256 + ct], s_m[384 + ct]));
-                    float Z = 0.f;
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float me = s_m[e * 128 + ct];
-                        if (me > -INFINITY) Z += s_z[e * 128 + ct] * ex2_approx(me - M);
-                    }
-                    __stcg(&partials[ct], make_float2(M, Z));
-                }
-                tc::named_barrier(1, ST_CONSUMERS);
-                // the barrier orders the block's stores before thread 0's release; the acquire side mirrors it
-                if (ct == 0) s_last = (atom_add_acq_rel_gpu(&p.sc_cnt[g], 1u) == (uint32_t)(team - 1)) ? 1u : 0u;
-                tc::named_barrier(1, ST_CONSUMERS);
-                if (s_last && ct < p.n_q) {
-                    const float2 *hp = reinterpret_cast<const float2 *>(p.sc_part) + (c.sc_part_off + (size_t)item.lh * team * 128);
-                    float M = -INFINITY;
-                    for (int ch = 0; ch < team; ++ch) M = fmaxf(M, __ldcg(&hp[(size_t)ch * 128 + ct]).x);
-                    float Z = 0.f;
-                    for (int ch = 0; ch < team; ++ch) {
-                        const float2 v = __ldcg(&hp[(size_t)ch * 128 + ct]);
-                        Z += v.y * ex2_approx(v.x - M);
-                    }
-                    float mp = M + lg2_approx(Z);
-                    if (!(Z > 0.f) || !isfinite(mp)) {
-                        atomicOr(p.status, OBF_DEV_NONFINITE);
-                        mp = __int_as_float(0x7fc00000);
-                    }
-                    // one 64-bit word per query: low = M'_t, high = 1 once it is valid
-                    st_relaxed_gpu_u64(reinterpret_cast<unsigned long long *>(p.sc_head) + (size_t)g * 128 + ct,
-                                       (1ull << 32) | __float_as_uint(mp));
-                }
+                it += item.nt;
+                // hand (m, z) of this column part to the messenger
+                if (n_a[buf] > 0) tc::mbar_wait(&bar_st_free[buf], (n_a[buf] - 1) & 1u, wc);
+                s_m[(buf * 4 + part) * 128 + row] = m;
+                s_z[(buf * 4 + part) * 128 + row] = z;
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(&bar_st_ready[buf]);
+                ++n_a[buf];
             }
-            // ======== pass B of round i - 1: pooled mass per key ========
+            // ======== pass B of round i - 1: pooled mass per key over queries [32 * part, +32) ========
             if (i >= 1 && score_item(p, i - 1, (int)blockIdx.x, item)) {
                 const CacheDev &c = p.c[item.cache];
-                const int g = c.head_base + item.lh;
-                const int T = c.T;
-                if (ct < 128) {
-                    float mp = INFINITY;                                   // exp2(-inf) = 0 for padding columns
-                    if (ct < p.n_q) {
-                        const unsigned long long *word = reinterpret_cast<const unsigned long long *>(p.sc_head) + (size_t)g * 128 + ct;
-                        const uint64_t t0 = tc::global_ns();
-                        unsigned long long v;
-                        while (((v = ld_relaxed_gpu_u64(word)) >> 32) == 0ull) {
-                            if (s_abort) break;
-                            if (tc::global_ns() - t0 > tc::WAIT_LIMIT_NS) {
-                                s_abort = 1u;
-                                atomicOr(p.status, OBF_DEV_TIMEOUT);
-                                break;
-                            }
-                        }
-                        mp = __uint_as_float((uint32_t)v);
-                    }
-                    s_mp[ct] = mp;
-                }
-                tc::named_barrier(1, ST_CONSUMERS);
+                const int T = c.T, buf = (i - 1) & 1;
+                tc::mbar_wait(&bar_mp_ready[buf], n_b[buf] & 1u, wc);
                 float mp[32];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    const float4 v = *reinterpret_cast<const float4 *>(&s_mp[part * 32 + e * 4]);
+                    const float4 v = *reinterpret_cast<const float4 *>(s_mp + buf * 128 + part * 32 + e * 4);
                     mp[4 * e] = v.x; mp[4 * e + 1] = v.y; mp[4 * e + 2] = v.z; mp[4 * e + 3] = v.w;
                 }
-                for (int t = 0; t < item.nt; ++t, ++it) {
-                    const int tb = it % ST_TBUF;
-                    tc::mbar_wait(&bar_t_full[tb], (it / ST_TBUF) & 1u, wc);
+#pragma unroll 1
+                for (int t = 0; t < item.nt; ++t) {
+                    // queries [32 * part, +32) of every tile of the chunk; the tile is released as soon as they are in registers
+                    const uint32_t ti = it + t;
+                    const int tb = ti % ST_TBUF;
+                    tc::mbar_wait(&bar_t_full[tb], (ti / ST_TBUF) & 1u, wc);
                     tc::tc_fence_after();
                     uint32_t rr[32];
-                    tc::tmem_ld32(tlane + (uint32_t)(tb * 128), rr);
+                    tc::tmem_ld32(tlane + (uint32_t)(tb * 128 + part * 32), rr);
                     tc::tmem_ld_wait();
                     tc::tc_fence_before();
                     __syncwarp();
@@ -351,21 +340,133 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                         a2 += ex2_approx(fmaf(__uint_as_float(rr[e + 2]), sc, -mp[e + 2]));
                         a3 += ex2_approx(fmaf(__uint_as_float(rr[e + 3]), sc, -mp[e + 3]));
                     }
-                    s_acc[(t * 4 + part) * 128 + row] = (a0 + a1) + (a2 + a3);
-                }
-                tc::named_barrier(1, ST_CONSUMERS);
-                {
-                    const int t = ct >> 7, key = ct & 127;
-                    const int j = item.chunk * ST_CHUNK + t * 128 + key;
-                    if (t < item.nt && j < T) {
-                        const float *sa = s_acc + t * 4 * 128 + key;
+                    // the four parts meet in shared memory; part (t mod 4) adds them up and writes the masses
+                    const uint32_t bit = 1u << tb;
+                    if (acc_used & bit) tc::mbar_wait(&bar_acc_free[tb], ((acc_par >> tb) & 1u) ^ 1u, wc);
+                    s_acc[(tb * 4 + part) * 128 + row] = (a0 + a1) + (a2 + a3);
+                    __syncwarp();
+                    if (lane == 0) tc::mbar_arrive(&bar_acc_ready[tb]);
+                    if (part == (t & 3)) {
+                        tc::mbar_wait(&bar_acc_ready[tb], (acc_par >> tb) & 1u, wc);
+                        const float *sa = s_acc + tb * 4 * 128 + row;
                         const float a = (sa[0] + sa[128]) + (sa[256] + sa[384]);
-                        if (!isfinite(a)) atomicOr(p.status, OBF_DEV_NONFINITE);
-                        p.scores[c.tok_off + (size_t)item.lh * T + j] = a;
-                        if (c.scores_out) c.scores_out[(size_t)item.lh * T + j] = a;
+                        __syncwarp();
+                        if (lane == 0) tc::mbar_arrive(&bar_acc_free[tb]);
+                        const int j = item.chunk * ST_CHUNK + t * 128 + row;
+                        if (j < T) {
+                            if (!isfinite(a)) atomicOr(p.status, OBF_DEV_NONFINITE);
+                            p.scores[c.tok_off + (size_t)item.lh * T + j] = a;
+                            if (c.scores_out) c.scores_out[(size_t)item.lh * T + j] = a;
+                        }
+                    }
+                    acc_used |= bit;
+                    acc_par ^= bit;
+                }
+                it += item.nt;
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(&bar_mp_free[buf]);
+                ++n_b[buf];
+            }
+        }
+    } else {
+        // ---------------- messenger ----------------
+        uint32_t n_a[2] = {0u, 0u}, n_b[2] = {0u, 0u};
+        for (int i = 0; i <= R; ++i) {
+            ScoreItem item;
+            // M' of the head that is pooled next, into shared memory
+            if (i >= 1 && score_item(p, i - 1, (int)blockIdx.x, item)) {
+                const int buf = (i - 1) & 1;
+                const int g = p.c[item.cache].head_base + item.lh;
+                if (n_b[buf] > 0) tc::mbar_wait(&bar_mp_free[buf], (n_b[buf] - 1) & 1u, wc, 32);
+                const unsigned long long *words = reinterpret_cast<const unsigned long long *>(p.sc_head) + (size_t)g * 128;
+                // the four words of this lane are polled together: one round trip, not four
+                unsigned long long v[4] = {0ull, 0ull, 0ull, 0ull};
+                const uint64_t t0 = tc::global_ns();
+                for (;;) {
+                    bool all = true;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        if (lane + 32 * k < p.n_q && (v[k] >> 32) == 0ull) v[k] = ld_relaxed_gpu_u64(words + lane + 32 * k);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        if (lane + 32 * k < p.n_q && (v[k] >> 32) == 0ull) all = false;
+                    if (all || s_abort) break;
+                    if (tc::global_ns() - t0 > tc::WAIT_LIMIT_NS) {
+                        s_abort = 1u;
+                        atomicOr(p.status, OBF_DEV_TIMEOUT);
+                        break;
+                    }
+                    __nanosleep(32);
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int t = lane + 32 * k;
+                    // exp2(-inf) = 0 for padding columns
+                    s_mp[buf * 128 + t] = t < p.n_q ? __uint_as_float((uint32_t)v[k]) : INFINITY;
+                }
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(&bar_mp_ready[buf]);
+                ++n_b[buf];
+            }
+            // statistics of the chunk the consumers have just finished
+            if (i < R && score_item(p, i, (int)blockIdx.x, item)) {
+                const CacheDev &c = p.c[item.cache];
+                const int buf = i & 1, team = c.sc_team;
+                const int g = c.head_base + item.lh;
+                tc::mbar_wait(&bar_st_ready[buf], n_a[buf] & 1u, wc, 32);
+                float2 *partials = reinterpret_cast<float2 *>(p.sc_part) + (c.sc_part_off + ((size_t)item.lh * team + item.chunk) * 128);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int t = lane + 32 * k;
+                    const float *sm = s_m + buf * 4 * 128 + t, *sz = s_z + buf * 4 * 128 + t;
+                    const float M = fmaxf(fmaxf(sm[0], sm[128]), fmaxf(sm[256], sm[384]));
+                    float Z = 0.f;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        if (sm[e * 128] > -INFINITY) Z += sz[e * 128] * ex2_approx(sm[e * 128] - M);
+                    if (t < p.n_q) __stcg(&partials[t], make_float2(M, Z));
+                }
+                __syncwarp();
+                uint32_t last = 0u;
+                if (lane == 0) {
+                    tc::mbar_arrive(&bar_st_free[buf]);
+                    // the warp barrier orders the lanes' stores before this release; the acquire side mirrors it
+                    last = (atom_add_acq_rel_gpu(&p.sc_cnt[g], 1u) == (uint32_t)(team - 1)) ? 1u : 0u;
+                }
+                last = __shfl_sync(0xffffffffu, last, 0);
+                ++n_a[buf];
+                if (last) {
+                    // this block is the last of its head: fold all chunks
+                    const float2 *hp = reinterpret_cast<const float2 *>(p.sc_part) + (c.sc_part_off + (size_t)item.lh * team * 128);
+                    unsigned long long *words = reinterpret_cast<unsigned long long *>(p.sc_head) + (size_t)g * 128;
+                    for (int t = lane; t < p.n_q; t += 32) {
+                        // one sweep over the chunks, eight loads in flight at a time
+                        float M = -INFINITY, Z = 0.f;
+                        for (int c0 = 0; c0 < team; c0 += 8) {
+                            float2 v[8];
+#pragma unroll
+                            for (int e = 0; e < 8; ++e)
+                                v[e] = c0 + e < team ? __ldcg(&hp[(size_t)(c0 + e) * 128 + t]) : make_float2(-INFINITY, 0.f);
+                            float Mn = M;
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) Mn = fmaxf(Mn, v[e].x);
+                            if (Mn > -INFINITY) {
+                                Z *= ex2_approx(M - Mn);
+#pragma unroll
+                                for (int e = 0; e < 8; ++e)
+                                    if (v[e].x > -INFINITY) Z += v[e].y * ex2_approx(v[e].x - Mn);
+                                M = Mn;
+                            }
+                        }
+                        float mp = M + lg2_approx(Z);
+                        if (!(Z > 0.f) || !isfinite(mp)) {
+                            atomicOr(p.status, OBF_DEV_NONFINITE);
+                            mp = __int_as_float(0x7fc00000);
+                        }
+                        // one 64-bit word per query: low = M'_t, high = 1 once it is valid
+                        st_relaxed_gpu_u64(words + t, (1ull << 32) | __float_as_uint(mp));
                     }
                 }
-                tc::named_barrier(1, ST_CONSUMERS);
             }
         }
     }

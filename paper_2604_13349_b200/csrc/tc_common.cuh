@@ -63,16 +63,20 @@ struct WaitCtx {
 
 // Waits until the phase of `bar` with the given parity has completed.  Returns
 // false (at once if the block already aborted, else after WAIT_LIMIT_NS) when the
-// wait was abandoned.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, const WaitCtx &w)
+// wait was abandoned.  A non-zero `sleep_ns` makes a single-thread role (producer,
+// MMA issuer) back off between polls so that it does not take issue slots from
+// the warps that compute.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, const WaitCtx &w, uint32_t sleep_ns = 0)
 {
     if (mbar_try(bar, parity)) return true;
     if (*w.abort_flag) return false;
     const uint64_t t0 = global_ns();
     for (;;) {
 #pragma unroll 1
-        for (int i = 0; i < 32; ++i)
+        for (int i = 0; i < 32; ++i) {
             if (mbar_try(bar, parity)) return true;
+            if (sleep_ns) __nanosleep(sleep_ns);
+        }
         if (*w.abort_flag) return false;
         if (global_ns() - t0 > WAIT_LIMIT_NS) {
             *w.abort_flag = 1u;
@@ -90,6 +94,13 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
 {
     asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
                  ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z) : "memory");
+}
+
+// Asks for the tile to be brought into the L2 cache; nothing lands in shared memory.
+__device__ __forceinline__ void tma_prefetch_l2_3d(const CUtensorMap *map, int x, int y, int z)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
+                 ::"l"(map), "r"(x), "r"(y), "r"(z) : "memory");
 }
 
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map)
