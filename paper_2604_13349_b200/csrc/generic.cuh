@@ -267,30 +267,200 @@ __global__ void __launch_bounds__(SEL_NT) k_select(const __grid_constant__ CallD
     }
 }
 
-// Step a3: K_out = K[idx], V_out = V[idx], one warp per retained row, 16-byte vectors.
-// grid = (ceil(k_eff_max/8), heads_total).
+// Step a2 for heads whose T keys fit in shared memory (the usual case): same result as
+// k_select, bit for bit, but the order-preserving keys are read from global memory
+// once.  The radix histogram is built with one shared-memory atomic per distinct digit
+// and warp; the ordered pass gives every warp a contiguous run of positions, so two
+// block-wide barriers suffice.
+constexpr int SEL_SMEM_MAX_T = 16384;
+
+__global__ void __launch_bounds__(SEL_NT) k_select_smem(const __grid_constant__ CallDev p)
+{
+    extern __shared__ uint32_t sel_keys[];
+    __shared__ uint32_t hist[256];
+    __shared__ uint32_t s_prefix, s_want;
+    __shared__ uint32_t wtot[32];
+    __shared__ float red[32];
+    int ci, lh;
+    locate(p, blockIdx.x, ci, lh);
+    const CacheDev &c = p.c[ci];
+    const int T = c.T, k = c.k_eff;
+    float *Af = p.scores + c.tok_off + (size_t)lh * T;
+    const uint32_t *A = reinterpret_cast<const uint32_t *>(Af);
+    uint8_t *keep = p.keep + c.tok_off + (size_t)lh * T;
+    int32_t *idx = c.idx_out + (size_t)lh * k;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    for (int j = tid; j < T; j += SEL_NT) sel_keys[j] = score_key_bits(A[j]);
+    if (tid == 0) { s_prefix = 0u; s_want = (uint32_t)k; }
+    uint32_t mask = 0u;
+    const int T_pad = (T + SEL_NT - 1) / SEL_NT * SEL_NT;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        if (tid < 256) hist[tid] = 0u;
+        __syncthreads();
+        const uint32_t prefix = s_prefix;
+        for (int j = tid; j < T_pad; j += SEL_NT) {
+            const uint32_t u = j < T ? sel_keys[j] : 0u;
+            const bool cand = j < T && (u & mask) == prefix;
+            const uint32_t digit = (u >> shift) & 255u;
+            // lanes that are no candidates form one group of their own, which adds nothing
+            const uint32_t peers = __match_any_sync(0xffffffffu, cand ? digit : 256u);
+            if (cand && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], (uint32_t)__popc(peers));
+        }
+        __syncthreads();
+        if (warp == 0) {
+            // lane l owns bins [8l, 8l+8); walk down from the top bin
+            uint32_t own = 0u;
+#pragma unroll
+            for (int b = 0; b < 8; ++b) own += hist[lane * 8 + b];
+            uint32_t above = own;                       // inclusive sum over lanes >= this one
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t n = __shfl_down_sync(0xffffffffu, above, o);
+                if (lane + o < 32) above += n;
+            }
+            const uint32_t want = s_want;
+            const uint32_t excl = above - own;          // keys in bins above this lane's
+            const bool mine = excl < want && want <= above;
+            const uint32_t who = __ballot_sync(0xffffffffu, mine);
+            // total < want cannot happen (want <= candidates); guard anyway: lowest bin
+            const int sel_lane = who ? 31 - __clz(who) : 0;
+            if (lane == sel_lane) {
+                uint32_t cum = who ? excl : 0u;
+                int b = 7;
+                for (; b > 0; --b) {
+                    const uint32_t h = hist[lane * 8 + b];
+                    if (cum + h >= want) break;
+                    cum += h;
+                }
+                s_want = want - cum;
+                s_prefix = prefix | ((uint32_t)(lane * 8 + b) << shift);
+            }
+        }
+        mask |= 255u << shift;
+        __syncthreads();
+    }
+    const uint32_t tau = s_prefix;       // key of the k-th largest mass
+    const uint32_t want = s_want;        // how many positions with key == tau are retained (>= 1)
+
+    // ordered pass: warp w owns positions [w * seg, (w + 1) * seg)
+    const int seg = ((T + 31) / 32 + 31) / 32 * 32;
+    const int j_begin = warp * seg, j_end = min(T, j_begin + seg);
+    uint32_t n_gt = 0u, n_eq = 0u;
+    for (int j0 = j_begin; j0 < j_end; j0 += 32) {
+        const int j = j0 + lane;
+        const uint32_t u = j < j_end ? sel_keys[j] : 0u;
+        n_gt += __popc(__ballot_sync(0xffffffffu, j < j_end && u > tau));
+        n_eq += __popc(__ballot_sync(0xffffffffu, j < j_end && u == tau));
+    }
+    if (lane == 0) wtot[warp] = n_gt | (n_eq << 16);
+    __syncthreads();
+    if (warp == 0) {
+        const uint32_t w = wtot[lane];
+        uint32_t inc = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t n = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += n;
+        }
+        wtot[lane] = inc - w;              // positions before this warp's run: greater (low half), equal (high half)
+    }
+    __syncthreads();
+    uint32_t run_gt = wtot[warp] & 0xFFFFu, run_eq = wtot[warp] >> 16;
+    float sk = 0.f, sd = 0.f, nx = -1.0f;
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    for (int j0 = j_begin; j0 < j_end; j0 += 32) {
+        const int j = j0 + lane;
+        const bool valid = j < j_end;
+        const uint32_t u = valid ? sel_keys[j] : 0u;
+        const bool gt = valid && u > tau, eq = valid && u == tau;
+        const uint32_t m_gt = __ballot_sync(0xffffffffu, gt), m_eq = __ballot_sync(0xffffffffu, eq);
+        const uint32_t gt_before = run_gt + __popc(m_gt & lt_mask), eq_before = run_eq + __popc(m_eq & lt_mask);
+        const bool kp = gt || (eq && eq_before < want);
+        if (valid) {
+            const float a = key_score(u);
+            keep[j] = kp ? 1 : 0;
+            if (kp) {
+                Af[j] = -1.0f;             // later passes need the mass of deleted tokens only
+                const uint32_t pos = gt_before + min(eq_before, want);
+                if (pos < (uint32_t)k) idx[pos] = j;
+                else atomicOr(p.status, OBF_DEV_INTERNAL);
+                sk += a;
+            } else { sd += a; nx = fmaxf(nx, a); }
+        }
+        run_gt += __popc(m_gt);
+        run_eq += __popc(m_eq);
+    }
+    const float a_keep = block_sum<SEL_NT>(sk, red);
+    const float a_del = block_sum<SEL_NT>(sd, red);
+    const float next = block_max<SEL_NT>(nx, red);
+    if (tid == 0) {
+        float *sm = p.sums + (size_t)blockIdx.x * 4;
+        sm[0] = a_keep; sm[1] = a_del; sm[2] = key_score(tau); sm[3] = next;
+        if (c.diag) {
+            obf_diag_t dg;
+            dg.a_keep = a_keep; dg.a_del = a_del; dg.alpha = a_del / (a_keep + p.eps);
+            dg.rcr = 0.f; dg.delta_norm = 0.f; dg.kth_score = key_score(tau); dg.next_score = next;
+            dg.lam_1 = dg.lam_rho = dg.lam_next = 0.f;
+            dg.span_rank = -1; dg.rho_eff = 0; dg.status = OBF_DEV_SKIPPED; dg.reserved = 0;
+            c.diag[lh] = dg;
+        }
+    }
+}
+
+// Step a3: K_out = K[idx], V_out = V[idx] as 16-byte vectors.  A block copies GATHER_ROWS
+// retained rows of one head; every thread moves one vector of four different rows of K
+// and of V, with all eight loads in flight before the first store.
+// grid = (ceil(k_eff_max / GATHER_ROWS), heads_total).
+constexpr int GATHER_ROWS = 64;
+
 template <int ROW_BYTES>
 __global__ void __launch_bounds__(256) k_gather(const __grid_constant__ CallDev p)
 {
+    constexpr int CH = ROW_BYTES / 16;             // vectors per row
+    constexpr int RPP = 256 / CH;                  // rows per pass of the block
+    constexpr int PASSES = GATHER_ROWS / RPP;
     int ci, lh;
     locate(p, blockIdx.y, ci, lh);
     const CacheDev &c = p.c[ci];
-    const int r = blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (r >= c.k_eff) return;
-    const int lane = threadIdx.x & 31;
-    const int j = c.idx_out[(size_t)lh * c.k_eff + r];
-    if ((unsigned)j >= (unsigned)c.T) {            // never dereference a position outside the cache
-        if (lane == 0) atomicOr(p.status, OBF_DEV_INTERNAL);
-        return;
-    }
-    constexpr int CH = ROW_BYTES / 16;
-    const uint4 *ks = reinterpret_cast<const uint4 *>(reinterpret_cast<const char *>(c.k) + ((size_t)lh * c.T + j) * ROW_BYTES);
-    const uint4 *vs = reinterpret_cast<const uint4 *>(reinterpret_cast<const char *>(c.v) + ((size_t)lh * c.T + j) * ROW_BYTES);
-    uint4 *kd = reinterpret_cast<uint4 *>(reinterpret_cast<char *>(c.k_out) + ((size_t)lh * c.k_eff + r) * ROW_BYTES);
-    uint4 *vd = reinterpret_cast<uint4 *>(reinterpret_cast<char *>(c.v_out) + ((size_t)lh * c.k_eff + r) * ROW_BYTES);
-    for (int ch = lane; ch < CH; ch += 32) {
-        kd[ch] = ks[ch];
-        vd[ch] = vs[ch];
+    const int r0 = blockIdx.x * GATHER_ROWS;
+    if (r0 >= c.k_eff) return;
+    const int ch = threadIdx.x % CH, rr = threadIdx.x / CH;
+    const char *kb = reinterpret_cast<const char *>(c.k) + (size_t)lh * c.T * ROW_BYTES;
+    const char *vb = reinterpret_cast<const char *>(c.v) + (size_t)lh * c.T * ROW_BYTES;
+    char *ko = reinterpret_cast<char *>(c.k_out) + (size_t)lh * c.k_eff * ROW_BYTES;
+    char *vo = reinterpret_cast<char *>(c.v_out) + (size_t)lh * c.k_eff * ROW_BYTES;
+    const int32_t *idx = c.idx_out + (size_t)lh * c.k_eff;
+#pragma unroll 1
+    for (int p0 = 0; p0 < PASSES; p0 += 4) {
+        int r[4], j[4];
+        uint4 kv[4], vv[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            r[u] = r0 + (p0 + u) * RPP + rr;
+            j[u] = -1;
+            if (p0 + u < PASSES && r[u] < c.k_eff) {
+                j[u] = idx[r[u]];
+                if ((unsigned)j[u] >= (unsigned)c.T) {     // never dereference a position outside the cache
+                    atomicOr(p.status, OBF_DEV_INTERNAL);
+                    j[u] = -1;
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (j[u] >= 0) {
+                kv[u] = *reinterpret_cast<const uint4 *>(kb + (size_t)j[u] * ROW_BYTES + ch * 16);
+                vv[u] = *reinterpret_cast<const uint4 *>(vb + (size_t)j[u] * ROW_BYTES + ch * 16);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (j[u] >= 0) {
+                *reinterpret_cast<uint4 *>(ko + (size_t)r[u] * ROW_BYTES + ch * 16) = kv[u];
+                *reinterpret_cast<uint4 *>(vo + (size_t)r[u] * ROW_BYTES + ch * 16) = vv[u];
+            }
+        }
     }
 }
 

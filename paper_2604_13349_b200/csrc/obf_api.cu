@@ -322,9 +322,15 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
         k_score_pool<TIN, D><<<g2, SC_NT, sm_sc, st>>>(cd);
         mark(st, "k_score_pool");
     }
-    k_select<<<heads, SEL_NT, 0, st>>>(cd);
+    if (T_max <= SEL_SMEM_MAX_T) {
+        const size_t sm_sel = (size_t)T_max * sizeof(uint32_t);
+        if ((s = set_smem(k_select_smem, sm_sel)) != OBF_OK) return s;
+        k_select_smem<<<heads, SEL_NT, sm_sel, st>>>(cd);
+    } else {
+        k_select<<<heads, SEL_NT, 0, st>>>(cd);
+    }
     mark(st, "k_select");
-    dim3 g4((k_max + 7) / 8, heads);
+    dim3 g4((k_max + GATHER_ROWS - 1) / GATHER_ROWS, heads);
     k_gather<D * (int)sizeof(TIN)><<<g4, 256, 0, st>>>(cd);
     mark(st, "k_gather");
     if (cd.rank > 0) {
