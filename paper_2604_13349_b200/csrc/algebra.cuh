@@ -134,7 +134,7 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
         }
         if (tid < D) {
             float s = 0.f;
-            for (int sp = 0; sp < n_del; ++sp) s += p.uvec[((size_t)g * S + sp) * D + tid];
+            for (int sp = 0; sp < n_del * p.u_groups; ++sp) s += p.uvec[((size_t)g * S * p.u_groups + sp) * D + tid];
             vu[tid] = s;
         }
         __syncthreads();

@@ -52,7 +52,7 @@ struct CallDev {
     int32_t splits;           // token splits of the Gram pass (shape-generic path)
     int32_t gram_slots;       // partial Gram matrices stored per head (stride of gram_d / gram_k / uvec)
     int32_t tc_per;           // tuned path: tiles per block of the Gram pass (0: shape-generic path)
-    int32_t pad_;
+    int32_t u_groups;         // partial u vectors stored per partial Gram matrix (1, tuned Gram pass: 2)
     long long tc_total_sub;   // tuned path: tiles in the call-wide tile sequence
     int32_t sc_nq;            // tuned score kernel: query rows of its tiles (0: shape-generic score kernels)
     int32_t sc_subs;          // 128-key tiles per chunk
@@ -70,7 +70,7 @@ struct CallDev {
     float *sums;              // [heads_total, 4] a_keep, a_del, kth, next
     float *gram_d;            // [heads_total, gram_slots, d, d] partial Gram of deleted values
     float *gram_k;            // [heads_total, gram_slots, d, d] partial Gram of retained values
-    float *uvec;              // [heads_total, gram_slots, d] partial sum_j A_j v_j over deleted j
+    float *uvec;              // [heads_total, gram_slots, u_groups, d] partial sum_j A_j v_j over deleted j
     float *delta;             // [heads_total, d]
     uint32_t *hflag;          // [heads_total] bit0: delta != 0 -> inject
 };

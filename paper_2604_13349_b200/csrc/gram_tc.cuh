@@ -14,12 +14,12 @@
 // (and one partial u), stored in slot (b - first block touching that head and kind).
 //
 // Block = 14 warps:
-//   warp 0        TMA producer: 128 x 128 bf16 tiles (two 128-byte-swizzled column halves) into a 5-stage ring
+//   warp 0        TMA producer: 128 x 128 bf16 tiles (two 128-byte-swizzled column halves) into a 6-stage ring
 //   warp 1        issues tcgen05.mma: G (+)= tile^T tile, both operands MN-major views of the same tile,
 //                 accumulators (128 lanes x 128 columns fp32) double-buffered in tensor memory
-//   warps 2..9    fix-up: zero the retained rows of a V tile in shared memory and accumulate u on the CUDA
-//                 cores; the attention mass of the tile after next (-1 marks a retained token) is
-//                 fetched while the current one is processed
+//   warps 2..9    fix-up, two groups of four warps taking tiles alternately: zero the retained rows of a
+//                 V tile in shared memory and accumulate u on the CUDA cores; the attention mass of the
+//                 group's next tile (-1 marks a retained token) is fetched while the current one is processed
 //   warps 10..13  epilogue: tensor memory -> partial Gram matrix in the workspace
 #pragma once
 
@@ -27,7 +27,7 @@
 
 namespace obf {
 
-constexpr int GT_STAGES = 5;
+constexpr int GT_STAGES = 6;
 constexpr int GT_TILE = 128;                       // tokens per tile
 constexpr int GT_TILE_BYTES = GT_TILE * 128 * 2;   // 32 KiB
 constexpr int GT_FIX_THREADS = 256;
@@ -113,7 +113,7 @@ __global__ void __launch_bounds__(GT_THREADS, 1) k_gram_tc(const __grid_constant
         s_abort = 0u;
         for (int s = 0; s < GT_STAGES; ++s) {
             tc::mbar_init(&bar_full[s], 1);
-            tc::mbar_init(&bar_ready[s], GT_FIX_THREADS / 32);
+            tc::mbar_init(&bar_ready[s], GT_FIX_THREADS / 64);
             tc::mbar_init(&bar_empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) { tc::mbar_init(&bar_acc_full[b], 1); tc::mbar_init(&bar_acc_empty[b], 4); }
@@ -183,74 +183,82 @@ __global__ void __launch_bounds__(GT_THREADS, 1) k_gram_tc(const __grid_constant
         }
     } else if (warp < 2 + GT_FIX_THREADS / 32) {
         // ---------------- fix-up: zero retained rows, accumulate u ----------------
+        // Two groups of four warps take the tiles of the run alternately, so that one group's
+        // tile can be fixed up while the other's is; each group keeps its own partial u.
         const int f = tid - 64;                    // 0..255
-        const int cg = f & 15, rg = f >> 4;        // 16-byte column group, row group (16 of them)
+        const int grp = f >> 7, fl = f & 127;      // group, thread within the group
+        const int cg = fl & 15, rg = fl >> 4;      // 16-byte column group, row group (8 of them)
         const uint32_t col_off = (uint32_t)(cg >> 3) * (GT_TILE_BYTES / 2);
-        // attention mass of token f of a tile as k_select left it: -1 marks a retained token (threads 0..127 fetch)
+        float *u_red_g = u_red + grp * 8 * 128;
+        const int bar_id = 1 + grp;
+        // attention mass of token fl of a tile as k_select left it: -1 marks a retained token
         auto fetch = [&](const TileInfo &ti) -> float {
-            if (ti.kind != 0 || f >= GT_TILE) return 0.f;
+            if (ti.kind != 0) return 0.f;
             const CacheDev &c = p.c[ti.cache];
-            const int j = ti.sub * GT_TILE + f;
+            const int j = ti.sub * GT_TILE + fl;
             if (j >= c.T) return 0.f;
             return __ldg(p.scores + c.tok_off + (size_t)ti.lh * c.T + j);
         };
         TileIter iter;
         iter.init(p, blockIdx.x);
-        TileInfo cur, nxt, nxt2;
+        // the group looks at every tile of the run (to see where segments start and end) but fixes up
+        // only tiles with index == grp (mod 2); the masses of its next tile are requested one step early
+        TileInfo cur, nxt;
         bool has_cur = iter.next(p, cur);
         bool has_nxt = has_cur && iter.next(p, nxt);
-        float a_cur = has_cur ? fetch(cur) : 0.f;
-        float a_nxt = has_nxt ? fetch(nxt) : 0.f;
-        float u[8];
         uint32_t it = 0;
+        float a_own = 0.f;                          // mass for the group's next own tile
+        if (has_cur && grp == 0) a_own = fetch(cur);
+        else if (has_nxt && grp == 1) a_own = fetch(nxt);
+        float u[8];
         while (has_cur) {
-            // the masses of the tile after next are requested now and used two tiles later
+            TileInfo nxt2;
             const bool has_nxt2 = has_nxt && iter.next(p, nxt2);
-            const int s = it % GT_STAGES;
-            if (f < GT_TILE) s_a[s * 128 + f] = a_cur;
-            a_cur = a_nxt;
-            a_nxt = has_nxt2 ? fetch(nxt2) : 0.f;
+            const bool own = (it & 1u) == (uint32_t)grp;
             if (cur.first) {
 #pragma unroll
                 for (int e = 0; e < 8; ++e) u[e] = 0.f;
             }
-            tc::mbar_wait(&bar_full[s], (it / GT_STAGES) & 1u, wc);
-            tc::named_barrier(1, GT_FIX_THREADS);      // s_a[s] is complete; nobody still reads the slot's previous use
-            if (cur.kind == 0) {
-                uint8_t *tile = tiles + s * GT_TILE_BYTES + col_off;
+            if (own) {
+                const int s = it % GT_STAGES;
+                s_a[s * 128 + fl] = a_own;
+                if (has_nxt2) a_own = fetch(nxt2);     // the group's next own tile; in flight while this one is processed
+                tc::mbar_wait(&bar_full[s], (it / GT_STAGES) & 1u, wc);
+                tc::named_barrier(bar_id, 128);        // s_a[s] is complete; nobody still reads the slot's previous use
+                if (cur.kind == 0) {
+                    uint8_t *tile = tiles + s * GT_TILE_BYTES + col_off;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int r = rg + 16 * i;
-                    const float a = s_a[s * 128 + r];
-                    const bool kept = a < 0.f;
-                    const float am = kept ? 0.f : a;
-                    uint4 *ptr = reinterpret_cast<uint4 *>(tile + r * 128 + (((cg & 7) ^ (r & 7)) << 4));
-                    const uint4 raw = *ptr;
-                    if (kept) *ptr = make_uint4(0u, 0u, 0u, 0u);
-                    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+                    for (int i = 0; i < 16; ++i) {
+                        const int r = rg + 8 * i;
+                        const float a = s_a[s * 128 + r];
+                        const bool kept = a < 0.f;
+                        const float am = kept ? 0.f : a;
+                        uint4 *ptr = reinterpret_cast<uint4 *>(tile + r * 128 + (((cg & 7) ^ (r & 7)) << 4));
+                        const uint4 raw = *ptr;
+                        if (kept) *ptr = make_uint4(0u, 0u, 0u, 0u);
+                        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        u[2 * e] = fmaf(am, __uint_as_float(w[e] << 16), u[2 * e]);
-                        u[2 * e + 1] = fmaf(am, __uint_as_float(w[e] & 0xFFFF0000u), u[2 * e + 1]);
+                        for (int e = 0; e < 4; ++e) {
+                            u[2 * e] = fmaf(am, __uint_as_float(w[e] << 16), u[2 * e]);
+                            u[2 * e + 1] = fmaf(am, __uint_as_float(w[e] & 0xFFFF0000u), u[2 * e + 1]);
+                        }
                     }
+                    tc::fence_async_smem();
                 }
-                tc::fence_async_smem();
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(&bar_ready[s]);
             }
-            __syncwarp();
-            if (lane == 0) tc::mbar_arrive(&bar_ready[s]);
             if (cur.kind == 0 && cur.last) {
-                // u over the 16 row groups, in a fixed order
+                // the group's u over its 8 row groups, in a fixed order
                 const int g = p.c[cur.cache].head_base + cur.lh;
-                tc::named_barrier(1, GT_FIX_THREADS);
+                tc::named_barrier(bar_id, 128);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) u_red[rg * 128 + cg * 8 + e] = u[e];
-                tc::named_barrier(1, GT_FIX_THREADS);
-                if (f < 128) {
-                    float sum = 0.f;
+                for (int e = 0; e < 8; ++e) u_red_g[rg * 128 + cg * 8 + e] = u[e];
+                tc::named_barrier(bar_id, 128);
+                float sum = 0.f;
 #pragma unroll
-                    for (int r = 0; r < 16; ++r) sum += u_red[r * 128 + f];
-                    p.uvec[((size_t)g * p.gram_slots + cur.slot) * D + f] = sum;
-                }
+                for (int r = 0; r < 8; ++r) sum += u_red_g[r * 128 + fl];
+                p.uvec[(((size_t)g * p.gram_slots + cur.slot) * 2 + grp) * D + fl] = sum;
             }
             cur = nxt;
             nxt = nxt2;
