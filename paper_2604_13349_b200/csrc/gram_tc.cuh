@@ -13,14 +13,14 @@
 // one (head, kind) inside a run is a segment and yields one partial Gram matrix
 // (and one partial u), stored in slot (b - first block touching that head and kind).
 //
-// Block = 14 warps:
+// Block = 18 warps:
 //   warp 0        TMA producer: 128 x 128 bf16 tiles (two 128-byte-swizzled column halves) into a 6-stage ring
 //   warp 1        issues tcgen05.mma: G (+)= tile^T tile, both operands MN-major views of the same tile,
 //                 accumulators (128 lanes x 128 columns fp32) double-buffered in tensor memory
-//   warps 2..9    fix-up, two groups of four warps taking tiles alternately: zero the retained rows of a
+//   warps 2..13   fix-up, three groups of four warps taking tiles in turn: zero the retained rows of a
 //                 V tile in shared memory and accumulate u on the CUDA cores; the attention mass of the
 //                 group's next tile (-1 marks a retained token) is fetched while the current one is processed
-//   warps 10..13  epilogue: tensor memory -> partial Gram matrix in the workspace
+//   warps 14..17  epilogue: tensor memory -> partial Gram matrix in the workspace
 #pragma once
 
 #include "tc_common.cuh"
@@ -30,10 +30,14 @@ namespace obf {
 constexpr int GT_STAGES = 6;
 constexpr int GT_TILE = 128;                       // tokens per tile
 constexpr int GT_TILE_BYTES = GT_TILE * 128 * 2;   // 32 KiB
-constexpr int GT_FIX_THREADS = 256;
+constexpr int GT_GROUPS = 3;                       // fix-up groups of four warps, taking tiles in turn
+// A ring stage must always be fixed up by the same group: a thread may wait for a barrier phase only if it
+// also waited for the phase before (waiting on a parity assumes the previous phase is over).
+static_assert(GT_STAGES % GT_GROUPS == 0, "every ring stage must belong to one fix-up group");
+constexpr int GT_FIX_THREADS = 128 * GT_GROUPS;
 constexpr int GT_THREADS = 64 + GT_FIX_THREADS + 128;
-constexpr size_t GT_SMEM_BYTES = 1024 + (size_t)GT_STAGES * GT_TILE_BYTES + 16 * 128 * sizeof(float) +
-                                 GT_STAGES * 128 * sizeof(float) + 256;
+constexpr size_t GT_SMEM_BYTES = 1024 + (size_t)GT_STAGES * GT_TILE_BYTES + GT_GROUPS * 8 * 128 * sizeof(float) +
+                                 GT_GROUPS * 2 * 128 * sizeof(float) + 256;
 
 // Walks the segments of one block's run of tiles.
 struct TileRun {
@@ -99,9 +103,9 @@ __global__ void __launch_bounds__(GT_THREADS, 1) k_gram_tc(const __grid_constant
     extern __shared__ uint8_t gt_smem_raw[];
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(gt_smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *tiles = base;                                                // GT_STAGES x 32 KiB, 1024-byte aligned
-    float *u_red = reinterpret_cast<float *>(tiles + GT_STAGES * GT_TILE_BYTES);   // [16][128]
-    // [GT_STAGES][128] per token of the tile: attention mass, -1 for a retained token, 0 beyond T
-    float *s_a = u_red + 16 * 128;
+    float *u_red = reinterpret_cast<float *>(tiles + GT_STAGES * GT_TILE_BYTES);   // [GT_GROUPS][8][128]
+    // [GT_GROUPS][2][128] per token of a group's current / next tile: attention mass, -1 for a retained token, 0 beyond T
+    float *s_a = u_red + GT_GROUPS * 8 * 128;
     __shared__ uint64_t bar_full[GT_STAGES], bar_ready[GT_STAGES], bar_empty[GT_STAGES];
     __shared__ uint64_t bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t s_tmem, s_abort;
@@ -113,7 +117,7 @@ __global__ void __launch_bounds__(GT_THREADS, 1) k_gram_tc(const __grid_constant
         s_abort = 0u;
         for (int s = 0; s < GT_STAGES; ++s) {
             tc::mbar_init(&bar_full[s], 1);
-            tc::mbar_init(&bar_ready[s], GT_FIX_THREADS / 64);
+            tc::mbar_init(&bar_ready[s], 4);
             tc::mbar_init(&bar_empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) { tc::mbar_init(&bar_acc_full[b], 1); tc::mbar_init(&bar_acc_empty[b], 4); }
@@ -183,9 +187,9 @@ __global__ void __launch_bounds__(GT_THREADS, 1) k_gram_tc(const __grid_constant
         }
     } else if (warp < 2 + GT_FIX_THREADS / 32) {
         // ---------------- fix-up: zero retained rows, accumulate u ----------------
-        // Two groups of four warps take the tiles of the run alternately, so that one group's
-        // tile can be fixed up while the other's is; each group keeps its own partial u.
-        const int f = tid - 64;                    // 0..255
+        // GT_GROUPS groups of four warps take the tiles of the run in turn, so that several tiles are
+        // fixed up at the same time; each group keeps its own partial u.
+        const int f = tid - 64;
         const int grp = f >> 7, fl = f & 127;      // group, thread within the group
         const int cg = fl & 15, rg = fl >> 4;      // 16-byte column group, row group (8 of them)
         const uint32_t col_off = (uint32_t)(cg >> 3) * (GT_TILE_BYTES / 2);
@@ -199,38 +203,41 @@ __global__ void __launch_bounds__(GT_THREADS, 1) k_gram_tc(const __grid_constant
             if (j >= c.T) return 0.f;
             return __ldg(p.scores + c.tok_off + (size_t)ti.lh * c.T + j);
         };
-        TileIter iter;
+        TileIter iter, ahead;
         iter.init(p, blockIdx.x);
+        ahead.init(p, blockIdx.x);
         // the group looks at every tile of the run (to see where segments start and end) but fixes up
-        // only tiles with index == grp (mod 2); the masses of its next tile are requested one step early
-        TileInfo cur, nxt;
+        // only tiles with index == grp (mod GT_GROUPS); the masses of its next tile are requested one tile early
+        TileInfo cur, pre;
         bool has_cur = iter.next(p, cur);
-        bool has_nxt = has_cur && iter.next(p, nxt);
-        uint32_t it = 0;
-        float a_own = 0.f;                          // mass for the group's next own tile
-        if (has_cur && grp == 0) a_own = fetch(cur);
-        else if (has_nxt && grp == 1) a_own = fetch(nxt);
+        // `ahead` stands on the group's next own tile
+        bool has_pre = true;
+        for (int sk = 0; sk <= grp && has_pre; ++sk) has_pre = ahead.next(p, pre);
+        float a_own = has_pre ? fetch(pre) : 0.f;   // mass for the group's next own tile
+        uint32_t it = 0, n_own = 0;
         float u[8];
+        float *s_ag = s_a + grp * 2 * 128;
         while (has_cur) {
-            TileInfo nxt2;
-            const bool has_nxt2 = has_nxt && iter.next(p, nxt2);
-            const bool own = (it & 1u) == (uint32_t)grp;
+            const bool own = (it % GT_GROUPS) == (uint32_t)grp;
             if (cur.first) {
 #pragma unroll
                 for (int e = 0; e < 8; ++e) u[e] = 0.f;
             }
             if (own) {
                 const int s = it % GT_STAGES;
-                s_a[s * 128 + fl] = a_own;
-                if (has_nxt2) a_own = fetch(nxt2);     // the group's next own tile; in flight while this one is processed
+                float *sa = s_ag + (n_own & 1u) * 128;
+                sa[fl] = a_own;
+                // the group's next own tile: its masses are in flight while this tile is processed
+                for (int sk = 0; sk < GT_GROUPS && has_pre; ++sk) has_pre = ahead.next(p, pre);
+                if (has_pre) a_own = fetch(pre);
                 tc::mbar_wait(&bar_full[s], (it / GT_STAGES) & 1u, wc);
-                tc::named_barrier(bar_id, 128);        // s_a[s] is complete; nobody still reads the slot's previous use
+                tc::named_barrier(bar_id, 128);        // sa is complete
                 if (cur.kind == 0) {
                     uint8_t *tile = tiles + s * GT_TILE_BYTES + col_off;
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
                         const int r = rg + 8 * i;
-                        const float a = s_a[s * 128 + r];
+                        const float a = sa[r];
                         const bool kept = a < 0.f;
                         const float am = kept ? 0.f : a;
                         uint4 *ptr = reinterpret_cast<uint4 *>(tile + r * 128 + (((cg & 7) ^ (r & 7)) << 4));
@@ -247,6 +254,7 @@ __global__ void __launch_bounds__(GT_THREADS, 1) k_gram_tc(const __grid_constant
                 }
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(&bar_ready[s]);
+                ++n_own;
             }
             if (cur.kind == 0 && cur.last) {
                 // the group's u over its 8 row groups, in a fixed order
@@ -258,12 +266,9 @@ __global__ void __launch_bounds__(GT_THREADS, 1) k_gram_tc(const __grid_constant
                 float sum = 0.f;
 #pragma unroll
                 for (int r = 0; r < 8; ++r) sum += u_red_g[r * 128 + fl];
-                p.uvec[(((size_t)g * p.gram_slots + cur.slot) * 2 + grp) * D + fl] = sum;
+                p.uvec[(((size_t)g * p.gram_slots + cur.slot) * GT_GROUPS + grp) * D + fl] = sum;
             }
-            cur = nxt;
-            nxt = nxt2;
-            has_cur = has_nxt;
-            has_nxt = has_nxt2;
+            has_cur = iter.next(p, cur);
             ++it;
         }
     } else {

@@ -203,7 +203,7 @@ static void make_layout(const obf_params_t *p, const obf_cache_t *caches, int32_
         const size_t gsz = (size_t)L.heads_total * L.gram_slots * d * d * sizeof(float);
         L.off_gram_d = o; o = align_up(o + gsz, 256);
         L.off_gram_k = o; o = align_up(o + gsz, 256);
-        L.off_uvec = o;   o = align_up(o + (size_t)L.heads_total * L.gram_slots * 2 * d * sizeof(float), 256);
+        L.off_uvec = o;   o = align_up(o + (size_t)L.heads_total * L.gram_slots * GT_GROUPS * d * sizeof(float), 256);
         L.off_delta = o;  o = align_up(o + (size_t)L.heads_total * d * sizeof(float), 256);
         L.off_hflag = o;  o = align_up(o + (size_t)L.heads_total * sizeof(uint32_t), 256);
     }
@@ -413,7 +413,7 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
     cd.splits = L.splits;
     cd.gram_slots = L.gram_slots;
     cd.tc_per = L.tc_per;
-    cd.u_groups = L.tc_per ? 2 : 1;
+    cd.u_groups = L.tc_per ? GT_GROUPS : 1;
     cd.tc_total_sub = L.tc_total_sub;
     cd.sc_nq = L.sc_on ? L.sc_nq : 0;
     cd.sc_subs = L.sc_subs;
