@@ -8,7 +8,8 @@
 // pivot stays above CHOL_PIVOT_TOL of the channel's own squared norm.  One block
 // per (cache, layer, KV head); right-looking blocked algorithm with 32-wide
 // panels: the diagonal block is factorised by one warp in registers, the panel
-// below it by one thread per row, the trailing matrix by 4x4 register tiles.
+// below it by one thread per row, the lower triangle of the trailing matrix by
+// 8x4 register tiles.
 // Result: bit 1 of hflag[head].
 #pragma once
 
@@ -22,7 +23,7 @@ constexpr uint32_t HFLAG_INJECT = 1u;      // delta != 0: the injection kernel h
 constexpr uint32_t HFLAG_SPAN_FULL = 2u;   // span(V_keep) = R^d
 
 template <int D>
-constexpr size_t span_smem_bytes() { return (size_t)(D * (D + 1) + 32 * 32 + 32 + D) * sizeof(float); }
+constexpr size_t span_smem_bytes() { return (size_t)(D * (D + 1) + 32 * 32 + 32 + D + 32) * sizeof(float); }
 
 template <int D>
 __global__ void __launch_bounds__(ST_NT) k_span_test(const __grid_constant__ CallDev p)
@@ -33,6 +34,7 @@ __global__ void __launch_bounds__(ST_NT) k_span_test(const __grid_constant__ Cal
     float *L11 = A + D * LD;           // 32 x 32 factor of the current diagonal block (16-byte aligned)
     float *rinv = L11 + NB * NB;       // 32 reciprocals of its diagonal
     float *d0 = rinv + NB;             // D original diagonal entries
+    float *colbuf = d0 + D;            // 32 entries: the current column of the diagonal block's factor
     __shared__ int s_ok;
 
     const int g = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -46,15 +48,30 @@ __global__ void __launch_bounds__(ST_NT) k_span_test(const __grid_constant__ Cal
     }
     const int n_part = gram_partial_count(p, c, lh, 1);
     const float *parts = p.gram_k + (size_t)g * p.gram_slots * D * D;
-    for (int e4 = tid; e4 < D * D / 4; e4 += ST_NT) {
-        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int e0 = tid; e0 < D * D / 4; e0 += 4 * ST_NT) {
+        float4 acc[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int sp = 0; sp < n_part; ++sp) {
-            const float4 v = *reinterpret_cast<const float4 *>(parts + (size_t)sp * D * D + e4 * 4);
-            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+            float4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int e4 = e0 + u * ST_NT;
+                v[u] = e4 < D * D / 4 ? *reinterpret_cast<const float4 *>(parts + (size_t)sp * D * D + e4 * 4)
+                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { acc[u].x += v[u].x; acc[u].y += v[u].y; acc[u].z += v[u].z; acc[u].w += v[u].w; }
         }
-        const int r = (e4 * 4) / D, cc = (e4 * 4) % D;
-        float *o = A + r * LD + cc;
-        o[0] = s.x; o[1] = s.y; o[2] = s.z; o[3] = s.w;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int e4 = e0 + u * ST_NT;
+            if (e4 < D * D / 4) {
+                const int r = (e4 * 4) / D, cc = (e4 * 4) % D;
+                float *o = A + r * LD + cc;
+                o[0] = acc[u].x; o[1] = acc[u].y; o[2] = acc[u].z; o[3] = acc[u].w;
+            }
+        }
     }
     if (tid == 0) s_ok = 1;
     __syncthreads();
@@ -74,14 +91,20 @@ __global__ void __launch_bounds__(ST_NT) k_span_test(const __grid_constant__ Cal
             for (int j = 0; j < NB; ++j) {
                 const float piv = __shfl_sync(0xffffffffu, a[j], j);
                 ok = ok && (piv > CHOL_PIVOT_TOL * d0[j0 + j]) && (piv > 0.f);
-                const float inv = rsqrtf(piv);
-                const float l = a[j] * inv;                  // lanes >= j: L[lane][j]
+                const float l = a[j] * __frsqrt_rn(piv);     // lanes >= j: L[lane][j]
                 a[j] = l;
+                // column j of L goes through shared memory: every lane then reads the entries it needs as vectors
+                colbuf[lane] = l;
+                __syncwarp();
 #pragma unroll
-                for (int cc = j + 1; cc < NB; ++cc) {
-                    const float lc = __shfl_sync(0xffffffffu, l, cc);   // L[cc][j]
-                    a[cc] = fmaf(-l, lc, a[cc]);
+                for (int c4 = (j + 1) / 4; c4 < NB / 4; ++c4) {
+                    const float4 lc = *reinterpret_cast<const float4 *>(&colbuf[4 * c4]);
+                    if (4 * c4 + 0 > j) a[4 * c4 + 0] = fmaf(-l, lc.x, a[4 * c4 + 0]);
+                    if (4 * c4 + 1 > j) a[4 * c4 + 1] = fmaf(-l, lc.y, a[4 * c4 + 1]);
+                    if (4 * c4 + 2 > j) a[4 * c4 + 2] = fmaf(-l, lc.z, a[4 * c4 + 2]);
+                    if (4 * c4 + 3 > j) a[4 * c4 + 3] = fmaf(-l, lc.w, a[4 * c4 + 3]);
                 }
+                __syncwarp();
             }
 #pragma unroll
             for (int cc = 0; cc < NB; ++cc) L11[lane * NB + cc] = cc <= lane ? a[cc] : 0.f;
@@ -93,47 +116,58 @@ __global__ void __launch_bounds__(ST_NT) k_span_test(const __grid_constant__ Cal
         __syncthreads();
         if (!s_ok) break;
         if (nrem > 0) {
-            // panel: L21 = A21 L11^-T, one thread per row
+            // panel: L21 = A21 L11^-T, one thread per row; once x_c is known every later entry of the
+            // row is updated independently, so the dependency chain is 32 steps long, not 496
             if (tid < nrem) {
                 float *row = A + (j0 + NB + tid) * LD + j0;
                 float x[NB];
 #pragma unroll
-                for (int cc = 0; cc < NB; ++cc) {
-                    float s = row[cc];
+                for (int cc = 0; cc < NB; ++cc) x[cc] = row[cc];
 #pragma unroll
-                    for (int k = 0; k < cc; ++k) s = fmaf(-x[k], L11[cc * NB + k], s);
-                    x[cc] = s * rinv[cc];
+                for (int cc = 0; cc < NB; ++cc) {
+                    x[cc] *= rinv[cc];
+#pragma unroll
+                    for (int c2 = cc + 1; c2 < NB; ++c2) x[c2] = fmaf(-x[cc], L11[c2 * NB + cc], x[c2]);
                 }
 #pragma unroll
                 for (int cc = 0; cc < NB; ++cc) row[cc] = x[cc];
             }
             __syncthreads();
-            // trailing matrix -= L21 L21^T, 4x4 tiles on interleaved rows (bank-conflict free)
-            const int nt = nrem / 4;
-            for (int t = tid; t < nt * nt; t += ST_NT) {
-                const int ti = t / nt, tj = t - ti * nt;
-                float acc[4][4];
+            // trailing matrix -= L21 L21^T.  Only the lower triangle is ever read again: the trailing matrix is
+            // cut into 32 x 32 blocks and a thread updates an 8 x 4 register tile of a block on or below the
+            // diagonal (rows r0 + 4a.., columns c0 + 8b.. interleaved inside the block, bank-conflict free).
+            const int nb = nrem / NB;                      // blocks per side
+            const int n_blk = nb * (nb + 1) / 2;           // blocks on or below the diagonal
+            for (int t = tid; t < n_blk * 32; t += ST_NT) {
+                const int blk = t >> 5, sub = t & 31;      // 32 threads per block: 4 row groups x 8 column groups
+                int bi = 0, rem = blk;
+                while (rem > bi) { rem -= bi + 1; ++bi; }  // block row bi, block column rem (rem <= bi)
+                const int bj = rem;
+                const int ri = sub >> 3, cj = sub & 7;     // rows ri + 4a (a < 8), columns cj + 8b (b < 4)
+                float acc[8][4];
 #pragma unroll
-                for (int a_ = 0; a_ < 4; ++a_)
+                for (int a_ = 0; a_ < 8; ++a_)
 #pragma unroll
                     for (int b_ = 0; b_ < 4; ++b_) acc[a_][b_] = 0.f;
-                const float *Li = A + (j0 + NB + ti) * LD + j0;
-                const float *Lj = A + (j0 + NB + tj) * LD + j0;
-#pragma unroll 8
+                const float *Li = A + (j0 + NB + bi * NB + ri) * LD + j0;
+                const float *Lj = A + (j0 + NB + bj * NB + cj) * LD + j0;
+#pragma unroll 4
                 for (int k = 0; k < NB; ++k) {
-                    float li[4], lj[4];
+                    float li[8], lj[4];
 #pragma unroll
-                    for (int a_ = 0; a_ < 4; ++a_) { li[a_] = Li[a_ * nt * LD + k]; lj[a_] = Lj[a_ * nt * LD + k]; }
+                    for (int a_ = 0; a_ < 8; ++a_) li[a_] = Li[a_ * 4 * LD + k];
 #pragma unroll
-                    for (int a_ = 0; a_ < 4; ++a_)
+                    for (int b_ = 0; b_ < 4; ++b_) lj[b_] = Lj[b_ * 8 * LD + k];
+#pragma unroll
+                    for (int a_ = 0; a_ < 8; ++a_)
 #pragma unroll
                         for (int b_ = 0; b_ < 4; ++b_) acc[a_][b_] = fmaf(li[a_], lj[b_], acc[a_][b_]);
                 }
 #pragma unroll
-                for (int a_ = 0; a_ < 4; ++a_)
+                for (int a_ = 0; a_ < 8; ++a_)
 #pragma unroll
                     for (int b_ = 0; b_ < 4; ++b_)
-                        A[(j0 + NB + ti + a_ * nt) * LD + j0 + NB + tj + b_ * nt] -= acc[a_][b_];
+                        A[(j0 + NB + bi * NB + ri + 4 * a_) * LD + j0 + NB + bj * NB + cj + 8 * b_] -= acc[a_][b_];
             }
             __syncthreads();
         }
