@@ -157,7 +157,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="c4")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -251,17 +251,35 @@ def main():
     kv_bytes = sum(hpc * c.T * d * e for c in w.caches)
     q_bytes = len(w.caches) * hpc * w.n_q * d * e
     out_bytes = sum(hpc * min(c.budget, c.T) * (2 * d * e + 4) for c in w.caches)
-    kernel_bytes = {"k_score_stats": kv_bytes + q_bytes, "k_score_pool": kv_bytes + q_bytes,
-                    "k_gram": kv_bytes, "k_gram_tc": kv_bytes, "k_score_tc": kv_bytes + q_bytes, "k_span_test": 0,
-                    "k_gather": 2 * out_bytes, "k_inject": out_bytes,
-                    "k_select": sum(hpc * c.T * 4 for c in w.caches),
-                    "k_obf_algebra": 0, "k_fused": step_bytes}.get(dom, step_bytes)
+    score_bytes = sum(hpc * c.T * 4 for c in w.caches)                 # the mass array A (fp32)
+    kernel_bytes = {"k_score_stats": kv_bytes + q_bytes, "k_score_pool": kv_bytes + q_bytes + score_bytes,
+                    "k_score_tc": kv_bytes + q_bytes + score_bytes,     # K and Q read once, A written
+                    "k_gram": kv_bytes, "k_gram_tc": kv_bytes,          # V read once
+                    "k_gather": 2 * out_bytes, "k_select": score_bytes,
+                    "k_span_test": 0, "k_obf_algebra": 0}.get(dom, step_bytes)
     achieved = kernel_bytes / (phase_acc[dom] * 1e-3) / 1e9
+    traffic = None
+    # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu summaries ("kernel workload bytes")
+    tpath = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    if os.path.exists(tpath):
+        with open(tpath) as f:
+            for ln in f:
+                parts = ln.split("#")[0].split()
+                if len(parts) == 3 and parts[0] == dom and parts[1] == w.name:
+                    traffic = int(parts[2])
+    # the attention-mass kernel evaluates 2 exponentials per (query, key): its own ceiling is the
+    # special-function unit (16 results per clock and SM), not HBM
+    n_exp = 2.0 * sum(hpc * c.T * w.n_q for c in w.caches)
+    sm_clock = (clocks or {}).get("sm_mhz") or 1965.0
+    sfu_peak = 16 * 148 * sm_clock * 1e6 / 1e9
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_kind": peak_kind, "traffic": None,
+                "frac": achieved / peak, "peak_kind": peak_kind, "traffic": traffic,
                 "kernel_ms": phase_acc[dom], "algorithmic_bytes_per_launch": kernel_bytes,
                 "whole_step_frac": (step_bytes / (ms_per_step * 1e-3) / 1e9) / peak,
                 "phases_ms": {k: round(v, 4) for k, v in phase_acc.items()}}
+    if dom == "k_score_tc":
+        roofline["sfu"] = {"unit": "Gexp/s", "achieved": n_exp / (phase_acc[dom] * 1e-3) / 1e9, "peak": sfu_peak,
+                           "frac": n_exp / (phase_acc[dom] * 1e-3) / 1e9 / sfu_peak}
 
     # end to end through the host entry point: pinned host buffers, copies inside the timed region
     e2e = None

@@ -195,6 +195,23 @@ def test_tuned_path_rank_deficient_values_with_budget_above_head_dim():
     assert torch.all(outs[0]["delta"].norm(dim=-1) > 1e-6)
 
 
+@pytest.mark.parametrize("T,budget", [(20000, 300), (80000, 200)])
+def test_long_prompts_take_the_fallback_kernels(T, budget):
+    # 20000 keys: more than the select kernel keeps in shared memory; 80000 keys: more chunks than the
+    # persistent score kernel has blocks, so the shape-generic score kernels run (the Gram pass stays tuned)
+    w = small("long", layers=1, kv_heads=1, G=4, n_obs=8, d=128, dtype="bf16", rank=1, caches=((T, budget),),
+              n_outlier=3, n_sink=4, heavy=8, seed=T % 97)
+    outs, reps, _ = run_and_check(w)
+    assert all(r.oracle_skipped for r in reps)              # budget >= head_dim with generic values: delta = 0
+
+
+def test_more_than_128_query_rows_use_the_generic_score_kernels_and_the_tuned_gram_pass():
+    w = small("wideq", layers=2, kv_heads=2, G=5, n_obs=32, d=128, dtype="bf16", rank=2, caches=((640, 24),),
+              n_outlier=3, seed=77)
+    outs, reps, _ = run_and_check(w)
+    assert all(not r.oracle_skipped for r in reps)
+
+
 def test_exact_ties_go_to_the_lowest_position():
     # duplicated keys give bit-identical masses on the GPU as well; ties must resolve to lower positions
     w = small("ties", d=64, dtype="f32", rank=0, caches=((96, 20),), heavy=0, kv_heads=1)
