@@ -167,7 +167,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                     const int qb = r % ST_QBUF;
                     if (pass == 0) {
                         // the buffer is free once the pooling MMAs of its previous user are done
-                        if (nq[qb] > 0 && !tc::mbar_wait(&bar_q_free[qb], (nq[qb] - 1) & 1u, wc, 32)) { dead = true; break; }
+                        if (nq[qb] > 0 && !tc::mbar_wait(&bar_q_free[qb], (nq[qb] - 1) & 1u, wc, 128)) { dead = true; break; }
                         const uint32_t qdst = tc::smem_u32(q_s + qb * ST_TILE_BYTES);
                         tc::mbar_expect_tx(&bar_q_full[qb], ST_TILE_BYTES);
                         tc::tma_load_3d(qdst, &tm.b[item.cache], &bar_q_full[qb], 0, 0, item.lh);
@@ -184,7 +184,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                     }
                     for (int t = 0; t < item.nt; ++t, ++it) {
                         const int s = it % ST_STAGES;
-                        if (!tc::mbar_wait(&bar_empty[s], ((it / ST_STAGES) & 1u) ^ 1u, wc, 32)) { dead = true; break; }
+                        if (!tc::mbar_wait(&bar_empty[s], ((it / ST_STAGES) & 1u) ^ 1u, wc, 128)) { dead = true; break; }
                         tc::mbar_expect_tx(&bar_full[s], ST_TILE_BYTES);
                         const uint32_t dst = tc::smem_u32(ring + s * ST_TILE_BYTES);
                         const int row0 = item.chunk * ST_CHUNK + t * 128;
@@ -195,9 +195,9 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
             }
             // nothing this thread started may still be in flight when the block exits
             for (uint32_t j = it > (uint32_t)ST_STAGES ? it - ST_STAGES : 0u; j < it; ++j)
-                tc::mbar_wait(&bar_full[j % ST_STAGES], (j / ST_STAGES) & 1u, wc, 32);
+                tc::mbar_wait(&bar_full[j % ST_STAGES], (j / ST_STAGES) & 1u, wc, 128);
             for (int b = 0; b < ST_QBUF; ++b)
-                if (nq[b] > 0) tc::mbar_wait(&bar_q_full[b], (nq[b] - 1) & 1u, wc, 32);
+                if (nq[b] > 0) tc::mbar_wait(&bar_q_full[b], (nq[b] - 1) & 1u, wc, 128);
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
@@ -262,7 +262,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                     // columns [32 * part, +32) of every tile of the chunk; the tile is released as soon as they are in registers
                     const uint32_t ti = it + t;
                     const int tb = ti % ST_TBUF;
-                    tc::mbar_wait(&bar_t_full[tb], (ti / ST_TBUF) & 1u, wc);
+                    tc::mbar_wait(&bar_t_full[tb], (ti / ST_TBUF) & 1u, wc, 20);
                     tc::tc_fence_after();
                     uint32_t rr[32];
                     tc::tmem_ld32(tlane + (uint32_t)(tb * 128 + part * 32), rr);
@@ -301,7 +301,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                 }
                 it += item.nt;
                 // hand (m, z) of this column part to the messenger
-                if (n_a[buf] > 0) tc::mbar_wait(&bar_st_free[buf], (n_a[buf] - 1) & 1u, wc);
+                if (n_a[buf] > 0) tc::mbar_wait(&bar_st_free[buf], (n_a[buf] - 1) & 1u, wc, 20);
                 s_m[(buf * 4 + part) * 128 + row] = m;
                 s_z[(buf * 4 + part) * 128 + row] = z;
                 __syncwarp();
@@ -312,7 +312,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
             if (i >= 1 && score_item(p, i - 1, (int)blockIdx.x, item)) {
                 const CacheDev &c = p.c[item.cache];
                 const int T = c.T, buf = (i - 1) & 1;
-                tc::mbar_wait(&bar_mp_ready[buf], n_b[buf] & 1u, wc);
+                tc::mbar_wait(&bar_mp_ready[buf], n_b[buf] & 1u, wc, 20);
                 float mp[32];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
@@ -324,7 +324,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                     // queries [32 * part, +32) of every tile of the chunk; the tile is released as soon as they are in registers
                     const uint32_t ti = it + t;
                     const int tb = ti % ST_TBUF;
-                    tc::mbar_wait(&bar_t_full[tb], (ti / ST_TBUF) & 1u, wc);
+                    tc::mbar_wait(&bar_t_full[tb], (ti / ST_TBUF) & 1u, wc, 20);
                     tc::tc_fence_after();
                     uint32_t rr[32];
                     tc::tmem_ld32(tlane + (uint32_t)(tb * 128 + part * 32), rr);
@@ -342,12 +342,12 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                     }
                     // the four parts meet in shared memory; part (t mod 4) adds them up and writes the masses
                     const uint32_t bit = 1u << tb;
-                    if (acc_used & bit) tc::mbar_wait(&bar_acc_free[tb], ((acc_par >> tb) & 1u) ^ 1u, wc);
+                    if (acc_used & bit) tc::mbar_wait(&bar_acc_free[tb], ((acc_par >> tb) & 1u) ^ 1u, wc, 20);
                     s_acc[(tb * 4 + part) * 128 + row] = (a0 + a1) + (a2 + a3);
                     __syncwarp();
                     if (lane == 0) tc::mbar_arrive(&bar_acc_ready[tb]);
                     if (part == (t & 3)) {
-                        tc::mbar_wait(&bar_acc_ready[tb], (acc_par >> tb) & 1u, wc);
+                        tc::mbar_wait(&bar_acc_ready[tb], (acc_par >> tb) & 1u, wc, 20);
                         const float *sa = s_acc + tb * 4 * 128 + row;
                         const float a = (sa[0] + sa[128]) + (sa[256] + sa[384]);
                         __syncwarp();

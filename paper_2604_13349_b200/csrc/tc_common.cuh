@@ -46,11 +46,13 @@ __device__ __forceinline__ void mbar_arrive(uint64_t *bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-__device__ __forceinline__ bool mbar_try(uint64_t *bar, uint32_t parity)
+// One test of the phase with the given parity.  The hardware may park the thread until the phase
+// completes or `suspend_ns` have passed, which keeps a waiting warp out of the issue slots.
+__device__ __forceinline__ bool mbar_try(uint64_t *bar, uint32_t parity, uint32_t suspend_ns = 20000u)
 {
     uint32_t ok;
-    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(suspend_ns) : "memory");
     return ok != 0;
 }
 

@@ -45,7 +45,7 @@ def run_and_check(w, rank=None, evict=False, heads=None, arrays=None, flags=0):
 
 
 # ---------------------------------------------------------------------------
-# BASELINE configurations that the oracle finishes whole
+# benchmark configurations that the oracle finishes whole
 # ---------------------------------------------------------------------------
 def test_c1_tiny_fp32_whole():
     outs, reps, _ = run_and_check(synth.workload("c1"))
@@ -271,7 +271,7 @@ def test_host_entry_point_matches_the_device_entry_point():
 
 
 # ---------------------------------------------------------------------------
-# BASELINE configurations at full size, in the benchmark's launch configuration,
+# benchmark configurations at full size, in the benchmark's launch configuration,
 # checked on sampled heads that the oracle computes one by one
 # ---------------------------------------------------------------------------
 @pytest.fixture(scope="module")

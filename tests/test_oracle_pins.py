@@ -370,7 +370,7 @@ def test_rank_deficient_values_with_budget_above_head_dim_still_inject():
 
 
 # --------------------------------------------------------------------------
-# the tiny BASELINE configuration end to end, whole-cache entry point
+# the tiny benchmark configuration end to end, whole-cache entry point
 # --------------------------------------------------------------------------
 def test_c1_whole_cache_matches_lapack_pipeline_per_head():
     w = synth.workload("c1")
