@@ -274,11 +274,13 @@ __global__ void __launch_bounds__(SEL_NT) k_select(const __grid_constant__ CallD
 // block-wide barriers suffice.
 constexpr int SEL_SMEM_MAX_T = 16384;
 
-__global__ void __launch_bounds__(SEL_NT) k_select_smem(const __grid_constant__ CallDev p)
+template <int NT>
+__global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ CallDev p)
 {
     extern __shared__ uint32_t sel_keys[];
     __shared__ uint32_t hist[256];
     __shared__ uint32_t s_prefix, s_want;
+    constexpr int NW = NT / 32;
     __shared__ uint32_t wtot[32];
     __shared__ float red[32];
     int ci, lh;
@@ -291,15 +293,15 @@ __global__ void __launch_bounds__(SEL_NT) k_select_smem(const __grid_constant__ 
     int32_t *idx = c.idx_out + (size_t)lh * k;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    for (int j = tid; j < T; j += SEL_NT) sel_keys[j] = score_key_bits(A[j]);
+    for (int j = tid; j < T; j += NT) sel_keys[j] = score_key_bits(A[j]);
     if (tid == 0) { s_prefix = 0u; s_want = (uint32_t)k; }
     uint32_t mask = 0u;
-    const int T_pad = (T + SEL_NT - 1) / SEL_NT * SEL_NT;
+    const int T_pad = (T + NT - 1) / NT * NT;
     for (int shift = 24; shift >= 0; shift -= 8) {
         if (tid < 256) hist[tid] = 0u;
         __syncthreads();
         const uint32_t prefix = s_prefix;
-        for (int j = tid; j < T_pad; j += SEL_NT) {
+        for (int j = tid; j < T_pad; j += NT) {
             const uint32_t u = j < T ? sel_keys[j] : 0u;
             const bool cand = j < T && (u & mask) == prefix;
             const uint32_t digit = (u >> shift) & 255u;
@@ -344,7 +346,7 @@ __global__ void __launch_bounds__(SEL_NT) k_select_smem(const __grid_constant__ 
     const uint32_t want = s_want;        // how many positions with key == tau are retained (>= 1)
 
     // ordered pass: warp w owns positions [w * seg, (w + 1) * seg)
-    const int seg = ((T + 31) / 32 + 31) / 32 * 32;
+    const int seg = ((T + NW - 1) / NW + 31) / 32 * 32;
     const int j_begin = warp * seg, j_end = min(T, j_begin + seg);
     uint32_t n_gt = 0u, n_eq = 0u;
     for (int j0 = j_begin; j0 < j_end; j0 += 32) {
@@ -356,7 +358,7 @@ __global__ void __launch_bounds__(SEL_NT) k_select_smem(const __grid_constant__ 
     if (lane == 0) wtot[warp] = n_gt | (n_eq << 16);
     __syncthreads();
     if (warp == 0) {
-        const uint32_t w = wtot[lane];
+        const uint32_t w = lane < NW ? wtot[lane] : 0u;
         uint32_t inc = w;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -391,9 +393,9 @@ __global__ void __launch_bounds__(SEL_NT) k_select_smem(const __grid_constant__ 
         run_gt += __popc(m_gt);
         run_eq += __popc(m_eq);
     }
-    const float a_keep = block_sum<SEL_NT>(sk, red);
-    const float a_del = block_sum<SEL_NT>(sd, red);
-    const float next = block_max<SEL_NT>(nx, red);
+    const float a_keep = block_sum<NT>(sk, red);
+    const float a_del = block_sum<NT>(sd, red);
+    const float next = block_max<NT>(nx, red);
     if (tid == 0) {
         float *sm = p.sums + (size_t)blockIdx.x * 4;
         sm[0] = a_keep; sm[1] = a_del; sm[2] = key_score(tau); sm[3] = next;

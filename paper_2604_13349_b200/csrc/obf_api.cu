@@ -324,8 +324,16 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
     }
     if (T_max <= SEL_SMEM_MAX_T) {
         const size_t sm_sel = (size_t)T_max * sizeof(uint32_t);
-        if ((s = set_smem(k_select_smem, sm_sel)) != OBF_OK) return s;
-        k_select_smem<<<heads, SEL_NT, sm_sel, st>>>(cd);
+        // blocks of 1024 threads fit twice on an SM; when the heads then need a second, nearly empty wave,
+        // blocks of 512 threads (four per SM) finish sooner
+        const int sms = sm_count();
+        if (heads > 2 * sms && heads <= 4 * sms) {
+            if ((s = set_smem(k_select_smem<512>, sm_sel)) != OBF_OK) return s;
+            k_select_smem<512><<<heads, 512, sm_sel, st>>>(cd);
+        } else {
+            if ((s = set_smem(k_select_smem<1024>, sm_sel)) != OBF_OK) return s;
+            k_select_smem<1024><<<heads, 1024, sm_sel, st>>>(cd);
+        }
     } else {
         k_select<<<heads, SEL_NT, 0, st>>>(cd);
     }

@@ -108,6 +108,40 @@ __device__ __forceinline__ unsigned long long ld_relaxed_gpu_u64(const unsigned 
     return v;
 }
 
+// Pass A on one thread's 32 logits of a tile: running maximum m (log2 domain) and sum z of
+// exp2(s c - m) of one query.  With MASKED only the first n_valid columns are keys.
+template <bool MASKED>
+__device__ __forceinline__ void stats_update(uint32_t (&rr)[32], int n_valid, float sc, float &m, float &z)
+{
+    if (MASKED) {
+#pragma unroll
+        for (int e = 0; e < 32; ++e)
+            if (e >= n_valid) rr[e] = 0xff800000u;                                     // -inf: no such key
+    }
+    float t0 = __uint_as_float(rr[0]), t1 = __uint_as_float(rr[1]);
+    float t2 = __uint_as_float(rr[2]), t3 = __uint_as_float(rr[3]);
+#pragma unroll
+    for (int e = 4; e < 32; e += 4) {
+        t0 = fmaxf(t0, __uint_as_float(rr[e]));
+        t1 = fmaxf(t1, __uint_as_float(rr[e + 1]));
+        t2 = fmaxf(t2, __uint_as_float(rr[e + 2]));
+        t3 = fmaxf(t3, __uint_as_float(rr[e + 3]));
+    }
+    const float mn = fmaxf(m, fmaxf(fmaxf(t0, t1), fmaxf(t2, t3)) * sc);
+    if (mn > -INFINITY) {
+        float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
+#pragma unroll
+        for (int e = 0; e < 32; e += 4) {
+            z0 += ex2_approx(fmaf(__uint_as_float(rr[e]), sc, -mn));
+            z1 += ex2_approx(fmaf(__uint_as_float(rr[e + 1]), sc, -mn));
+            z2 += ex2_approx(fmaf(__uint_as_float(rr[e + 2]), sc, -mn));
+            z3 += ex2_approx(fmaf(__uint_as_float(rr[e + 3]), sc, -mn));
+        }
+        z = z * ex2_approx(m - mn) + ((z0 + z1) + (z2 + z3));
+        m = mn;
+    }
+}
+
 __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constant__ CallDev p, const __grid_constant__ TcMaps tm)
 {
     extern __shared__ uint8_t st_smem_raw[];
@@ -271,33 +305,9 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                     __syncwarp();
                     if (lane == 0) tc::mbar_arrive(&bar_t_empty[tb]);
                     const int key0 = item.chunk * ST_CHUNK + t * 128 + part * 32;         // key of column 0 of this block
-                    if (key0 + 32 > T) {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e)
-                            if (key0 + e >= T) rr[e] = 0xff800000u;                        // -inf: no such key
-                    }
-                    float t0_ = __uint_as_float(rr[0]), t1_ = __uint_as_float(rr[1]);
-                    float t2_ = __uint_as_float(rr[2]), t3_ = __uint_as_float(rr[3]);
-#pragma unroll
-                    for (int e = 4; e < 32; e += 4) {
-                        t0_ = fmaxf(t0_, __uint_as_float(rr[e]));
-                        t1_ = fmaxf(t1_, __uint_as_float(rr[e + 1]));
-                        t2_ = fmaxf(t2_, __uint_as_float(rr[e + 2]));
-                        t3_ = fmaxf(t3_, __uint_as_float(rr[e + 3]));
-                    }
-                    const float mn = fmaxf(m, fmaxf(fmaxf(t0_, t1_), fmaxf(t2_, t3_)) * sc);
-                    if (mn > -INFINITY) {
-                        float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
-#pragma unroll
-                        for (int e = 0; e < 32; e += 4) {
-                            z0 += ex2_approx(fmaf(__uint_as_float(rr[e]), sc, -mn));
-                            z1 += ex2_approx(fmaf(__uint_as_float(rr[e + 1]), sc, -mn));
-                            z2 += ex2_approx(fmaf(__uint_as_float(rr[e + 2]), sc, -mn));
-                            z3 += ex2_approx(fmaf(__uint_as_float(rr[e + 3]), sc, -mn));
-                        }
-                        z = z * ex2_approx(m - mn) + ((z0 + z1) + (z2 + z3));
-                        m = mn;
-                    }
+                    // two copies of the update: the one that masks missing keys runs for a head's ragged last tile only
+                    if (key0 + 32 > T) stats_update<true>(rr, T - key0, sc, m, z);
+                    else stats_update<false>(rr, 32, sc, m, z);
                 }
                 it += item.nt;
                 // hand (m, z) of this column part to the messenger
