@@ -238,6 +238,9 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
         if (lane == 0) {
             constexpr uint32_t IDESC = tc::idesc_bf16(128, 128, 0, 0);
             uint32_t it = 0, nq[ST_QBUF] = {0u, 0u, 0u};
+            // ring stage and accumulator tile of the next tile, with the parity of their current use
+            uint32_t st = 0, st_par = 0, tb = 0, tb_par = 0;
+            const uint32_t ring_addr = tc::smem_u32(ring);
             bool dead = false;
             for (int i = 0; i <= R && !dead; ++i) {
                 for (int pass = 0; pass < 2 && !dead; ++pass) {
@@ -247,29 +250,30 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                     if (!score_item(p, r, (int)blockIdx.x, item)) continue;
                     const int qb = r % ST_QBUF;
                     if (pass == 0) {
-                        if (!tc::mbar_wait(&bar_q_full[qb], nq[qb] & 1u, wc, 32)) { dead = true; break; }
+                        if (!tc::mbar_wait(&bar_q_full[qb], nq[qb] & 1u, wc)) { dead = true; break; }
                         ++nq[qb];
                     }
-                    const uint32_t qaddr = tc::smem_u32(q_s + qb * ST_TILE_BYTES);
+                    // operand descriptors: the k-step only moves the start address (in 16-byte units, low word)
+                    const uint64_t dq0 = tc::smem_desc_sw128(tc::smem_u32(q_s + qb * ST_TILE_BYTES), 16, 1024);
                     for (int t = 0; t < item.nt; ++t, ++it) {
-                        const int s = it % ST_STAGES, tb = it % ST_TBUF;
-                        if (!tc::mbar_wait(&bar_t_empty[tb], ((it / ST_TBUF) & 1u) ^ 1u, wc, 32)) { dead = true; break; }
-                        if (!tc::mbar_wait(&bar_full[s], (it / ST_STAGES) & 1u, wc, 32)) { dead = true; break; }
+                        if (!tc::mbar_wait(&bar_t_empty[tb], tb_par ^ 1u, wc)) { dead = true; break; }
+                        if (!tc::mbar_wait(&bar_full[st], st_par, wc)) { dead = true; break; }
                         tc::tc_fence_after();
-                        const uint32_t kaddr = tc::smem_u32(ring + s * ST_TILE_BYTES);
+                        const uint64_t dk0 = tc::smem_desc_sw128(ring_addr + st * ST_TILE_BYTES, 16, 1024);
                         const uint32_t acc = tmem + (uint32_t)(tb * 128);
+                        // pass A: queries on the lanes (S = Q K^T); pass B: keys on the lanes (S^T = K Q^T)
+                        const uint64_t da0 = pass == 0 ? dq0 : dk0, db0 = pass == 0 ? dk0 : dq0;
 #pragma unroll
                         for (int kk = 0; kk < 8; ++kk) {
                             // 16 channels per instruction: 32 bytes along the swizzled row, second half after 4 steps
-                            const uint32_t off = (kk >> 2) * (ST_TILE_BYTES / 2) + (kk & 3) * 32;
-                            const uint64_t dk = tc::smem_desc_sw128(kaddr + off, 16, 1024);
-                            const uint64_t dq = tc::smem_desc_sw128(qaddr + off, 16, 1024);
-                            // pass A: queries on the lanes (S = Q K^T); pass B: keys on the lanes (S^T = K Q^T)
-                            if (pass == 0) tc::umma_bf16(acc, dq, dk, IDESC, kk > 0 ? 1u : 0u);
-                            else tc::umma_bf16(acc, dk, dq, IDESC, kk > 0 ? 1u : 0u);
+                            constexpr uint32_t HALF16 = (ST_TILE_BYTES / 2) >> 4;
+                            const uint64_t off16 = (uint64_t)((kk >> 2) * HALF16 + (kk & 3) * 2);
+                            tc::umma_bf16(acc, da0 + off16, db0 + off16, IDESC, kk > 0 ? 1u : 0u);
                         }
-                        tc::umma_commit(&bar_empty[s]);
+                        tc::umma_commit(&bar_empty[st]);
                         tc::umma_commit(&bar_t_full[tb]);
+                        if (++st == ST_STAGES) { st = 0; st_par ^= 1u; }
+                        if (++tb == ST_TBUF) { tb = 0; tb_par ^= 1u; }
                     }
                     if (pass == 1) tc::umma_commit(&bar_q_free[qb]);
                 }
