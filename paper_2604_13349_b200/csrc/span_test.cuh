@@ -23,18 +23,19 @@ constexpr uint32_t HFLAG_INJECT = 1u;      // delta != 0: the injection kernel h
 constexpr uint32_t HFLAG_SPAN_FULL = 2u;   // span(V_keep) = R^d
 
 template <int D>
-constexpr size_t span_smem_bytes() { return (size_t)(D * (D + 1) + 32 * 32 + 32 + D + 32) * sizeof(float); }
+constexpr size_t span_smem_bytes() { return (size_t)(D * (D + 1) + 32 * 33 + 32 + D + 64 + 256 + 3) * sizeof(float); }
 
 template <int D>
-__global__ void __launch_bounds__(ST_NT) k_span_test(const __grid_constant__ CallDev p)
+__global__ void __launch_bounds__(ST_NT, 3) k_span_test(const __grid_constant__ CallDev p)
 {
-    constexpr int LD = D + 1, NB = 32;
+    constexpr int LD = D + 1, NB = 32, L11_LD = NB + 1;
     extern __shared__ float st_sm[];
     float *A = st_sm;                  // D x LD, lower triangle is what counts
     float *L11 = A + D * LD;           // 32 x 32 factor of the current diagonal block (16-byte aligned)
-    float *rinv = L11 + NB * NB;       // 32 reciprocals of its diagonal
+    float *rinv = L11 + NB * L11_LD;   // 32 reciprocals of its diagonal
     float *d0 = rinv + NB;             // D original diagonal entries
-    float *colbuf = d0 + D;            // 32 entries: the current column of the diagonal block's factor
+    float *pvt = d0 + D;               // 8 x 8 pivot block of the diagonal block (16-byte aligned)
+    float *lrow = pvt + 64;            // 32 x 8: the newest 8 columns of the factor, row by row
     __shared__ int s_ok;
 
     const int g = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -57,8 +58,10 @@ __global__ void __launch_bounds__(ST_NT) k_span_test(const __grid_constant__ Cal
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const int e4 = e0 + u * ST_NT;
-                v[u] = e4 < D * D / 4 ? *reinterpret_cast<const float4 *>(parts + (size_t)sp * D * D + e4 * 4)
-                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+                // only the lower triangle is ever read: skip the 4-element groups right of the diagonal
+                const bool lower = e4 < D * D / 4 && (e4 * 4) % D <= (e4 * 4) / D;
+                v[u] = lower ? *reinterpret_cast<const float4 *>(parts + (size_t)sp * D * D + e4 * 4)
+                             : make_float4(0.f, 0.f, 0.f, 0.f);
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) { acc[u].x += v[u].x; acc[u].y += v[u].y; acc[u].z += v[u].z; acc[u].w += v[u].w; }
@@ -82,35 +85,75 @@ __global__ void __launch_bounds__(ST_NT) k_span_test(const __grid_constant__ Cal
     for (int j0 = 0; j0 < D; j0 += NB) {
         const int nrem = D - j0 - NB;                      // rows below the diagonal block
         if (warp == 0) {
-            // lane i owns row i of the diagonal block
+            // Lane i owns row i of the diagonal block in registers.  The block is factorised 8 columns at a
+            // time: the 8 x 8 pivot block is published through shared memory and factorised by EVERY lane
+            // in registers (redundantly, so no lane waits for another inside those 8 columns); each lane
+            // then solves its own 8 entries and the lanes exchange them once for the rank-8 update.
             float a[NB];
 #pragma unroll
             for (int cc = 0; cc < NB; ++cc) a[cc] = cc <= lane ? A[(j0 + lane) * LD + j0 + cc] : 0.f;
             bool ok = true;
 #pragma unroll
-            for (int j = 0; j < NB; ++j) {
-                const float piv = __shfl_sync(0xffffffffu, a[j], j);
-                ok = ok && (piv > CHOL_PIVOT_TOL * d0[j0 + j]) && (piv > 0.f);
-                const float l = a[j] * __frsqrt_rn(piv);     // lanes >= j: L[lane][j]
-                a[j] = l;
-                // column j of L goes through shared memory: every lane then reads the entries it needs as vectors
-                colbuf[lane] = l;
-                __syncwarp();
-#pragma unroll
-                for (int c4 = (j + 1) / 4; c4 < NB / 4; ++c4) {
-                    const float4 lc = *reinterpret_cast<const float4 *>(&colbuf[4 * c4]);
-                    if (4 * c4 + 0 > j) a[4 * c4 + 0] = fmaf(-l, lc.x, a[4 * c4 + 0]);
-                    if (4 * c4 + 1 > j) a[4 * c4 + 1] = fmaf(-l, lc.y, a[4 * c4 + 1]);
-                    if (4 * c4 + 2 > j) a[4 * c4 + 2] = fmaf(-l, lc.z, a[4 * c4 + 2]);
-                    if (4 * c4 + 3 > j) a[4 * c4 + 3] = fmaf(-l, lc.w, a[4 * c4 + 3]);
+            for (int c0 = 0; c0 < NB; c0 += 8) {
+                // rows c0..c0+7 publish their entries of the pivot block (lower triangle is what counts)
+                if (lane >= c0 && lane < c0 + 8) {
+                    float4 *dst = reinterpret_cast<float4 *>(pvt + (lane - c0) * 8);
+                    dst[0] = make_float4(a[c0], a[c0 + 1], a[c0 + 2], a[c0 + 3]);
+                    dst[1] = make_float4(a[c0 + 4], a[c0 + 5], a[c0 + 6], a[c0 + 7]);
                 }
                 __syncwarp();
+                float l8[8][8];                                // factor of the pivot block, row-major, lower
+#pragma unroll
+                for (int r = 0; r < 8; ++r) {
+                    const float4 v0 = *reinterpret_cast<const float4 *>(pvt + r * 8);
+                    const float4 v1 = *reinterpret_cast<const float4 *>(pvt + r * 8 + 4);
+                    l8[r][0] = v0.x; l8[r][1] = v0.y; l8[r][2] = v0.z; l8[r][3] = v0.w;
+                    l8[r][4] = v1.x; l8[r][5] = v1.y; l8[r][6] = v1.z; l8[r][7] = v1.w;
+                }
+                float inv8[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const float piv = l8[k][k];
+                    ok = ok && (piv > CHOL_PIVOT_TOL * d0[j0 + c0 + k]) && (piv > 0.f);
+                    asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(inv8[k]) : "f"(piv));
+                    if (lane == 0) rinv[c0 + k] = inv8[k];
+#pragma unroll
+                    for (int r = k; r < 8; ++r) l8[r][k] *= inv8[k];
+#pragma unroll
+                    for (int c2 = k + 1; c2 < 8; ++c2)
+#pragma unroll
+                        for (int r = c2; r < 8; ++r) l8[r][c2] = fmaf(-l8[r][k], l8[c2][k], l8[r][c2]);
+                }
+                // this lane's 8 entries of L: forward substitution against the pivot block's factor
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    float v = a[c0 + k];
+#pragma unroll
+                    for (int mm = 0; mm < k; ++mm) v = fmaf(-a[c0 + mm], l8[k][mm], v);
+                    a[c0 + k] = v * inv8[k];
+                }
+                if (c0 + 8 < NB) {
+                    // exchange the 8 entries of every row, then the rank-8 update of the columns to the right
+                    float4 *dst = reinterpret_cast<float4 *>(lrow + lane * 8);
+                    dst[0] = make_float4(a[c0], a[c0 + 1], a[c0 + 2], a[c0 + 3]);
+                    dst[1] = make_float4(a[c0 + 4], a[c0 + 5], a[c0 + 6], a[c0 + 7]);
+                    __syncwarp();
+#pragma unroll
+                    for (int cc = c0 + 8; cc < NB; ++cc) {
+                        const float4 w0 = *reinterpret_cast<const float4 *>(lrow + cc * 8);
+                        const float4 w1 = *reinterpret_cast<const float4 *>(lrow + cc * 8 + 4);
+                        float v = a[cc];
+                        v = fmaf(-a[c0], w0.x, v); v = fmaf(-a[c0 + 1], w0.y, v);
+                        v = fmaf(-a[c0 + 2], w0.z, v); v = fmaf(-a[c0 + 3], w0.w, v);
+                        v = fmaf(-a[c0 + 4], w1.x, v); v = fmaf(-a[c0 + 5], w1.y, v);
+                        v = fmaf(-a[c0 + 6], w1.z, v); v = fmaf(-a[c0 + 7], w1.w, v);
+                        a[cc] = v;
+                    }
+                    __syncwarp();
+                }
             }
 #pragma unroll
-            for (int cc = 0; cc < NB; ++cc) L11[lane * NB + cc] = cc <= lane ? a[cc] : 0.f;
-#pragma unroll
-            for (int cc = 0; cc < NB; ++cc)
-                if (cc == lane) rinv[lane] = 1.0f / a[cc];
+            for (int cc = 0; cc < NB; ++cc) L11[lane * L11_LD + cc] = cc <= lane ? a[cc] : 0.f;
             if (!ok && lane == 0) s_ok = 0;
         }
         __syncthreads();
@@ -127,7 +170,7 @@ __global__ void __launch_bounds__(ST_NT) k_span_test(const __grid_constant__ Cal
                 for (int cc = 0; cc < NB; ++cc) {
                     x[cc] *= rinv[cc];
 #pragma unroll
-                    for (int c2 = cc + 1; c2 < NB; ++c2) x[c2] = fmaf(-x[cc], L11[c2 * NB + cc], x[c2]);
+                    for (int c2 = cc + 1; c2 < NB; ++c2) x[c2] = fmaf(-x[cc], L11[c2 * L11_LD + cc], x[c2]);
                 }
 #pragma unroll
                 for (int cc = 0; cc < NB; ++cc) row[cc] = x[cc];
