@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
     float *s_z = s_m + 2 * 4 * 128;                                // [2][4 parts][128 queries] chunk sums
     float *s_mp = s_z + 2 * 4 * 128;                               // [2][128] M'_t of the head being pooled
     float *s_acc = s_mp + 2 * 128;                                 // [ST_TBUF][4 parts][128 keys] pooled partial masses
-    __shared__ uint64_t bar_q_full[ST_QBUF], bar_q_free[ST_QBUF], bar_full[ST_STAGES], bar_empty[ST_STAGES];
+    __shared__ uint64_t bar_q_full[ST_QBUF], bar_q_free[ST_QBUF], bar_full[ST_STAGES];
     __shared__ uint64_t bar_t_full[ST_TBUF], bar_t_empty[ST_TBUF];
     // pooled partial masses of an accumulator tile: written by the four column parts, summed by one of them
     __shared__ uint64_t bar_acc_ready[ST_TBUF], bar_acc_free[ST_TBUF];
@@ -166,7 +166,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
     if (tid == 0) {
         s_abort = 0u;
         for (int b = 0; b < ST_QBUF; ++b) { tc::mbar_init(&bar_q_full[b], 1); tc::mbar_init(&bar_q_free[b], 1); }
-        for (int s = 0; s < ST_STAGES; ++s) { tc::mbar_init(&bar_full[s], 1); tc::mbar_init(&bar_empty[s], 1); }
+        for (int s = 0; s < ST_STAGES; ++s) tc::mbar_init(&bar_full[s], 1);
         for (int s = 0; s < ST_TBUF; ++s) {
             tc::mbar_init(&bar_t_full[s], 1);
             tc::mbar_init(&bar_t_empty[s], ST_CONSUMERS / 32);
@@ -218,7 +218,12 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                     }
                     for (int t = 0; t < item.nt; ++t, ++it) {
                         const int s = it % ST_STAGES;
-                        if (!tc::mbar_wait(&bar_empty[s], ((it / ST_STAGES) & 1u) ^ 1u, wc, 128)) { dead = true; break; }
+                        // the stage is free once the MMAs of the tile that used it last are done: that is the
+                        // same event that hands the accumulator tile to the consumers
+                        if (it >= (uint32_t)ST_STAGES) {
+                            const uint32_t j = it - ST_STAGES;
+                            if (!tc::mbar_wait(&bar_t_full[j % ST_TBUF], (j / ST_TBUF) & 1u, wc, 128)) { dead = true; break; }
+                        }
                         tc::mbar_expect_tx(&bar_full[s], ST_TILE_BYTES);
                         const uint32_t dst = tc::smem_u32(ring + s * ST_TILE_BYTES);
                         const int row0 = item.chunk * ST_CHUNK + t * 128;
@@ -270,7 +275,6 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                             const uint64_t off16 = (uint64_t)((kk >> 2) * HALF16 + (kk & 3) * 2);
                             tc::umma_bf16(acc, da0 + off16, db0 + off16, IDESC, kk > 0 ? 1u : 0u);
                         }
-                        tc::umma_commit(&bar_empty[st]);
                         tc::umma_commit(&bar_t_full[tb]);
                         if (++st == ST_STAGES) { st = 0; st_par ^= 1u; }
                         if (++tb == ST_TBUF) { tb = 0; tb_par ^= 1u; }
@@ -333,6 +337,22 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                     const float4 v = *reinterpret_cast<const float4 *>(s_mp + buf * 128 + part * 32 + e * 4);
                     mp[4 * e] = v.x; mp[4 * e + 1] = v.y; mp[4 * e + 2] = v.z; mp[4 * e + 3] = v.w;
                 }
+                // sum of the four parts of accumulator tile tb (tile t of the chunk), by the part that owns the tile
+                auto finish_tile = [&](int t, int tb, uint32_t par) {
+                    tc::mbar_wait(&bar_acc_ready[tb], par, wc, 20);
+                    const float *sa = s_acc + tb * 4 * 128 + row;
+                    const float a = (sa[0] + sa[128]) + (sa[256] + sa[384]);
+                    __syncwarp();
+                    if (lane == 0) tc::mbar_arrive(&bar_acc_free[tb]);
+                    const int j = item.chunk * ST_CHUNK + t * 128 + row;
+                    if (j < T) {
+                        if (!isfinite(a)) atomicOr(p.status, OBF_DEV_NONFINITE);
+                        p.scores[c.tok_off + (size_t)item.lh * T + j] = a;
+                        if (c.scores_out) c.scores_out[(size_t)item.lh * T + j] = a;
+                    }
+                };
+                int pend_t = -1, pend_tb = 0;
+                uint32_t pend_par = 0u;
 #pragma unroll 1
                 for (int t = 0; t < item.nt; ++t) {
                     // queries [32 * part, +32) of every tile of the chunk; the tile is released as soon as they are in registers
@@ -354,28 +374,21 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                         a2 += ex2_approx(fmaf(__uint_as_float(rr[e + 2]), sc, -mp[e + 2]));
                         a3 += ex2_approx(fmaf(__uint_as_float(rr[e + 3]), sc, -mp[e + 3]));
                     }
-                    // the four parts meet in shared memory; part (t mod 4) adds them up and writes the masses
+                    // the four parts meet in shared memory; part (t mod 4) adds them up and writes the masses,
+                    // one tile later, when the other parts' sums have long arrived
                     const uint32_t bit = 1u << tb;
                     if (acc_used & bit) tc::mbar_wait(&bar_acc_free[tb], ((acc_par >> tb) & 1u) ^ 1u, wc, 20);
                     s_acc[(tb * 4 + part) * 128 + row] = (a0 + a1) + (a2 + a3);
                     __syncwarp();
                     if (lane == 0) tc::mbar_arrive(&bar_acc_ready[tb]);
-                    if (part == (t & 3)) {
-                        tc::mbar_wait(&bar_acc_ready[tb], (acc_par >> tb) & 1u, wc, 20);
-                        const float *sa = s_acc + tb * 4 * 128 + row;
-                        const float a = (sa[0] + sa[128]) + (sa[256] + sa[384]);
-                        __syncwarp();
-                        if (lane == 0) tc::mbar_arrive(&bar_acc_free[tb]);
-                        const int j = item.chunk * ST_CHUNK + t * 128 + row;
-                        if (j < T) {
-                            if (!isfinite(a)) atomicOr(p.status, OBF_DEV_NONFINITE);
-                            p.scores[c.tok_off + (size_t)item.lh * T + j] = a;
-                            if (c.scores_out) c.scores_out[(size_t)item.lh * T + j] = a;
-                        }
-                    }
+                    if (pend_t >= 0) finish_tile(pend_t, pend_tb, pend_par);
+                    pend_t = part == (t & 3) ? t : -1;
+                    pend_tb = tb;
+                    pend_par = (acc_par >> tb) & 1u;
                     acc_used |= bit;
                     acc_par ^= bit;
                 }
+                if (pend_t >= 0) finish_tile(pend_t, pend_tb, pend_par);
                 it += item.nt;
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(&bar_mp_free[buf]);
