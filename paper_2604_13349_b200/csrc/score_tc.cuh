@@ -20,18 +20,21 @@
 // A head's T keys are cut into chunks of 4 tiles of 128 keys; a head's chunks are worked
 // on by a team of blocks in the same round.  Rounds are dealt as
 // (head, chunk) = (round * heads_per_round + block / team, block % team), and a block
-// runs A(0), then A(r), B(r-1) for r = 1.., then B(last): a chunk's second visit comes
-// one chunk of work after its first, when every block of its team has long published.
+// runs A(i), B(i - ST_LAG) for i = 0, 1, ..: a chunk's second visit comes two rounds after
+// its first, when every block of its team has long published, also when the team's
+// blocks sit on both dies and every step of the hand-over is a slow round trip.
 // The wait for M' is bounded like every other wait (tc_common.cuh).
 //
-// Block = 19 warps: warp 0 TMA producer (Q once per chunk, one round ahead; K tiles through a
-// 3-stage ring, asked into L2 one round ahead), warp 1 MMA issuer (accumulators in a 4-deep ring of 128 tensor-memory columns),
+// Block = 20 warps: warp 0 TMA producer (K tiles through a 4-stage ring, asked into L2 one
+// round ahead; Q of a pass is loaded while the pass before it runs, into the buffer of its
+// kind: one for the statistics passes, one for the pooling passes, which read Q again),
+// warp 1 MMA issuer (accumulators in a 4-deep ring of 128 tensor-memory columns),
 // warps 2..17 consumers: warp (quarter, part) reads lanes [32*quarter, +32) and columns
 // [32*part, +32) of every accumulator tile, which frees the tile as soon as the 16 warps
-// have it in registers; warp 18 is the messenger: it publishes the
-// chunk statistics the consumers leave in shared memory, folds a head's chunks when it
-// is the last to arrive, and fetches M' for the next pooling pass, so that the
-// consumers never wait for global memory.
+// have it in registers; warp 18 publishes the chunk statistics the consumers leave in shared
+// memory and folds a head's chunks when its block is the last to arrive; warp 19 fetches M'
+// for the coming pooling passes as early as its two buffers allow, so that the consumers
+// never wait for global memory.
 #pragma once
 
 #include "tc_common.cuh"
@@ -40,39 +43,65 @@ namespace obf {
 
 constexpr int ST_TILES = 4;                         // 128-key tiles per chunk
 constexpr int ST_CHUNK = ST_TILES * 128;
-constexpr int ST_STAGES = 3;                        // K tiles in flight in shared memory
-constexpr int ST_QBUF = 3;                          // Q tiles: rounds r, r - 1 (being pooled) and r + 1 (arriving)
+constexpr int ST_STAGES = 4;                        // K tiles in flight in shared memory
 constexpr int ST_TBUF = 4;                          // accumulator tiles in tensor memory
+constexpr int ST_LAG = 2;                           // rounds between a chunk's statistics pass and its pooling pass
 constexpr int ST_TILE_BYTES = 128 * 128 * 2;
 constexpr int ST_CONSUMERS = 512;
-constexpr int ST_THREADS = 64 + ST_CONSUMERS + 32;
+constexpr int ST_THREADS = 64 + ST_CONSUMERS + 64;
 constexpr int ST_MAX_NQ = 128;
 constexpr float ST_LOG2E = 1.4426950408889634f;
-constexpr size_t ST_SMEM_BYTES = 1024 + (size_t)ST_QBUF * ST_TILE_BYTES + (size_t)ST_STAGES * ST_TILE_BYTES +
-                                 (2 * 2 * 4 * 128 + 2 * 128 + ST_TBUF * 4 * 128) * sizeof(float) + 64;
+constexpr size_t ST_SMEM_BYTES = 1024 + (size_t)2 * ST_TILE_BYTES + (size_t)ST_STAGES * ST_TILE_BYTES +
+                                 (2 * 2 * 4 * 128 + 2 * 128 + 2 * ST_TILES * 4 * 128) * sizeof(float) + 64;
+static_assert(ST_STAGES == ST_TBUF, "a ring stage is released by the accumulator barrier of the same index");
 
 struct ScoreItem {
-    int cache, lh, chunk, nt;      // nt: tiles of the chunk that hold at least one key
+    int r, cache, lh, chunk, nt;   // r: round; nt: tiles of the chunk that hold at least one key
 };
 
-// Work of block `block` in round `r`; false when the block idles in that round.
-__device__ __forceinline__ bool score_item(const CallDev &p, int r, int block, ScoreItem &it)
+// What a block needs of a cache to find its work of a round (kept in shared memory).
+struct ScoreTab {
+    int round_base, hpr, hi, chunk, T;   // hi, chunk: this block's head slot and chunk inside a round of the cache
+};
+
+// Work of this block in round `r`; false when the block idles in that round.
+__device__ __forceinline__ bool score_item(const CallDev &p, const ScoreTab *tab, int r, ScoreItem &it)
 {
     int ci = 0;
 #pragma unroll 1
     for (int i = 1; i < p.n_caches; ++i)
-        if (r >= p.c[i].sc_round_base) ci = i;
-    const CacheDev &c = p.c[ci];
-    const int hi = block / c.sc_team;
-    if (hi >= c.sc_hpr) return false;
-    const int lh = (r - c.sc_round_base) * c.sc_hpr + hi;
+        if (r >= tab[i].round_base) ci = i;
+    const ScoreTab c = tab[ci];
+    if (c.hi >= c.hpr) return false;
+    const int lh = (r - c.round_base) * c.hpr + c.hi;
     if (lh >= p.heads_per_cache) return false;
+    it.r = r;
     it.cache = ci;
     it.lh = lh;
-    it.chunk = block - hi * c.sc_team;
-    const int tiles = (c.T - it.chunk * ST_CHUNK + 127) / 128;
+    it.chunk = c.chunk;
+    const int tiles = (c.T - c.chunk * ST_CHUNK + 127) >> 7;
     it.nt = tiles < ST_TILES ? tiles : ST_TILES;
     return true;
+}
+
+// The passes of a block in the order it runs them: A(i), B(i - ST_LAG) for i = 0, 1, ..
+struct PassIter {
+    int i = 0, ph = 0;
+};
+
+// Next pass with work for this block: kind 0 = statistics, 1 = pooling.
+__device__ __forceinline__ bool next_pass(const CallDev &p, const ScoreTab *tab, int R, PassIter &s, ScoreItem &item, int &kind)
+{
+    while (s.i < R + ST_LAG) {
+        const int ph = s.ph, r = ph == 0 ? s.i : s.i - ST_LAG;
+        if (ph == 0) s.ph = 1;
+        else { s.ph = 0; ++s.i; }
+        if (r < 0 || r >= R) continue;
+        if (!score_item(p, tab, r, item)) continue;
+        kind = ph;
+        return true;
+    }
+    return false;
 }
 
 __device__ __forceinline__ float ex2_approx(float x)
@@ -146,17 +175,18 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
 {
     extern __shared__ uint8_t st_smem_raw[];
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(st_smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t *q_s = base;                                           // ST_QBUF x [128 x 128] bf16 (round mod ST_QBUF), two 64-column halves each
-    uint8_t *ring = q_s + ST_QBUF * ST_TILE_BYTES;                       // ST_STAGES x 32 KiB
+    uint8_t *q_s = base;                                           // 2 x [128 x 128] bf16: Q of a statistics pass, Q of a pooling pass; two 64-column halves each
+    uint8_t *ring = q_s + 2 * ST_TILE_BYTES;                       // ST_STAGES x 32 KiB
     float *s_m = reinterpret_cast<float *>(ring + ST_STAGES * ST_TILE_BYTES);   // [2][4 parts][128 queries] chunk maxima
     float *s_z = s_m + 2 * 4 * 128;                                // [2][4 parts][128 queries] chunk sums
     float *s_mp = s_z + 2 * 4 * 128;                               // [2][128] M'_t of the head being pooled
-    float *s_acc = s_mp + 2 * 128;                                 // [ST_TBUF][4 parts][128 keys] pooled partial masses
-    __shared__ uint64_t bar_q_full[ST_QBUF], bar_q_free[ST_QBUF], bar_full[ST_STAGES];
+    float *s_acc = s_mp + 2 * 128;                                 // [2][ST_TILES][4 parts][128 keys] pooled partial masses of a pass
+    __shared__ uint64_t bar_q_full[2], bar_q_free[2], bar_full[ST_STAGES];
     __shared__ uint64_t bar_t_full[ST_TBUF], bar_t_empty[ST_TBUF];
-    // pooled partial masses of an accumulator tile: written by the four column parts, summed by one of them
-    __shared__ uint64_t bar_acc_ready[ST_TBUF], bar_acc_free[ST_TBUF];
+    // pooled partial masses of a pooling pass: written by the four column parts, summed one tile into the next pass
+    __shared__ uint64_t bar_acc_ready[2], bar_acc_free[2];
     __shared__ uint64_t bar_st_ready[2], bar_st_free[2], bar_mp_ready[2], bar_mp_free[2];
+    __shared__ ScoreTab s_tab[OBF_MAX_CACHES];
     __shared__ uint32_t s_tmem, s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -165,21 +195,31 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
 
     if (tid == 0) {
         s_abort = 0u;
-        for (int b = 0; b < ST_QBUF; ++b) { tc::mbar_init(&bar_q_full[b], 1); tc::mbar_init(&bar_q_free[b], 1); }
+        for (int b = 0; b < 2; ++b) { tc::mbar_init(&bar_q_full[b], 1); tc::mbar_init(&bar_q_free[b], 1); }
         for (int s = 0; s < ST_STAGES; ++s) tc::mbar_init(&bar_full[s], 1);
         for (int s = 0; s < ST_TBUF; ++s) {
             tc::mbar_init(&bar_t_full[s], 1);
             tc::mbar_init(&bar_t_empty[s], ST_CONSUMERS / 32);
-            tc::mbar_init(&bar_acc_ready[s], ST_CONSUMERS / 32);
-            tc::mbar_init(&bar_acc_free[s], 4);
         }
         for (int b = 0; b < 2; ++b) {
+            tc::mbar_init(&bar_acc_ready[b], ST_CONSUMERS / 32);
+            tc::mbar_init(&bar_acc_free[b], ST_CONSUMERS / 32);
             tc::mbar_init(&bar_st_ready[b], ST_CONSUMERS / 32);
             tc::mbar_init(&bar_st_free[b], 1);
             tc::mbar_init(&bar_mp_ready[b], 1);
             tc::mbar_init(&bar_mp_free[b], ST_CONSUMERS / 32);
         }
         tc::mbar_init_fence();
+    }
+    if (tid >= 64 && tid < 64 + p.n_caches) {
+        const CacheDev &c = p.c[tid - 64];
+        ScoreTab e;
+        e.round_base = c.sc_round_base;
+        e.hpr = c.sc_hpr;
+        e.hi = (int)blockIdx.x / c.sc_team;
+        e.chunk = (int)blockIdx.x - e.hi * c.sc_team;
+        e.T = c.T;
+        s_tab[tid - 64] = e;
     }
     if (warp == 1) tc::tmem_alloc(&s_tmem, 512);
     tc::tc_fence_before();
@@ -190,114 +230,135 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            uint32_t it = 0, nq[ST_QBUF] = {0u, 0u, 0u};
+            uint32_t it = 0, nq[2] = {0u, 0u};
             bool dead = false;
-            for (int i = 0; i <= R && !dead; ++i) {
-                for (int pass = 0; pass < 2 && !dead; ++pass) {
-                    const int r = pass == 0 ? i : i - 1;
-                    if (r < 0 || r >= R) continue;
-                    ScoreItem item;
-                    if (!score_item(p, r, (int)blockIdx.x, item)) continue;
-                    const int qb = r % ST_QBUF;
-                    if (pass == 0) {
-                        // the buffer is free once the pooling MMAs of its previous user are done
-                        if (nq[qb] > 0 && !tc::mbar_wait(&bar_q_free[qb], (nq[qb] - 1) & 1u, wc, 128)) { dead = true; break; }
-                        const uint32_t qdst = tc::smem_u32(q_s + qb * ST_TILE_BYTES);
-                        tc::mbar_expect_tx(&bar_q_full[qb], ST_TILE_BYTES);
-                        tc::tma_load_3d(qdst, &tm.b[item.cache], &bar_q_full[qb], 0, 0, item.lh);
-                        tc::tma_load_3d(qdst + ST_TILE_BYTES / 2, &tm.b[item.cache], &bar_q_full[qb], 64, 0, item.lh);
-                        ++nq[qb];
-                        // the next round's first visit comes from HBM: ask for its tiles now
-                        ScoreItem nx;
-                        if (r + 1 < R && score_item(p, r + 1, (int)blockIdx.x, nx)) {
-                            for (int t = 0; t < nx.nt; ++t) {
-                                tc::tma_prefetch_l2_3d(&tm.a[nx.cache], 0, nx.chunk * ST_CHUNK + t * 128, nx.lh);
-                                tc::tma_prefetch_l2_3d(&tm.a[nx.cache], 64, nx.chunk * ST_CHUNK + t * 128, nx.lh);
-                            }
+            // Q of a pass goes to the buffer of its kind once the MMAs of that buffer's last user are done
+            auto load_q = [&](const ScoreItem &item, int kind) -> bool {
+                if (nq[kind] > 0 && !tc::mbar_wait(&bar_q_free[kind], (nq[kind] - 1) & 1u, wc, 64)) return false;
+                const uint32_t qdst = tc::smem_u32(q_s + kind * ST_TILE_BYTES);
+                tc::mbar_expect_tx(&bar_q_full[kind], ST_TILE_BYTES);
+                tc::tma_load_3d(qdst, &tm.b[item.cache], &bar_q_full[kind], 0, 0, item.lh);
+                tc::tma_load_3d(qdst + ST_TILE_BYTES / 2, &tm.b[item.cache], &bar_q_full[kind], 64, 0, item.lh);
+                ++nq[kind];
+                return true;
+            };
+            PassIter pi;
+            ScoreItem item, nxt;
+            int kind = 0, nkind = 0;
+            bool have = next_pass(p, s_tab, R, pi, item, kind);
+            if (have) load_q(item, kind);
+            while (have && !dead) {
+                if (kind == 0) {
+                    // the next statistics pass reads its tiles from HBM: ask for them now
+                    ScoreItem nx;
+                    if (item.r + 1 < R && score_item(p, s_tab, item.r + 1, nx)) {
+                        for (int t = 0; t < nx.nt; ++t) {
+                            tc::tma_prefetch_l2_3d(&tm.a[nx.cache], 0, nx.chunk * ST_CHUNK + t * 128, nx.lh);
+                            tc::tma_prefetch_l2_3d(&tm.a[nx.cache], 64, nx.chunk * ST_CHUNK + t * 128, nx.lh);
                         }
-                    }
-                    for (int t = 0; t < item.nt; ++t, ++it) {
-                        const int s = it % ST_STAGES;
-                        // the stage is free once the MMAs of the tile that used it last are done: that is the
-                        // same event that hands the accumulator tile to the consumers
-                        if (it >= (uint32_t)ST_STAGES) {
-                            const uint32_t j = it - ST_STAGES;
-                            if (!tc::mbar_wait(&bar_t_full[j % ST_TBUF], (j / ST_TBUF) & 1u, wc, 128)) { dead = true; break; }
-                        }
-                        tc::mbar_expect_tx(&bar_full[s], ST_TILE_BYTES);
-                        const uint32_t dst = tc::smem_u32(ring + s * ST_TILE_BYTES);
-                        const int row0 = item.chunk * ST_CHUNK + t * 128;
-                        tc::tma_load_3d(dst, &tm.a[item.cache], &bar_full[s], 0, row0, item.lh);
-                        tc::tma_load_3d(dst + ST_TILE_BYTES / 2, &tm.a[item.cache], &bar_full[s], 64, row0, item.lh);
                     }
                 }
+                for (int t = 0; t < item.nt; ++t, ++it) {
+                    const int s = it % ST_STAGES;
+                    // the stage is free once the MMAs of the tile that used it last are done: that is the
+                    // same event that hands the accumulator tile to the consumers
+                    if (it >= (uint32_t)ST_STAGES) {
+                        const uint32_t j = it - ST_STAGES;
+                        if (!tc::mbar_wait(&bar_t_full[j % ST_TBUF], (j / ST_TBUF) & 1u, wc, 64)) { dead = true; break; }
+                    }
+                    tc::mbar_expect_tx(&bar_full[s], ST_TILE_BYTES);
+                    const uint32_t dst = tc::smem_u32(ring + s * ST_TILE_BYTES);
+                    const int row0 = item.chunk * ST_CHUNK + t * 128;
+                    tc::tma_load_3d(dst, &tm.a[item.cache], &bar_full[s], 0, row0, item.lh);
+                    tc::tma_load_3d(dst + ST_TILE_BYTES / 2, &tm.a[item.cache], &bar_full[s], 64, row0, item.lh);
+                }
+                if (dead) break;
+                // Q of the next pass, while the tiles just asked for are worked on
+                have = next_pass(p, s_tab, R, pi, nxt, nkind);
+                if (have && !load_q(nxt, nkind)) dead = true;
+                item = nxt;
+                kind = nkind;
             }
             // nothing this thread started may still be in flight when the block exits
             for (uint32_t j = it > (uint32_t)ST_STAGES ? it - ST_STAGES : 0u; j < it; ++j)
-                tc::mbar_wait(&bar_full[j % ST_STAGES], (j / ST_STAGES) & 1u, wc, 128);
-            for (int b = 0; b < ST_QBUF; ++b)
-                if (nq[b] > 0) tc::mbar_wait(&bar_q_full[b], (nq[b] - 1) & 1u, wc, 128);
+                tc::mbar_wait(&bar_full[j % ST_STAGES], (j / ST_STAGES) & 1u, wc, 64);
+            for (int b = 0; b < 2; ++b)
+                if (nq[b] > 0) tc::mbar_wait(&bar_q_full[b], (nq[b] - 1) & 1u, wc, 64);
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
             constexpr uint32_t IDESC = tc::idesc_bf16(128, 128, 0, 0);
-            uint32_t it = 0, nq[ST_QBUF] = {0u, 0u, 0u};
-            // ring stage and accumulator tile of the next tile, with the parity of their current use
-            uint32_t st = 0, st_par = 0, tb = 0, tb_par = 0;
+            uint32_t nq[2] = {0u, 0u};
+            // ring stage / accumulator tile of the next tile (same index), with the parity of its current use
+            uint32_t tb = 0, tb_par = 0;
             const uint32_t ring_addr = tc::smem_u32(ring);
             bool dead = false;
-            for (int i = 0; i <= R && !dead; ++i) {
-                for (int pass = 0; pass < 2 && !dead; ++pass) {
-                    const int r = pass == 0 ? i : i - 1;
-                    if (r < 0 || r >= R) continue;
-                    ScoreItem item;
-                    if (!score_item(p, r, (int)blockIdx.x, item)) continue;
-                    const int qb = r % ST_QBUF;
-                    if (pass == 0) {
-                        if (!tc::mbar_wait(&bar_q_full[qb], nq[qb] & 1u, wc)) { dead = true; break; }
-                        ++nq[qb];
-                    }
-                    // operand descriptors: the k-step only moves the start address (in 16-byte units, low word)
-                    const uint64_t dq0 = tc::smem_desc_sw128(tc::smem_u32(q_s + qb * ST_TILE_BYTES), 16, 1024);
-                    for (int t = 0; t < item.nt; ++t, ++it) {
-                        if (!tc::mbar_wait(&bar_t_empty[tb], tb_par ^ 1u, wc)) { dead = true; break; }
-                        if (!tc::mbar_wait(&bar_full[st], st_par, wc)) { dead = true; break; }
-                        tc::tc_fence_after();
-                        const uint64_t dk0 = tc::smem_desc_sw128(ring_addr + st * ST_TILE_BYTES, 16, 1024);
-                        const uint32_t acc = tmem + (uint32_t)(tb * 128);
-                        // pass A: queries on the lanes (S = Q K^T); pass B: keys on the lanes (S^T = K Q^T)
-                        const uint64_t da0 = pass == 0 ? dq0 : dk0, db0 = pass == 0 ? dk0 : dq0;
+            PassIter pi;
+            ScoreItem item;
+            int kind = 0;
+            while (!dead && next_pass(p, s_tab, R, pi, item, kind)) {
+                if (!tc::mbar_wait(&bar_q_full[kind], nq[kind] & 1u, wc)) break;
+                ++nq[kind];
+                // operand descriptors: the k-step only moves the start address (in 16-byte units, low word)
+                const uint64_t dq0 = tc::smem_desc_sw128(tc::smem_u32(q_s + kind * ST_TILE_BYTES), 16, 1024);
+                for (int t = 0; t < item.nt; ++t) {
+                    if (!tc::mbar_wait(&bar_t_empty[tb], tb_par ^ 1u, wc)) { dead = true; break; }
+                    if (!tc::mbar_wait(&bar_full[tb], tb_par, wc)) { dead = true; break; }
+                    tc::tc_fence_after();
+                    const uint64_t dk0 = tc::smem_desc_sw128(ring_addr + tb * ST_TILE_BYTES, 16, 1024);
+                    const uint32_t acc = tmem + (uint32_t)(tb * 128);
+                    // pass A: queries on the lanes (S = Q K^T); pass B: keys on the lanes (S^T = K Q^T)
+                    const uint64_t da0 = kind == 0 ? dq0 : dk0, db0 = kind == 0 ? dk0 : dq0;
 #pragma unroll
-                        for (int kk = 0; kk < 8; ++kk) {
-                            // 16 channels per instruction: 32 bytes along the swizzled row, second half after 4 steps
-                            constexpr uint32_t HALF16 = (ST_TILE_BYTES / 2) >> 4;
-                            const uint64_t off16 = (uint64_t)((kk >> 2) * HALF16 + (kk & 3) * 2);
-                            tc::umma_bf16(acc, da0 + off16, db0 + off16, IDESC, kk > 0 ? 1u : 0u);
-                        }
-                        tc::umma_commit(&bar_t_full[tb]);
-                        if (++st == ST_STAGES) { st = 0; st_par ^= 1u; }
-                        if (++tb == ST_TBUF) { tb = 0; tb_par ^= 1u; }
+                    for (int kk = 0; kk < 8; ++kk) {
+                        // 16 channels per instruction: 32 bytes along the swizzled row, second half after 4 steps
+                        constexpr uint32_t HALF16 = (ST_TILE_BYTES / 2) >> 4;
+                        const uint64_t off16 = (uint64_t)((kk >> 2) * HALF16 + (kk & 3) * 2);
+                        tc::umma_bf16(acc, da0 + off16, db0 + off16, IDESC, kk > 0 ? 1u : 0u);
                     }
-                    if (pass == 1) tc::umma_commit(&bar_q_free[qb]);
+                    tc::umma_commit(&bar_t_full[tb]);
+                    if (++tb == ST_TBUF) { tb = 0; tb_par ^= 1u; }
                 }
+                if (!dead) tc::umma_commit(&bar_q_free[kind]);
             }
         }
     } else if (warp < 2 + ST_CONSUMERS / 32) {
         // ---------------- consumers ----------------
         const int q = warp & 3;                        // tensor-memory lane quarter this warp may touch
-        const int part = (warp - 2) >> 2;              // which tile of a chunk
+        const int part = (warp - 2) >> 2;              // columns [32 * part, +32) of every tile; sums tile `part` of a pooling pass
         const int row = q * 32 + lane;                 // lane of the accumulator tile: a query (pass A) or a key (pass B)
         const uint32_t tlane = tmem + ((uint32_t)(q * 32) << 16);
         const float sc = ST_LOG2E * rsqrtf(128.0f);
-        uint32_t it = 0, n_a[2] = {0u, 0u}, n_b[2] = {0u, 0u};
-        uint32_t acc_used = 0u, acc_par = 0u;          // per accumulator tile: s_acc slot used before, parity of its uses
+        uint32_t it = 0, n_a[2] = {0u, 0u}, n_b[2] = {0u, 0u}, n_pool = 0u;
 
-        for (int i = 0; i <= R; ++i) {
+        // a pooling pass whose partial masses wait in shared memory for their sum
+        bool pend = false;
+        uint32_t pend_buf = 0u, pend_par = 0u;
+        int pend_T = 0, pend_j = 0, pend_nt = 0;
+        float *pend_dst = nullptr, *pend_out = nullptr;
+        auto finish_pool = [&]() {
+            tc::mbar_wait(&bar_acc_ready[pend_buf], pend_par, wc, 20);
+            float a = 0.f;
+            if (part < pend_nt) {
+                const float *sa = s_acc + ((pend_buf * ST_TILES + part) * 4) * 128 + row;
+                a = (sa[0] + sa[128]) + (sa[256] + sa[384]);
+            }
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(&bar_acc_free[pend_buf]);
+            if (part < pend_nt && pend_j < pend_T) {
+                if (!isfinite(a)) atomicOr(p.status, OBF_DEV_NONFINITE);
+                pend_dst[pend_j] = a;
+                if (pend_out) pend_out[pend_j] = a;
+            }
+            pend = false;
+        };
+
+        for (int i = 0; i < R + ST_LAG; ++i) {
             // ======== pass A of round i: maximum and sum per query over columns [32 * part, +32) of the chunk's tiles ========
             ScoreItem item;
-            if (i < R && score_item(p, i, (int)blockIdx.x, item)) {
-                const int T = p.c[item.cache].T, buf = i & 1;
+            if (i < R && score_item(p, s_tab, i, item)) {
+                const int T = s_tab[item.cache].T, buf = i & 1;
                 float m = -INFINITY, z = 0.f;
 #pragma unroll 1
                 for (int t = 0; t < item.nt; ++t) {
@@ -316,6 +377,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                     // two copies of the update: the one that masks missing keys runs for a head's ragged last tile only
                     if (key0 + 32 > T) stats_update<true>(rr, T - key0, sc, m, z);
                     else stats_update<false>(rr, 32, sc, m, z);
+                    if (pend) finish_pool();
                 }
                 it += item.nt;
                 // hand (m, z) of this column part to the messenger
@@ -326,10 +388,10 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                 if (lane == 0) tc::mbar_arrive(&bar_st_ready[buf]);
                 ++n_a[buf];
             }
-            // ======== pass B of round i - 1: pooled mass per key over queries [32 * part, +32) ========
-            if (i >= 1 && score_item(p, i - 1, (int)blockIdx.x, item)) {
+            // ======== pass B of round i - ST_LAG: pooled mass per key over queries [32 * part, +32) ========
+            if (i >= ST_LAG && score_item(p, s_tab, i - ST_LAG, item)) {
                 const CacheDev &c = p.c[item.cache];
-                const int T = c.T, buf = (i - 1) & 1;
+                const int T = s_tab[item.cache].T, buf = (i - ST_LAG) & 1;
                 tc::mbar_wait(&bar_mp_ready[buf], n_b[buf] & 1u, wc, 20);
                 float mp[32];
 #pragma unroll
@@ -337,22 +399,8 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                     const float4 v = *reinterpret_cast<const float4 *>(s_mp + buf * 128 + part * 32 + e * 4);
                     mp[4 * e] = v.x; mp[4 * e + 1] = v.y; mp[4 * e + 2] = v.z; mp[4 * e + 3] = v.w;
                 }
-                // sum of the four parts of accumulator tile tb (tile t of the chunk), by the part that owns the tile
-                auto finish_tile = [&](int t, int tb, uint32_t par) {
-                    tc::mbar_wait(&bar_acc_ready[tb], par, wc, 20);
-                    const float *sa = s_acc + tb * 4 * 128 + row;
-                    const float a = (sa[0] + sa[128]) + (sa[256] + sa[384]);
-                    __syncwarp();
-                    if (lane == 0) tc::mbar_arrive(&bar_acc_free[tb]);
-                    const int j = item.chunk * ST_CHUNK + t * 128 + row;
-                    if (j < T) {
-                        if (!isfinite(a)) atomicOr(p.status, OBF_DEV_NONFINITE);
-                        p.scores[c.tok_off + (size_t)item.lh * T + j] = a;
-                        if (c.scores_out) c.scores_out[(size_t)item.lh * T + j] = a;
-                    }
-                };
-                int pend_t = -1, pend_tb = 0;
-                uint32_t pend_par = 0u;
+                // this pass's partial masses go to the buffer the pass before the last one used
+                const uint32_t ab = n_pool & 1u, use = n_pool >> 1;
 #pragma unroll 1
                 for (int t = 0; t < item.nt; ++t) {
                     // queries [32 * part, +32) of every tile of the chunk; the tile is released as soon as they are in registers
@@ -374,127 +422,146 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                         a2 += ex2_approx(fmaf(__uint_as_float(rr[e + 2]), sc, -mp[e + 2]));
                         a3 += ex2_approx(fmaf(__uint_as_float(rr[e + 3]), sc, -mp[e + 3]));
                     }
-                    // the four parts meet in shared memory; part (t mod 4) adds them up and writes the masses,
-                    // one tile later, when the other parts' sums have long arrived
-                    const uint32_t bit = 1u << tb;
-                    if (acc_used & bit) tc::mbar_wait(&bar_acc_free[tb], ((acc_par >> tb) & 1u) ^ 1u, wc, 20);
-                    s_acc[(tb * 4 + part) * 128 + row] = (a0 + a1) + (a2 + a3);
-                    __syncwarp();
-                    if (lane == 0) tc::mbar_arrive(&bar_acc_ready[tb]);
-                    if (pend_t >= 0) finish_tile(pend_t, pend_tb, pend_par);
-                    pend_t = part == (t & 3) ? t : -1;
-                    pend_tb = tb;
-                    pend_par = (acc_par >> tb) & 1u;
-                    acc_used |= bit;
-                    acc_par ^= bit;
+                    if (pend) finish_pool();                       // the pass before this one, one tile late
+                    if (t == 0 && use > 0) tc::mbar_wait(&bar_acc_free[ab], (use - 1) & 1u, wc, 20);
+                    s_acc[((ab * ST_TILES + t) * 4 + part) * 128 + row] = (a0 + a1) + (a2 + a3);
                 }
-                if (pend_t >= 0) finish_tile(pend_t, pend_tb, pend_par);
                 it += item.nt;
                 __syncwarp();
-                if (lane == 0) tc::mbar_arrive(&bar_mp_free[buf]);
+                if (lane == 0) {
+                    tc::mbar_arrive(&bar_acc_ready[ab]);
+                    tc::mbar_arrive(&bar_mp_free[buf]);
+                }
                 ++n_b[buf];
+                ++n_pool;
+                // the four parts' sums of tile `part` become this warp's keys' masses after the next tile
+                pend = true;
+                pend_buf = ab;
+                pend_par = use & 1u;
+                pend_T = T;
+                pend_nt = item.nt;
+                pend_j = item.chunk * ST_CHUNK + part * 128 + row;
+                pend_dst = p.scores + c.tok_off + (size_t)item.lh * T;
+                pend_out = c.scores_out ? c.scores_out + (size_t)item.lh * T : nullptr;
+            }
+        }
+        if (pend) finish_pool();
+    } else if (warp == 2 + ST_CONSUMERS / 32) {
+        // ---------------- publisher: chunk statistics out, a head's chunks folded by the last block to arrive ----------------
+        uint32_t n_a[2] = {0u, 0u};
+        for (int i = 0; i < R; ++i) {
+            ScoreItem item;
+            if (!score_item(p, s_tab, i, item)) continue;
+            const CacheDev &c = p.c[item.cache];
+            const int buf = i & 1, team = c.sc_team;
+            const int g = c.head_base + item.lh;
+            tc::mbar_wait(&bar_st_ready[buf], n_a[buf] & 1u, wc, 32);
+            float2 *partials = reinterpret_cast<float2 *>(p.sc_part) + (c.sc_part_off + ((size_t)item.lh * team + item.chunk) * 128);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int t = lane + 32 * k;
+                const float *sm = s_m + buf * 4 * 128 + t, *sz = s_z + buf * 4 * 128 + t;
+                const float M = fmaxf(fmaxf(sm[0], sm[128]), fmaxf(sm[256], sm[384]));
+                float Z = 0.f;
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (sm[e * 128] > -INFINITY) Z += sz[e * 128] * ex2_approx(sm[e * 128] - M);
+                if (t < p.n_q) __stcg(&partials[t], make_float2(M, Z));
+            }
+            __syncwarp();
+            uint32_t last = 0u;
+            if (lane == 0) {
+                tc::mbar_arrive(&bar_st_free[buf]);
+                // the warp barrier orders the lanes' stores before this release; the acquire side mirrors it
+                last = (atom_add_acq_rel_gpu(&p.sc_cnt[g], 1u) == (uint32_t)(team - 1)) ? 1u : 0u;
+            }
+            last = __shfl_sync(0xffffffffu, last, 0);
+            ++n_a[buf];
+            if (last) {
+                // this block is the last of its head: fold all chunks, eight chunks of the lane's four queries per sweep
+                // (32 loads in flight: the fold is a few round trips long, whatever the team's size)
+                const float2 *hp = reinterpret_cast<const float2 *>(p.sc_part) + (c.sc_part_off + (size_t)item.lh * team * 128);
+                unsigned long long *words = reinterpret_cast<unsigned long long *>(p.sc_head) + (size_t)g * 128;
+                float M[4], Z[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) { M[k] = -INFINITY; Z[k] = 0.f; }
+                for (int c0 = 0; c0 < team; c0 += 8) {
+                    float2 v[4][8];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+#pragma unroll
+                        for (int e = 0; e < 8; ++e)
+                            v[k][e] = (c0 + e < team && lane + 32 * k < p.n_q) ? __ldcg(&hp[(size_t)(c0 + e) * 128 + lane + 32 * k])
+                                                                               : make_float2(-INFINITY, 0.f);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        float Mn = M[k];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) Mn = fmaxf(Mn, v[k][e].x);
+                        if (Mn > -INFINITY) {
+                            Z[k] *= ex2_approx(M[k] - Mn);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e)
+                                if (v[k][e].x > -INFINITY) Z[k] += v[k][e].y * ex2_approx(v[k][e].x - Mn);
+                            M[k] = Mn;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int t = lane + 32 * k;
+                    if (t >= p.n_q) continue;
+                    float mp = M[k] + lg2_approx(Z[k]);
+                    if (!(Z[k] > 0.f) || !isfinite(mp)) {
+                        atomicOr(p.status, OBF_DEV_NONFINITE);
+                        mp = __int_as_float(0x7fc00000);
+                    }
+                    // one 64-bit word per query: low = M'_t, high = 1 once it is valid
+                    st_relaxed_gpu_u64(words + t, (1ull << 32) | __float_as_uint(mp));
+                }
             }
         }
     } else {
-        // ---------------- messenger ----------------
-        uint32_t n_a[2] = {0u, 0u}, n_b[2] = {0u, 0u};
-        for (int i = 0; i <= R; ++i) {
+        // ---------------- fetcher: M' of the heads to be pooled, into shared memory as early as the buffers allow ----------------
+        uint32_t n_b[2] = {0u, 0u};
+        for (int r = 0; r < R; ++r) {
             ScoreItem item;
-            // M' of the head that is pooled next, into shared memory
-            if (i >= 1 && score_item(p, i - 1, (int)blockIdx.x, item)) {
-                const int buf = (i - 1) & 1;
-                const int g = p.c[item.cache].head_base + item.lh;
-                if (n_b[buf] > 0) tc::mbar_wait(&bar_mp_free[buf], (n_b[buf] - 1) & 1u, wc, 32);
-                const unsigned long long *words = reinterpret_cast<const unsigned long long *>(p.sc_head) + (size_t)g * 128;
-                // the four words of this lane are polled together: one round trip, not four
-                unsigned long long v[4] = {0ull, 0ull, 0ull, 0ull};
-                const uint64_t t0 = tc::global_ns();
-                for (;;) {
-                    bool all = true;
+            if (!score_item(p, s_tab, r, item)) continue;
+            const int buf = r & 1;
+            const int g = p.c[item.cache].head_base + item.lh;
+            if (n_b[buf] > 0) tc::mbar_wait(&bar_mp_free[buf], (n_b[buf] - 1) & 1u, wc, 32);
+            const unsigned long long *words = reinterpret_cast<const unsigned long long *>(p.sc_head) + (size_t)g * 128;
+            // the four words of this lane are polled together: one round trip, not four
+            unsigned long long v[4] = {0ull, 0ull, 0ull, 0ull};
+            const uint64_t t0 = tc::global_ns();
+            for (;;) {
+                bool all = true;
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        if (lane + 32 * k < p.n_q && (v[k] >> 32) == 0ull) v[k] = ld_relaxed_gpu_u64(words + lane + 32 * k);
+                for (int k = 0; k < 4; ++k)
+                    if (lane + 32 * k < p.n_q && (v[k] >> 32) == 0ull) v[k] = ld_relaxed_gpu_u64(words + lane + 32 * k);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        if (lane + 32 * k < p.n_q && (v[k] >> 32) == 0ull) all = false;
-                    if (all || s_abort) break;
-                    if (tc::global_ns() - t0 > tc::WAIT_LIMIT_NS) {
+                for (int k = 0; k < 4; ++k)
+                    if (lane + 32 * k < p.n_q && (v[k] >> 32) == 0ull) all = false;
+                // the warp leaves the loop as one: votes, not per-lane exits
+                if (__all_sync(0xffffffffu, all) || __any_sync(0xffffffffu, *(volatile uint32_t *)&s_abort != 0u)) break;
+                if (__any_sync(0xffffffffu, tc::global_ns() - t0 > tc::WAIT_LIMIT_NS)) {
+                    if (lane == 0) {
                         s_abort = 1u;
                         atomicOr(p.status, OBF_DEV_TIMEOUT);
-                        break;
                     }
-                    __nanosleep(32);
+                    break;
                 }
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const int t = lane + 32 * k;
-                    // exp2(-inf) = 0 for padding columns
-                    s_mp[buf * 128 + t] = t < p.n_q ? __uint_as_float((uint32_t)v[k]) : INFINITY;
-                }
-                __syncwarp();
-                if (lane == 0) tc::mbar_arrive(&bar_mp_ready[buf]);
-                ++n_b[buf];
+                __nanosleep(64);
             }
-            // statistics of the chunk the consumers have just finished
-            if (i < R && score_item(p, i, (int)blockIdx.x, item)) {
-                const CacheDev &c = p.c[item.cache];
-                const int buf = i & 1, team = c.sc_team;
-                const int g = c.head_base + item.lh;
-                tc::mbar_wait(&bar_st_ready[buf], n_a[buf] & 1u, wc, 32);
-                float2 *partials = reinterpret_cast<float2 *>(p.sc_part) + (c.sc_part_off + ((size_t)item.lh * team + item.chunk) * 128);
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const int t = lane + 32 * k;
-                    const float *sm = s_m + buf * 4 * 128 + t, *sz = s_z + buf * 4 * 128 + t;
-                    const float M = fmaxf(fmaxf(sm[0], sm[128]), fmaxf(sm[256], sm[384]));
-                    float Z = 0.f;
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        if (sm[e * 128] > -INFINITY) Z += sz[e * 128] * ex2_approx(sm[e * 128] - M);
-                    if (t < p.n_q) __stcg(&partials[t], make_float2(M, Z));
-                }
-                __syncwarp();
-                uint32_t last = 0u;
-                if (lane == 0) {
-                    tc::mbar_arrive(&bar_st_free[buf]);
-                    // the warp barrier orders the lanes' stores before this release; the acquire side mirrors it
-                    last = (atom_add_acq_rel_gpu(&p.sc_cnt[g], 1u) == (uint32_t)(team - 1)) ? 1u : 0u;
-                }
-                last = __shfl_sync(0xffffffffu, last, 0);
-                ++n_a[buf];
-                if (last) {
-                    // this block is the last of its head: fold all chunks
-                    const float2 *hp = reinterpret_cast<const float2 *>(p.sc_part) + (c.sc_part_off + (size_t)item.lh * team * 128);
-                    unsigned long long *words = reinterpret_cast<unsigned long long *>(p.sc_head) + (size_t)g * 128;
-                    for (int t = lane; t < p.n_q; t += 32) {
-                        // one sweep over the chunks, eight loads in flight at a time
-                        float M = -INFINITY, Z = 0.f;
-                        for (int c0 = 0; c0 < team; c0 += 8) {
-                            float2 v[8];
-#pragma unroll
-                            for (int e = 0; e < 8; ++e)
-                                v[e] = c0 + e < team ? __ldcg(&hp[(size_t)(c0 + e) * 128 + t]) : make_float2(-INFINITY, 0.f);
-                            float Mn = M;
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) Mn = fmaxf(Mn, v[e].x);
-                            if (Mn > -INFINITY) {
-                                Z *= ex2_approx(M - Mn);
-#pragma unroll
-                                for (int e = 0; e < 8; ++e)
-                                    if (v[e].x > -INFINITY) Z += v[e].y * ex2_approx(v[e].x - Mn);
-                                M = Mn;
-                            }
-                        }
-                        float mp = M + lg2_approx(Z);
-                        if (!(Z > 0.f) || !isfinite(mp)) {
-                            atomicOr(p.status, OBF_DEV_NONFINITE);
-                            mp = __int_as_float(0x7fc00000);
-                        }
-                        // one 64-bit word per query: low = M'_t, high = 1 once it is valid
-                        st_relaxed_gpu_u64(words + t, (1ull << 32) | __float_as_uint(mp));
-                    }
-                }
+            for (int k = 0; k < 4; ++k) {
+                const int t = lane + 32 * k;
+                // exp2(-inf) = 0 for padding columns
+                s_mp[buf * 128 + t] = t < p.n_q ? __uint_as_float((uint32_t)v[k]) : INFINITY;
             }
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(&bar_mp_ready[buf]);
+            ++n_b[buf];
         }
     }
 
