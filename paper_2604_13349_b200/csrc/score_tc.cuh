@@ -20,21 +20,21 @@
 // A head's T keys are cut into chunks of 4 tiles of 128 keys; a head's chunks are worked
 // on by a team of blocks in the same round.  Rounds are dealt as
 // (head, chunk) = (round * heads_per_round + block / team, block % team), and a block
-// runs A(i), B(i - ST_LAG) for i = 0, 1, ..: a chunk's second visit comes two rounds after
-// its first, when every block of its team has long published, also when the team's
-// blocks sit on both dies and every step of the hand-over is a slow round trip.
+// runs A(i), B(i - ST_LAG) for i = 0, 1, ..: a chunk's second visit comes one round after
+// its first, when every block of its team has published (a longer lag pushes the chunk out
+// of the L2 cache before its second visit).
 // The wait for M' is bounded like every other wait (tc_common.cuh).
 //
 // Block = 20 warps: warp 0 TMA producer (K tiles through a 4-stage ring, asked into L2 one
 // round ahead; Q of a pass is loaded while the pass before it runs, into the buffer of its
 // kind: one for the statistics passes, one for the pooling passes, which read Q again),
-// warp 1 MMA issuer (accumulators in a 4-deep ring of 128 tensor-memory columns),
+// warps 1 and 19 MMA issuers, alternate tiles (accumulators in a 4-deep ring of 128 tensor-memory columns),
 // warps 2..17 consumers: warp (quarter, part) reads lanes [32*quarter, +32) and columns
 // [32*part, +32) of every accumulator tile, which frees the tile as soon as the 16 warps
-// have it in registers; warp 18 publishes the chunk statistics the consumers leave in shared
-// memory and folds a head's chunks when its block is the last to arrive; warp 19 fetches M'
-// for the coming pooling passes as early as its two buffers allow, so that the consumers
-// never wait for global memory.
+// have it in registers; warp 18 is the messenger: it publishes the chunk statistics the
+// consumers leave in shared memory, folds a head's chunks when its block is the last to
+// arrive, and then fetches the head's M' for the pooling pass a round later, so that the
+// consumers never wait for global memory.
 #pragma once
 
 #include "tc_common.cuh"
@@ -45,7 +45,7 @@ constexpr int ST_TILES = 4;                         // 128-key tiles per chunk
 constexpr int ST_CHUNK = ST_TILES * 128;
 constexpr int ST_STAGES = 4;                        // K tiles in flight in shared memory
 constexpr int ST_TBUF = 4;                          // accumulator tiles in tensor memory
-constexpr int ST_LAG = 2;                           // rounds between a chunk's statistics pass and its pooling pass
+constexpr int ST_LAG = 1;                           // rounds between a chunk's statistics pass and its pooling pass
 constexpr int ST_TILE_BYTES = 128 * 128 * 2;
 constexpr int ST_CONSUMERS = 512;
 constexpr int ST_THREADS = 64 + ST_CONSUMERS + 64;
@@ -195,7 +195,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
 
     if (tid == 0) {
         s_abort = 0u;
-        for (int b = 0; b < 2; ++b) { tc::mbar_init(&bar_q_full[b], 1); tc::mbar_init(&bar_q_free[b], 1); }
+        for (int b = 0; b < 2; ++b) { tc::mbar_init(&bar_q_full[b], 1); tc::mbar_init(&bar_q_free[b], 2); }
         for (int s = 0; s < ST_STAGES; ++s) tc::mbar_init(&bar_full[s], 1);
         for (int s = 0; s < ST_TBUF; ++s) {
             tc::mbar_init(&bar_t_full[s], 1);
@@ -285,13 +285,16 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
             for (int b = 0; b < 2; ++b)
                 if (nq[b] > 0) tc::mbar_wait(&bar_q_full[b], (nq[b] - 1) & 1u, wc, 64);
         }
-    } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
+    } else if (warp == 1 || warp == ST_THREADS / 32 - 1) {
+        // ---------------- MMA issuers: two threads, alternate tiles ----------------
+        // What an issuer does for a tile (two barrier tests, eight instructions that each hold the thread
+        // for about 100 cycles, a commit) takes longer than the tensor cores need for the tile; two
+        // issuers on separate warps overlap that.  Tiles are independent: different accumulators and ring
+        // stages, and a commit only covers its own thread's instructions.
         if (lane == 0) {
             constexpr uint32_t IDESC = tc::idesc_bf16(128, 128, 0, 0);
-            uint32_t nq[2] = {0u, 0u};
-            // ring stage / accumulator tile of the next tile (same index), with the parity of its current use
-            uint32_t tb = 0, tb_par = 0;
+            const uint32_t me = warp == 1 ? 0u : 1u;
+            uint32_t it = 0, nq[2] = {0u, 0u};
             const uint32_t ring_addr = tc::smem_u32(ring);
             bool dead = false;
             PassIter pi;
@@ -302,12 +305,18 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                 ++nq[kind];
                 // operand descriptors: the k-step only moves the start address (in 16-byte units, low word)
                 const uint64_t dq0 = tc::smem_desc_sw128(tc::smem_u32(q_s + kind * ST_TILE_BYTES), 16, 1024);
+                bool issued = false;
                 for (int t = 0; t < item.nt; ++t) {
-                    if (!tc::mbar_wait(&bar_t_empty[tb], tb_par ^ 1u, wc)) { dead = true; break; }
-                    if (!tc::mbar_wait(&bar_full[tb], tb_par, wc)) { dead = true; break; }
+                    const uint32_t ti = it + t;
+                    if ((ti & 1u) != me) continue;
+                    // accumulator tile and ring stage share their index and the parity of their use
+                    const uint32_t tb = ti % ST_TBUF, par = (ti / ST_TBUF) & 1u;
+                    const bool e_ok = tc::mbar_test(&bar_t_empty[tb], par ^ 1u), f_ok = tc::mbar_test(&bar_full[tb], par);
+                    if (!e_ok && !tc::mbar_wait(&bar_t_empty[tb], par ^ 1u, wc)) { dead = true; break; }
+                    if (!f_ok && !tc::mbar_wait(&bar_full[tb], par, wc)) { dead = true; break; }
                     tc::tc_fence_after();
                     const uint64_t dk0 = tc::smem_desc_sw128(ring_addr + tb * ST_TILE_BYTES, 16, 1024);
-                    const uint32_t acc = tmem + (uint32_t)(tb * 128);
+                    const uint32_t acc = tmem + tb * 128u;
                     // pass A: queries on the lanes (S = Q K^T); pass B: keys on the lanes (S^T = K Q^T)
                     const uint64_t da0 = kind == 0 ? dq0 : dk0, db0 = kind == 0 ? dk0 : dq0;
 #pragma unroll
@@ -318,9 +327,14 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                         tc::umma_bf16(acc, da0 + off16, db0 + off16, IDESC, kk > 0 ? 1u : 0u);
                     }
                     tc::umma_commit(&bar_t_full[tb]);
-                    if (++tb == ST_TBUF) { tb = 0; tb_par ^= 1u; }
+                    issued = true;
                 }
-                if (!dead) tc::umma_commit(&bar_q_free[kind]);
+                it += item.nt;
+                // the Q buffer is free when both issuers' instructions of the pass are done
+                if (!dead) {
+                    if (issued) tc::umma_commit(&bar_q_free[kind]);
+                    else tc::mbar_arrive(&bar_q_free[kind]);
+                }
             }
         }
     } else if (warp < 2 + ST_CONSUMERS / 32) {
@@ -446,9 +460,9 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
             }
         }
         if (pend) finish_pool();
-    } else if (warp == 2 + ST_CONSUMERS / 32) {
-        // ---------------- publisher: chunk statistics out, a head's chunks folded by the last block to arrive ----------------
-        uint32_t n_a[2] = {0u, 0u};
+    } else {
+        // ---------------- messenger: chunk statistics out, a head's chunks folded by the last block to arrive, M' in ----------------
+        uint32_t n_a[2] = {0u, 0u}, n_b[2] = {0u, 0u};
         for (int i = 0; i < R; ++i) {
             ScoreItem item;
             if (!score_item(p, s_tab, i, item)) continue;
@@ -520,48 +534,43 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                     st_relaxed_gpu_u64(words + t, (1ull << 32) | __float_as_uint(mp));
                 }
             }
-        }
-    } else {
-        // ---------------- fetcher: M' of the heads to be pooled, into shared memory as early as the buffers allow ----------------
-        uint32_t n_b[2] = {0u, 0u};
-        for (int r = 0; r < R; ++r) {
-            ScoreItem item;
-            if (!score_item(p, s_tab, r, item)) continue;
-            const int buf = r & 1;
-            const int g = p.c[item.cache].head_base + item.lh;
-            if (n_b[buf] > 0) tc::mbar_wait(&bar_mp_free[buf], (n_b[buf] - 1) & 1u, wc, 32);
-            const unsigned long long *words = reinterpret_cast<const unsigned long long *>(p.sc_head) + (size_t)g * 128;
-            // the four words of this lane are polled together: one round trip, not four
-            unsigned long long v[4] = {0ull, 0ull, 0ull, 0ull};
-            const uint64_t t0 = tc::global_ns();
-            for (;;) {
-                bool all = true;
+            // M'_t of this head for the pooling pass one round on; the team has a round to get there
+            {
+                const int fb = i & 1;
+                if (n_b[fb] > 0) tc::mbar_wait(&bar_mp_free[fb], (n_b[fb] - 1) & 1u, wc, 32);
+                const unsigned long long *words = reinterpret_cast<const unsigned long long *>(p.sc_head) + (size_t)g * 128;
+                // the four words of this lane are polled together: one round trip, not four
+                unsigned long long v[4] = {0ull, 0ull, 0ull, 0ull};
+                const uint64_t t0 = tc::global_ns();
+                for (;;) {
+                    bool all = true;
 #pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    if (lane + 32 * k < p.n_q && (v[k] >> 32) == 0ull) v[k] = ld_relaxed_gpu_u64(words + lane + 32 * k);
+                    for (int k = 0; k < 4; ++k)
+                        if (lane + 32 * k < p.n_q && (v[k] >> 32) == 0ull) v[k] = ld_relaxed_gpu_u64(words + lane + 32 * k);
 #pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    if (lane + 32 * k < p.n_q && (v[k] >> 32) == 0ull) all = false;
-                // the warp leaves the loop as one: votes, not per-lane exits
-                if (__all_sync(0xffffffffu, all) || __any_sync(0xffffffffu, *(volatile uint32_t *)&s_abort != 0u)) break;
-                if (__any_sync(0xffffffffu, tc::global_ns() - t0 > tc::WAIT_LIMIT_NS)) {
-                    if (lane == 0) {
-                        s_abort = 1u;
-                        atomicOr(p.status, OBF_DEV_TIMEOUT);
+                    for (int k = 0; k < 4; ++k)
+                        if (lane + 32 * k < p.n_q && (v[k] >> 32) == 0ull) all = false;
+                    // the warp leaves the loop as one: votes, not per-lane exits
+                    if (__all_sync(0xffffffffu, all) || __any_sync(0xffffffffu, *(volatile uint32_t *)&s_abort != 0u)) break;
+                    if (__any_sync(0xffffffffu, tc::global_ns() - t0 > tc::WAIT_LIMIT_NS)) {
+                        if (lane == 0) {
+                            s_abort = 1u;
+                            atomicOr(p.status, OBF_DEV_TIMEOUT);
+                        }
+                        break;
                     }
-                    break;
+                    __nanosleep(64);
                 }
-                __nanosleep(64);
-            }
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const int t = lane + 32 * k;
-                // exp2(-inf) = 0 for padding columns
-                s_mp[buf * 128 + t] = t < p.n_q ? __uint_as_float((uint32_t)v[k]) : INFINITY;
+                for (int k = 0; k < 4; ++k) {
+                    const int t = lane + 32 * k;
+                    // exp2(-inf) = 0 for padding columns
+                    s_mp[fb * 128 + t] = t < p.n_q ? __uint_as_float((uint32_t)v[k]) : INFINITY;
+                }
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(&bar_mp_ready[fb]);
+                ++n_b[fb];
             }
-            __syncwarp();
-            if (lane == 0) tc::mbar_arrive(&bar_mp_ready[buf]);
-            ++n_b[buf];
         }
     }
 

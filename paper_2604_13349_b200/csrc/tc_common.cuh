@@ -56,6 +56,16 @@ __device__ __forceinline__ bool mbar_try(uint64_t *bar, uint32_t parity, uint32_
     return ok != 0;
 }
 
+// Non-blocking test of the phase with the given parity.  Two of these issued back to back overlap
+// their latency, which a pair of parked tests does not.
+__device__ __forceinline__ bool mbar_test(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+
 // What a block shares to give up cleanly: the abort flag lives in shared memory,
 // the status word in the workspace.
 struct WaitCtx {
