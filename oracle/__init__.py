@@ -70,6 +70,11 @@ def lib():
         _lib.obf_oracle_compress.argtypes = [fp, fp, fp, ci, ci, ci, ci, ci, ci, ci, ci,
                                              ctypes.c_double, ip, dp, dp, dp, ctypes.POINTER(Diag)]
         _lib.obf_oracle_compress.restype = ci
+        _lib.obf_oracle_layer.argtypes = [fp, fp, fp, ci, ci, ci, ci, ci, ci, ctypes.c_double,
+                                          ip, dp, dp, dp, dp, dp, ctypes.POINTER(Diag)]
+        _lib.obf_oracle_layer.restype = ci
+        _lib.obf_oracle_compress_layerwise.argtypes = _lib.obf_oracle_compress.argtypes
+        _lib.obf_oracle_compress_layerwise.restype = ci
         _lib.obf_oracle_num_threads.argtypes = []
         _lib.obf_oracle_num_threads.restype = ci
     return _lib
@@ -159,9 +164,38 @@ def head(K, V, Q, budget: int, rank: int, eps: float = 1e-12) -> Dict[str, objec
             "rbar": rbar, "Delta": Delta, "eigvals": eig, "proj": proj, "diag": dg.asdict()}
 
 
+def layer(K, V, Q, budget: int, rank: int, eps: float = 1e-12) -> Dict[str, object]:
+    """Layerwise selector (Algorithm 2, granularity L) + Algorithm 3 on one layer.
+
+    K, V [kv_heads,T,d]; Q [kv_heads,n_q,d].  The retained positions are TopK_B of the masses summed over
+    the KV heads and are shared by the heads; the back-fill runs per head with the head's own masses.
+    Returns idx [kv_heads,k], K_out, V_out (float64), S (summed masses), A [kv_heads,T], delta, diag (per head).
+    """
+    K, V, Q = _f32(K), _f32(V), _f32(Q)
+    H, T, d = K.shape
+    k = min(budget, T)
+    idx = np.empty((H, max(k, 1)), dtype=np.int32)
+    K_out = np.zeros((H, max(k, 1), d), dtype=np.float64)
+    V_out = np.zeros((H, max(k, 1), d), dtype=np.float64)
+    S = np.empty(T, dtype=np.float64)
+    A = np.empty((H, T), dtype=np.float64)
+    delta = np.zeros((H, d), dtype=np.float64)
+    diags = (Diag * H)()
+    cd = ctypes.c_double
+    k2 = lib().obf_oracle_layer(
+        _p(K, ctypes.c_float), _p(V, ctypes.c_float), _p(Q, ctypes.c_float),
+        H, T, d, Q.shape[1], budget, rank, eps,
+        _p(idx, ctypes.c_int32), _p(K_out, cd), _p(V_out, cd), _p(S, cd), _p(A, cd), _p(delta, cd), diags)
+    assert k2 == k
+    return {"idx": idx[:, :k].copy(), "K_out": K_out[:, :k], "V_out": V_out[:, :k], "S": S, "A": A,
+            "delta": delta, "diag": [diags[h].asdict() for h in range(H)]}
+
+
 def compress(K, V, Q, q_heads: int, n_obs: int, budget: int, rank: int,
-             eps: float = 1e-12) -> Dict[str, object]:
-    """A whole cache: K, V [layers, kv_heads, T, d]; Q [layers, q_heads, n_obs, d]."""
+             eps: float = 1e-12, layerwise: bool = False) -> Dict[str, object]:
+    """A whole cache: K, V [layers, kv_heads, T, d]; Q [layers, q_heads, n_obs, d].
+
+    layerwise: one retained set per layer (masses summed over its KV heads) instead of one per head."""
     K, V, Q = _f32(K), _f32(V), _f32(Q)
     layers, kv_heads, T, d = K.shape
     k = min(budget, T)
@@ -172,7 +206,8 @@ def compress(K, V, Q, q_heads: int, n_obs: int, budget: int, rank: int,
     delta = np.zeros((layers, kv_heads, d), dtype=np.float64)
     diags = (Diag * heads)()
     cd = ctypes.c_double
-    lib().obf_oracle_compress(
+    fn = lib().obf_oracle_compress_layerwise if layerwise else lib().obf_oracle_compress
+    fn(
         _p(K, ctypes.c_float), _p(V, ctypes.c_float), _p(Q, ctypes.c_float),
         layers, kv_heads, q_heads, n_obs, T, d, budget, rank, eps,
         _p(idx, ctypes.c_int32), _p(K_out, cd), _p(V_out, cd), _p(delta, cd), diags)

@@ -1,6 +1,6 @@
 /*
- * CPU oracle for relay-boundary prompt-KV compression: headwise attention-mass
- * eviction followed by Orthogonal BackFill (OBF).
+ * CPU oracle for relay-boundary prompt-KV compression: headwise (or layerwise)
+ * attention-mass eviction followed by Orthogonal BackFill (OBF).
  *
  * THIS IS TEST INFRASTRUCTURE, NOT THE PRODUCT.  It is a plain, slow, fp64,
  * step-by-step statement of the paper's definitions (Eq. 1-7, Algorithms 2-3),
@@ -16,6 +16,9 @@
  *               closed form, library softmax, permutation equivariance
  *   top-k       pinned: brute-force full sort on tiny inputs, library stable
  *               argsort, planted exact ties
+ *   layerwise   pinned: one KV head reduces to the headwise result, identical
+ *               heads reduce to the headwise result, library argsort of the
+ *               summed masses, retained set shared by the heads of a layer
  *   gather      pinned: bitwise copies
  *   span basis  pinned: orthonormality, annihilation of V_keep, library
  *               pseudo-inverse projector, library matrix rank
@@ -261,23 +264,52 @@ void obf_oracle_sym_eig(double *S, int n, double *lam, double *E)
  * proj [d*d] (C^T C, the projector onto the residual principal subspace), diag.
  * Returns k_eff.
  */
+static int backfill_given_selection(const float *K, const float *V, const double *A_in,
+                                    int T, int d, int k, int rank, double eps,
+                                    const int32_t *idx, double kth_score, double next_score,
+                                    double *K_out, double *V_out,
+                                    double *delta_out, double *rbar_out, double *Delta_out,
+                                    double *eigvals_out, double *proj_out, obf_oracle_diag_t *diag);
+
 int obf_oracle_head(const float *K, const float *V, const float *Q,
                     int T, int d, int n_q, int budget, int rank, double eps,
                     int32_t *idx, double *K_out, double *V_out,
                     double *A_out, double *delta_out, double *rbar_out, double *Delta_out,
                     double *eigvals_out, double *proj_out, obf_oracle_diag_t *diag)
 {
-    obf_oracle_diag_t dg;
-    memset(&dg, 0, sizeof(dg));
-    dg.next_score = -1.0;
-
     /* O1: attention mass */
     double *A = (double *)malloc((size_t)T * sizeof(double));
     obf_oracle_scores(K, Q, T, d, n_q, A);
     if (A_out) memcpy(A_out, A, (size_t)T * sizeof(double));
 
     /* O2: headwise TopK_B, ascending index list */
-    int k = obf_oracle_topk(A, T, budget, idx, &dg.kth_score, &dg.next_score);
+    double kth = 0.0, next = -1.0;
+    int k = obf_oracle_topk(A, T, budget, idx, &kth, &next);
+
+    backfill_given_selection(K, V, A, T, d, k, rank, eps, idx, kth, next, K_out, V_out,
+                             delta_out, rbar_out, Delta_out, eigvals_out, proj_out, diag);
+    free(A);
+    return k;
+}
+
+/*
+ * Everything after the selection (last step of Algorithm 2, then Algorithm 3) for one (layer, KV head):
+ * A_in are this head's own attention masses, idx the k retained positions (ascending), whichever
+ * granularity chose them.  kth_score / next_score are passed through to the diagnostics.
+ */
+static int backfill_given_selection(const float *K, const float *V, const double *A_in,
+                                    int T, int d, int k, int rank, double eps,
+                                    const int32_t *idx, double kth_score, double next_score,
+                                    double *K_out, double *V_out,
+                                    double *delta_out, double *rbar_out, double *Delta_out,
+                                    double *eigvals_out, double *proj_out, obf_oracle_diag_t *diag)
+{
+    obf_oracle_diag_t dg;
+    memset(&dg, 0, sizeof(dg));
+    dg.kth_score = kth_score;
+    dg.next_score = next_score;
+    double *A = (double *)malloc((size_t)T * sizeof(double));
+    memcpy(A, A_in, (size_t)T * sizeof(double));
 
     /* O3: gather (Algorithm 2, last step) */
     for (int r = 0; r < k; ++r)
@@ -434,6 +466,66 @@ int obf_oracle_compress(const float *K, const float *V, const float *Q,
                         K_out + (size_t)lh * k * d, V_out + (size_t)lh * k * d,
                         NULL, delta_out ? delta_out + (size_t)lh * d : NULL, NULL, NULL, NULL, NULL,
                         diag_out ? diag_out + lh : NULL);
+    }
+    return k;
+}
+
+/* ------------------------------------------------------------------ */
+/* Layerwise granularity (Algorithm 2, granularity L) + Algorithm 3     */
+/* ------------------------------------------------------------------ */
+/*
+ * One layer: K, V [kv_heads, T, d]; Q [kv_heads, n_q, d].  The retained set is
+ * TopK_B of the masses summed over the layer's KV heads (retention rule of
+ * Section 3.2, second form) and is shared by all heads of the layer; the gather
+ * and Orthogonal BackFill then run per head with that head's own masses
+ * (Eq. 4 and Eq. 6 are written per (l, h)).  Outputs are [kv_heads, k_eff, ...];
+ * S_out (may be NULL) receives the T summed masses, A_out (may be NULL) the
+ * [kv_heads, T] per-head masses.  Returns k_eff.
+ */
+int obf_oracle_layer(const float *K, const float *V, const float *Q,
+                     int kv_heads, int T, int d, int n_q, int budget, int rank, double eps,
+                     int32_t *idx_out, double *K_out, double *V_out,
+                     double *S_out, double *A_out, double *delta_out, obf_oracle_diag_t *diag_out)
+{
+    double *A = (double *)malloc((size_t)kv_heads * T * sizeof(double));
+    double *S = (double *)calloc((size_t)T, sizeof(double));
+    for (int h = 0; h < kv_heads; ++h) {
+        obf_oracle_scores(K + (size_t)h * T * d, Q + (size_t)h * n_q * d, T, d, n_q, A + (size_t)h * T);
+        for (int j = 0; j < T; ++j) S[j] += A[(size_t)h * T + j];
+    }
+    if (S_out) memcpy(S_out, S, (size_t)T * sizeof(double));
+    if (A_out) memcpy(A_out, A, (size_t)kv_heads * T * sizeof(double));
+    const int kmax = budget < T ? budget : T;
+    int32_t *idx = (int32_t *)malloc((size_t)(kmax > 0 ? kmax : 1) * sizeof(int32_t));
+    double kth = 0.0, next = -1.0;
+    const int k = obf_oracle_topk(S, T, budget, idx, &kth, &next);
+    for (int h = 0; h < kv_heads; ++h) {
+        memcpy(idx_out + (size_t)h * k, idx, (size_t)k * sizeof(int32_t));
+        backfill_given_selection(K + (size_t)h * T * d, V + (size_t)h * T * d, A + (size_t)h * T, T, d, k, rank, eps,
+                                 idx, kth, next, K_out + (size_t)h * k * d, V_out + (size_t)h * k * d,
+                                 delta_out ? delta_out + (size_t)h * d : NULL, NULL, NULL, NULL, NULL,
+                                 diag_out ? diag_out + h : NULL);
+    }
+    free(idx); free(S); free(A);
+    return k;
+}
+
+/* A whole cache with the layerwise selector; arrays as in obf_oracle_compress. */
+int obf_oracle_compress_layerwise(const float *K, const float *V, const float *Q,
+                                  int layers, int kv_heads, int q_heads, int n_obs, int T, int d,
+                                  int budget, int rank, double eps,
+                                  int32_t *idx_out, double *K_out, double *V_out,
+                                  double *delta_out, obf_oracle_diag_t *diag_out)
+{
+    const int G = q_heads / kv_heads;
+    const int n_q = G * n_obs;
+    const int k = budget < T ? budget : T;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int l = 0; l < layers; ++l) {
+        const size_t lh = (size_t)l * kv_heads;
+        obf_oracle_layer(K + lh * T * d, V + lh * T * d, Q + lh * n_q * d, kv_heads, T, d, n_q, budget, rank, eps,
+                         idx_out + lh * k, K_out + lh * k * d, V_out + lh * k * d, NULL, NULL,
+                         delta_out ? delta_out + lh * d : NULL, diag_out ? diag_out + lh : NULL);
     }
     return k;
 }

@@ -388,3 +388,104 @@ def test_c1_whole_cache_matches_lapack_pipeline_per_head():
         # the planted heavy hitters must be among the retained positions
         k1, _, _ = synth.gen_head(w, 0, 0, h)
         assert np.array_equal(k1, arr["K"][0, h])
+
+
+# --------------------------------------------------------------------------
+# layerwise selector (retention rule, second form; Algorithm 2 with granularity L)
+# --------------------------------------------------------------------------
+def lib_obf_given_idx(V, A, idx, rank, eps=1e-12):
+    """Algorithm 3 through LAPACK routines for a retained set chosen elsewhere."""
+    T = V.shape[0]
+    keep = np.zeros(T, bool); keep[idx] = True
+    Vd = V.astype(np.float64)
+    Vk, Vdel = Vd[keep], Vd[~keep]
+    if rank <= 0 or Vdel.shape[0] == 0:
+        return np.zeros(V.shape[1]), Vk
+    R = Vdel - Vdel @ (np.linalg.pinv(Vk) @ Vk)
+    if (R ** 2).sum() <= 1e-12 * (Vdel ** 2).sum():
+        return np.zeros(V.shape[1]), Vk
+    _, s, Vt = np.linalg.svd(R, full_matrices=False)
+    rho = min(rank, int((s ** 2 > V.shape[1] * np.finfo(float).eps * s[0] ** 2).sum()))
+    C = Vt[:rho]
+    a_del, a_keep = A[~keep].sum(), A[keep].sum()
+    rbar = (A[~keep] / (a_del + eps)) @ R
+    delta = a_del / (a_keep + eps) * ((rbar @ C.T) @ C)
+    return delta, Vk + delta
+
+
+def rand_layer(seed, H, T, d, n_q):
+    g = np.random.default_rng(seed)
+    K = g.standard_normal((H, T, d)).astype(np.float32)
+    V = g.standard_normal((H, T, d)).astype(np.float32)
+    Q = g.standard_normal((H, n_q, d)).astype(np.float32)
+    K[:, g.choice(T, 3, replace=False)] *= 3.0
+    return K, V, Q
+
+
+@pytest.mark.parametrize("seed,H,T,d,n_q,budget,rank", [(0, 2, 48, 16, 4, 6, 1), (1, 4, 96, 32, 8, 12, 2),
+                                                         (2, 3, 40, 8, 4, 40, 2), (3, 8, 64, 16, 8, 5, 4)])
+def test_layerwise_selects_on_summed_masses_and_backfills_per_head(seed, H, T, d, n_q, budget, rank):
+    K, V, Q = rand_layer(seed, H, T, d, n_q)
+    out = oracle.layer(K, V, Q, budget, rank)
+    A = np.stack([lib_scores(K[h], Q[h]) for h in range(H)])
+    S = A.sum(axis=0)
+    np.testing.assert_allclose(out["S"], S, rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(out["A"], A, rtol=1e-12, atol=1e-15)
+    want = brute_topk(S, budget)                                # brute force over the summed masses
+    assert np.array_equal(want, np.sort(np.argsort(-S, kind="stable")[:min(budget, T)]))
+    for h in range(H):
+        assert np.array_equal(out["idx"][h], want)              # one set, shared by the heads of the layer
+        assert np.array_equal(out["K_out"][h], K[h][want].astype(np.float64))
+        delta, v_out = lib_obf_given_idx(V[h], A[h], want, rank)
+        scale = max(1.0, np.abs(delta).max())
+        np.testing.assert_allclose(out["delta"][h], delta, atol=1e-9 * scale)
+        np.testing.assert_allclose(out["V_out"][h], v_out, atol=1e-9 * scale)
+        dg = out["diag"][h]
+        keep = np.zeros(T, bool); keep[want] = True
+        assert dg["a_keep"] == pytest.approx(A[h][keep].sum(), rel=1e-12)     # the head's own masses (Eq. 6)
+        assert dg["a_del"] == pytest.approx(A[h][~keep].sum(), rel=1e-12, abs=1e-300)
+
+
+def test_layerwise_with_one_kv_head_is_the_headwise_result():
+    K, V, Q = rand_layer(7, 1, 80, 16, 6)
+    lay = oracle.layer(K, V, Q, 9, 2)
+    hd = oracle.head(K[0], V[0], Q[0], 9, 2)
+    assert np.array_equal(lay["idx"][0], hd["idx"])
+    assert np.array_equal(lay["V_out"][0], hd["V_out"])
+    assert np.array_equal(lay["delta"][0], hd["delta"])
+
+
+def test_layerwise_with_identical_heads_is_the_headwise_result():
+    K1, V1, Q1 = rand_layer(8, 1, 72, 16, 6)
+    K, V, Q = np.repeat(K1, 4, 0), np.repeat(V1, 4, 0), np.repeat(Q1, 4, 0)
+    lay = oracle.layer(K, V, Q, 10, 1)
+    hd = oracle.head(K1[0], V1[0], Q1[0], 10, 1)
+    for h in range(4):
+        assert np.array_equal(lay["idx"][h], hd["idx"])          # summing equal masses keeps their order
+        np.testing.assert_allclose(lay["V_out"][h], hd["V_out"], atol=1e-12)
+
+
+def test_layerwise_differs_from_headwise_when_heads_disagree():
+    # two heads whose heavy keys sit at different positions: headwise keeps each head's own, layerwise the union's top
+    g = np.random.default_rng(11)
+    H, T, d = 2, 32, 8
+    K = 0.01 * g.standard_normal((H, T, d)).astype(np.float32)
+    V = g.standard_normal((H, T, d)).astype(np.float32)
+    Q = np.ones((H, 2, d), np.float32)
+    K[0, 3] = 4.0; K[1, 20] = 4.0; K[0, 9] = 2.0; K[1, 9] = 2.0
+    lay = oracle.layer(K, V, Q, 2, 0)
+    assert oracle.head(K[0], V[0], Q[0], 2, 0)["idx"].tolist() == [3, 9]
+    assert oracle.head(K[1], V[1], Q[1], 2, 0)["idx"].tolist() == [9, 20]
+    assert lay["idx"][0].tolist() == lay["idx"][1].tolist() == [3, 20]       # 3 and 20 each carry one head's top mass
+
+
+def test_layerwise_whole_cache_matches_per_layer_calls():
+    w = synth.workload("c1")
+    a = synth.gen_cache(w, 0)
+    d, n_q = w.head.head_dim, w.n_q
+    out = oracle.compress(a["K"], a["V"], a["Q"], w.q_heads, w.n_obs, w.caches[0].budget, w.rank, layerwise=True)
+    Qv = a["Q"].reshape(w.layers, w.kv_heads, n_q, d)
+    for l in range(w.layers):
+        lay = oracle.layer(a["K"][l], a["V"][l], Qv[l], w.caches[0].budget, w.rank)
+        assert np.array_equal(out["idx"][l], lay["idx"])
+        assert np.array_equal(out["V_out"][l], lay["V_out"])
