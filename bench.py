@@ -106,7 +106,7 @@ def cpu_baseline(w, arrays0, seconds_target: float = 15.0):
         l = layers_done
         k, v, q = conv(K[l:l + 1]), conv(V[l:l + 1]), conv(Q[l:l + 1])
         t0 = time.perf_counter()
-        oracle.compress(k, v, q, w.q_heads, w.n_obs, w.caches[0].budget, w.rank)
+        oracle.compress(k, v, q, w.q_heads, w.n_obs, w.caches[0].budget, w.rank, layerwise=w.layerwise)
         t_total += time.perf_counter() - t0
         layers_done += 1
     gbs = per_layer_bytes * layers_done / t_total / 1e9
@@ -134,10 +134,10 @@ def run_reference(args):
     step_bytes = w.kv_heads * (2 * T * w.head.head_dim * w.elem_bytes + w.n_q * w.head.head_dim * w.elem_bytes
                                + 2 * ke * w.head.head_dim * w.elem_bytes + 4 * ke)
     for _ in range(args.warmup):
-        oracle.compress(k, v, q, w.q_heads, w.n_obs, w.caches[0].budget, w.rank)
+        oracle.compress(k, v, q, w.q_heads, w.n_obs, w.caches[0].budget, w.rank, layerwise=w.layerwise)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        oracle.compress(k, v, q, w.q_heads, w.n_obs, w.caches[0].budget, w.rank)
+        oracle.compress(k, v, q, w.q_heads, w.n_obs, w.caches[0].budget, w.rank, layerwise=w.layerwise)
     dt = time.perf_counter() - t0
     val = step_bytes * args.steps / dt / 1e9
     sample = "each step = layer 0 of cache 0 of %s (%d heads, T=%d)" % (w.name, w.kv_heads, T)
@@ -184,7 +184,8 @@ def main():
 
     w = synth.workload(args.workload)
     params = P.make_params(w.layers, w.kv_heads, w.q_heads, w.head.head_dim, w.n_obs, w.rank,
-                           P.OBF_F32 if w.dtype == "f32" else P.OBF_BF16, 1e-12, 0)
+                           P.OBF_F32 if w.dtype == "f32" else P.OBF_BF16, 1e-12,
+                           P.binding.OBF_FLAG_LAYERWISE if w.layerwise else 0)
     tdt = torch.float32 if w.dtype == "f32" else torch.bfloat16
 
     def as_t(a):
@@ -321,7 +322,7 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": w.name, "layers": w.layers, "kv_heads": w.kv_heads, "q_heads": w.q_heads,
-                       "head_dim": d, "n_obs": w.n_obs, "rank": w.rank,
+                       "head_dim": d, "n_obs": w.n_obs, "rank": w.rank, "selector": "layerwise" if w.layerwise else "headwise",
                        "T": [c.T for c in w.caches], "budget": [c.budget for c in w.caches],
                        "l2": "inputs_larger_than_l2" if 2 * kv_bytes > 126e6 else "inputs_fit_l2",
                        "parallelism": "replicas" if world > 1 else "single_gpu"},

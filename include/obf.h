@@ -75,6 +75,11 @@ typedef enum { OBF_F32 = 0, OBF_BF16 = 1 } obf_dtype_t;
 
 /* obf_params_t.flags */
 #define OBF_FLAG_GENERIC_PATH 0x1u /* run the shape-generic kernels even where the tuned bf16 path applies */
+#define OBF_FLAG_LAYERWISE    0x2u /* layerwise selector (Section 3.2 retention rule, second form; Algorithm 2,
+                                      granularity L): the retained positions of a layer are TopK_B of the masses
+                                      summed over its KV heads and are shared by those heads (idx_out repeats them
+                                      per head); gather and OBF then run per head with the head's own masses.
+                                      Needs every T <= 16384, else OBF_ERR_UNSUPPORTED                          */
 
 #define OBF_MAX_CACHES 32          /* caches per call                                              */
 #define OBF_MAX_T (1 << 20)        /* prompt positions per cache                                   */

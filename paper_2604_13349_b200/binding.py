@@ -33,6 +33,7 @@ OBF_DEV_SKIPPED = 0x100
 OBF_DEV_SPAN_FULL = 0x200
 
 OBF_FLAG_GENERIC_PATH = 0x1
+OBF_FLAG_LAYERWISE = 0x2        # one retained set per layer (masses summed over its KV heads)
 OBF_MAX_CACHES = 32
 
 EXPORTS = ("obf_workspace_bytes", "obf_compress", "evict_only", "obf_host_arena_bytes",

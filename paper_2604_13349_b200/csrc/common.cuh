@@ -62,9 +62,12 @@ struct CallDev {
     float *sc_head;           // per (head, query of 128): one 64-bit word, low = M + log2(Z) over all keys, high = 1 when valid
     uint32_t *sc_cnt;         // per head: chunks that have published
     float eps;
+    int32_t kv_heads;         // KV heads per layer
+    int32_t layerwise;        // 1: one retained set per layer (masses summed over its KV heads)
     // workspace
     uint32_t *status;
     float *scores;            // [sum heads*T] attention mass (Eq. 1)
+    float *lscores;           // layerwise selector: [sum layers*T] masses summed over a layer's KV heads (cache offset tok_off / kv_heads)
     uint8_t *keep;            // [sum heads*T] 1 = retained
     float *stats;             // [heads_total, n_q, 2] softmax row max (log2 domain) and normaliser
     float *sums;              // [heads_total, 4] a_keep, a_del, kth, next

@@ -274,7 +274,24 @@ __global__ void __launch_bounds__(SEL_NT) k_select(const __grid_constant__ CallD
 // block-wide barriers suffice.
 constexpr int SEL_SMEM_MAX_T = 16384;
 
-template <int NT>
+// Layerwise selector, first half (Section 3.2, retention rule, second form): the masses of a layer's KV heads
+// added up per position, head 0 first.  grid = (ceil(T_max / 256), layers of all caches).
+__global__ void __launch_bounds__(256) k_layer_sum(const __grid_constant__ CallDev p)
+{
+    int ci, lh;
+    locate(p, blockIdx.y * p.kv_heads, ci, lh);
+    const CacheDev &c = p.c[ci];
+    const int j = blockIdx.x * 256 + threadIdx.x;
+    if (j >= c.T) return;
+    const float *A = p.scores + c.tok_off + (size_t)lh * c.T + j;
+    float s = 0.f;
+    for (int h = 0; h < p.kv_heads; ++h) s += A[(size_t)h * c.T];
+    p.lscores[c.tok_off / p.kv_heads + (size_t)(lh / p.kv_heads) * c.T + j] = s;
+}
+
+// With LAYER the block is a layer: it selects on the layer's summed masses and then writes the shared
+// positions, the keep flags and the demand sums (of the head's own masses) for each of the layer's heads.
+template <int NT, bool LAYER = false>
 __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ CallDev p)
 {
     extern __shared__ uint32_t sel_keys[];
@@ -284,11 +301,12 @@ __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ Call
     __shared__ uint32_t wtot[32];
     __shared__ float red[32];
     int ci, lh;
-    locate(p, blockIdx.x, ci, lh);
+    locate(p, LAYER ? blockIdx.x * p.kv_heads : blockIdx.x, ci, lh);      // LAYER: lh is the layer's first head
     const CacheDev &c = p.c[ci];
     const int T = c.T, k = c.k_eff;
     float *Af = p.scores + c.tok_off + (size_t)lh * T;
-    const uint32_t *A = reinterpret_cast<const uint32_t *>(Af);
+    const uint32_t *A = LAYER ? reinterpret_cast<const uint32_t *>(p.lscores + c.tok_off / p.kv_heads + (size_t)(lh / p.kv_heads) * T)
+                              : reinterpret_cast<const uint32_t *>(Af);
     uint8_t *keep = p.keep + c.tok_off + (size_t)lh * T;
     int32_t *idx = c.idx_out + (size_t)lh * k;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -379,7 +397,14 @@ __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ Call
         const uint32_t m_gt = __ballot_sync(0xffffffffu, gt), m_eq = __ballot_sync(0xffffffffu, eq);
         const uint32_t gt_before = run_gt + __popc(m_gt & lt_mask), eq_before = run_eq + __popc(m_eq & lt_mask);
         const bool kp = gt || (eq && eq_before < want);
-        if (valid) {
+        if (LAYER) {
+            // the verdict of a position, kept for the per-head sweep below: its output slot, or "deleted"
+            if (valid) {
+                const uint32_t pos = gt_before + min(eq_before, want);
+                if (kp && pos >= (uint32_t)k) atomicOr(p.status, OBF_DEV_INTERNAL);
+                sel_keys[j] = (kp && pos < (uint32_t)k) ? pos : 0xFFFFFFFFu;
+            }
+        } else if (valid) {
             const float a = key_score(u);
             keep[j] = kp ? 1 : 0;
             if (kp) {
@@ -392,6 +417,47 @@ __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ Call
         }
         run_gt += __popc(m_gt);
         run_eq += __popc(m_eq);
+    }
+    if (LAYER) {
+        __syncthreads();
+        // the largest summed mass among the deleted positions, for the diagnostics
+        for (int j = tid; j < T; j += NT)
+            if (sel_keys[j] == 0xFFFFFFFFu) nx = fmaxf(nx, __uint_as_float(A[j]));
+        const float next = block_max<NT>(nx, red);
+        for (int h = 0; h < p.kv_heads; ++h) {
+            float *Ah = Af + (size_t)h * T;
+            uint8_t *keep_h = keep + (size_t)h * T;
+            int32_t *idx_h = idx + (size_t)h * k;
+            sk = 0.f; sd = 0.f;
+            for (int j = tid; j < T; j += NT) {
+                const uint32_t pos = sel_keys[j];
+                const float a = Ah[j];
+                const bool kp = pos != 0xFFFFFFFFu;
+                keep_h[j] = kp ? 1 : 0;
+                if (kp) {
+                    Ah[j] = -1.0f;             // later passes need the mass of deleted tokens only
+                    idx_h[pos] = j;
+                    sk += a;
+                } else {
+                    sd += a;
+                }
+            }
+            const float a_keep = block_sum<NT>(sk, red);
+            const float a_del = block_sum<NT>(sd, red);
+            if (tid == 0) {
+                float *sm = p.sums + (size_t)(c.head_base + lh + h) * 4;
+                sm[0] = a_keep; sm[1] = a_del; sm[2] = key_score(tau); sm[3] = next;
+                if (c.diag) {
+                    obf_diag_t dg;
+                    dg.a_keep = a_keep; dg.a_del = a_del; dg.alpha = a_del / (a_keep + p.eps);
+                    dg.rcr = 0.f; dg.delta_norm = 0.f; dg.kth_score = key_score(tau); dg.next_score = next;
+                    dg.lam_1 = dg.lam_rho = dg.lam_next = 0.f;
+                    dg.span_rank = -1; dg.rho_eff = 0; dg.status = OBF_DEV_SKIPPED; dg.reserved = 0;
+                    c.diag[lh + h] = dg;
+                }
+            }
+        }
+        return;
     }
     const float a_keep = block_sum<NT>(sk, red);
     const float a_del = block_sum<NT>(sd, red);

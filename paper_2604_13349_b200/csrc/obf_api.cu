@@ -37,7 +37,7 @@ static inline void mark(cudaStream_t st, const char *name)
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-    size_t off_status, off_scores, off_keep, off_stats, off_sums;
+    size_t off_status, off_scores, off_keep, off_stats, off_sums, off_lscores;
     size_t off_gram_d, off_gram_k, off_uvec, off_delta, off_hflag;
     size_t total;
     int splits;
@@ -110,6 +110,8 @@ static obf_status_t validate_shapes(const obf_params_t *p, const obf_cache_t *ca
     for (int i = 0; i < n; ++i) {
         if (caches[i].T < 1 || caches[i].T > OBF_MAX_T) return OBF_ERR_INVALID_ARG;
         if (caches[i].budget < 1) return OBF_ERR_INVALID_ARG;
+        // the layerwise selector keeps a layer's summed masses in shared memory
+        if ((p->flags & OBF_FLAG_LAYERWISE) && caches[i].T > SEL_SMEM_MAX_T) return OBF_ERR_UNSUPPORTED;
     }
     return OBF_OK;
 }
@@ -191,6 +193,8 @@ static void make_layout(const obf_params_t *p, const obf_cache_t *caches, int32_
     L.off_keep = o;   o = align_up(o + tok, 256);
     L.off_stats = o;  o = align_up(o + (size_t)L.heads_total * n_q * 2 * sizeof(float), 256);
     L.off_sums = o;   o = align_up(o + (size_t)L.heads_total * 4 * sizeof(float), 256);
+    L.off_lscores = o;
+    if (p->flags & OBF_FLAG_LAYERWISE) o = align_up(o + tok / p->kv_heads * sizeof(float), 256);
     L.off_sc_part = L.off_sc_head = L.off_sc_sync = o;
     if (L.sc_on) {
         L.off_sc_part = o; o = align_up(o + L.sc_part_pairs * 2 * sizeof(float), 256);
@@ -322,7 +326,16 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
         k_score_pool<TIN, D><<<g2, SC_NT, sm_sc, st>>>(cd);
         mark(st, "k_score_pool");
     }
-    if (T_max <= SEL_SMEM_MAX_T) {
+    if (cd.layerwise) {
+        // one block per layer: masses of the layer's KV heads added up, selection on the sums, outputs per head
+        const int n_layers = heads / cd.kv_heads;
+        const size_t sm_sel = (size_t)T_max * sizeof(uint32_t);
+        dim3 gl((T_max + 255) / 256, n_layers);
+        k_layer_sum<<<gl, 256, 0, st>>>(cd);
+        mark(st, "k_layer_sum");
+        if ((s = set_smem(k_select_smem<1024, true>, sm_sel)) != OBF_OK) return s;
+        k_select_smem<1024, true><<<n_layers, 1024, sm_sel, st>>>(cd);
+    } else if (T_max <= SEL_SMEM_MAX_T) {
         const size_t sm_sel = (size_t)T_max * sizeof(uint32_t);
         // blocks of 1024 threads fit twice on an SM; when the heads then need a second, nearly empty wave,
         // blocks of 512 threads (four per SM) finish sooner
@@ -433,6 +446,9 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
     cd.keep = reinterpret_cast<uint8_t *>(ws + L.off_keep);
     cd.stats = reinterpret_cast<float *>(ws + L.off_stats);
     cd.sums = reinterpret_cast<float *>(ws + L.off_sums);
+    cd.lscores = reinterpret_cast<float *>(ws + L.off_lscores);
+    cd.kv_heads = p->kv_heads;
+    cd.layerwise = (p->flags & OBF_FLAG_LAYERWISE) ? 1 : 0;
     cd.sc_part = reinterpret_cast<float *>(ws + L.off_sc_part);
     cd.sc_head = reinterpret_cast<float *>(ws + L.off_sc_head);
     cd.sc_cnt = reinterpret_cast<uint32_t *>(ws + L.off_sc_sync);

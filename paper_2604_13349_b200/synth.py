@@ -101,6 +101,7 @@ class Workload:
     dtype: str                    # "f32" or "bf16"
     head: HeadSpec
     caches: Tuple[CacheSpec, ...]
+    layerwise: bool = False       # layerwise selector: one retained set per layer
 
     @property
     def G(self) -> int:
@@ -233,6 +234,8 @@ def _make_workloads() -> Dict[str, Workload]:
         name="c4", seed=3, layers=40, kv_heads=8, q_heads=32, n_obs=32, rank=4, dtype="bf16",
         head=hs_full, caches=(CacheSpec(T=8192, budget=811),))
     out["c4_evict"] = dataclasses.replace(out["c4"], name="c4_evict", rank=0)
+    # the layerwise selector with the rank the paper pairs it with (L-OBF, pca_rank 4)
+    out["c4_layer"] = dataclasses.replace(out["c4"], name="c4_layer", layerwise=True)
     Ts = _ragged_T(4, 4)
     out["c5"] = Workload(
         name="c5", seed=4, layers=36, kv_heads=8, q_heads=32, n_obs=32, rank=2, dtype="bf16",

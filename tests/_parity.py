@@ -73,14 +73,22 @@ class HeadReport:
 def check_head(dtype: str, K: np.ndarray, V: np.ndarray, Q: np.ndarray, budget: int, rank: int,
                g_idx: np.ndarray, g_kbits: np.ndarray, g_vbits: np.ndarray, g_v: np.ndarray,
                g_scores: Optional[np.ndarray], g_delta: Optional[np.ndarray], g_diag: Optional[dict],
-               in_kbits: np.ndarray, in_vbits: np.ndarray, name: str = "") -> HeadReport:
-    """K, V, Q: float32 values of one head (bf16 already up-cast).  g_*: the CUDA path's outputs."""
+               in_kbits: np.ndarray, in_vbits: np.ndarray, name: str = "",
+               ref: Optional[dict] = None, sel_scores: Optional[np.ndarray] = None,
+               tie_band: float = TIE_BAND) -> HeadReport:
+    """K, V, Q: float32 values of one head (bf16 already up-cast).  g_*: the CUDA path's outputs.
+
+    ref: the oracle's result for this head when it was not chosen headwise (layerwise selector), with
+    sel_scores the masses the selection ran on and tie_band the band on those."""
     rep = HeadReport()
     T, d = K.shape
     k = min(budget, T)
-    ref = oracle.head(K, V, Q, budget, rank)
+    if ref is None:
+        ref = oracle.head(K, V, Q, budget, rank)
     A = ref["A"]
     dg = ref["diag"]
+    if sel_scores is None:
+        sel_scores = A
 
     # -- a1: attention mass ------------------------------------------------
     if g_scores is not None:
@@ -93,14 +101,14 @@ def check_head(dtype: str, K: np.ndarray, V: np.ndarray, Q: np.ndarray, budget: 
     assert g_idx.shape == (k,)
     assert np.all(np.diff(g_idx) > 0), "%s: positions not strictly ascending" % name
     assert g_idx.min() >= 0 and g_idx.max() < T
-    band = np.abs(A - dg["kth_score"]) <= TIE_BAND
+    band = np.abs(sel_scores - dg["kth_score"]) <= tie_band
     rep.in_band = int(band.sum())
     gset, oset = set(g_idx.tolist()), set(ref["idx"].tolist())
     outside = ~band
     g_out = {j for j in gset if outside[j]}
     o_out = {j for j in oset if outside[j]}
     assert g_out == o_out, "%s: retained sets differ outside the %.0e tie band: %s" % (
-        name, TIE_BAND, sorted(g_out ^ o_out)[:8])
+        name, tie_band, sorted(g_out ^ o_out)[:8])
     rep.band_mismatch = gset != oset
 
     # -- a3: gather is bit-exact -------------------------------------------------
@@ -170,6 +178,42 @@ def check_cache(w: synth.Workload, ci: int, arrays: Dict[str, np.ndarray], out: 
             diags[l * w.kv_heads + h] if diags else None, kb, vb,
             name="%s cache %d layer %d head %d" % (name or w.name, ci, l, h))
         reps.append(rep)
+    return reps
+
+
+def check_cache_layerwise(w: synth.Workload, ci: int, arrays: Dict[str, np.ndarray], out: Dict[str, torch.Tensor],
+                          layers: Sequence[int], rank: Optional[int] = None, name: str = "") -> List[HeadReport]:
+    """Layerwise selector: every head of a layer against the oracle's layer result.  The tie band is the
+    headwise one times the number of KV heads (the selection runs on a sum of that many masses)."""
+    rank = w.rank if rank is None else rank
+    d, n_q, H = w.head.head_dim, w.n_q, w.kv_heads
+    budget = w.caches[ci].budget
+    Qv = arrays["Q"].reshape(w.layers, H, n_q, d)
+    diags = P.parse_diag(out["diag"]) if out.get("diag") is not None else None
+    bits = np.int16 if w.dtype == "bf16" else np.int32
+    reps = []
+    for l in layers:
+        K = f32_view(arrays["K"][l], w.dtype)
+        V = f32_view(arrays["V"][l], w.dtype)
+        Q = f32_view(Qv[l], w.dtype)
+        lay = oracle.layer(K, V, Q, budget, rank)
+        g_idx_all = out["idx"][l].cpu().numpy()
+        for h in range(1, H):
+            assert np.array_equal(g_idx_all[h], g_idx_all[0]), "layer %d: heads do not share their positions" % l
+        for h in range(H):
+            ref = {"A": lay["A"][h], "idx": lay["idx"][h], "delta": lay["delta"][h], "V_out": lay["V_out"][h],
+                   "diag": lay["diag"][h]}
+            rep = check_head(
+                w.dtype, K[h], V[h], Q[h], budget, rank,
+                g_idx_all[h], out_bits(out["K_out"][l, h]), out_bits(out["V_out"][l, h]),
+                out_to_f32(out["V_out"][l, h]),
+                out["scores"][l, h].cpu().numpy() if out.get("scores") is not None else None,
+                out["delta"][l, h].cpu().numpy() if out.get("delta") is not None else None,
+                diags[l * H + h] if diags else None,
+                arrays["K"][l, h].view(bits), arrays["V"][l, h].view(bits),
+                name="%s cache %d layer %d head %d (layerwise)" % (name or w.name, ci, l, h),
+                ref=ref, sel_scores=lay["S"], tie_band=TIE_BAND * H)
+            reps.append(rep)
     return reps
 
 

@@ -302,3 +302,57 @@ def test_paper_regime_budget_32_sampled_heads():
     w = synth.workload("pa")
     outs, reps, _ = run_and_check(w, heads=[(0, 0), (9, 4), (35, 7)])
     assert all(not r.oracle_skipped for r in reps)
+
+
+# ---------------------------------------------------------------------------
+# layerwise selector: one retained set per layer, back-fill per head
+# ---------------------------------------------------------------------------
+def run_and_check_layerwise(w, arrays=None, flags=0, evict=False):
+    arrays = arrays or [synth.gen_cache(w, ci) for ci in range(len(w.caches))]
+    outs, _, st = par.run_gpu(w, arrays, evict=evict, flags=flags | P.binding.OBF_FLAG_LAYERWISE)
+    assert st & 0xFF == 0, "device status %#x" % st
+    reps = []
+    for ci in range(len(w.caches)):
+        reps += par.check_cache_layerwise(w, ci, arrays[ci], outs[ci], range(w.layers), rank=0 if evict else None)
+    print("\n[%s layerwise] %s" % (w.name, par.summarize(reps)))
+    return outs, reps, arrays
+
+
+@pytest.mark.parametrize("dtype,d", [("f32", 64), ("bf16", 64), ("f32", 128)])
+def test_layerwise_small_budgets_backfill_every_head(dtype, d):
+    w = small("lw", layers=3, kv_heads=4, G=2, n_obs=5, d=d, dtype=dtype, rank=2, caches=((220, 14), (97, 9)), seed=33)
+    outs, reps, _ = run_and_check_layerwise(w)
+    assert all(not r.oracle_skipped for r in reps)              # budget < head_dim: OBF is active everywhere
+
+
+def test_layerwise_c1_and_its_eviction_only_form():
+    w = synth.workload("c1")
+    a, reps, arrays = run_and_check_layerwise(w)
+    assert all(not r.oracle_skipped for r in reps)
+    b, _, _ = run_and_check_layerwise(w, arrays=arrays, evict=True)
+    for x, y in zip(a, b):
+        assert torch.equal(x["idx"], y["idx"]) and torch.equal(x["K_out"], y["K_out"])
+
+
+@pytest.mark.parametrize("caches", [((300, 20), (130, 129), (777, 100)), ((2048, 205),)])
+def test_layerwise_on_the_tensor_core_path(caches):
+    w = small("lw_tuned", layers=2, kv_heads=3, G=2, n_obs=9, d=128, dtype="bf16", rank=4, caches=caches,
+              n_outlier=3, n_sink=2, seed=51 + len(caches))
+    a, reps, arrays = run_and_check_layerwise(w)
+    b, _, _ = run_and_check_layerwise(w, arrays=arrays, flags=P.binding.OBF_FLAG_GENERIC_PATH)
+    for x, y in zip(a, b):
+        assert torch.equal(x["K_out"], y["K_out"])
+
+
+def test_layerwise_with_one_kv_head_equals_headwise():
+    w = small("lw1", layers=2, kv_heads=1, G=4, n_obs=4, d=64, dtype="f32", rank=1, caches=((150, 11),), seed=3)
+    a, _, arrays = run_and_check_layerwise(w)
+    b, _, _ = run_and_check(w, arrays=arrays)
+    assert torch.equal(a[0]["idx"], b[0]["idx"]) and torch.equal(a[0]["V_out"], b[0]["V_out"])
+
+
+def test_layerwise_rejects_prompts_that_do_not_fit_shared_memory():
+    w = small("lw_long", layers=1, kv_heads=2, d=64, dtype="f32", rank=0, caches=((20000, 8),))
+    arrays = [synth.gen_cache(w, 0)]
+    with pytest.raises(Exception):
+        par.run_gpu(w, arrays, flags=P.binding.OBF_FLAG_LAYERWISE)
