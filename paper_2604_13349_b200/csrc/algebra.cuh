@@ -13,9 +13,13 @@
 //      left of it exceeds 1e-4 of its own norm.
 //   3. P = I - Q^T Q,  M = P G_del P = R^T R  (Eq. 3 in Gram form, App. H),
 //      r_bar = P u / (A_del + eps)  (Eq. 4).
-//   4. Symmetric eigen-decomposition of M by parallel-order Jacobi rotations run
-//      to convergence; C = eigenvectors of the `rank` largest eigenvalues above
-//      1e-5 of the largest.
+//   4. C = eigenvectors of the `rank` largest eigenvalues of M above 1e-5 of the
+//      largest.  For rank <= ALG_TRI_MAX_RANK: Householder reduction of M to
+//      tridiagonal form, the rank + 1 largest eigenvalues by bisection on Sturm
+//      counts, their vectors by inverse iteration (neighbours closer than 1e-3 of
+//      the largest eigenvalue are kept orthogonal during the iteration), mapped
+//      back through the reflectors.  For larger ranks: full eigen-decomposition by
+//      parallel-order Jacobi rotations run to convergence.
 //   5. Delta = C^T C r_bar (Eq. 5), delta = A_del / (A_keep + eps) * Delta (Eq. 6),
 //      V_out = V_keep + delta on the head's retained rows (Eq. 7).
 #pragma once
@@ -30,6 +34,25 @@ constexpr float SPAN_ROW_TOL = 1e-4f;
 constexpr float RCR_SKIP_TOL = 1e-6f;
 constexpr float EIG_RANK_TOL = 1e-5f;
 constexpr int JACOBI_MAX_SWEEPS = 30;
+constexpr int ALG_TRI_MAX_RANK = 8;     // up to this rank only rank + 1 eigenpairs are computed
+constexpr int ALG_TRI_NE = ALG_TRI_MAX_RANK + 1;
+constexpr float EIG_CLUSTER_TOL = 1e-3f; // eigenvalues closer than this (relative to the largest) are orthogonalised explicitly
+
+// Number of eigenvalues of the symmetric tridiagonal matrix (diagonal a, off-diagonal b) that are smaller than x:
+// the negative pivots of the LDL^T factorisation of T - x I.
+template <int D>
+__device__ __forceinline__ int sturm_count(const float *a, const float *b, float x, float pivmin)
+{
+    float q = a[0] - x;
+    int cnt = q < 0.f ? 1 : 0;
+#pragma unroll 4
+    for (int i = 1; i < D; ++i) {
+        if (fabsf(q) < pivmin) q = -pivmin;
+        q = a[i] - x - b[i - 1] * b[i - 1] / q;
+        cnt += q < 0.f ? 1 : 0;
+    }
+    return cnt;
+}
 
 template <int D>
 constexpr size_t algebra_smem_bytes() { return (size_t)(3 * D * (D + 1) + 6 * D + 64) * sizeof(float) + 2 * D * sizeof(int); }
@@ -175,7 +198,216 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
         rcr = trM / (trG + p.eps);
         if (!(rcr >= RCR_SKIP_TOL)) { done = true; status |= OBF_DEV_SKIPPED; }
 
-        // ---- 4. Jacobi eigen-decomposition of M (B2), eigenvectors in B1 -----
+        // ---- 4a. few eigenpairs wanted: tridiagonal form, bisection, inverse iteration ----
+        if (!done && p.rank <= ALG_TRI_MAX_RANK) {
+            const int lane = tid & 31, warp = tid >> 5;
+            const int ne = min(min(p.rank, D) + 1, D);             // eigenpairs computed: the wanted ones and the next
+            float *ta = B0, *tb = B0 + D;                          // diagonal, off-diagonal (tb[i] couples i and i + 1)
+            float *tlam = tb + D;                                  // ALG_TRI_NE eigenvalues, largest first
+            float *tz = tlam + 16;                                 // [ALG_TRI_NE][D] eigenvectors
+            float *twk = tz + ALG_TRI_NE * D;                      // [ALG_TRI_NE][5][D] factors of T - lambda I
+            // Householder reduction: reflector k (a unit vector, row k of B1) zeroes column k below the sub-diagonal
+            const float tiny2 = 1e-20f * trM * trM;
+#pragma unroll 1
+            for (int k = 0; k < D - 2; ++k) {
+                const float xi = (tid > k && tid < D) ? B2[tid * LD + k] : 0.f;
+                const float nrm2 = block_sum<ALG_NT>(xi * xi, red);
+                const float x0 = B2[(k + 1) * LD + k];
+                const float nrm = sqrtf(nrm2);
+                const float al = x0 >= 0.f ? -nrm : nrm;
+                const float vn2 = 2.f * nrm * (nrm + fabsf(x0));   // |x - al e_0|^2
+                const bool skip = !(nrm2 - x0 * x0 > tiny2) || !(vn2 > 0.f);   // nothing below the sub-diagonal
+                if (tid < D) {
+                    float v = 0.f;
+                    if (!skip && tid > k) v = (tid == k + 1 ? x0 - al : xi) * rsqrtf(vn2);
+                    B1[k * LD + tid] = v;
+                }
+                if (tid == 0) { ta[k] = B2[k * LD + k]; tb[k] = skip ? x0 : al; }
+                __syncthreads();
+                if (skip) continue;
+                const float *v = B1 + k * LD;
+                {                                                   // pvec = 2 M v on the trailing block -> vc
+                    const int i = tid >> 2, part = tid & 3;
+                    float sacc = 0.f;
+                    if (i > k && i < D) {
+                        const float *mi = B2 + i * LD;
+                        for (int cc = k + 1 + part; cc < D; cc += 4) sacc = fmaf(mi[cc], v[cc], sacc);
+                    }
+                    sacc += __shfl_xor_sync(0xffffffffu, sacc, 1);
+                    sacc += __shfl_xor_sync(0xffffffffu, sacc, 2);
+                    if (part == 0 && i < D) vc[i] = i > k ? 2.f * sacc : 0.f;
+                }
+                __syncthreads();
+                const float kk = block_sum<ALG_NT>(tid < D ? v[tid] * vc[tid] : 0.f, red);
+                if (tid < D) vw[tid] = vc[tid] - kk * v[tid];       // w = pvec - (v . pvec) v
+                __syncthreads();
+                for (int e = tid; e < D * D; e += ALG_NT) {         // M <- H M H = M - v w^T - w v^T
+                    const int i = e / D, j = e % D;
+                    if (i > k && j > k) B2[i * LD + j] -= v[i] * vw[j] + vw[i] * v[j];
+                }
+                __syncthreads();
+            }
+            if (tid == 0) {
+                ta[D - 2] = B2[(D - 2) * LD + D - 2]; tb[D - 2] = B2[(D - 1) * LD + D - 2];
+                ta[D - 1] = B2[(D - 1) * LD + D - 1]; tb[D - 1] = 0.f;
+            }
+            if (tid < D) B1[(D - 2) * LD + tid] = 0.f;              // no reflector for the last two columns
+            __syncthreads();
+            // bounds of the spectrum (Gershgorin) and the pivot floor of the Sturm counts
+            float gl = INFINITY, gh = -INFINITY, b2 = 0.f;
+            if (tid < D) {
+                const float r = (tid > 0 ? fabsf(tb[tid - 1]) : 0.f) + fabsf(tb[tid]);
+                gl = ta[tid] - r; gh = ta[tid] + r; b2 = tb[tid] * tb[tid];
+            }
+            const float g_hi = block_max<ALG_NT>(gh, red), g_lo = -block_max<ALG_NT>(-gl, red);
+            const float pivmin = 1e-30f * fmaxf(1.f, block_max<ALG_NT>(b2, red));
+            const float span = fmaxf(g_hi - g_lo, 1e-30f);
+            // eigenvalue j (largest first) by 32-way multisection, one warp per eigenvalue
+            if (warp < ne) {
+                const int want = D - 1 - warp;                      // it has exactly `want` eigenvalues below it
+                float lo = g_lo - 1e-3f * span, hi = g_hi + 1e-3f * span;
+#pragma unroll 1
+                for (int round = 0; round < 7; ++round) {
+                    const float x = lo + (hi - lo) * (float)(lane + 1) * (1.f / 33.f);
+                    const bool below = sturm_count<D>(ta, tb, x, pivmin) <= want;     // x is not above the eigenvalue
+                    const int nl = __popc(__ballot_sync(0xffffffffu, below));        // counts are monotone in x
+                    const float x_lo = __shfl_sync(0xffffffffu, x, max(nl - 1, 0));
+                    const float x_hi = __shfl_sync(0xffffffffu, x, min(nl, 31));
+                    if (nl > 0) lo = x_lo;
+                    if (nl < 32) hi = x_hi;
+                }
+                if (lane == 0) tlam[warp] = 0.5f * (lo + hi);
+            }
+            __syncthreads();
+            const float l1 = tlam[0];
+            // inverse iteration on T: factor T - lambda_j I once (LU with row interchanges), three solves
+            if (warp < ne && lane == 0) {
+                const float lam = tlam[warp];
+                float *dd = twk + (warp * 5) * D, *dl = dd + D, *du = dl + D, *du2 = du + D, *pv = du2 + D;
+                const float pert = 4e-7f * fmaxf(fabsf(g_hi), fabsf(g_lo)) + 1e-30f;
+                for (int i = 0; i < D; ++i) { dd[i] = ta[i] - lam; dl[i] = tb[i]; du[i] = tb[i]; du2[i] = 0.f; }
+                for (int i = 0; i < D - 1; ++i) {
+                    if (fabsf(dd[i]) >= fabsf(dl[i])) {
+                        if (dd[i] == 0.f) dd[i] = pert;
+                        const float f = dl[i] / dd[i];
+                        dl[i] = f; dd[i + 1] -= f * du[i]; pv[i] = 0.f;
+                    } else {
+                        const float f = dd[i] / dl[i];
+                        dd[i] = dl[i]; dl[i] = f;
+                        const float t = du[i];
+                        du[i] = dd[i + 1]; dd[i + 1] = t - f * dd[i + 1];
+                        if (i < D - 2) { du2[i] = du[i + 1]; du[i + 1] = -f * du[i + 1]; }
+                        pv[i] = 1.f;
+                    }
+                }
+                if (dd[D - 1] == 0.f) dd[D - 1] = pert;
+                for (int i = 0; i < D; ++i)
+                    if (fabsf(dd[i]) < pert) dd[i] = dd[i] < 0.f ? -pert : pert;
+            }
+            if (warp < ne) {
+                float *y = tz + warp * D;
+                for (int i = lane; i < D; i += 32) {                // a start vector without structure
+                    const uint32_t hsh = ((uint32_t)i * 2654435761u + (uint32_t)warp * 40503u + 12345u) >> 8;
+                    y[i] = (float)(hsh & 0xFFFFu) * (1.f / 65536.f) - 0.5f;
+                }
+            }
+            __syncthreads();
+#pragma unroll 1
+            for (int itn = 0; itn < 3; ++itn) {
+                if (warp < ne && lane == 0) {
+                    float *y = tz + warp * D;
+                    const float *dd = twk + (warp * 5) * D, *dl = dd + D, *du = dl + D, *du2 = du + D, *pv = du2 + D;
+                    for (int i = 0; i < D - 1; ++i) {
+                        if (pv[i] == 0.f) y[i + 1] -= dl[i] * y[i];
+                        else { const float t = y[i]; y[i] = y[i + 1]; y[i + 1] = t - dl[i] * y[i]; }
+                    }
+                    y[D - 1] /= dd[D - 1];
+                    y[D - 2] = (y[D - 2] - du[D - 2] * y[D - 1]) / dd[D - 2];
+                    for (int i = D - 3; i >= 0; --i) y[i] = (y[i] - du[i] * y[i + 1] - du2[i] * y[i + 2]) / dd[i];
+                    float mx = 0.f;
+                    for (int i = 0; i < D; ++i) mx = fmaxf(mx, fabsf(y[i]));
+                    const float sc1 = mx > 0.f ? 1.f / mx : 1.f;
+                    for (int i = 0; i < D; ++i) y[i] *= sc1;
+                }
+                __syncthreads();
+                if (warp == 0) {
+                    // in order of the eigenvalues: orthogonal to the close neighbours before it, unit length
+                    for (int j = 0; j < ne; ++j) {
+                        float *y = tz + j * D;
+                        for (int i2 = 0; i2 < j; ++i2) {
+                            if (fabsf(tlam[i2] - tlam[j]) > EIG_CLUSTER_TOL * fabsf(l1)) continue;
+                            const float *z = tz + i2 * D;
+                            float dsum = 0.f;
+                            for (int cc = lane; cc < D; cc += 32) dsum = fmaf(y[cc], z[cc], dsum);
+                            dsum = warp_sum(dsum);
+                            for (int cc = lane; cc < D; cc += 32) y[cc] -= dsum * z[cc];
+                            __syncwarp();
+                        }
+                        float n2 = 0.f;
+                        for (int cc = lane; cc < D; cc += 32) n2 = fmaf(y[cc], y[cc], n2);
+                        n2 = warp_sum(n2);
+                        const float inv = n2 > 0.f ? rsqrtf(n2) : 0.f;
+                        for (int cc = lane; cc < D; cc += 32) y[cc] *= inv;
+                        __syncwarp();
+                    }
+                }
+                __syncthreads();
+            }
+            // back through the reflectors: z = H_0 H_1 ... H_{D-3} y, one warp per vector
+            if (warp < ne) {
+                float *y = tz + warp * D;
+#pragma unroll 1
+                for (int k = D - 3; k >= 0; --k) {
+                    const float *v = B1 + k * LD;
+                    float dsum = 0.f;
+                    for (int cc = lane; cc < D; cc += 32) dsum = fmaf(v[cc], y[cc], dsum);
+                    dsum = 2.f * warp_sum(dsum);
+                    for (int cc = lane; cc < D; cc += 32) y[cc] -= dsum * v[cc];
+                    __syncwarp();
+                }
+            }
+            __syncthreads();
+            // ---- 5a. Delta, delta from the wanted eigenvectors ----------------------------------
+            const int rmax = min(p.rank, D);
+            rho = 0;
+            while (rho < rmax && rho < ne && tlam[rho] > EIG_RANK_TOL * l1 && tlam[rho] > 0.f) ++rho;
+            lam1 = l1; lam_rho = rho > 0 ? tlam[rho - 1] : 0.f; lam_next = rho < ne ? fmaxf(tlam[rho], 0.f) : 0.f;
+            if (tid < rho) {
+                float sacc = 0.f;
+                for (int cc = 0; cc < D; ++cc) sacc = fmaf(tz[tid * D + cc], vu[cc], sacc);
+                vc[tid] = sacc;
+            }
+            __syncthreads();
+            float dl = 0.f;
+            if (tid < D) {
+                float sacc = 0.f;
+                for (int t = 0; t < rho; ++t) sacc = fmaf(vc[t], tz[t * D + tid], sacc);
+                dl = alpha * sacc;
+            }
+            const float dn2 = block_sum<ALG_NT>(dl * dl, red);
+            dnorm = sqrtf(dn2);
+            if (!isfinite(dn2)) { status |= OBF_DEV_NONFINITE | OBF_DEV_SKIPPED; dnorm = 0.f; }
+            else if (rho == 0 || dn2 == 0.f) status |= OBF_DEV_SKIPPED;
+            else {
+                if (tid < D) {
+                    p.delta[(size_t)g * D + tid] = dl;
+                    if (c.delta_out) c.delta_out[(size_t)lh * D + tid] = dl;
+                    vw[tid] = dl;
+                }
+                if (tid == 0) p.hflag[g] = HFLAG_INJECT;
+                __syncthreads();
+                // Eq. 7: V_out = V_keep + delta on every retained row; the fp32 sum is rounded once
+                TIN *rows = reinterpret_cast<TIN *>(c.v_out) + (size_t)lh * k * D;
+                for (int e = tid; e < k * D; e += ALG_NT) {
+                    const float sum = to_f32(rows[e]) + vw[e % D];
+                    if constexpr (sizeof(TIN) == 4) rows[e] = sum;
+                    else rows[e] = __float2bfloat16_rn(sum);
+                }
+            }
+            done = true;
+        }
+
+        // ---- 4b. Jacobi eigen-decomposition of M (B2), eigenvectors in B1 -----
         if (!done) {
             // rotations below the fp32 noise level of the largest eigenvalue never settle: stop there
             const float floor_abs = 2e-7f * block_max<ALG_NT>(tid < D ? B2[tid * LD + tid] : 0.f, red);
