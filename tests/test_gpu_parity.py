@@ -356,3 +356,36 @@ def test_layerwise_rejects_prompts_that_do_not_fit_shared_memory():
     arrays = [synth.gen_cache(w, 0)]
     with pytest.raises(Exception):
         par.run_gpu(w, arrays, flags=P.binding.OBF_FLAG_LAYERWISE)
+
+
+# ---------------------------------------------------------------------------
+# eigen-solve of the small-rank path: a residual spectrum with a tie at the top
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("rank", [1, 2, 3])
+def test_residual_with_two_equal_leading_singular_values(rank):
+    # The retained values live in the first 10 channels; every deleted value adds a component along channel 20
+    # or channel 21, with the same energy on both and no correlation between them: the residual has two equal
+    # leading singular values and nothing else.  Rank 2 and 3 have a unique answer (Delta = r_bar); rank 1 does
+    # not (any direction of that plane is a leading singular vector), so only the invariants are checked for it.
+    w = small("tie", d=64, dtype="f32", rank=rank, caches=((240, 12),), heavy=0, kv_heads=2, seed=77)
+    arrays = [synth.gen_cache(w, 0)]
+    a = arrays[0]
+    Qv = a["Q"].reshape(1, 2, w.n_q, 64)
+    g = np.random.default_rng(9)
+    V = np.zeros_like(a["V"])
+    for h in range(2):
+        A = oracle.scores(a["K"][0, h], Qv[0, h])
+        keep = np.zeros(240, bool); keep[oracle.topk(A, 12)[0]] = True
+        V[0, h, :, :10] = g.standard_normal((240, 10)).astype(np.float32)
+        dele = np.flatnonzero(~keep)
+        half = len(dele) // 2
+        V[0, h, dele[:half], 20] = 0.5                       # same count, same magnitude, disjoint supports
+        V[0, h, dele[half:2 * half], 21] = 0.5
+    a["V"] = V
+    outs, reps, _ = run_and_check(w, arrays=arrays)
+    assert all(not r.oracle_skipped for r in reps)
+    d = outs[0]["delta"].cpu().numpy()
+    assert np.all(np.abs(d[..., :10]) < 1e-5) and np.all(np.abs(d[..., 22:]) < 1e-5)
+    if rank >= 2:
+        assert all(r.gap_rel > 0.5 for r in reps)            # the plane itself is well separated from the rest
+        assert np.all(np.linalg.norm(d, axis=-1) > 1e-4)
