@@ -105,7 +105,7 @@ typedef struct {              /* per (layer, KV head) diagnostics (App. K.2 name
     int32_t span_rank;        /* numerical dimension m of span(V_keep) (-1: not evaluated)          */
     int32_t rho_eff;          /* number of principal directions actually used                       */
     uint32_t status;          /* OBF_DEV_* bits                                                     */
-    int32_t reserved;
+    float revr;               /* sum of the rho_eff kept eigenvalues of R^T R over their total  [REVR]; PCR is 1 - rcr */
 } obf_diag_t;
 
 typedef struct {              /* one agent's prompt cache; T and budget may differ between caches   */

@@ -56,6 +56,7 @@ typedef struct {
     int32_t rho_eff;     /* min(pca_rank, numerical rank of R)                              */
     int32_t n_del;       /* number of deleted positions                                     */
     int32_t skipped;     /* 1 if OBF was skipped for this head (footnote to Eq. 7)          */
+    double revr;         /* kept share of the residual's squared singular values (REVR, App. K.2) */
 } obf_oracle_diag_t;
 
 /* ------------------------------------------------------------------ */
@@ -396,6 +397,9 @@ static int backfill_given_selection(const float *K, const float *V, const double
     dg.lam_1 = lam[0];
     dg.lam_rho = rho > 0 ? lam[rho - 1] : 0.0;
     dg.lam_next = rho < d ? lam[rho] : 0.0;
+    { double kept = 0.0, all = 0.0;
+      for (int i = 0; i < d; ++i) { all += lam[i]; if (i < rho) kept += lam[i]; }
+      dg.revr = kept / (all + eps); }
 
     /* O10: attention-weighted residual mean, Eq. 4 */
     double *rbar = (double *)calloc((size_t)d, sizeof(double));

@@ -89,7 +89,7 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
 
     uint32_t status = 0u;
     int m = 0;
-    float rcr = 0.f, lam1 = 0.f, lam_rho = 0.f, lam_next = 0.f, dnorm = 0.f;
+    float rcr = 0.f, lam1 = 0.f, lam_rho = 0.f, lam_next = 0.f, dnorm = 0.f, revr = 0.f;
     int rho = 0;
     bool done = false;
 
@@ -372,6 +372,8 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
             rho = 0;
             while (rho < rmax && rho < ne && tlam[rho] > EIG_RANK_TOL * l1 && tlam[rho] > 0.f) ++rho;
             lam1 = l1; lam_rho = rho > 0 ? tlam[rho - 1] : 0.f; lam_next = rho < ne ? fmaxf(tlam[rho], 0.f) : 0.f;
+            for (int t = 0; t < rho; ++t) revr += tlam[t];
+            revr /= trM + p.eps;                                    // trace of M = sum of all its eigenvalues
             if (tid < rho) {
                 float sacc = 0.f;
                 for (int cc = 0; cc < D; ++cc) sacc = fmaf(tz[tid * D + cc], vu[cc], sacc);
@@ -474,20 +476,21 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
                 float l1 = 0.f;
                 for (int i = 0; i < D; ++i) l1 = fmaxf(l1, vl[i]);
                 int n = 0;
-                float last = 0.f;
+                float last = 0.f, kept = 0.f;
                 const int rmax = min(p.rank, D);
                 while (n < rmax) {
                     int b = -1; float best = EIG_RANK_TOL * l1;
                     for (int i = 0; i < D; ++i) if (vl[i] > best) { best = vl[i]; b = i; }
                     if (b < 0) break;
-                    isel[n++] = b; last = vl[b]; vl[b] = -1.f;
+                    isel[n++] = b; last = vl[b]; kept += vl[b]; vl[b] = -1.f;
                 }
                 float nxt = 0.f;
                 for (int i = 0; i < D; ++i) nxt = fmaxf(nxt, vl[i]);
-                misc[1] = l1; misc[2] = last; misc[3] = nxt; misc[4] = (float)n;
+                misc[1] = l1; misc[2] = last; misc[3] = nxt; misc[4] = (float)n; misc[5] = kept;
             }
             __syncthreads();
             lam1 = misc[1]; lam_rho = misc[2]; lam_next = misc[3]; rho = (int)misc[4];
+            revr = misc[5] / (trM + p.eps);
             if (tid < rho) {
                 const int col = isel[tid];
                 float s = 0.f;
@@ -531,6 +534,7 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
             dg->rcr = rcr; dg->delta_norm = dnorm;
             dg->lam_1 = lam1; dg->lam_rho = lam_rho; dg->lam_next = lam_next;
             dg->span_rank = m; dg->rho_eff = rho; dg->status = status;
+            dg->revr = revr;
         }
     }
 }

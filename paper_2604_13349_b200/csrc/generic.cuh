@@ -261,7 +261,7 @@ __global__ void __launch_bounds__(SEL_NT) k_select(const __grid_constant__ CallD
             dg.a_keep = a_keep; dg.a_del = a_del; dg.alpha = a_del / (a_keep + p.eps);
             dg.rcr = 0.f; dg.delta_norm = 0.f; dg.kth_score = key_score(tau); dg.next_score = next;
             dg.lam_1 = dg.lam_rho = dg.lam_next = 0.f;
-            dg.span_rank = -1; dg.rho_eff = 0; dg.status = OBF_DEV_SKIPPED; dg.reserved = 0;
+            dg.span_rank = -1; dg.rho_eff = 0; dg.status = OBF_DEV_SKIPPED; dg.revr = 0.f;
             c.diag[lh] = dg;
         }
     }
@@ -452,7 +452,7 @@ __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ Call
                     dg.a_keep = a_keep; dg.a_del = a_del; dg.alpha = a_del / (a_keep + p.eps);
                     dg.rcr = 0.f; dg.delta_norm = 0.f; dg.kth_score = key_score(tau); dg.next_score = next;
                     dg.lam_1 = dg.lam_rho = dg.lam_next = 0.f;
-                    dg.span_rank = -1; dg.rho_eff = 0; dg.status = OBF_DEV_SKIPPED; dg.reserved = 0;
+                    dg.span_rank = -1; dg.rho_eff = 0; dg.status = OBF_DEV_SKIPPED; dg.revr = 0.f;
                     c.diag[lh + h] = dg;
                 }
             }
@@ -470,7 +470,7 @@ __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ Call
             dg.a_keep = a_keep; dg.a_del = a_del; dg.alpha = a_del / (a_keep + p.eps);
             dg.rcr = 0.f; dg.delta_norm = 0.f; dg.kth_score = key_score(tau); dg.next_score = next;
             dg.lam_1 = dg.lam_rho = dg.lam_next = 0.f;
-            dg.span_rank = -1; dg.rho_eff = 0; dg.status = OBF_DEV_SKIPPED; dg.reserved = 0;
+            dg.span_rank = -1; dg.rho_eff = 0; dg.status = OBF_DEV_SKIPPED; dg.revr = 0.f;
             c.diag[lh] = dg;
         }
     }

@@ -144,6 +144,10 @@ def check_head(dtype: str, K: np.ndarray, V: np.ndarray, Q: np.ndarray, budget: 
         if np.linalg.norm(gd) > 0:
             assert np.abs(Vk @ gd).max() / (np.linalg.norm(Vk, 2) * np.linalg.norm(gd)) <= 1e-4
             assert np.linalg.norm(gd) <= scale * (1 + 1e-3)
+    if g_diag is not None and "revr" in dg:
+        # kept share of the residual's squared singular values: a ratio of well-conditioned eigenvalue sums
+        assert abs(g_diag["revr"] - dg["revr"]) <= 1e-4, "%s: REVR %.6f vs %.6f" % (name, g_diag["revr"], dg["revr"])
+        assert abs(g_diag["rcr"] - dg["rcr"]) <= 1e-4 * max(1.0, dg["rcr"])
     verr = np.abs(g_v.astype(np.float64) - ref["V_out"])
     rep.v_err = float(verr.max())
     if gap >= 1e-3:

@@ -280,6 +280,10 @@ def test_obf_matches_lapack_pipeline(seed, T, d, n_q, budget, rank):
     np.testing.assert_allclose(r["rbar"], ref["rbar"], atol=1e-11)
     np.testing.assert_allclose(r["eigvals"][:len(ref["sing"])], ref["sing"] ** 2,
                                atol=1e-9 * ref["sing"][0] ** 2)
+    # diagnostics of App. K.2: kept share of the squared singular values (REVR), residual content ratio (RCR)
+    rho = r["diag"]["rho_eff"]
+    assert r["diag"]["revr"] == pytest.approx((ref["sing"][:rho] ** 2).sum() / (ref["sing"] ** 2).sum(), rel=1e-9)
+    assert r["diag"]["rcr"] == pytest.approx(ref["rcr"], rel=1e-9)
     np.testing.assert_allclose(r["proj"], ref["proj"], atol=1e-8)      # sign/rotation free comparison
     np.testing.assert_allclose(r["Delta"], ref["Delta"], atol=1e-9)
     np.testing.assert_allclose(r["delta"], ref["delta"], atol=1e-9)
