@@ -323,6 +323,8 @@ __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ Call
             const uint32_t u = j < T ? sel_keys[j] : 0u;
             const bool cand = j < T && (u & mask) == prefix;
             const uint32_t digit = (u >> shift) & 255u;
+            // after the first passes few keys are still candidates: most warps have none and skip the matching
+            if (!__any_sync(0xffffffffu, cand)) continue;
             // lanes that are no candidates form one group of their own, which adds nothing
             const uint32_t peers = __match_any_sync(0xffffffffu, cand ? digit : 256u);
             if (cand && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], (uint32_t)__popc(peers));
