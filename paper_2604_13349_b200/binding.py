@@ -293,4 +293,5 @@ def compress_caches(params: ObfParams, caches_in: Sequence[Dict[str, object]], *
     (evict_only if evict else obf_compress)(params, cs, workspace, stream=stream)
     for o in outs:
         o["workspace"] = workspace
+        o["cache_structs"] = cs                 # for a repeated call on the same buffers (profiling)
     return outs

@@ -57,7 +57,7 @@ struct CallDev {
     int32_t sc_nq;            // tuned score kernel: query rows of its tiles (0: shape-generic score kernels)
     int32_t sc_subs;          // 128-key tiles per chunk
     int32_t sc_rounds;        // rounds of the persistent score kernel
-    int32_t pad3_;
+    int32_t sc_qt;            // tuned score kernel: 128-row query tiles per head (1 or 2)
     float *sc_part;           // per (head, chunk, query of 128): chunk maximum and normaliser
     float *sc_head;           // per (head, query of 128): one 64-bit word, low = M + log2(Z) over all keys, high = 1 when valid
     uint32_t *sc_cnt;         // per head: chunks that have published
@@ -67,6 +67,7 @@ struct CallDev {
     // workspace
     uint32_t *status;
     float *scores;            // [sum heads*T] attention mass (Eq. 1)
+    float *scores2;           // tuned score kernel with two query tiles: masses of the second tile, added into `scores` afterwards
     float *lscores;           // layerwise selector: [sum layers*T] masses summed over a layer's KV heads (cache offset tok_off / kv_heads)
     uint8_t *keep;            // [sum heads*T] 1 = retained
     float *stats;             // [heads_total, n_q, 2] softmax row max (log2 domain) and normaliser

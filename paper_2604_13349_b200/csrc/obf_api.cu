@@ -37,7 +37,7 @@ static inline void mark(cudaStream_t st, const char *name)
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-    size_t off_status, off_scores, off_keep, off_stats, off_sums, off_lscores;
+    size_t off_status, off_scores, off_keep, off_stats, off_sums, off_lscores, off_scores2;
     size_t off_gram_d, off_gram_k, off_uvec, off_delta, off_hflag;
     size_t total;
     int splits;
@@ -53,7 +53,7 @@ struct Layout {
     long long sub_base[OBF_MAX_CACHES];
     // tensor-core score kernel
     bool sc_on;
-    int sc_nq, sc_subs, sc_blocks, sc_rounds;
+    int sc_nq, sc_subs, sc_blocks, sc_rounds, sc_qt;
     int sc_team[OBF_MAX_CACHES], sc_hpr[OBF_MAX_CACHES], sc_round_base[OBF_MAX_CACHES];
     size_t sc_part_off[OBF_MAX_CACHES], sc_part_pairs;
     size_t off_sc_part, off_sc_head, off_sc_sync;
@@ -159,8 +159,13 @@ static void make_layout(const obf_params_t *p, const obf_cache_t *caches, int32_
     }
     L.sc_on = false;
     L.sc_nq = L.sc_subs = L.sc_blocks = L.sc_rounds = 0;
+    L.sc_qt = 1;
     L.sc_part_pairs = 0;
     if (L.tuned && n_q <= ST_MAX_NQ) {
+        // more than 128 query rows per head: two work items per head, one per 128 rows
+        L.sc_qt = (n_q + 127) / 128;
+        const int hpc_real = hpc;
+        const int hpc = hpc_real * L.sc_qt;
         // chunks of ST_TILES 128-key tiles, one per block and round; a head's team must fit in one round
         L.sc_nq = 128;
         L.sc_subs = ST_TILES;
@@ -193,14 +198,16 @@ static void make_layout(const obf_params_t *p, const obf_cache_t *caches, int32_
     L.off_keep = o;   o = align_up(o + tok, 256);
     L.off_stats = o;  o = align_up(o + (size_t)L.heads_total * n_q * 2 * sizeof(float), 256);
     L.off_sums = o;   o = align_up(o + (size_t)L.heads_total * 4 * sizeof(float), 256);
+    L.off_scores2 = o;
+    if (L.sc_on && L.sc_qt == 2) o = align_up(o + tok * sizeof(float), 256);
     L.off_lscores = o;
     if (p->flags & OBF_FLAG_LAYERWISE) o = align_up(o + tok / p->kv_heads * sizeof(float), 256);
     L.off_sc_part = L.off_sc_head = L.off_sc_sync = o;
     if (L.sc_on) {
         L.off_sc_part = o; o = align_up(o + L.sc_part_pairs * 2 * sizeof(float), 256);
         // sc_head and sc_cnt are cleared together before every launch
-        L.off_sc_head = o; o = align_up(o + (size_t)L.heads_total * 128 * sizeof(unsigned long long), 256);
-        L.off_sc_sync = o; o = align_up(o + (size_t)L.heads_total * sizeof(uint32_t), 256);
+        L.off_sc_head = o; o = align_up(o + (size_t)L.heads_total * L.sc_qt * 128 * sizeof(unsigned long long), 256);
+        L.off_sc_sync = o; o = align_up(o + (size_t)L.heads_total * L.sc_qt * sizeof(uint32_t), 256);
     }
     L.off_gram_d = L.off_gram_k = L.off_uvec = L.off_delta = L.off_hflag = o;
     if (rank > 0) {
@@ -302,9 +309,16 @@ static obf_status_t launch_score_tc(const CallDev &cd, const Layout &L, cudaStre
     }
     const size_t smem = ST_SMEM_BYTES;
     OBF_CUDA_TRY(cudaFuncSetAttribute(k_score_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    OBF_CUDA_TRY(cudaMemsetAsync(cd.sc_head, 0, (L.off_sc_sync - L.off_sc_head) + (size_t)cd.heads_total * sizeof(uint32_t), st));
+    OBF_CUDA_TRY(cudaMemsetAsync(cd.sc_head, 0, (L.off_sc_sync - L.off_sc_head) + (size_t)cd.heads_total * L.sc_qt * sizeof(uint32_t), st));
     k_score_tc<<<L.sc_blocks, ST_THREADS, smem, st>>>(cd, maps);
     mark(st, "k_score_tc");
+    if (L.sc_qt == 2) {
+        int T_max = 1;
+        for (int i = 0; i < cd.n_caches; ++i) T_max = cd.c[i].T > T_max ? cd.c[i].T : T_max;
+        dim3 gj((T_max + 255) / 256, cd.heads_total);
+        k_score_join<<<gj, 256, 0, st>>>(cd);
+        mark(st, "k_score_join");
+    }
     return OBF_OK;
 }
 
@@ -437,6 +451,7 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
     cd.u_groups = L.tc_per ? GT_GROUPS : 1;
     cd.tc_total_sub = L.tc_total_sub;
     cd.sc_nq = L.sc_on ? L.sc_nq : 0;
+    cd.sc_qt = L.sc_on ? L.sc_qt : 1;
     cd.sc_subs = L.sc_subs;
     cd.sc_rounds = L.sc_rounds;
     cd.eps = p->eps;
@@ -447,6 +462,7 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
     cd.stats = reinterpret_cast<float *>(ws + L.off_stats);
     cd.sums = reinterpret_cast<float *>(ws + L.off_sums);
     cd.lscores = reinterpret_cast<float *>(ws + L.off_lscores);
+    cd.scores2 = reinterpret_cast<float *>(ws + L.off_scores2);
     cd.kv_heads = p->kv_heads;
     cd.layerwise = (p->flags & OBF_FLAG_LAYERWISE) ? 1 : 0;
     cd.sc_part = reinterpret_cast<float *>(ws + L.off_sc_part);

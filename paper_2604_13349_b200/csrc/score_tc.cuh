@@ -1,5 +1,6 @@
 // Tuned attention-mass kernel (step a1, Eq. 1 with the softmax of App. L.1) for bf16
-// caches with head_dim 128 and up to 128 query rows per KV head.
+// caches with head_dim 128 and up to 256 query rows per KV head (above 128 rows a head is
+// worked on as two items of up to 128 rows whose masses are added afterwards).
 //
 //   A_j = sum_t softmax_j(q_t . K_j / sqrt(d)),  t over the n_q query rows of the KV head.
 //
@@ -49,14 +50,15 @@ constexpr int ST_LAG = 1;                           // rounds between a chunk's 
 constexpr int ST_TILE_BYTES = 128 * 128 * 2;
 constexpr int ST_CONSUMERS = 512;
 constexpr int ST_THREADS = 64 + ST_CONSUMERS + 64;
-constexpr int ST_MAX_NQ = 128;
+constexpr int ST_MAX_NQ = 256;                      // two query tiles of 128 rows
 constexpr float ST_LOG2E = 1.4426950408889634f;
 constexpr size_t ST_SMEM_BYTES = 1024 + (size_t)2 * ST_TILE_BYTES + (size_t)ST_STAGES * ST_TILE_BYTES +
                                  (2 * 2 * 4 * 128 + 2 * 128 + 2 * ST_TILES * 4 * 128) * sizeof(float) + 64;
 static_assert(ST_STAGES == ST_TBUF, "a ring stage is released by the accumulator barrier of the same index");
 
 struct ScoreItem {
-    int r, cache, lh, chunk, nt;   // r: round; nt: tiles of the chunk that hold at least one key
+    int r, cache, lh, chunk, nt;   // r: round; lh: KV head in the cache; nt: tiles of the chunk that hold at least one key
+    int lv, qt;                    // lv = lh * query tiles + qt: the (head, query tile) pair; qt: which 128 query rows
 };
 
 // What a block needs of a cache to find its work of a round (kept in shared memory).
@@ -73,11 +75,15 @@ __device__ __forceinline__ bool score_item(const CallDev &p, const ScoreTab *tab
         if (r >= tab[i].round_base) ci = i;
     const ScoreTab c = tab[ci];
     if (c.hi >= c.hpr) return false;
-    const int lh = (r - c.round_base) * c.hpr + c.hi;
-    if (lh >= p.heads_per_cache) return false;
+    // a head with more than 128 query rows is dealt as two items, one per 128 rows: softmax rows are independent,
+    // so the head's masses are the sum of the two items' masses
+    const int lv = (r - c.round_base) * c.hpr + c.hi;
+    if (lv >= p.heads_per_cache * p.sc_qt) return false;
     it.r = r;
     it.cache = ci;
-    it.lh = lh;
+    it.lv = lv;
+    it.lh = p.sc_qt == 2 ? lv >> 1 : lv;
+    it.qt = p.sc_qt == 2 ? lv & 1 : 0;
     it.chunk = c.chunk;
     const int tiles = (c.T - c.chunk * ST_CHUNK + 127) >> 7;
     it.nt = tiles < ST_TILES ? tiles : ST_TILES;
@@ -237,8 +243,8 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                 if (nq[kind] > 0 && !tc::mbar_wait(&bar_q_free[kind], (nq[kind] - 1) & 1u, wc, 64)) return false;
                 const uint32_t qdst = tc::smem_u32(q_s + kind * ST_TILE_BYTES);
                 tc::mbar_expect_tx(&bar_q_full[kind], ST_TILE_BYTES);
-                tc::tma_load_3d(qdst, &tm.b[item.cache], &bar_q_full[kind], 0, 0, item.lh);
-                tc::tma_load_3d(qdst + ST_TILE_BYTES / 2, &tm.b[item.cache], &bar_q_full[kind], 64, 0, item.lh);
+                tc::tma_load_3d(qdst, &tm.b[item.cache], &bar_q_full[kind], 0, item.qt * 128, item.lh);      // rows past n_q read as zero
+                tc::tma_load_3d(qdst + ST_TILE_BYTES / 2, &tm.b[item.cache], &bar_q_full[kind], 64, item.qt * 128, item.lh);
                 ++nq[kind];
                 return true;
             };
@@ -455,8 +461,9 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                 pend_T = T;
                 pend_nt = item.nt;
                 pend_j = item.chunk * ST_CHUNK + part * 128 + row;
-                pend_dst = p.scores + c.tok_off + (size_t)item.lh * T;
-                pend_out = c.scores_out ? c.scores_out + (size_t)item.lh * T : nullptr;
+                // with two query tiles per head each writes its own plane; a small kernel adds them up afterwards
+                pend_dst = (item.qt ? p.scores2 : p.scores) + c.tok_off + (size_t)item.lh * T;
+                pend_out = (c.scores_out && p.sc_qt == 1) ? c.scores_out + (size_t)item.lh * T : nullptr;
             }
         }
         if (pend) finish_pool();
@@ -468,9 +475,10 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
             if (!score_item(p, s_tab, i, item)) continue;
             const CacheDev &c = p.c[item.cache];
             const int buf = i & 1, team = c.sc_team;
-            const int g = c.head_base + item.lh;
+            const int g = c.head_base * p.sc_qt + item.lv;                     // index of the (head, query tile) pair
+            const int nq = min(128, p.n_q - 128 * item.qt);                    // query rows of this item
             tc::mbar_wait(&bar_st_ready[buf], n_a[buf] & 1u, wc, 32);
-            float2 *partials = reinterpret_cast<float2 *>(p.sc_part) + (c.sc_part_off + ((size_t)item.lh * team + item.chunk) * 128);
+            float2 *partials = reinterpret_cast<float2 *>(p.sc_part) + (c.sc_part_off + ((size_t)item.lv * team + item.chunk) * 128);
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 const int t = lane + 32 * k;
@@ -480,7 +488,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
                     if (sm[e * 128] > -INFINITY) Z += sz[e * 128] * ex2_approx(sm[e * 128] - M);
-                if (t < p.n_q) __stcg(&partials[t], make_float2(M, Z));
+                if (t < nq) __stcg(&partials[t], make_float2(M, Z));
             }
             __syncwarp();
             uint32_t last = 0u;
@@ -494,7 +502,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
             if (last) {
                 // this block is the last of its head: fold all chunks, eight chunks of the lane's four queries per sweep
                 // (32 loads in flight: the fold is a few round trips long, whatever the team's size)
-                const float2 *hp = reinterpret_cast<const float2 *>(p.sc_part) + (c.sc_part_off + (size_t)item.lh * team * 128);
+                const float2 *hp = reinterpret_cast<const float2 *>(p.sc_part) + (c.sc_part_off + (size_t)item.lv * team * 128);
                 unsigned long long *words = reinterpret_cast<unsigned long long *>(p.sc_head) + (size_t)g * 128;
                 float M[4], Z[4];
 #pragma unroll
@@ -505,7 +513,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                     for (int k = 0; k < 4; ++k)
 #pragma unroll
                         for (int e = 0; e < 8; ++e)
-                            v[k][e] = (c0 + e < team && lane + 32 * k < p.n_q) ? __ldcg(&hp[(size_t)(c0 + e) * 128 + lane + 32 * k])
+                            v[k][e] = (c0 + e < team && lane + 32 * k < nq) ? __ldcg(&hp[(size_t)(c0 + e) * 128 + lane + 32 * k])
                                                                                : make_float2(-INFINITY, 0.f);
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
@@ -524,7 +532,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     const int t = lane + 32 * k;
-                    if (t >= p.n_q) continue;
+                    if (t >= nq) continue;
                     float mp = M[k] + lg2_approx(Z[k]);
                     if (!(Z[k] > 0.f) || !isfinite(mp)) {
                         atomicOr(p.status, OBF_DEV_NONFINITE);
@@ -546,10 +554,10 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                     bool all = true;
 #pragma unroll
                     for (int k = 0; k < 4; ++k)
-                        if (lane + 32 * k < p.n_q && (v[k] >> 32) == 0ull) v[k] = ld_relaxed_gpu_u64(words + lane + 32 * k);
+                        if (lane + 32 * k < nq && (v[k] >> 32) == 0ull) v[k] = ld_relaxed_gpu_u64(words + lane + 32 * k);
 #pragma unroll
                     for (int k = 0; k < 4; ++k)
-                        if (lane + 32 * k < p.n_q && (v[k] >> 32) == 0ull) all = false;
+                        if (lane + 32 * k < nq && (v[k] >> 32) == 0ull) all = false;
                     // the warp leaves the loop as one: votes, not per-lane exits
                     if (__all_sync(0xffffffffu, all) || __any_sync(0xffffffffu, *(volatile uint32_t *)&s_abort != 0u)) break;
                     if (__any_sync(0xffffffffu, tc::global_ns() - t0 > tc::WAIT_LIMIT_NS)) {
@@ -565,7 +573,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                 for (int k = 0; k < 4; ++k) {
                     const int t = lane + 32 * k;
                     // exp2(-inf) = 0 for padding columns
-                    s_mp[fb * 128 + t] = t < p.n_q ? __uint_as_float((uint32_t)v[k]) : INFINITY;
+                    s_mp[fb * 128 + t] = t < nq ? __uint_as_float((uint32_t)v[k]) : INFINITY;
                 }
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(&bar_mp_ready[fb]);
@@ -577,6 +585,21 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
     tc::tc_fence_before();
     __syncthreads();
     if (warp == 1) tc::tmem_dealloc(tmem, 512);
+}
+
+// Heads with two query tiles: the masses of the second tile's rows are added to the first tile's.
+// grid = (ceil(T_max / 256), heads_total).
+__global__ void __launch_bounds__(256) k_score_join(const __grid_constant__ CallDev p)
+{
+    int ci, lh;
+    locate(p, blockIdx.y, ci, lh);
+    const CacheDev &c = p.c[ci];
+    const int j = blockIdx.x * 256 + threadIdx.x;
+    if (j >= c.T) return;
+    const size_t e = c.tok_off + (size_t)lh * c.T + j;
+    const float a = p.scores[e] + p.scores2[e];
+    p.scores[e] = a;
+    if (c.scores_out) c.scores_out[(size_t)lh * c.T + j] = a;
 }
 
 }  // namespace obf

@@ -205,11 +205,29 @@ def test_long_prompts_take_the_fallback_kernels(T, budget):
     assert all(r.oracle_skipped for r in reps)              # budget >= head_dim with generic values: delta = 0
 
 
-def test_more_than_128_query_rows_use_the_generic_score_kernels_and_the_tuned_gram_pass():
-    w = small("wideq", layers=2, kv_heads=2, G=5, n_obs=32, d=128, dtype="bf16", rank=2, caches=((640, 24),),
-              n_outlier=3, seed=77)
-    outs, reps, _ = run_and_check(w)
+@pytest.mark.parametrize("G,n_obs,caches", [(5, 32, ((640, 24),)),          # 160 rows: two query tiles per head
+                                            (4, 40, ((1024, 32), (300, 20), (2048, 32))),   # the paper's 40 latent steps
+                                            (8, 32, ((700, 40),)),          # 256 rows: two full tiles
+                                            (2, 65, ((513, 30),))])         # 130 rows: second tile nearly empty
+def test_between_129_and_256_query_rows_take_two_query_tiles_per_head(G, n_obs, caches):
+    w = small("wideq", layers=2, kv_heads=3, G=G, n_obs=n_obs, d=128, dtype="bf16", rank=2, caches=caches,
+              n_outlier=3, seed=77 + G)
+    a, reps, arrays = run_and_check(w)
     assert all(not r.oracle_skipped for r in reps)
+    names = [n for n, _ in P.obf_compress_profiled(par.params_for(w), a[0]["cache_structs"], a[0]["workspace"])]
+    assert "k_score_tc" in names and "k_score_join" in names
+    b, _, _ = run_and_check(w, arrays=arrays, flags=P.binding.OBF_FLAG_GENERIC_PATH)
+    for x, y in zip(a, b):
+        assert torch.equal(x["K_out"], y["K_out"])
+
+
+def test_more_than_256_query_rows_use_the_generic_score_kernels_and_the_tuned_gram_pass():
+    w = small("widerq", layers=1, kv_heads=2, G=9, n_obs=32, d=128, dtype="bf16", rank=2, caches=((640, 24),),
+              n_outlier=3, seed=78)
+    outs, reps, arrays = run_and_check(w)
+    assert all(not r.oracle_skipped for r in reps)
+    names = [n for n, _ in P.obf_compress_profiled(par.params_for(w), outs[0]["cache_structs"], outs[0]["workspace"])]
+    assert "k_score_stats" in names and "k_gram_tc" in names
 
 
 def test_exact_ties_go_to_the_lowest_position():
