@@ -162,21 +162,39 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
         }
         __syncthreads();
         const float trG = block_sum<ALG_NT>(tid < D ? B2[tid * LD + tid] : 0.f, red);
-        for (int e = tid; e < D * D; e += ALG_NT) {            // W = G_del P  -> B0
-            const int a = e / D, b = e % D;
-            float s = 0.f;
-#pragma unroll 8
-            for (int cc = 0; cc < D; ++cc) s = fmaf(B2[a * LD + cc], B1[cc * LD + b], s);
-            B0[a * LD + b] = s;
-        }
+        // two D x D x D products, a 4 x 8 register tile per thread (rows a0 + 0..3, columns b0 + 32 * 0..7:
+        // the lanes of a warp read consecutive columns, and a row's value is a broadcast)
+        auto matmul = [&](const float *X, const float *Y, float *Z) {
+            constexpr int TILES_B = D / 8 < 32 ? D / 8 : 32;      // threads across the columns
+            constexpr int NB = D / TILES_B;                       // columns per thread
+            for (int t = tid; t < (D / 4) * TILES_B; t += ALG_NT) {
+                const int a0 = (t / TILES_B) * 4, b0 = t % TILES_B;
+                float acc[4][NB];
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int j = 0; j < NB; ++j) acc[i][j] = 0.f;
+#pragma unroll 4
+                for (int cc = 0; cc < D; ++cc) {
+                    float x[4], y[NB];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) x[i] = X[(a0 + i) * LD + cc];
+#pragma unroll
+                    for (int j = 0; j < NB; ++j) y[j] = Y[cc * LD + b0 + j * TILES_B];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+#pragma unroll
+                        for (int j = 0; j < NB; ++j) acc[i][j] = fmaf(x[i], y[j], acc[i][j]);
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int j = 0; j < NB; ++j) Z[(a0 + i) * LD + b0 + j * TILES_B] = acc[i][j];
+            }
+        };
+        matmul(B2, B1, B0);                                     // W = G_del P  -> B0
         __syncthreads();
-        for (int e = tid; e < D * D; e += ALG_NT) {            // M = P W -> B2
-            const int a = e / D, b = e % D;
-            float s = 0.f;
-#pragma unroll 8
-            for (int cc = 0; cc < D; ++cc) s = fmaf(B1[a * LD + cc], B0[cc * LD + b], s);
-            B2[a * LD + b] = s;
-        }
+        matmul(B1, B0, B2);                                     // M = P W -> B2
         if (tid < D) {                                          // r_bar = P u / (A_del + eps)
             float s = 0.f;
             for (int cc = 0; cc < D; ++cc) s = fmaf(B1[tid * LD + cc], vu[cc], s);
@@ -226,24 +244,24 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
                 __syncthreads();
                 if (skip) continue;
                 const float *v = B1 + k * LD;
-                {                                                   // pvec = 2 M v on the trailing block -> vc
-                    const int i = tid >> 2, part = tid & 3;
+                // pvec = 2 M v on the trailing block -> vc: a warp takes whole rows, its lanes consecutive columns
+                if (tid <= k) vc[tid] = 0.f;
+                for (int i = k + 1 + warp; i < D; i += ALG_NT / 32) {
+                    const float *mi = B2 + i * LD;
                     float sacc = 0.f;
-                    if (i > k && i < D) {
-                        const float *mi = B2 + i * LD;
-                        for (int cc = k + 1 + part; cc < D; cc += 4) sacc = fmaf(mi[cc], v[cc], sacc);
-                    }
-                    sacc += __shfl_xor_sync(0xffffffffu, sacc, 1);
-                    sacc += __shfl_xor_sync(0xffffffffu, sacc, 2);
-                    if (part == 0 && i < D) vc[i] = i > k ? 2.f * sacc : 0.f;
+                    for (int cc = k + 1 + lane; cc < D; cc += 32) sacc = fmaf(mi[cc], v[cc], sacc);
+                    sacc = warp_sum(sacc);
+                    if (lane == 0) vc[i] = 2.f * sacc;
                 }
                 __syncthreads();
                 const float kk = block_sum<ALG_NT>(tid < D ? v[tid] * vc[tid] : 0.f, red);
                 if (tid < D) vw[tid] = vc[tid] - kk * v[tid];       // w = pvec - (v . pvec) v
                 __syncthreads();
-                for (int e = tid; e < D * D; e += ALG_NT) {         // M <- H M H = M - v w^T - w v^T
-                    const int i = e / D, j = e % D;
-                    if (i > k && j > k) B2[i * LD + j] -= v[i] * vw[j] + vw[i] * v[j];
+                // M <- H M H = M - v w^T - w v^T on the trailing block: a warp takes whole rows, its lanes consecutive columns
+                for (int i = k + 1 + warp; i < D; i += ALG_NT / 32) {
+                    const float vi = v[i], wi = vw[i];
+                    float *mi = B2 + i * LD;
+                    for (int j = k + 1 + lane; j < D; j += 32) mi[j] -= vi * vw[j] + wi * v[j];
                 }
                 __syncthreads();
             }
