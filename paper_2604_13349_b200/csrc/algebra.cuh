@@ -226,42 +226,87 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
             float *twk = tz + ALG_TRI_NE * D;                      // [ALG_TRI_NE][5][D] factors of T - lambda I
             // Householder reduction: reflector k (a unit vector, row k of B1) zeroes column k below the sub-diagonal
             const float tiny2 = 1e-20f * trM * trM;
+            // Three block barriers per column: the two reductions of a step (column norm, v . pvec) are taken by
+            // every warp for itself rather than by the block, and w = pvec - (v . pvec) v is formed on the fly.
+            constexpr int RPW = (D + ALG_NT / 32 - 1) / (ALG_NT / 32);   // rows a warp handles per sweep
 #pragma unroll 1
             for (int k = 0; k < D - 2; ++k) {
-                const float xi = (tid > k && tid < D) ? B2[tid * LD + k] : 0.f;
-                const float nrm2 = block_sum<ALG_NT>(xi * xi, red);
+                float part = 0.f;
+                for (int i = k + 2 + lane; i < D; i += 32) { const float x = B2[i * LD + k]; part = fmaf(x, x, part); }
+                const float below2 = warp_sum(part);               // squares below the sub-diagonal entry
                 const float x0 = B2[(k + 1) * LD + k];
+                const float nrm2 = below2 + x0 * x0;
                 const float nrm = sqrtf(nrm2);
                 const float al = x0 >= 0.f ? -nrm : nrm;
                 const float vn2 = 2.f * nrm * (nrm + fabsf(x0));   // |x - al e_0|^2
-                const bool skip = !(nrm2 - x0 * x0 > tiny2) || !(vn2 > 0.f);   // nothing below the sub-diagonal
+                const bool skip = !(below2 > tiny2) || !(vn2 > 0.f);   // nothing below the sub-diagonal
                 if (tid < D) {
                     float v = 0.f;
-                    if (!skip && tid > k) v = (tid == k + 1 ? x0 - al : xi) * rsqrtf(vn2);
+                    if (!skip && tid > k) v = (tid == k + 1 ? x0 - al : B2[tid * LD + k]) * rsqrtf(vn2);
                     B1[k * LD + tid] = v;
                 }
                 if (tid == 0) { ta[k] = B2[k * LD + k]; tb[k] = skip ? x0 : al; }
                 __syncthreads();
                 if (skip) continue;
                 const float *v = B1 + k * LD;
-                // pvec = 2 M v on the trailing block -> vc: a warp takes whole rows, its lanes consecutive columns
-                if (tid <= k) vc[tid] = 0.f;
-                for (int i = k + 1 + warp; i < D; i += ALG_NT / 32) {
-                    const float *mi = B2 + i * LD;
-                    float sacc = 0.f;
-                    for (int cc = k + 1 + lane; cc < D; cc += 32) sacc = fmaf(mi[cc], v[cc], sacc);
-                    sacc = warp_sum(sacc);
-                    if (lane == 0) vc[i] = 2.f * sacc;
+                {                                                   // pvec = 2 M v on the trailing block -> vc
+                    float acc[RPW];
+#pragma unroll
+                    for (int r = 0; r < RPW; ++r) acc[r] = 0.f;
+                    // rows of this warp inside the trailing block (the same for all its lanes: real branches below)
+                    const int nr = (D - (k + 1 + warp) + ALG_NT / 32 - 1) / (ALG_NT / 32);
+                    for (int cc = k + 1 + lane; cc < D; cc += 32) {
+                        const float vcc = v[cc];
+#pragma unroll
+                        for (int r = 0; r < RPW; ++r) {
+                            if (r >= nr) break;
+                            acc[r] = fmaf(B2[(k + 1 + warp + r * (ALG_NT / 32)) * LD + cc], vcc, acc[r]);
+                        }
+                    }
+#pragma unroll
+                    for (int r = 0; r < RPW; ++r) {
+                        if (r >= nr) break;
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) acc[r] += __shfl_xor_sync(0xffffffffu, acc[r], o);
+                        if (lane == 0) vc[k + 1 + warp + r * (ALG_NT / 32)] = 2.f * acc[r];
+                    }
                 }
                 __syncthreads();
-                const float kk = block_sum<ALG_NT>(tid < D ? v[tid] * vc[tid] : 0.f, red);
-                if (tid < D) vw[tid] = vc[tid] - kk * v[tid];       // w = pvec - (v . pvec) v
-                __syncthreads();
-                // M <- H M H = M - v w^T - w v^T on the trailing block: a warp takes whole rows, its lanes consecutive columns
-                for (int i = k + 1 + warp; i < D; i += ALG_NT / 32) {
-                    const float vi = v[i], wi = vw[i];
-                    float *mi = B2 + i * LD;
-                    for (int j = k + 1 + lane; j < D; j += 32) mi[j] -= vi * vw[j] + wi * v[j];
+                float kpart = 0.f;
+                for (int cc = k + 1 + lane; cc < D; cc += 32) kpart = fmaf(v[cc], vc[cc], kpart);
+                const float kk = warp_sum(kpart);                   // v . pvec, the same sum in every warp
+                // M <- H M H = M - v w^T - w v^T with w = pvec - kk v, on the trailing block
+                // (all loads of a thread's elements are issued before the first store: the loop bodies are short)
+                {
+                    constexpr int CPL = (D + 31) / 32;             // columns per lane
+                    float vj[CPL], wj[CPL];
+#pragma unroll
+                    for (int cI = 0; cI < CPL; ++cI) {
+                        const int j = k + 1 + lane + 32 * cI;
+                        vj[cI] = j < D ? v[j] : 0.f;
+                        wj[cI] = j < D ? vc[j] - kk * vj[cI] : 0.f;
+                    }
+                    const int nr = (D - (k + 1 + warp) + ALG_NT / 32 - 1) / (ALG_NT / 32);   // rows of this warp in the block
+                    const int nc = (D - (k + 1) + 31) / 32;                                  // 32-column groups in the block
+#pragma unroll
+                    for (int r = 0; r < RPW; ++r) {
+                        if (r >= nr) break;
+                        const int i = k + 1 + warp + r * (ALG_NT / 32);
+                        const float vi = v[i], wi = vc[i] - kk * vi;
+                        float m_[CPL];
+#pragma unroll
+                        for (int cI = 0; cI < CPL; ++cI) {
+                            if (cI >= nc) break;
+                            const int j = k + 1 + lane + 32 * cI;
+                            m_[cI] = j < D ? B2[i * LD + j] : 0.f;
+                        }
+#pragma unroll
+                        for (int cI = 0; cI < CPL; ++cI) {
+                            if (cI >= nc) break;
+                            const int j = k + 1 + lane + 32 * cI;
+                            if (j < D) B2[i * LD + j] = m_[cI] - (vi * wj[cI] + wi * vj[cI]);
+                        }
+                    }
                 }
                 __syncthreads();
             }
