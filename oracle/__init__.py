@@ -60,6 +60,8 @@ def lib():
         _lib.obf_oracle_scores.restype = None
         _lib.obf_oracle_topk.argtypes = [dp, ci, ci, ip, dp, dp]
         _lib.obf_oracle_topk.restype = ci
+        _lib.obf_oracle_topk_sink.argtypes = [dp, ci, ci, ci, ip, dp, dp]
+        _lib.obf_oracle_topk_sink.restype = ci
         _lib.obf_oracle_span_basis.argtypes = [dp, ci, ci, dp]
         _lib.obf_oracle_span_basis.restype = ci
         _lib.obf_oracle_sym_eig.argtypes = [dp, ci, dp, dp]
@@ -67,11 +69,13 @@ def lib():
         _lib.obf_oracle_head.argtypes = [fp, fp, fp, ci, ci, ci, ci, ci, ctypes.c_double,
                                          ip, dp, dp, dp, dp, dp, dp, dp, dp, ctypes.POINTER(Diag)]
         _lib.obf_oracle_head.restype = ci
+        _lib.obf_oracle_head_sink.argtypes = _lib.obf_oracle_head.argtypes + [ci]
+        _lib.obf_oracle_head_sink.restype = ci
         _lib.obf_oracle_compress.argtypes = [fp, fp, fp, ci, ci, ci, ci, ci, ci, ci, ci,
-                                             ctypes.c_double, ip, dp, dp, dp, ctypes.POINTER(Diag)]
+                                             ctypes.c_double, ip, dp, dp, dp, ctypes.POINTER(Diag), ci]
         _lib.obf_oracle_compress.restype = ci
         _lib.obf_oracle_layer.argtypes = [fp, fp, fp, ci, ci, ci, ci, ci, ci, ctypes.c_double,
-                                          ip, dp, dp, dp, dp, dp, ctypes.POINTER(Diag)]
+                                          ip, dp, dp, dp, dp, dp, ctypes.POINTER(Diag), ci]
         _lib.obf_oracle_layer.restype = ci
         _lib.obf_oracle_compress_layerwise.argtypes = _lib.obf_oracle_compress.argtypes
         _lib.obf_oracle_compress_layerwise.restype = ci
@@ -106,15 +110,23 @@ def scores(K, Q) -> np.ndarray:
     return A
 
 
-def topk(A, budget: int):
-    """Ascending retained positions, plus the k-th and (k+1)-th largest masses."""
+def k_eff(T: int, budget: int, n_sink: int = 0) -> int:
+    """Retained positions: the protected prefix plus at most `budget` of the others."""
+    s = max(0, min(n_sink, T))
+    return s + min(budget, T - s)
+
+
+def topk(A, budget: int, n_sink: int = 0):
+    """Ascending retained positions, plus the smallest retained and largest deleted mass among the candidates.
+
+    n_sink: the first n_sink positions are protected: retained besides the budget, no candidates."""
     A = _f64(A)
     T = A.shape[0]
-    k = min(budget, T)
-    idx = np.empty(max(k, 1), dtype=np.int32)
+    idx = np.empty(max(T, 1), dtype=np.int32)
     kth, nxt = ctypes.c_double(), ctypes.c_double()
-    k2 = lib().obf_oracle_topk(_p(A, ctypes.c_double), T, budget, _p(idx, ctypes.c_int32),
-                               ctypes.byref(kth), ctypes.byref(nxt))
+    k2 = lib().obf_oracle_topk_sink(_p(A, ctypes.c_double), T, budget, n_sink, _p(idx, ctypes.c_int32),
+                                    ctypes.byref(kth), ctypes.byref(nxt))
+    assert k2 == k_eff(T, budget, n_sink)
     return idx[:k2].copy(), kth.value, nxt.value
 
 
@@ -137,7 +149,7 @@ def sym_eig(S):
     return lam, E
 
 
-def head(K, V, Q, budget: int, rank: int, eps: float = 1e-12) -> Dict[str, object]:
+def head(K, V, Q, budget: int, rank: int, eps: float = 1e-12, n_sink: int = 0) -> Dict[str, object]:
     """Algorithm 2 (headwise) + Algorithm 3 on one (layer, KV head).
 
     K, V [T,d]; Q [n_q,d] (float32 values; bf16 inputs up-cast exactly).
@@ -145,7 +157,7 @@ def head(K, V, Q, budget: int, rank: int, eps: float = 1e-12) -> Dict[str, objec
     """
     K, V, Q = _f32(K), _f32(V), _f32(Q)
     T, d = K.shape
-    k = min(budget, T)
+    k = k_eff(T, budget, n_sink)
     idx = np.empty(max(k, 1), dtype=np.int32)
     K_out = np.zeros((max(k, 1), d), dtype=np.float64)
     V_out = np.zeros((max(k, 1), d), dtype=np.float64)
@@ -154,17 +166,17 @@ def head(K, V, Q, budget: int, rank: int, eps: float = 1e-12) -> Dict[str, objec
     proj = np.empty((d, d))
     dg = Diag()
     cd = ctypes.c_double
-    k2 = lib().obf_oracle_head(
+    k2 = lib().obf_oracle_head_sink(
         _p(K, ctypes.c_float), _p(V, ctypes.c_float), _p(Q, ctypes.c_float),
         T, d, Q.shape[0], budget, rank, eps,
         _p(idx, ctypes.c_int32), _p(K_out, cd), _p(V_out, cd), _p(A, cd), _p(delta, cd),
-        _p(rbar, cd), _p(Delta, cd), _p(eig, cd), _p(proj, cd), ctypes.byref(dg))
+        _p(rbar, cd), _p(Delta, cd), _p(eig, cd), _p(proj, cd), ctypes.byref(dg), n_sink)
     assert k2 == k
     return {"idx": idx[:k].copy(), "K_out": K_out[:k], "V_out": V_out[:k], "A": A, "delta": delta,
             "rbar": rbar, "Delta": Delta, "eigvals": eig, "proj": proj, "diag": dg.asdict()}
 
 
-def layer(K, V, Q, budget: int, rank: int, eps: float = 1e-12) -> Dict[str, object]:
+def layer(K, V, Q, budget: int, rank: int, eps: float = 1e-12, n_sink: int = 0) -> Dict[str, object]:
     """Layerwise selector (Algorithm 2, granularity L) + Algorithm 3 on one layer.
 
     K, V [kv_heads,T,d]; Q [kv_heads,n_q,d].  The retained positions are TopK_B of the masses summed over
@@ -173,7 +185,7 @@ def layer(K, V, Q, budget: int, rank: int, eps: float = 1e-12) -> Dict[str, obje
     """
     K, V, Q = _f32(K), _f32(V), _f32(Q)
     H, T, d = K.shape
-    k = min(budget, T)
+    k = k_eff(T, budget, n_sink)
     idx = np.empty((H, max(k, 1)), dtype=np.int32)
     K_out = np.zeros((H, max(k, 1), d), dtype=np.float64)
     V_out = np.zeros((H, max(k, 1), d), dtype=np.float64)
@@ -185,20 +197,20 @@ def layer(K, V, Q, budget: int, rank: int, eps: float = 1e-12) -> Dict[str, obje
     k2 = lib().obf_oracle_layer(
         _p(K, ctypes.c_float), _p(V, ctypes.c_float), _p(Q, ctypes.c_float),
         H, T, d, Q.shape[1], budget, rank, eps,
-        _p(idx, ctypes.c_int32), _p(K_out, cd), _p(V_out, cd), _p(S, cd), _p(A, cd), _p(delta, cd), diags)
+        _p(idx, ctypes.c_int32), _p(K_out, cd), _p(V_out, cd), _p(S, cd), _p(A, cd), _p(delta, cd), diags, n_sink)
     assert k2 == k
     return {"idx": idx[:, :k].copy(), "K_out": K_out[:, :k], "V_out": V_out[:, :k], "S": S, "A": A,
             "delta": delta, "diag": [diags[h].asdict() for h in range(H)]}
 
 
 def compress(K, V, Q, q_heads: int, n_obs: int, budget: int, rank: int,
-             eps: float = 1e-12, layerwise: bool = False) -> Dict[str, object]:
+             eps: float = 1e-12, layerwise: bool = False, n_sink: int = 0) -> Dict[str, object]:
     """A whole cache: K, V [layers, kv_heads, T, d]; Q [layers, q_heads, n_obs, d].
 
     layerwise: one retained set per layer (masses summed over its KV heads) instead of one per head."""
     K, V, Q = _f32(K), _f32(V), _f32(Q)
     layers, kv_heads, T, d = K.shape
-    k = min(budget, T)
+    k = k_eff(T, budget, n_sink)
     heads = layers * kv_heads
     idx = np.empty((layers, kv_heads, k), dtype=np.int32)
     K_out = np.zeros((layers, kv_heads, k, d), dtype=np.float64)
@@ -210,6 +222,6 @@ def compress(K, V, Q, q_heads: int, n_obs: int, budget: int, rank: int,
     fn(
         _p(K, ctypes.c_float), _p(V, ctypes.c_float), _p(Q, ctypes.c_float),
         layers, kv_heads, q_heads, n_obs, T, d, budget, rank, eps,
-        _p(idx, ctypes.c_int32), _p(K_out, cd), _p(V_out, cd), _p(delta, cd), diags)
+        _p(idx, ctypes.c_int32), _p(K_out, cd), _p(V_out, cd), _p(delta, cd), diags, n_sink)
     return {"idx": idx, "K_out": K_out, "V_out": V_out, "delta": delta,
             "diag": [diags[i].asdict() for i in range(heads)]}

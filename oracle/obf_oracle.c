@@ -16,6 +16,8 @@
  *               closed form, library softmax, permutation equivariance
  *   top-k       pinned: brute-force full sort on tiny inputs, library stable
  *               argsort, planted exact ties
+ *   sink prefix pinned: protected positions always retained, the rest equals
+ *               the plain top-k of the remaining positions (library argsort)
  *   layerwise   pinned: one KV head reduces to the headwise result, identical
  *               heads reduce to the headwise result, library argsort of the
  *               summed masses, retained set shared by the heads of a layer
@@ -110,24 +112,39 @@ static int cmp_int_asc(const void *x, const void *y)
 }
 
 /*
- * Order positions by (mass descending, position ascending), keep the first
- * k_eff = min(budget, T), return them as an ascending index list (Section 3.1:
- * a retained cache is a subsequence i_1 < ... < i_m).  kth/next receive the
- * k_eff-th and (k_eff+1)-th largest masses (next = -1 when k_eff == T).
+ * The first n_sink positions are protected (the sink prefix of App. F, "Right
+ * padding": the compressors protect the first s indices of the cache); they are
+ * no candidates of the selection (the eligible set of Section 3.2 leaves them
+ * out) and are retained besides the budget.  The other positions are ordered by
+ * (mass descending, position ascending) and the first min(budget, T - n_sink)
+ * of them are kept.  Returns k_eff = min(n_sink, T) + that many, the retained
+ * positions as an ascending index list (Section 3.1: a retained cache is a
+ * subsequence i_1 < ... < i_m).  kth/next receive the smallest retained and the
+ * largest deleted mass among the candidates (-1 when there is none).
  */
+int obf_oracle_topk_sink(const double *A, int T, int budget, int n_sink, int32_t *idx, double *kth, double *next)
+{
+    int s = n_sink < T ? n_sink : T;
+    if (s < 0) s = 0;
+    const int nc = T - s;                                  /* candidates */
+    int kc = budget < nc ? budget : nc;
+    if (kc < 0) kc = 0;
+    score_pos_t *sp = (score_pos_t *)malloc((size_t)(nc > 0 ? nc : 1) * sizeof(score_pos_t));
+    for (int j = s; j < T; ++j) { sp[j - s].a = A[j]; sp[j - s].j = j; }
+    qsort(sp, (size_t)nc, sizeof(score_pos_t), cmp_score_desc_index_asc);
+    for (int r = 0; r < s; ++r) idx[r] = r;
+    for (int r = 0; r < kc; ++r) idx[s + r] = sp[r].j;
+    if (kth)  *kth  = kc > 0 ? sp[kc - 1].a : -1.0;
+    if (next) *next = kc < nc ? sp[kc].a : -1.0;
+    qsort(idx, (size_t)(s + kc), sizeof(int32_t), cmp_int_asc);
+    free(sp);
+    return s + kc;
+}
+
+/* TopK_B with every position eligible. */
 int obf_oracle_topk(const double *A, int T, int budget, int32_t *idx, double *kth, double *next)
 {
-    int k = budget < T ? budget : T;
-    if (k < 0) k = 0;
-    score_pos_t *sp = (score_pos_t *)malloc((size_t)T * sizeof(score_pos_t));
-    for (int j = 0; j < T; ++j) { sp[j].a = A[j]; sp[j].j = j; }
-    qsort(sp, (size_t)T, sizeof(score_pos_t), cmp_score_desc_index_asc);
-    for (int r = 0; r < k; ++r) idx[r] = sp[r].j;
-    if (kth)  *kth  = k > 0 ? sp[k - 1].a : -1.0;
-    if (next) *next = k < T ? sp[k].a : -1.0;
-    qsort(idx, (size_t)k, sizeof(int32_t), cmp_int_asc);
-    free(sp);
-    return k;
+    return obf_oracle_topk_sink(A, T, budget, 0, idx, kth, next);
 }
 
 /* ------------------------------------------------------------------ */
@@ -272,11 +289,11 @@ static int backfill_given_selection(const float *K, const float *V, const double
                                     double *delta_out, double *rbar_out, double *Delta_out,
                                     double *eigvals_out, double *proj_out, obf_oracle_diag_t *diag);
 
-int obf_oracle_head(const float *K, const float *V, const float *Q,
-                    int T, int d, int n_q, int budget, int rank, double eps,
-                    int32_t *idx, double *K_out, double *V_out,
-                    double *A_out, double *delta_out, double *rbar_out, double *Delta_out,
-                    double *eigvals_out, double *proj_out, obf_oracle_diag_t *diag)
+int obf_oracle_head_sink(const float *K, const float *V, const float *Q,
+                         int T, int d, int n_q, int budget, int rank, double eps,
+                         int32_t *idx, double *K_out, double *V_out,
+                         double *A_out, double *delta_out, double *rbar_out, double *Delta_out,
+                         double *eigvals_out, double *proj_out, obf_oracle_diag_t *diag, int n_sink)
 {
     /* O1: attention mass */
     double *A = (double *)malloc((size_t)T * sizeof(double));
@@ -285,12 +302,22 @@ int obf_oracle_head(const float *K, const float *V, const float *Q,
 
     /* O2: headwise TopK_B, ascending index list */
     double kth = 0.0, next = -1.0;
-    int k = obf_oracle_topk(A, T, budget, idx, &kth, &next);
+    int k = obf_oracle_topk_sink(A, T, budget, n_sink, idx, &kth, &next);
 
     backfill_given_selection(K, V, A, T, d, k, rank, eps, idx, kth, next, K_out, V_out,
                              delta_out, rbar_out, Delta_out, eigvals_out, proj_out, diag);
     free(A);
     return k;
+}
+
+int obf_oracle_head(const float *K, const float *V, const float *Q,
+                    int T, int d, int n_q, int budget, int rank, double eps,
+                    int32_t *idx, double *K_out, double *V_out,
+                    double *A_out, double *delta_out, double *rbar_out, double *Delta_out,
+                    double *eigvals_out, double *proj_out, obf_oracle_diag_t *diag)
+{
+    return obf_oracle_head_sink(K, V, Q, T, d, n_q, budget, rank, eps, idx, K_out, V_out, A_out, delta_out, rbar_out,
+                                Delta_out, eigvals_out, proj_out, diag, 0);
 }
 
 /*
@@ -454,22 +481,23 @@ int obf_oracle_compress(const float *K, const float *V, const float *Q,
                         int layers, int kv_heads, int q_heads, int n_obs, int T, int d,
                         int budget, int rank, double eps,
                         int32_t *idx_out, double *K_out, double *V_out,
-                        double *delta_out, obf_oracle_diag_t *diag_out)
+                        double *delta_out, obf_oracle_diag_t *diag_out, int n_sink)
 {
     const int G = q_heads / kv_heads;
     const int n_q = G * n_obs;
-    const int k = budget < T ? budget : T;
+    const int sink = n_sink < T ? (n_sink > 0 ? n_sink : 0) : T;
+    const int k = sink + (budget < T - sink ? budget : T - sink);
     const int heads = layers * kv_heads;
 #pragma omp parallel for schedule(dynamic, 1)
     for (int lh = 0; lh < heads; ++lh) {
         const float *Kh = K + (size_t)lh * T * d;
         const float *Vh = V + (size_t)lh * T * d;
         const float *Qh = Q + (size_t)lh * n_q * d;
-        obf_oracle_head(Kh, Vh, Qh, T, d, n_q, budget, rank, eps,
-                        idx_out + (size_t)lh * k,
-                        K_out + (size_t)lh * k * d, V_out + (size_t)lh * k * d,
-                        NULL, delta_out ? delta_out + (size_t)lh * d : NULL, NULL, NULL, NULL, NULL,
-                        diag_out ? diag_out + lh : NULL);
+        obf_oracle_head_sink(Kh, Vh, Qh, T, d, n_q, budget, rank, eps,
+                             idx_out + (size_t)lh * k,
+                             K_out + (size_t)lh * k * d, V_out + (size_t)lh * k * d,
+                             NULL, delta_out ? delta_out + (size_t)lh * d : NULL, NULL, NULL, NULL, NULL,
+                             diag_out ? diag_out + lh : NULL, n_sink);
     }
     return k;
 }
@@ -489,7 +517,7 @@ int obf_oracle_compress(const float *K, const float *V, const float *Q,
 int obf_oracle_layer(const float *K, const float *V, const float *Q,
                      int kv_heads, int T, int d, int n_q, int budget, int rank, double eps,
                      int32_t *idx_out, double *K_out, double *V_out,
-                     double *S_out, double *A_out, double *delta_out, obf_oracle_diag_t *diag_out)
+                     double *S_out, double *A_out, double *delta_out, obf_oracle_diag_t *diag_out, int n_sink)
 {
     double *A = (double *)malloc((size_t)kv_heads * T * sizeof(double));
     double *S = (double *)calloc((size_t)T, sizeof(double));
@@ -499,10 +527,9 @@ int obf_oracle_layer(const float *K, const float *V, const float *Q,
     }
     if (S_out) memcpy(S_out, S, (size_t)T * sizeof(double));
     if (A_out) memcpy(A_out, A, (size_t)kv_heads * T * sizeof(double));
-    const int kmax = budget < T ? budget : T;
-    int32_t *idx = (int32_t *)malloc((size_t)(kmax > 0 ? kmax : 1) * sizeof(int32_t));
+    int32_t *idx = (int32_t *)malloc((size_t)T * sizeof(int32_t));
     double kth = 0.0, next = -1.0;
-    const int k = obf_oracle_topk(S, T, budget, idx, &kth, &next);
+    const int k = obf_oracle_topk_sink(S, T, budget, n_sink, idx, &kth, &next);
     for (int h = 0; h < kv_heads; ++h) {
         memcpy(idx_out + (size_t)h * k, idx, (size_t)k * sizeof(int32_t));
         backfill_given_selection(K + (size_t)h * T * d, V + (size_t)h * T * d, A + (size_t)h * T, T, d, k, rank, eps,
@@ -519,17 +546,18 @@ int obf_oracle_compress_layerwise(const float *K, const float *V, const float *Q
                                   int layers, int kv_heads, int q_heads, int n_obs, int T, int d,
                                   int budget, int rank, double eps,
                                   int32_t *idx_out, double *K_out, double *V_out,
-                                  double *delta_out, obf_oracle_diag_t *diag_out)
+                                  double *delta_out, obf_oracle_diag_t *diag_out, int n_sink)
 {
     const int G = q_heads / kv_heads;
     const int n_q = G * n_obs;
-    const int k = budget < T ? budget : T;
+    const int sink = n_sink < T ? (n_sink > 0 ? n_sink : 0) : T;
+    const int k = sink + (budget < T - sink ? budget : T - sink);
 #pragma omp parallel for schedule(dynamic, 1)
     for (int l = 0; l < layers; ++l) {
         const size_t lh = (size_t)l * kv_heads;
         obf_oracle_layer(K + lh * T * d, V + lh * T * d, Q + lh * n_q * d, kv_heads, T, d, n_q, budget, rank, eps,
                          idx_out + lh * k, K_out + lh * k * d, V_out + lh * k * d, NULL, NULL,
-                         delta_out ? delta_out + lh * d : NULL, diag_out ? diag_out + lh : NULL);
+                         delta_out ? delta_out + lh * d : NULL, diag_out ? diag_out + lh : NULL, n_sink);
     }
     return k;
 }

@@ -493,3 +493,48 @@ def test_layerwise_whole_cache_matches_per_layer_calls():
         lay = oracle.layer(a["K"][l], a["V"][l], Qv[l], w.caches[0].budget, w.rank)
         assert np.array_equal(out["idx"][l], lay["idx"])
         assert np.array_equal(out["V_out"][l], lay["V_out"])
+
+
+# --------------------------------------------------------------------------
+# protected sink prefix (the first s positions are retained besides the budget and are no candidates)
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("seed,T,budget,n_sink", [(0, 50, 7, 4), (1, 50, 7, 0), (2, 12, 20, 4), (3, 9, 3, 9), (4, 6, 2, 10)])
+def test_sink_prefix_is_retained_besides_the_budget(seed, T, budget, n_sink):
+    g = np.random.default_rng(seed)
+    A = g.random(T)
+    A[:2] = 0.0                                            # protected even when nothing attends to them
+    idx, kth, nxt = oracle.topk(A, budget, n_sink)
+    s = min(n_sink, T)
+    rest = np.arange(s, T)
+    want_rest = rest[np.argsort(-A[rest], kind="stable")[:min(budget, T - s)]]      # library sort of the candidates
+    want = np.sort(np.concatenate([np.arange(s), want_rest])).astype(np.int32)
+    assert np.array_equal(idx, want)
+    assert len(idx) == oracle.k_eff(T, budget, n_sink) == s + min(budget, T - s)
+    if len(want_rest):
+        assert kth == A[want_rest].min()
+    deleted = np.setdiff1d(rest, want_rest)
+    assert nxt == (A[deleted].max() if len(deleted) else -1.0)
+
+
+def test_sink_prefix_head_backfill_uses_the_union_as_retained_set():
+    K, V, Q = rand_head(12, 90, 16, 6, heavy=3)
+    out = oracle.head(K, V, Q, budget=6, rank=2, n_sink=4)
+    A = lib_scores(K, Q)
+    assert out["idx"][:4].tolist() == [0, 1, 2, 3] and len(out["idx"]) == 10
+    delta, v_out = lib_obf_given_idx(V, A, out["idx"], 2)
+    np.testing.assert_allclose(out["delta"], delta, atol=1e-9)
+    np.testing.assert_allclose(out["V_out"], v_out, atol=1e-9)
+    keep = np.zeros(90, bool); keep[out["idx"]] = True
+    assert out["diag"]["a_keep"] == pytest.approx(A[keep].sum(), rel=1e-12)       # sink masses count as retained demand
+    plain = oracle.head(K, V, Q, budget=6, rank=2)
+    assert np.array_equal(oracle.head(K, V, Q, budget=6, rank=2, n_sink=0)["idx"], plain["idx"])
+
+
+def test_sink_prefix_with_the_layerwise_selector():
+    K, V, Q = rand_layer(13, 3, 70, 16, 5)
+    lay = oracle.layer(K, V, Q, 8, 1, n_sink=4)
+    S = sum(lib_scores(K[h], Q[h]) for h in range(3))
+    rest = np.arange(4, 70)
+    want = np.sort(np.concatenate([np.arange(4), rest[np.argsort(-S[rest], kind="stable")[:8]]]))
+    for h in range(3):
+        assert np.array_equal(lay["idx"][h], want)
