@@ -81,6 +81,14 @@ typedef enum { OBF_F32 = 0, OBF_BF16 = 1 } obf_dtype_t;
                                       per head); gather and OBF then run per head with the head's own masses.
                                       Needs every T <= 16384, else OBF_ERR_UNSUPPORTED                          */
 
+#define OBF_FLAG_SINK(n) (((uint32_t)(n) & 0xFFu) << 8)
+                                   /* protected sink prefix (App. F of the paper: the compressors protect the first s
+                                      indices of the cache; the eligible set of Section 3.2 leaves the sink out): the
+                                      first n <= 255 positions of every cache are retained besides the budget and are no
+                                      candidates of the selection, so k_eff = min(n, T) + min(budget, T - min(n, T));
+                                      size the outputs with that k_eff                                            */
+#define OBF_FLAG_SINK_OF(flags) (((flags) >> 8) & 0xFFu)
+
 #define OBF_MAX_CACHES 32          /* caches per call                                              */
 #define OBF_MAX_T (1 << 20)        /* prompt positions per cache                                   */
 

@@ -34,6 +34,17 @@ OBF_DEV_SPAN_FULL = 0x200
 
 OBF_FLAG_GENERIC_PATH = 0x1
 OBF_FLAG_LAYERWISE = 0x2        # one retained set per layer (masses summed over its KV heads)
+
+
+def OBF_FLAG_SINK(n: int) -> int:
+    """Protected sink prefix: the first n <= 255 positions are retained besides the budget."""
+    return (int(n) & 0xFF) << 8
+
+
+def k_eff(T: int, budget: int, flags: int = 0) -> int:
+    """Rows of K_out / V_out / idx per head for a cache of T positions."""
+    s = min((flags >> 8) & 0xFF, T)
+    return s + min(int(budget), T - s)
 OBF_MAX_CACHES = 32
 
 EXPORTS = ("obf_workspace_bytes", "obf_compress", "evict_only", "obf_host_arena_bytes",
@@ -272,7 +283,7 @@ def compress_caches(params: ObfParams, caches_in: Sequence[Dict[str, object]], *
         assert K.is_cuda and K.is_contiguous() and V.is_contiguous() and Q.is_contiguous()
         assert K.dtype == dt and V.dtype == dt and Q.dtype == dt
         T = K.shape[2]
-        ke = min(int(ci["budget"]), T)
+        ke = k_eff(T, ci["budget"], params.flags)
         dev = K.device
         o = {
             "K_out": torch.empty((params.layers, params.kv_heads, ke, params.head_dim), dtype=dt, device=dev),

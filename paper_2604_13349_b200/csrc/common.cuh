@@ -64,6 +64,7 @@ struct CallDev {
     float eps;
     int32_t kv_heads;         // KV heads per layer
     int32_t layerwise;        // 1: one retained set per layer (masses summed over its KV heads)
+    int32_t n_sink;           // protected prefix: the first n_sink positions are retained besides the budget
     // workspace
     uint32_t *status;
     float *scores;            // [sum heads*T] attention mass (Eq. 1)
@@ -193,6 +194,12 @@ __device__ __forceinline__ float block_max(float v, float *red)
 __device__ __forceinline__ uint32_t score_key_bits(uint32_t u)
 {
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// Selection key of position j: protected positions sort above every mass.
+__device__ __forceinline__ uint32_t select_key(const CallDev &p, int j, uint32_t mass_bits)
+{
+    return j < p.n_sink ? 0xFFFFFFFFu : score_key_bits(mass_bits);
 }
 
 __device__ __forceinline__ float key_score(uint32_t k)

@@ -182,7 +182,7 @@ __global__ void __launch_bounds__(SEL_NT) k_select(const __grid_constant__ CallD
         __syncthreads();
         const uint32_t prefix = s_prefix;
         for (int j = tid; j < T; j += SEL_NT) {
-            const uint32_t u = score_key_bits(A[j]);
+            const uint32_t u = select_key(p, j, A[j]);
             if ((u & mask) == prefix) atomicAdd(&hist[(u >> shift) & 255u], 1u);
         }
         __syncthreads();
@@ -209,7 +209,7 @@ __global__ void __launch_bounds__(SEL_NT) k_select(const __grid_constant__ CallD
         const bool valid = j < T;
         const uint32_t abits = valid ? A[j] : 0u;
         const float a = __uint_as_float(abits);
-        const uint32_t u = valid ? score_key_bits(abits) : 0u;
+        const uint32_t u = valid ? select_key(p, j, abits) : 0u;
         const bool gt = valid && u > tau, eq = valid && u == tau;
         uint32_t v = (gt ? 1u : 0u) | (eq ? 0x10000u : 0u);
         uint32_t inc = v;
@@ -255,11 +255,11 @@ __global__ void __launch_bounds__(SEL_NT) k_select(const __grid_constant__ CallD
     const float next = block_max<SEL_NT>(nx, red);
     if (tid == 0) {
         float *s = p.sums + (size_t)blockIdx.x * 4;
-        s[0] = a_keep; s[1] = a_del; s[2] = key_score(tau); s[3] = next;
+        s[0] = a_keep; s[1] = a_del; s[2] = tau == 0xFFFFFFFFu ? INFINITY : key_score(tau); s[3] = next;
         if (c.diag) {
             obf_diag_t dg;
             dg.a_keep = a_keep; dg.a_del = a_del; dg.alpha = a_del / (a_keep + p.eps);
-            dg.rcr = 0.f; dg.delta_norm = 0.f; dg.kth_score = key_score(tau); dg.next_score = next;
+            dg.rcr = 0.f; dg.delta_norm = 0.f; dg.kth_score = tau == 0xFFFFFFFFu ? INFINITY : key_score(tau); dg.next_score = next;
             dg.lam_1 = dg.lam_rho = dg.lam_next = 0.f;
             dg.span_rank = -1; dg.rho_eff = 0; dg.status = OBF_DEV_SKIPPED; dg.revr = 0.f;
             c.diag[lh] = dg;
@@ -311,7 +311,7 @@ __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ Call
     int32_t *idx = c.idx_out + (size_t)lh * k;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    for (int j = tid; j < T; j += NT) sel_keys[j] = score_key_bits(A[j]);
+    for (int j = tid; j < T; j += NT) sel_keys[j] = select_key(p, j, A[j]);
     if (tid == 0) { s_prefix = 0u; s_want = (uint32_t)k; }
     uint32_t mask = 0u;
     const int T_pad = (T + NT - 1) / NT * NT;
@@ -407,7 +407,7 @@ __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ Call
                 sel_keys[j] = (kp && pos < (uint32_t)k) ? pos : 0xFFFFFFFFu;
             }
         } else if (valid) {
-            const float a = key_score(u);
+            const float a = j < p.n_sink ? __uint_as_float(A[j]) : key_score(u);     // a protected position's key is not its mass
             keep[j] = kp ? 1 : 0;
             if (kp) {
                 Af[j] = -1.0f;             // later passes need the mass of deleted tokens only
@@ -448,11 +448,11 @@ __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ Call
             const float a_del = block_sum<NT>(sd, red);
             if (tid == 0) {
                 float *sm = p.sums + (size_t)(c.head_base + lh + h) * 4;
-                sm[0] = a_keep; sm[1] = a_del; sm[2] = key_score(tau); sm[3] = next;
+                sm[0] = a_keep; sm[1] = a_del; sm[2] = tau == 0xFFFFFFFFu ? INFINITY : key_score(tau); sm[3] = next;
                 if (c.diag) {
                     obf_diag_t dg;
                     dg.a_keep = a_keep; dg.a_del = a_del; dg.alpha = a_del / (a_keep + p.eps);
-                    dg.rcr = 0.f; dg.delta_norm = 0.f; dg.kth_score = key_score(tau); dg.next_score = next;
+                    dg.rcr = 0.f; dg.delta_norm = 0.f; dg.kth_score = tau == 0xFFFFFFFFu ? INFINITY : key_score(tau); dg.next_score = next;
                     dg.lam_1 = dg.lam_rho = dg.lam_next = 0.f;
                     dg.span_rank = -1; dg.rho_eff = 0; dg.status = OBF_DEV_SKIPPED; dg.revr = 0.f;
                     c.diag[lh + h] = dg;
@@ -466,11 +466,11 @@ __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ Call
     const float next = block_max<NT>(nx, red);
     if (tid == 0) {
         float *sm = p.sums + (size_t)blockIdx.x * 4;
-        sm[0] = a_keep; sm[1] = a_del; sm[2] = key_score(tau); sm[3] = next;
+        sm[0] = a_keep; sm[1] = a_del; sm[2] = tau == 0xFFFFFFFFu ? INFINITY : key_score(tau); sm[3] = next;
         if (c.diag) {
             obf_diag_t dg;
             dg.a_keep = a_keep; dg.a_del = a_del; dg.alpha = a_del / (a_keep + p.eps);
-            dg.rcr = 0.f; dg.delta_norm = 0.f; dg.kth_score = key_score(tau); dg.next_score = next;
+            dg.rcr = 0.f; dg.delta_norm = 0.f; dg.kth_score = tau == 0xFFFFFFFFu ? INFINITY : key_score(tau); dg.next_score = next;
             dg.lam_1 = dg.lam_rho = dg.lam_next = 0.f;
             dg.span_rank = -1; dg.rho_eff = 0; dg.status = OBF_DEV_SKIPPED; dg.revr = 0.f;
             c.diag[lh] = dg;

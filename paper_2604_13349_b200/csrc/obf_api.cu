@@ -95,6 +95,13 @@ static int choose_splits(int heads_total, int T_max)
     return s;
 }
 
+// Retained positions of a cache: the protected prefix plus at most `budget` of the other positions.
+static inline int k_eff_of(const obf_params_t *p, const obf_cache_t &c)
+{
+    const int s = (int)OBF_FLAG_SINK_OF(p->flags) < c.T ? (int)OBF_FLAG_SINK_OF(p->flags) : c.T;
+    return s + (c.budget < c.T - s ? c.budget : c.T - s);
+}
+
 static obf_status_t validate_shapes(const obf_params_t *p, const obf_cache_t *caches, int32_t n, int rank)
 {
     if (!p || !caches) return OBF_ERR_INVALID_ARG;
@@ -137,7 +144,7 @@ static void make_layout(const obf_params_t *p, const obf_cache_t *caches, int32_
     if (L.tuned && rank > 0) {
         long long total = 0;
         for (int i = 0; i < n; ++i) {
-            const int T = caches[i].T, ke = caches[i].budget < T ? caches[i].budget : T;
+            const int T = caches[i].T, ke = k_eff_of(p, caches[i]);
             L.nsub_del[i] = (T + GT_TILE - 1) / GT_TILE;
             L.nsub_keep[i] = (ke >= d && T > ke) ? (ke + GT_TILE - 1) / GT_TILE : 0;
             L.sub_base[i] = total;
@@ -426,7 +433,7 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
         c.k_out = caches[i].k_out; c.v_out = caches[i].v_out; c.idx_out = caches[i].idx_out;
         c.diag = caches[i].diag_out; c.scores_out = caches[i].scores_out; c.delta_out = caches[i].delta_out;
         c.T = caches[i].T;
-        c.k_eff = caches[i].budget < caches[i].T ? caches[i].budget : caches[i].T;
+        c.k_eff = k_eff_of(p, caches[i]);
         c.head_base = i * hpc;
         c.tok_off = L.tok_off[i];
         c.nsub_del = L.tc_per ? L.nsub_del[i] : 0;
@@ -465,6 +472,7 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
     cd.scores2 = reinterpret_cast<float *>(ws + L.off_scores2);
     cd.kv_heads = p->kv_heads;
     cd.layerwise = (p->flags & OBF_FLAG_LAYERWISE) ? 1 : 0;
+    cd.n_sink = (int32_t)OBF_FLAG_SINK_OF(p->flags);
     cd.sc_part = reinterpret_cast<float *>(ws + L.off_sc_part);
     cd.sc_head = reinterpret_cast<float *>(ws + L.off_sc_head);
     cd.sc_cnt = reinterpret_cast<uint32_t *>(ws + L.off_sc_sync);
@@ -531,7 +539,7 @@ static void host_arena_layout(const obf_params_t *p, const obf_cache_t *caches, 
     const size_t hpc = (size_t)p->layers * p->kv_heads, d = p->head_dim;
     size_t o = 0;
     for (int i = 0; i < n; ++i) {
-        const size_t T = caches[i].T, ke = caches[i].budget < caches[i].T ? caches[i].budget : caches[i].T;
+        const size_t T = caches[i].T, ke = (size_t)k_eff_of(p, caches[i]);
         H.k[i] = o; o = align_up(o + hpc * T * d * e, 256);
         H.v[i] = o; o = align_up(o + hpc * T * d * e, 256);
         H.q[i] = o; o = align_up(o + (size_t)p->layers * p->q_heads * p->n_obs * d * e, 256);
@@ -598,7 +606,7 @@ obf_status_t obf_compress_host(const obf_params_t *params, const obf_cache_t *ca
     if (s != OBF_OK) return s;
     for (int i = 0; i < n_caches; ++i) {
         const obf_cache_t &c = caches[i];
-        const size_t T = c.T, ke = c.budget < c.T ? c.budget : c.T;
+        const size_t T = c.T, ke = (size_t)k_eff_of(params, c);
         OBF_CUDA_TRY(cudaMemcpyAsync(c.k_out, base + H.k_out[i], hpc * ke * d * e, cudaMemcpyDeviceToHost, st));
         OBF_CUDA_TRY(cudaMemcpyAsync(c.v_out, base + H.v_out[i], hpc * ke * d * e, cudaMemcpyDeviceToHost, st));
         OBF_CUDA_TRY(cudaMemcpyAsync(c.idx_out, base + H.idx[i], hpc * ke * 4, cudaMemcpyDeviceToHost, st));

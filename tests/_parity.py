@@ -75,14 +75,14 @@ def check_head(dtype: str, K: np.ndarray, V: np.ndarray, Q: np.ndarray, budget: 
                g_scores: Optional[np.ndarray], g_delta: Optional[np.ndarray], g_diag: Optional[dict],
                in_kbits: np.ndarray, in_vbits: np.ndarray, name: str = "",
                ref: Optional[dict] = None, sel_scores: Optional[np.ndarray] = None,
-               tie_band: float = TIE_BAND) -> HeadReport:
+               tie_band: float = TIE_BAND, k_expected: Optional[int] = None) -> HeadReport:
     """K, V, Q: float32 values of one head (bf16 already up-cast).  g_*: the CUDA path's outputs.
 
     ref: the oracle's result for this head when it was not chosen headwise (layerwise selector), with
     sel_scores the masses the selection ran on and tie_band the band on those."""
     rep = HeadReport()
     T, d = K.shape
-    k = min(budget, T)
+    k = min(budget, T) if k_expected is None else k_expected
     if ref is None:
         ref = oracle.head(K, V, Q, budget, rank)
     A = ref["A"]

@@ -407,3 +407,63 @@ def test_residual_with_two_equal_leading_singular_values(rank):
     if rank >= 2:
         assert all(r.gap_rel > 0.5 for r in reps)            # the plane itself is well separated from the rest
         assert np.all(np.linalg.norm(d, axis=-1) > 1e-4)
+
+
+# ---------------------------------------------------------------------------
+# protected sink prefix: the first s positions are retained besides the budget
+# ---------------------------------------------------------------------------
+def check_sink(w, n_sink, outs, arrays, layerwise=False, rank=None):
+    rank = w.rank if rank is None else rank
+    d, n_q, H = w.head.head_dim, w.n_q, w.kv_heads
+    bits = np.int16 if w.dtype == "bf16" else np.int32
+    reps = []
+    for ci in range(len(w.caches)):
+        a, out = arrays[ci], outs[ci]
+        budget = w.caches[ci].budget
+        Qv = a["Q"].reshape(w.layers, H, n_q, d)
+        diags = P.parse_diag(out["diag"])
+        for l in range(w.layers):
+            K, V, Q = par.f32_view(a["K"][l], w.dtype), par.f32_view(a["V"][l], w.dtype), par.f32_view(Qv[l], w.dtype)
+            lay = oracle.layer(K, V, Q, budget, rank, n_sink=n_sink) if layerwise else None
+            for h in range(H):
+                if layerwise:
+                    ref = {"A": lay["A"][h], "idx": lay["idx"][h], "delta": lay["delta"][h], "V_out": lay["V_out"][h],
+                           "diag": lay["diag"][h]}
+                    sel, band = lay["S"].copy(), par.TIE_BAND * H
+                else:
+                    ref = oracle.head(K[h], V[h], Q[h], budget, rank, n_sink=n_sink)
+                    sel, band = ref["A"].copy(), par.TIE_BAND
+                sel[:n_sink] = np.inf                               # protected positions are never in the tie band
+                g_idx = out["idx"][l, h].cpu().numpy()
+                assert g_idx[:min(n_sink, K.shape[1])].tolist() == list(range(min(n_sink, K.shape[1])))
+                reps.append(par.check_head(
+                    w.dtype, K[h], V[h], Q[h], budget, rank, g_idx, par.out_bits(out["K_out"][l, h]),
+                    par.out_bits(out["V_out"][l, h]), par.out_to_f32(out["V_out"][l, h]),
+                    out["scores"][l, h].cpu().numpy(), out["delta"][l, h].cpu().numpy(), diags[l * H + h],
+                    a["K"][l, h].view(bits), a["V"][l, h].view(bits), name="sink cache %d layer %d head %d" % (ci, l, h),
+                    ref=ref, sel_scores=sel, tie_band=band, k_expected=oracle.k_eff(K.shape[1], budget, n_sink)))
+    return reps
+
+
+@pytest.mark.parametrize("dtype,d,caches,layerwise", [
+    ("f32", 64, ((200, 12), (90, 9)), False), ("bf16", 128, ((300, 20), (777, 100), (130, 129)), False),
+    ("f32", 64, ((200, 12),), True), ("bf16", 128, ((512, 28),), True)])
+def test_sink_prefix_is_retained_besides_the_budget(dtype, d, caches, layerwise):
+    w = small("sink", layers=2, kv_heads=3, G=2, n_obs=6, d=d, dtype=dtype, rank=2, caches=caches, seed=91, n_sink=0)
+    arrays = [synth.gen_cache(w, ci) for ci in range(len(w.caches))]
+    flags = P.binding.OBF_FLAG_SINK(4) | (P.binding.OBF_FLAG_LAYERWISE if layerwise else 0)
+    outs, _, st = par.run_gpu(w, arrays, flags=flags)
+    assert st & 0xFF == 0
+    for ci, (T, b) in enumerate(caches):
+        assert outs[ci]["idx"].shape[-1] == min(4, T) + min(b, T - min(4, T))
+    reps = check_sink(w, 4, outs, arrays, layerwise=layerwise)
+    print("\n[sink] %s" % par.summarize(reps))
+
+
+def test_sink_prefix_longer_than_the_prompt_keeps_everything():
+    w = small("sink_all", d=64, dtype="f32", rank=1, caches=((6, 3),), heavy=0)
+    arrays = [synth.gen_cache(w, 0)]
+    outs, _, st = par.run_gpu(w, arrays, flags=P.binding.OBF_FLAG_SINK(10))
+    assert st & 0xFF == 0
+    assert outs[0]["idx"].shape[-1] == 6
+    assert torch.equal(outs[0]["idx"][0, 0].cpu(), torch.arange(6, dtype=torch.int32))
