@@ -107,8 +107,8 @@ typedef struct {              /* per (layer, KV head) diagnostics (App. K.2 name
     float alpha;              /* a_del / (a_keep + eps)                              [DR]           */
     float rcr;                /* ||R||_F^2 / (||V_del||_F^2 + eps)                   [RCR]          */
     float delta_norm;         /* ||delta||_2                                         [IVN]          */
-    float kth_score;          /* k_eff-th largest A_j                                               */
-    float next_score;         /* (k_eff+1)-th largest A_j, -1 if none                               */
+    float kth_score;          /* smallest retained mass among the candidates of the selection       */
+    float next_score;         /* largest deleted mass, -1 if nothing is deleted                     */
     float lam_1, lam_rho, lam_next; /* eigenvalues of R^T R: largest, last kept, first dropped      */
     int32_t span_rank;        /* numerical dimension m of span(V_keep) (-1: not evaluated)          */
     int32_t rho_eff;          /* number of principal directions actually used                       */
@@ -120,7 +120,7 @@ typedef struct {              /* one agent's prompt cache; T and budget may diff
     const void *k, *v;        /* [layers, kv_heads, T, head_dim]                                    */
     const void *q_obs;        /* [layers, q_heads, n_obs, head_dim]                                 */
     int32_t T;                /* prompt positions, 1 <= T <= OBF_MAX_T                              */
-    int32_t budget;           /* >= 1; k_eff = min(budget, T)                                       */
+    int32_t budget;           /* >= 1; k_eff = min(budget, T) (more with OBF_FLAG_SINK, see there)  */
     void *k_out, *v_out;      /* [layers, kv_heads, k_eff, head_dim]                                */
     int32_t *idx_out;         /* [layers, kv_heads, k_eff]                                          */
     obf_diag_t *diag_out;     /* optional [layers, kv_heads], or NULL                               */
