@@ -71,6 +71,8 @@ def lib():
         _lib.obf_oracle_head.restype = ci
         _lib.obf_oracle_head_sink.argtypes = _lib.obf_oracle_head.argtypes + [ci]
         _lib.obf_oracle_head_sink.restype = ci
+        _lib.obf_oracle_head_ex.argtypes = _lib.obf_oracle_head.argtypes + [ci, ci]
+        _lib.obf_oracle_head_ex.restype = ci
         _lib.obf_oracle_compress.argtypes = [fp, fp, fp, ci, ci, ci, ci, ci, ci, ci, ci,
                                              ctypes.c_double, ip, dp, dp, dp, ctypes.POINTER(Diag), ci]
         _lib.obf_oracle_compress.restype = ci
@@ -149,10 +151,13 @@ def sym_eig(S):
     return lam, E
 
 
-def head(K, V, Q, budget: int, rank: int, eps: float = 1e-12, n_sink: int = 0) -> Dict[str, object]:
+def head(K, V, Q, budget: int, rank: int, eps: float = 1e-12, n_sink: int = 0,
+         fast_iters: int = 0) -> Dict[str, object]:
     """Algorithm 2 (headwise) + Algorithm 3 on one (layer, KV head).
 
     K, V [T,d]; Q [n_q,d] (float32 values; bf16 inputs up-cast exactly).
+    fast_iters > 0: the subspace comes from that many Gram subspace iterations (App. H) started at the first
+    rows of the identity, instead of the exact eigenvectors.
     Returns idx, K_out, V_out (float64), A, delta, rbar, Delta, eigvals, proj, diag.
     """
     K, V, Q = _f32(K), _f32(V), _f32(Q)
@@ -166,11 +171,11 @@ def head(K, V, Q, budget: int, rank: int, eps: float = 1e-12, n_sink: int = 0) -
     proj = np.empty((d, d))
     dg = Diag()
     cd = ctypes.c_double
-    k2 = lib().obf_oracle_head_sink(
+    k2 = lib().obf_oracle_head_ex(
         _p(K, ctypes.c_float), _p(V, ctypes.c_float), _p(Q, ctypes.c_float),
         T, d, Q.shape[0], budget, rank, eps,
         _p(idx, ctypes.c_int32), _p(K_out, cd), _p(V_out, cd), _p(A, cd), _p(delta, cd),
-        _p(rbar, cd), _p(Delta, cd), _p(eig, cd), _p(proj, cd), ctypes.byref(dg), n_sink)
+        _p(rbar, cd), _p(Delta, cd), _p(eig, cd), _p(proj, cd), ctypes.byref(dg), n_sink, fast_iters)
     assert k2 == k
     return {"idx": idx[:k].copy(), "K_out": K_out[:k], "V_out": V_out[:k], "A": A, "delta": delta,
             "rbar": rbar, "Delta": Delta, "eigvals": eig, "proj": proj, "diag": dg.asdict()}

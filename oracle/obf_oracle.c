@@ -287,13 +287,31 @@ static int backfill_given_selection(const float *K, const float *V, const double
                                     const int32_t *idx, double kth_score, double next_score,
                                     double *K_out, double *V_out,
                                     double *delta_out, double *rbar_out, double *Delta_out,
-                                    double *eigvals_out, double *proj_out, obf_oracle_diag_t *diag);
+                                    double *eigvals_out, double *proj_out, obf_oracle_diag_t *diag, int fast_iters);
+
+int obf_oracle_head_ex(const float *K, const float *V, const float *Q,
+                       int T, int d, int n_q, int budget, int rank, double eps,
+                       int32_t *idx, double *K_out, double *V_out,
+                       double *A_out, double *delta_out, double *rbar_out, double *Delta_out,
+                       double *eigvals_out, double *proj_out, obf_oracle_diag_t *diag, int n_sink, int fast_iters);
 
 int obf_oracle_head_sink(const float *K, const float *V, const float *Q,
                          int T, int d, int n_q, int budget, int rank, double eps,
                          int32_t *idx, double *K_out, double *V_out,
                          double *A_out, double *delta_out, double *rbar_out, double *Delta_out,
                          double *eigvals_out, double *proj_out, obf_oracle_diag_t *diag, int n_sink)
+{
+    return obf_oracle_head_ex(K, V, Q, T, d, n_q, budget, rank, eps, idx, K_out, V_out, A_out, delta_out, rbar_out,
+                              Delta_out, eigvals_out, proj_out, diag, n_sink, 0);
+}
+
+/* fast_iters > 0: the principal subspace comes from that many steps of the Gram subspace iteration of App. H
+ * instead of the exact eigen-decomposition (see backfill_given_selection). */
+int obf_oracle_head_ex(const float *K, const float *V, const float *Q,
+                       int T, int d, int n_q, int budget, int rank, double eps,
+                       int32_t *idx, double *K_out, double *V_out,
+                       double *A_out, double *delta_out, double *rbar_out, double *Delta_out,
+                       double *eigvals_out, double *proj_out, obf_oracle_diag_t *diag, int n_sink, int fast_iters)
 {
     /* O1: attention mass */
     double *A = (double *)malloc((size_t)T * sizeof(double));
@@ -305,7 +323,7 @@ int obf_oracle_head_sink(const float *K, const float *V, const float *Q,
     int k = obf_oracle_topk_sink(A, T, budget, n_sink, idx, &kth, &next);
 
     backfill_given_selection(K, V, A, T, d, k, rank, eps, idx, kth, next, K_out, V_out,
-                             delta_out, rbar_out, Delta_out, eigvals_out, proj_out, diag);
+                             delta_out, rbar_out, Delta_out, eigvals_out, proj_out, diag, fast_iters);
     free(A);
     return k;
 }
@@ -330,7 +348,7 @@ static int backfill_given_selection(const float *K, const float *V, const double
                                     const int32_t *idx, double kth_score, double next_score,
                                     double *K_out, double *V_out,
                                     double *delta_out, double *rbar_out, double *Delta_out,
-                                    double *eigvals_out, double *proj_out, obf_oracle_diag_t *diag)
+                                    double *eigvals_out, double *proj_out, obf_oracle_diag_t *diag, int fast_iters)
 {
     obf_oracle_diag_t dg;
     memset(&dg, 0, sizeof(dg));
@@ -427,6 +445,66 @@ static int backfill_given_selection(const float *K, const float *V, const double
     { double kept = 0.0, all = 0.0;
       for (int i = 0; i < d; ++i) { all += lam[i]; if (i < rho) kept += lam[i]; }
       dg.revr = kept / (all + eps); }
+
+    /*
+     * App. H ("fast path"): instead of the eigenvectors, C_0 with orthonormal rows, then
+     * C_{t+1} = orth(C_t G) for t = 0 .. fast_iters - 1 with G = R^T R.  The paper leaves C_0 open; here it is the
+     * first rows of the identity.  orth() is Gram-Schmidt over the rows in order, twice, which spans what a thin QR
+     * spans; a row that has nothing left after its predecessors were removed is dropped.
+     */
+    if (fast_iters > 0) {
+        int rho_f = rank < d - m ? rank : d - m;          /* rank(R) <= d - m */
+        double *Gc = (double *)calloc((size_t)d * d, sizeof(double));
+        for (int n = 0; n < N; ++n) {
+            const double *r = R + (size_t)n * d;
+            for (int a = 0; a < d; ++a) { double ra = r[a]; for (int b = 0; b < d; ++b) Gc[(size_t)a * d + b] += ra * r[b]; }
+        }
+        double *C = (double *)calloc((size_t)(rho_f > 0 ? rho_f : 1) * d, sizeof(double));
+        double *Y = (double *)calloc((size_t)(rho_f > 0 ? rho_f : 1) * d, sizeof(double));
+        for (int i = 0; i < rho_f; ++i) C[(size_t)i * d + i] = 1.0;
+        for (int t = 0; t < fast_iters; ++t) {
+            for (int i = 0; i < rho_f; ++i)
+                for (int b = 0; b < d; ++b) {
+                    double acc = 0.0;
+                    for (int a = 0; a < d; ++a) acc += C[(size_t)i * d + a] * Gc[(size_t)a * d + b];
+                    Y[(size_t)i * d + b] = acc;
+                }
+            int kept = 0;
+            for (int i = 0; i < rho_f; ++i) {
+                double *y = Y + (size_t)i * d;
+                double n0 = 0.0; for (int c = 0; c < d; ++c) n0 += y[c] * y[c];
+                for (int pass = 0; pass < 2; ++pass)
+                    for (int j = 0; j < kept; ++j) {
+                        const double *q = C + (size_t)j * d;
+                        double dot = 0.0; for (int c = 0; c < d; ++c) dot += y[c] * q[c];
+                        for (int c = 0; c < d; ++c) y[c] -= dot * q[c];
+                    }
+                double n1 = 0.0; for (int c = 0; c < d; ++c) n1 += y[c] * y[c];
+                if (n1 > 1e-24 * n0 && n1 > 0.0) {
+                    double inv = 1.0 / sqrt(n1);
+                    for (int c = 0; c < d; ++c) C[(size_t)kept * d + c] = y[c] * inv;
+                    ++kept;
+                }
+            }
+            rho_f = kept;
+        }
+        dg.rho_eff = rho_f;
+        /* eigenvalue fields: Rayleigh quotients of the rows of C; REVR from them */
+        double kept_sum = 0.0, tr = 0.0;
+        for (int a = 0; a < d; ++a) tr += Gc[(size_t)a * d + a];
+        dg.lam_1 = dg.lam_rho = dg.lam_next = 0.0;
+        for (int i = 0; i < rho_f; ++i) {
+            double rq = 0.0;
+            for (int a = 0; a < d; ++a) { double acc = 0.0; for (int b = 0; b < d; ++b) acc += Gc[(size_t)a * d + b] * C[(size_t)i * d + b]; rq += C[(size_t)i * d + a] * acc; }
+            kept_sum += rq;
+            if (i == 0) dg.lam_1 = rq;
+            if (i == rho_f - 1) dg.lam_rho = rq;
+        }
+        dg.revr = kept_sum / (tr + eps);
+        for (int i = 0; i < rho_f; ++i) memcpy(E + (size_t)i * d, C + (size_t)i * d, (size_t)d * sizeof(double));
+        rho = rho_f;
+        free(Y); free(C); free(Gc);
+    }
 
     /* O10: attention-weighted residual mean, Eq. 4 */
     double *rbar = (double *)calloc((size_t)d, sizeof(double));
@@ -535,7 +613,7 @@ int obf_oracle_layer(const float *K, const float *V, const float *Q,
         backfill_given_selection(K + (size_t)h * T * d, V + (size_t)h * T * d, A + (size_t)h * T, T, d, k, rank, eps,
                                  idx, kth, next, K_out + (size_t)h * k * d, V_out + (size_t)h * k * d,
                                  delta_out ? delta_out + (size_t)h * d : NULL, NULL, NULL, NULL, NULL,
-                                 diag_out ? diag_out + h : NULL);
+                                 diag_out ? diag_out + h : NULL, 0);
     }
     free(idx); free(S); free(A);
     return k;

@@ -538,3 +538,60 @@ def test_sink_prefix_with_the_layerwise_selector():
     want = np.sort(np.concatenate([np.arange(4), rest[np.argsort(-S[rest], kind="stable")[:8]]]))
     for h in range(3):
         assert np.array_equal(lay["idx"][h], want)
+
+
+# --------------------------------------------------------------------------
+# fixed-iteration Gram subspace path (App. H)
+# --------------------------------------------------------------------------
+def lib_fast_path(K, V, Q, budget, rank, iters, eps=1e-12):
+    """The same iteration through numpy's thin QR (a library orth), from the first rows of the identity."""
+    A = lib_scores(K, Q)
+    T, d = V.shape
+    idx = np.sort(np.argsort(-A, kind="stable")[:min(budget, T)])
+    keep = np.zeros(T, bool); keep[idx] = True
+    Vd = V.astype(np.float64)
+    Vk, Vdel = Vd[keep], Vd[~keep]
+    Pi = np.linalg.pinv(Vk) @ Vk
+    R = Vdel - Vdel @ Pi
+    G = R.T @ R
+    m = np.linalg.matrix_rank(Vk)
+    rho = min(rank, d - m)
+    C = np.eye(d)[:rho]
+    for _ in range(iters):
+        Qm, _ = np.linalg.qr((C @ G).T)                    # thin QR: columns of Qm span the rows of C G
+        C = Qm.T
+    a_del, a_keep = A[~keep].sum(), A[keep].sum()
+    rbar = (A[~keep] / (a_del + eps)) @ R
+    Delta = (rbar @ C.T) @ C
+    return {"proj": C.T @ C, "Delta": Delta, "delta": a_del / (a_keep + eps) * Delta, "G": G, "rho": rho}
+
+
+@pytest.mark.parametrize("seed,T,d,n_q,budget,rank,iters", [(0, 120, 16, 6, 5, 2, 3), (1, 200, 32, 8, 12, 4, 3),
+                                                            (2, 90, 16, 4, 6, 1, 1), (3, 150, 24, 6, 20, 8, 3)])
+def test_fast_path_matches_the_same_iteration_through_library_qr(seed, T, d, n_q, budget, rank, iters):
+    K, V, Q = rand_head(seed, T, d, n_q, heavy=3)
+    r = oracle.head(K, V, Q, budget, rank, fast_iters=iters)
+    ref = lib_fast_path(K, V, Q, budget, rank, iters)
+    assert r["diag"]["rho_eff"] == ref["rho"]
+    np.testing.assert_allclose(r["Delta"], ref["Delta"], atol=1e-9 * max(1.0, np.abs(ref["Delta"]).max()))
+    np.testing.assert_allclose(r["delta"], ref["delta"], atol=1e-9 * max(1.0, np.abs(ref["delta"]).max()))
+    Vk = V[r["idx"]].astype(np.float64)
+    assert np.abs(Vk @ r["delta"]).max() <= 1e-9 * np.linalg.norm(Vk, 2) * max(np.linalg.norm(r["delta"]), 1e-300)
+
+
+def test_fast_path_reaches_the_exact_subspace_when_the_spectrum_has_a_gap():
+    # a residual with two dominant directions (planted, 30 times the rest of the values)
+    g = np.random.default_rng(5)
+    T, d = 160, 16
+    K = g.standard_normal((T, d)).astype(np.float32); Q = g.standard_normal((5, d)).astype(np.float32)
+    V = g.standard_normal((T, d)).astype(np.float32)
+    V[:, 8] *= 30.0; V[:, 9] *= 30.0
+    V[oracle.topk(oracle.scores(K, Q), 4)[0], 8:10] = 0.0   # the retained values stay out of the planted plane
+    exact = oracle.head(K, V, Q, 4, 2)
+    fast = oracle.head(K, V, Q, 4, 2, fast_iters=3)
+    # one iteration contracts the error by about lambda_3 / lambda_2 ~ 1/580: three leave ~1e-6, five ~1e-11
+    np.testing.assert_allclose(fast["delta"], exact["delta"], atol=1e-5 * np.abs(exact["delta"]).max())
+    np.testing.assert_allclose(oracle.head(K, V, Q, 4, 2, fast_iters=5)["delta"], exact["delta"],
+                               atol=1e-9 * np.abs(exact["delta"]).max())
+    assert np.linalg.norm(oracle.head(K, V, Q, 4, 2, fast_iters=1)["delta"] - exact["delta"]) > \
+        np.linalg.norm(fast["delta"] - exact["delta"])
