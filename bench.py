@@ -185,7 +185,8 @@ def main():
     w = synth.workload(args.workload)
     params = P.make_params(w.layers, w.kv_heads, w.q_heads, w.head.head_dim, w.n_obs, w.rank,
                            P.OBF_F32 if w.dtype == "f32" else P.OBF_BF16, 1e-12,
-                           P.binding.OBF_FLAG_LAYERWISE if w.layerwise else 0)
+                           (P.binding.OBF_FLAG_LAYERWISE if w.layerwise else 0)
+                           | (P.binding.OBF_FLAG_FAST_PATH if w.fast_path else 0))
     tdt = torch.float32 if w.dtype == "f32" else torch.bfloat16
 
     def as_t(a):

@@ -81,6 +81,11 @@ typedef enum { OBF_F32 = 0, OBF_BF16 = 1 } obf_dtype_t;
                                       per head); gather and OBF then run per head with the head's own masses.
                                       Needs every T <= 16384, else OBF_ERR_UNSUPPORTED                          */
 
+#define OBF_FLAG_FAST_PATH    0x4u /* the principal subspace of the residual comes from three steps of the Gram
+                                      subspace iteration of App. H, C <- orth(C R^T R), started at the first rows of
+                                      the identity (the paper leaves the start open), instead of the exact
+                                      eigenvectors: an approximation whose error depends on the residual's spectrum.
+                                      diag: lam_1 / lam_rho are Rayleigh quotients, lam_next is 0                  */
 #define OBF_FLAG_SINK(n) (((uint32_t)(n) & 0xFFu) << 8)
                                    /* protected sink prefix (App. F of the paper: the compressors protect the first s
                                       indices of the cache; the eligible set of Section 3.2 leaves the sink out): the

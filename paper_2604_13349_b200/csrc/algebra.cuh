@@ -216,6 +216,106 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
         rcr = trM / (trG + p.eps);
         if (!(rcr >= RCR_SKIP_TOL)) { done = true; status |= OBF_DEV_SKIPPED; }
 
+        // ---- 4f. fast path of App. H: C <- orth(C M), a fixed number of times, from the first rows of the identity ----
+        if (!done && p.fast_iters > 0) {
+            const int lane = tid & 31, warp = tid >> 5;
+            int rho_f = min(min(p.rank, D), D - m);               // rank(R) <= d - m
+            float *C = B0, *Y = B1;                                // rows of length D (stride LD)
+            for (int e = tid; e < rho_f * D; e += ALG_NT) C[(e / D) * LD + (e % D)] = (e / D == e % D) ? 1.f : 0.f;
+            __syncthreads();
+#pragma unroll 1
+            for (int itn = 0; itn < p.fast_iters; ++itn) {
+                for (int e = tid; e < rho_f * D; e += ALG_NT) {    // Y = C M
+                    const int i = e / D, b = e % D;
+                    float sacc = 0.f;
+#pragma unroll 8
+                    for (int a = 0; a < D; ++a) sacc = fmaf(C[i * LD + a], B2[a * LD + b], sacc);
+                    Y[i * LD + b] = sacc;
+                }
+                __syncthreads();
+                // orth: Gram-Schmidt over the rows in order, twice; a row with nothing left is dropped (warp 0)
+                if (warp == 0) {
+                    int kept = 0;
+                    for (int i = 0; i < rho_f; ++i) {
+                        float *y = Y + i * LD;
+                        float n0 = 0.f;
+                        for (int cc = lane; cc < D; cc += 32) n0 = fmaf(y[cc], y[cc], n0);
+                        n0 = warp_sum(n0);
+                        for (int pass = 0; pass < 2; ++pass)
+                            for (int j = 0; j < kept; ++j) {
+                                const float *qv = C + j * LD;
+                                float dsum = 0.f;
+                                for (int cc = lane; cc < D; cc += 32) dsum = fmaf(y[cc], qv[cc], dsum);
+                                dsum = warp_sum(dsum);
+                                for (int cc = lane; cc < D; cc += 32) y[cc] -= dsum * qv[cc];
+                                __syncwarp();
+                            }
+                        float n1 = 0.f;
+                        for (int cc = lane; cc < D; cc += 32) n1 = fmaf(y[cc], y[cc], n1);
+                        n1 = warp_sum(n1);
+                        if (n1 > 1e-10f * n0 && n1 > 0.f) {
+                            const float inv = rsqrtf(n1);
+                            for (int cc = lane; cc < D; cc += 32) C[kept * LD + cc] = y[cc] * inv;
+                            ++kept;
+                        }
+                        __syncwarp();
+                    }
+                    if (lane == 0) misc[6] = (float)kept;
+                }
+                __syncthreads();
+                rho_f = (int)misc[6];
+            }
+            rho = rho_f;
+            // Rayleigh quotients of the rows (for the diagnostics), then Delta and delta
+            if (warp < 16) {
+                for (int i = warp; i < rho; i += 16) {
+                    float rq = 0.f;
+                    for (int a = lane; a < D; a += 32) {
+                        float sacc = 0.f;
+                        for (int b = 0; b < D; ++b) sacc = fmaf(B2[a * LD + b], C[i * LD + b], sacc);
+                        rq = fmaf(C[i * LD + a], sacc, rq);
+                    }
+                    rq = warp_sum(rq);
+                    if (lane == 0) vl[i] = rq;
+                }
+            }
+            if (tid < rho) {
+                float sacc = 0.f;
+                for (int cc = 0; cc < D; ++cc) sacc = fmaf(C[tid * LD + cc], vu[cc], sacc);
+                vc[tid] = sacc;
+            }
+            __syncthreads();
+            for (int t = 0; t < rho; ++t) revr += vl[t];
+            revr /= trM + p.eps;
+            lam1 = rho > 0 ? vl[0] : 0.f; lam_rho = rho > 0 ? vl[rho - 1] : 0.f; lam_next = 0.f;
+            float dl = 0.f;
+            if (tid < D) {
+                float sacc = 0.f;
+                for (int t = 0; t < rho; ++t) sacc = fmaf(vc[t], C[t * LD + tid], sacc);
+                dl = alpha * sacc;
+            }
+            const float dn2 = block_sum<ALG_NT>(dl * dl, red);
+            dnorm = sqrtf(dn2);
+            if (!isfinite(dn2)) { status |= OBF_DEV_NONFINITE | OBF_DEV_SKIPPED; dnorm = 0.f; }
+            else if (rho == 0 || dn2 == 0.f) status |= OBF_DEV_SKIPPED;
+            else {
+                if (tid < D) {
+                    p.delta[(size_t)g * D + tid] = dl;
+                    if (c.delta_out) c.delta_out[(size_t)lh * D + tid] = dl;
+                    vw[tid] = dl;
+                }
+                if (tid == 0) p.hflag[g] = HFLAG_INJECT;
+                __syncthreads();
+                TIN *rows = reinterpret_cast<TIN *>(c.v_out) + (size_t)lh * k * D;
+                for (int e = tid; e < k * D; e += ALG_NT) {        // Eq. 7, the fp32 sum rounded once
+                    const float sum = to_f32(rows[e]) + vw[e % D];
+                    if constexpr (sizeof(TIN) == 4) rows[e] = sum;
+                    else rows[e] = __float2bfloat16_rn(sum);
+                }
+            }
+            done = true;
+        }
+
         // ---- 4a. few eigenpairs wanted: tridiagonal form, bisection, inverse iteration ----
         if (!done && p.rank <= ALG_TRI_MAX_RANK) {
             const int lane = tid & 31, warp = tid >> 5;

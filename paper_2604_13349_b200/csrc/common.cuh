@@ -65,6 +65,7 @@ struct CallDev {
     int32_t kv_heads;         // KV heads per layer
     int32_t layerwise;        // 1: one retained set per layer (masses summed over its KV heads)
     int32_t n_sink;           // protected prefix: the first n_sink positions are retained besides the budget
+    int32_t fast_iters;       // > 0: that many Gram subspace iterations instead of the exact eigenvectors
     // workspace
     uint32_t *status;
     float *scores;            // [sum heads*T] attention mass (Eq. 1)

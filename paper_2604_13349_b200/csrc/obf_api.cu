@@ -473,6 +473,7 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
     cd.kv_heads = p->kv_heads;
     cd.layerwise = (p->flags & OBF_FLAG_LAYERWISE) ? 1 : 0;
     cd.n_sink = (int32_t)OBF_FLAG_SINK_OF(p->flags);
+    cd.fast_iters = (p->flags & OBF_FLAG_FAST_PATH) ? 3 : 0;
     cd.sc_part = reinterpret_cast<float *>(ws + L.off_sc_part);
     cd.sc_head = reinterpret_cast<float *>(ws + L.off_sc_head);
     cd.sc_cnt = reinterpret_cast<uint32_t *>(ws + L.off_sc_sync);

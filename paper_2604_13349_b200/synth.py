@@ -102,6 +102,7 @@ class Workload:
     head: HeadSpec
     caches: Tuple[CacheSpec, ...]
     layerwise: bool = False       # layerwise selector: one retained set per layer
+    fast_path: bool = False       # three Gram subspace iterations instead of the exact eigenvectors
 
     @property
     def G(self) -> int:
@@ -249,6 +250,8 @@ def _make_workloads() -> Dict[str, Workload]:
     out["pb"] = Workload(
         name="pb", seed=6, layers=36, kv_heads=8, q_heads=32, n_obs=40, rank=4, dtype="bf16",
         head=hs_paper, caches=(CacheSpec(T=2048, budget=32),))
+    # the paper's own approximation of the subspace (App. H), on the paper-regime shape
+    out["pa_fast"] = dataclasses.replace(out["pa"], name="pa_fast", fast_path=True)
     return out
 
 
