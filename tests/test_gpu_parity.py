@@ -310,6 +310,14 @@ def test_c4_full_size_evict_only_sampled_heads(c4_arrays):
     run_and_check(synth.workload("c4_evict"), evict=True, heads=[(3, 1), (39, 6)], arrays=c4_arrays)
 
 
+def test_c4_full_size_layerwise_sampled_layers(c4_arrays):
+    w = synth.workload("c4_layer")
+    outs, _, st = par.run_gpu(w, c4_arrays, flags=P.binding.OBF_FLAG_LAYERWISE)
+    assert st & 0xFF == 0
+    reps = par.check_cache_layerwise(w, 0, c4_arrays[0], outs[0], [0, 39])
+    print("\n[c4_layer] %s" % par.summarize(reps))
+
+
 def test_c5_ragged_relay_batch_sampled_heads():
     w = synth.workload("c5")
     run_and_check(w, heads=[(0, 0), (35, 7)])
