@@ -484,7 +484,9 @@ __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ Call
 // grid = (ceil(k_eff_max / GATHER_ROWS), heads_total).
 constexpr int GATHER_ROWS = 64;
 
-template <int ROW_BYTES>
+// WHICH: 3 = keys and values, 1 = values only, 2 = keys only (the keys are needed by nothing that follows in
+// the call, so their copy can run beside the later kernels).
+template <int ROW_BYTES, int WHICH = 3>
 __global__ void __launch_bounds__(256) k_gather(const __grid_constant__ CallDev p)
 {
     constexpr int CH = ROW_BYTES / 16;             // vectors per row
@@ -520,15 +522,15 @@ __global__ void __launch_bounds__(256) k_gather(const __grid_constant__ CallDev 
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             if (j[u] >= 0) {
-                kv[u] = *reinterpret_cast<const uint4 *>(kb + (size_t)j[u] * ROW_BYTES + ch * 16);
-                vv[u] = *reinterpret_cast<const uint4 *>(vb + (size_t)j[u] * ROW_BYTES + ch * 16);
+                if (WHICH & 2) kv[u] = *reinterpret_cast<const uint4 *>(kb + (size_t)j[u] * ROW_BYTES + ch * 16);
+                if (WHICH & 1) vv[u] = *reinterpret_cast<const uint4 *>(vb + (size_t)j[u] * ROW_BYTES + ch * 16);
             }
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             if (j[u] >= 0) {
-                *reinterpret_cast<uint4 *>(ko + (size_t)r[u] * ROW_BYTES + ch * 16) = kv[u];
-                *reinterpret_cast<uint4 *>(vo + (size_t)r[u] * ROW_BYTES + ch * 16) = vv[u];
+                if (WHICH & 2) *reinterpret_cast<uint4 *>(ko + (size_t)r[u] * ROW_BYTES + ch * 16) = kv[u];
+                if (WHICH & 1) *reinterpret_cast<uint4 *>(vo + (size_t)r[u] * ROW_BYTES + ch * 16) = vv[u];
             }
         }
     }
