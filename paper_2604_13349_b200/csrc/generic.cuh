@@ -289,8 +289,9 @@ __global__ void __launch_bounds__(256) k_layer_sum(const __grid_constant__ CallD
     p.lscores[c.tok_off / p.kv_heads + (size_t)(lh / p.kv_heads) * c.T + j] = s;
 }
 
-// With LAYER the block is a layer: it selects on the layer's summed masses and then writes the shared
-// positions, the keep flags and the demand sums (of the head's own masses) for each of the layer's heads.
+// With LAYER every head's block selects on its layer's summed masses (the layer's heads repeat the same
+// selection side by side rather than one block writing all of them in turn) and then writes the shared
+// positions, the keep flags and the demand sums of the head's own masses.
 template <int NT, bool LAYER = false>
 __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ CallDev p)
 {
@@ -301,7 +302,7 @@ __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ Call
     __shared__ uint32_t wtot[32];
     __shared__ float red[32];
     int ci, lh;
-    locate(p, LAYER ? blockIdx.x * p.kv_heads : blockIdx.x, ci, lh);      // LAYER: lh is the layer's first head
+    locate(p, blockIdx.x, ci, lh);
     const CacheDev &c = p.c[ci];
     const int T = c.T, k = c.k_eff;
     float *Af = p.scores + c.tok_off + (size_t)lh * T;
@@ -426,10 +427,10 @@ __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ Call
         for (int j = tid; j < T; j += NT)
             if (sel_keys[j] == 0xFFFFFFFFu) nx = fmaxf(nx, __uint_as_float(A[j]));
         const float next = block_max<NT>(nx, red);
-        for (int h = 0; h < p.kv_heads; ++h) {
-            float *Ah = Af + (size_t)h * T;
-            uint8_t *keep_h = keep + (size_t)h * T;
-            int32_t *idx_h = idx + (size_t)h * k;
+        {
+            float *Ah = Af;
+            uint8_t *keep_h = keep;
+            int32_t *idx_h = idx;
             sk = 0.f; sd = 0.f;
             for (int j = tid; j < T; j += NT) {
                 const uint32_t pos = sel_keys[j];
@@ -447,7 +448,7 @@ __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ Call
             const float a_keep = block_sum<NT>(sk, red);
             const float a_del = block_sum<NT>(sd, red);
             if (tid == 0) {
-                float *sm = p.sums + (size_t)(c.head_base + lh + h) * 4;
+                float *sm = p.sums + (size_t)blockIdx.x * 4;
                 sm[0] = a_keep; sm[1] = a_del; sm[2] = tau == 0xFFFFFFFFu ? INFINITY : key_score(tau); sm[3] = next;
                 if (c.diag) {
                     obf_diag_t dg;
@@ -455,7 +456,7 @@ __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ Call
                     dg.rcr = 0.f; dg.delta_norm = 0.f; dg.kth_score = tau == 0xFFFFFFFFu ? INFINITY : key_score(tau); dg.next_score = next;
                     dg.lam_1 = dg.lam_rho = dg.lam_next = 0.f;
                     dg.span_rank = -1; dg.rho_eff = 0; dg.status = OBF_DEV_SKIPPED; dg.revr = 0.f;
-                    c.diag[lh + h] = dg;
+                    c.diag[lh] = dg;
                 }
             }
         }

@@ -374,14 +374,20 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
         mark(st, "k_score_pool");
     }
     if (cd.layerwise) {
-        // one block per layer: masses of the layer's KV heads added up, selection on the sums, outputs per head
+        // masses of a layer's KV heads added up, then every head's block selects on its layer's sums
         const int n_layers = heads / cd.kv_heads;
         const size_t sm_sel = (size_t)T_max * sizeof(uint32_t);
         dim3 gl((T_max + 255) / 256, n_layers);
         k_layer_sum<<<gl, 256, 0, st>>>(cd);
         mark(st, "k_layer_sum");
-        if ((s = set_smem(k_select_smem<1024, true>, sm_sel)) != OBF_OK) return s;
-        k_select_smem<1024, true><<<n_layers, 1024, sm_sel, st>>>(cd);
+        const int sms = sm_count();
+        if (heads > 2 * sms && heads <= 4 * sms) {
+            if ((s = set_smem(k_select_smem<512, true>, sm_sel)) != OBF_OK) return s;
+            k_select_smem<512, true><<<heads, 512, sm_sel, st>>>(cd);
+        } else {
+            if ((s = set_smem(k_select_smem<1024, true>, sm_sel)) != OBF_OK) return s;
+            k_select_smem<1024, true><<<heads, 1024, sm_sel, st>>>(cd);
+        }
     } else if (T_max <= SEL_SMEM_MAX_T) {
         const size_t sm_sel = (size_t)T_max * sizeof(uint32_t);
         // blocks of 1024 threads fit twice on an SM; when the heads then need a second, nearly empty wave,
