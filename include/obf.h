@@ -170,10 +170,14 @@ obf_status_t obf_host_arena_bytes(const obf_params_t *params, const obf_cache_t 
  * relay hand-off when the cache is staged on the host).  Every pointer inside
  * `caches` is a host pointer (pinned memory makes the copies asynchronous);
  * `device_arena` is device memory of at least obf_host_arena_bytes(),
- * 256-byte aligned.  Enqueues host->device copies of k, v, q_obs, the
- * compression, and device->host copies of k_out, v_out, idx_out (and of
- * diag_out / delta_out / scores_out when non-NULL) on `stream`, then waits for
- * the stream.
+ * 256-byte aligned.  Copies k, v, q_obs to the device, compresses, and copies
+ * k_out, v_out, idx_out (and the optional outputs that are not NULL) back,
+ * as a pipeline over slabs of layers: the copies run on two streams that
+ * the library creates on first use (per host thread and device), the
+ * kernels on `stream`; work already enqueued on `stream` is waited for
+ * first.  Returns after everything has finished.  The injected vectors can
+ * differ from obf_compress on the same data in the last fp32 digits (a slab
+ * adds its partial sums up in another order than the whole call).
  */
 obf_status_t obf_compress_host(const obf_params_t *params, const obf_cache_t *caches, int32_t n_caches,
                                void *device_arena, size_t arena_bytes, void *stream);

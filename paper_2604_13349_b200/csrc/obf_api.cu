@@ -13,6 +13,7 @@
 namespace obf {
 
 static thread_local int32_t g_last_launches = 0;
+static thread_local bool g_keep_status = false;
 
 // Optional per-launch timing (obf_compress_profiled): an event after every launch.
 struct Profiler {
@@ -534,7 +535,7 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
     cd.hflag = reinterpret_cast<uint32_t *>(ws + L.off_hflag);
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    OBF_CUDA_TRY(cudaMemsetAsync(cd.status, 0, 256, st));
+    if (!g_keep_status) OBF_CUDA_TRY(cudaMemsetAsync(cd.status, 0, 256, st));     // a slab of a larger job adds to the job's status
     if (g_prof.active) cudaEventRecord(g_prof.ev[0], st);
 
     if (p->dtype == OBF_F32) {
@@ -619,6 +620,38 @@ obf_status_t obf_host_arena_bytes(const obf_params_t *params, const obf_cache_t 
     return OBF_OK;
 }
 
+// Streams and events of the host-staged call: copies in, copies out, and per slab of layers the two
+// hand-overs (inputs on the device, results ready).  Created on first use per host thread and device.
+constexpr int HOST_SLABS_MAX = 8;
+struct HostPipe {
+    cudaStream_t cin = nullptr, cout = nullptr;
+    cudaEvent_t start = nullptr, in_done[HOST_SLABS_MAX], comp_done[HOST_SLABS_MAX], out_done = nullptr;
+    int device = -1;
+};
+
+static HostPipe *host_pipe()
+{
+    static thread_local HostPipe hp[16];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 16) return nullptr;
+    HostPipe &h = hp[dev];
+    if (h.device != dev) {
+        bool ok = cudaStreamCreateWithFlags(&h.cin, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&h.cout, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&h.start, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&h.out_done, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; ok && i < HOST_SLABS_MAX; ++i)
+            ok = cudaEventCreateWithFlags(&h.in_done[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&h.comp_done[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) { cudaGetLastError(); return nullptr; }
+        h.device = dev;
+    }
+    return &h;
+}
+
+// The layers are cut into slabs that go through copy-in, compute and copy-out as a pipeline: the PCIe link
+// carries slab s + 1 in and slab s - 1 out while the kernels work on slab s (layers are independent and
+// contiguous in every array).  The kernels of all slabs run on the caller's stream, one slab after the other.
 obf_status_t obf_compress_host(const obf_params_t *params, const obf_cache_t *caches, int32_t n_caches,
                                void *device_arena, size_t arena_bytes, void *stream)
 {
@@ -635,40 +668,67 @@ obf_status_t obf_compress_host(const obf_params_t *params, const obf_cache_t *ca
     char *base = static_cast<char *>(device_arena);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t e = params->dtype == OBF_F32 ? 4 : 2;
-    const size_t hpc = (size_t)params->layers * params->kv_heads, d = params->head_dim;
-    obf_cache_t dev[OBF_MAX_CACHES];
-    for (int i = 0; i < n_caches; ++i) {
-        const obf_cache_t &c = caches[i];
-        const size_t T = c.T;
-        dev[i] = c;
-        dev[i].k = base + H.k[i]; dev[i].v = base + H.v[i]; dev[i].q_obs = base + H.q[i];
-        dev[i].k_out = base + H.k_out[i]; dev[i].v_out = base + H.v_out[i];
-        dev[i].idx_out = reinterpret_cast<int32_t *>(base + H.idx[i]);
-        dev[i].diag_out = c.diag_out ? reinterpret_cast<obf_diag_t *>(base + H.diag[i]) : nullptr;
-        dev[i].scores_out = c.scores_out ? reinterpret_cast<float *>(base + H.scores[i]) : nullptr;
-        dev[i].delta_out = c.delta_out ? reinterpret_cast<float *>(base + H.delta[i]) : nullptr;
-        OBF_CUDA_TRY(cudaMemcpyAsync(base + H.k[i], c.k, hpc * T * d * e, cudaMemcpyHostToDevice, st));
-        OBF_CUDA_TRY(cudaMemcpyAsync(base + H.v[i], c.v, hpc * T * d * e, cudaMemcpyHostToDevice, st));
-        OBF_CUDA_TRY(cudaMemcpyAsync(base + H.q[i], c.q_obs,
-                                     (size_t)params->layers * params->q_heads * params->n_obs * d * e,
-                                     cudaMemcpyHostToDevice, st));
+    const size_t H_kv = (size_t)params->kv_heads, d = params->head_dim;
+    HostPipe *hp = host_pipe();
+    if (!hp) return OBF_ERR_CUDA;
+    const int n_slabs = params->layers < 4 ? params->layers : 4;
+    // nothing of this call may start before what the caller's stream already holds (an earlier call on the arena)
+    OBF_CUDA_TRY(cudaEventRecord(hp->start, st));
+    OBF_CUDA_TRY(cudaStreamWaitEvent(hp->cin, hp->start, 0));
+    OBF_CUDA_TRY(cudaStreamWaitEvent(hp->cout, hp->start, 0));
+    for (int sl = 0; sl < n_slabs; ++sl) {
+        const size_t l0 = (size_t)params->layers * sl / n_slabs, l1 = (size_t)params->layers * (sl + 1) / n_slabs;
+        const size_t nl = l1 - l0;
+        obf_params_t ps = *params;
+        ps.layers = (int32_t)nl;
+        obf_cache_t dev[OBF_MAX_CACHES];
+        for (int i = 0; i < n_caches; ++i) {
+            const obf_cache_t &c = caches[i];
+            const size_t T = c.T, ke = (size_t)k_eff_of(params, c);
+            const size_t kv_l = H_kv * T * d * e, q_l = (size_t)params->q_heads * params->n_obs * d * e;
+            const size_t o_l = H_kv * ke * d * e;
+            dev[i] = c;
+            dev[i].k = base + H.k[i] + l0 * kv_l; dev[i].v = base + H.v[i] + l0 * kv_l; dev[i].q_obs = base + H.q[i] + l0 * q_l;
+            dev[i].k_out = base + H.k_out[i] + l0 * o_l; dev[i].v_out = base + H.v_out[i] + l0 * o_l;
+            dev[i].idx_out = reinterpret_cast<int32_t *>(base + H.idx[i]) + l0 * H_kv * ke;
+            dev[i].diag_out = c.diag_out ? reinterpret_cast<obf_diag_t *>(base + H.diag[i]) + l0 * H_kv : nullptr;
+            dev[i].scores_out = c.scores_out ? reinterpret_cast<float *>(base + H.scores[i]) + l0 * H_kv * T : nullptr;
+            dev[i].delta_out = c.delta_out ? reinterpret_cast<float *>(base + H.delta[i]) + l0 * H_kv * d : nullptr;
+            OBF_CUDA_TRY(cudaMemcpyAsync(const_cast<void *>(dev[i].k), static_cast<const char *>(c.k) + l0 * kv_l, nl * kv_l,
+                                         cudaMemcpyHostToDevice, hp->cin));
+            OBF_CUDA_TRY(cudaMemcpyAsync(const_cast<void *>(dev[i].v), static_cast<const char *>(c.v) + l0 * kv_l, nl * kv_l,
+                                         cudaMemcpyHostToDevice, hp->cin));
+            OBF_CUDA_TRY(cudaMemcpyAsync(const_cast<void *>(dev[i].q_obs), static_cast<const char *>(c.q_obs) + l0 * q_l,
+                                         nl * q_l, cudaMemcpyHostToDevice, hp->cin));
+        }
+        OBF_CUDA_TRY(cudaEventRecord(hp->in_done[sl], hp->cin));
+        OBF_CUDA_TRY(cudaStreamWaitEvent(st, hp->in_done[sl], 0));
+        g_keep_status = sl > 0;
+        s = run(&ps, dev, n_caches, ps.rank, base + H.ws, H.ws_bytes, stream);
+        g_keep_status = false;
+        if (s != OBF_OK) { cudaStreamSynchronize(hp->cin); cudaStreamSynchronize(st); cudaStreamSynchronize(hp->cout); return s; }
+        OBF_CUDA_TRY(cudaEventRecord(hp->comp_done[sl], st));
+        OBF_CUDA_TRY(cudaStreamWaitEvent(hp->cout, hp->comp_done[sl], 0));
+        for (int i = 0; i < n_caches; ++i) {
+            const obf_cache_t &c = caches[i];
+            const size_t T = c.T, ke = (size_t)k_eff_of(params, c);
+            const size_t o_l = H_kv * ke * d * e;
+            OBF_CUDA_TRY(cudaMemcpyAsync(static_cast<char *>(c.k_out) + l0 * o_l, dev[i].k_out, nl * o_l, cudaMemcpyDeviceToHost, hp->cout));
+            OBF_CUDA_TRY(cudaMemcpyAsync(static_cast<char *>(c.v_out) + l0 * o_l, dev[i].v_out, nl * o_l, cudaMemcpyDeviceToHost, hp->cout));
+            OBF_CUDA_TRY(cudaMemcpyAsync(c.idx_out + l0 * H_kv * ke, dev[i].idx_out, nl * H_kv * ke * 4, cudaMemcpyDeviceToHost, hp->cout));
+            if (c.diag_out)
+                OBF_CUDA_TRY(cudaMemcpyAsync(c.diag_out + l0 * H_kv, dev[i].diag_out, nl * H_kv * sizeof(obf_diag_t),
+                                             cudaMemcpyDeviceToHost, hp->cout));
+            if (c.scores_out)
+                OBF_CUDA_TRY(cudaMemcpyAsync(c.scores_out + l0 * H_kv * T, dev[i].scores_out, nl * H_kv * T * 4,
+                                             cudaMemcpyDeviceToHost, hp->cout));
+            if (c.delta_out)
+                OBF_CUDA_TRY(cudaMemcpyAsync(c.delta_out + l0 * H_kv * d, dev[i].delta_out, nl * H_kv * d * 4,
+                                             cudaMemcpyDeviceToHost, hp->cout));
+        }
     }
-    s = run(params, dev, n_caches, params->rank, base + H.ws, H.ws_bytes, stream);
-    if (s != OBF_OK) return s;
-    for (int i = 0; i < n_caches; ++i) {
-        const obf_cache_t &c = caches[i];
-        const size_t T = c.T, ke = (size_t)k_eff_of(params, c);
-        OBF_CUDA_TRY(cudaMemcpyAsync(c.k_out, base + H.k_out[i], hpc * ke * d * e, cudaMemcpyDeviceToHost, st));
-        OBF_CUDA_TRY(cudaMemcpyAsync(c.v_out, base + H.v_out[i], hpc * ke * d * e, cudaMemcpyDeviceToHost, st));
-        OBF_CUDA_TRY(cudaMemcpyAsync(c.idx_out, base + H.idx[i], hpc * ke * 4, cudaMemcpyDeviceToHost, st));
-        if (c.diag_out)
-            OBF_CUDA_TRY(cudaMemcpyAsync(c.diag_out, base + H.diag[i], hpc * sizeof(obf_diag_t),
-                                         cudaMemcpyDeviceToHost, st));
-        if (c.scores_out)
-            OBF_CUDA_TRY(cudaMemcpyAsync(c.scores_out, base + H.scores[i], hpc * T * 4, cudaMemcpyDeviceToHost, st));
-        if (c.delta_out)
-            OBF_CUDA_TRY(cudaMemcpyAsync(c.delta_out, base + H.delta[i], hpc * d * 4, cudaMemcpyDeviceToHost, st));
-    }
+    OBF_CUDA_TRY(cudaEventRecord(hp->out_done, hp->cout));
+    OBF_CUDA_TRY(cudaStreamWaitEvent(st, hp->out_done, 0));
     OBF_CUDA_TRY(cudaStreamSynchronize(st));
     return OBF_OK;
 }

@@ -288,6 +288,40 @@ def test_host_entry_point_matches_the_device_entry_point():
     assert torch.equal(oD, outs[0]["delta"].cpu())
 
 
+@pytest.mark.parametrize("layers", [1, 5, 9])
+def test_host_entry_point_pipelines_slabs_of_layers_for_ragged_batches(layers):
+    # layer counts that the slabs do not divide evenly, two caches of different lengths, bf16 on the tuned path
+    w = small("host", layers=layers, kv_heads=2, G=2, n_obs=8, d=128, dtype="bf16", rank=2,
+              caches=((300, 20), (700, 140)), n_outlier=3, seed=19 + layers)
+    arrays = [synth.gen_cache(w, ci) for ci in range(2)]
+    outs, _, st = par.run_gpu(w, arrays)
+    assert st & 0xFF == 0
+    params = par.params_for(w)
+    host, cs = [], []
+    for ci, (T, b) in enumerate(((300, 20), (700, 140))):
+        a = arrays[ci]
+        h = {n: torch.from_numpy(a[n].view(np.int16)).view(torch.bfloat16).pin_memory() for n in ("K", "V", "Q")}
+        h["oK"] = torch.empty((layers, 2, b, 128), dtype=torch.bfloat16).pin_memory()
+        h["oV"] = torch.empty((layers, 2, b, 128), dtype=torch.bfloat16).pin_memory()
+        h["oI"] = torch.empty((layers, 2, b), dtype=torch.int32).pin_memory()
+        h["oS"] = torch.empty((layers, 2, T), dtype=torch.float32).pin_memory()
+        h["oD"] = torch.empty((layers, 2, 128), dtype=torch.float32).pin_memory()
+        host.append(h)
+        cs.append(P.make_cache(h["K"], h["V"], h["Q"], T, b, h["oK"], h["oV"], h["oI"], None, h["oS"], h["oD"]))
+    arena = torch.empty(P.obf_host_arena_bytes(params, cs), dtype=torch.uint8, device="cuda")
+    for _ in range(2):                                      # twice: the second call reuses the arena and the streams
+        P.obf_compress_host(params, cs, arena)
+    for ci in range(2):
+        h = host[ci]
+        assert torch.equal(h["oI"], outs[ci]["idx"].cpu())
+        assert torch.equal(h["oK"].view(torch.int16), outs[ci]["K_out"].cpu().view(torch.int16))
+        assert torch.allclose(h["oV"].float(), outs[ci]["V_out"].cpu().float(), rtol=1e-2, atol=1e-5)
+        assert torch.equal(h["oS"], outs[ci]["scores"].cpu())
+        # the streaming pass cuts its tile sequence by the size of the call, so a slab adds its partial Gram
+        # matrices up in another order than the whole call: delta agrees to fp32 rounding, not bit for bit
+        assert torch.allclose(h["oD"], outs[ci]["delta"].cpu(), rtol=1e-4, atol=1e-6)
+
+
 # ---------------------------------------------------------------------------
 # benchmark configurations at full size, in the benchmark's launch configuration,
 # checked on sampled heads that the oracle computes one by one
