@@ -147,6 +147,9 @@ obf_status_t obf_workspace_bytes(const obf_params_t *params, const obf_cache_t *
  * are host structs (copied before return); `workspace` is device memory of at
  * least obf_workspace_bytes(), 256-byte aligned, private to this call until
  * the enqueued work completes; `stream` is a cudaStream_t passed as void*.
+ * With rank > 0 the copy of the retained keys runs on a stream of the library
+ * (created on first use per host thread and device) that forks from and joins
+ * `stream` inside the call: everything the call does is ordered on `stream`.
  */
 obf_status_t obf_compress(const obf_params_t *params, const obf_cache_t *caches, int32_t n_caches,
                           void *workspace, size_t workspace_bytes, void *stream);
