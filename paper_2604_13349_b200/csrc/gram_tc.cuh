@@ -27,6 +27,7 @@
 
 namespace obf {
 
+constexpr int GT_KEEP_TILES_MAX = 2;                // retained-row tiles per head that enter G_keep (span test)
 constexpr int GT_STAGES = 6;
 constexpr int GT_TILE = 128;                       // tokens per tile
 constexpr int GT_TILE_BYTES = GT_TILE * 128 * 2;   // 32 KiB

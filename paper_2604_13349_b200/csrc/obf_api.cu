@@ -173,7 +173,11 @@ static void make_layout(const obf_params_t *p, const obf_cache_t *caches, int32_
         for (int i = 0; i < n; ++i) {
             const int T = caches[i].T, ke = k_eff_of(p, caches[i]);
             L.nsub_del[i] = (T + GT_TILE - 1) / GT_TILE;
+            // The span test only has to certify span(V_keep) = R^d, and any subset of the retained rows that spans
+            // R^d does: the first two tiles (256 rows >= head_dim) are enough.  A head whose subset fails the test
+            // goes through the full Gram-Schmidt basis over all its retained rows, like every head with k < d.
             L.nsub_keep[i] = (ke >= d && T > ke) ? (ke + GT_TILE - 1) / GT_TILE : 0;
+            if (L.nsub_keep[i] > GT_KEEP_TILES_MAX) L.nsub_keep[i] = GT_KEEP_TILES_MAX;
             L.sub_base[i] = total;
             total += (long long)hpc * (L.nsub_del[i] + L.nsub_keep[i]);
         }
