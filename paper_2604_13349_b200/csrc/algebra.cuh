@@ -103,8 +103,10 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
         for (int i = 0; i < k && m < D; ++i) {
             if (tid < D) vw[tid] = to_f32(vk[(size_t)i * D + tid]);
             __syncthreads();
-            const float w0 = tid < D ? vw[tid] : 0.f;
-            const float n0 = sqrtf(block_sum<ALG_NT>(w0 * w0, red));
+            // the two norms of a row are taken by every warp for itself (same sum, same order): no block reduction
+            float np0 = 0.f;
+            for (int cc = (tid & 31); cc < D; cc += 32) np0 = fmaf(vw[cc], vw[cc], np0);
+            const float n0 = sqrtf(warp_sum(np0));
             for (int pass = 0; pass < 2; ++pass) {
                 {
                     const int j = tid >> 2, part = tid & 3;
@@ -132,7 +134,9 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
                 __syncthreads();
             }
             const float w1 = tid < D ? vw[tid] : 0.f;
-            const float n1 = sqrtf(block_sum<ALG_NT>(w1 * w1, red));
+            float np1 = 0.f;
+            for (int cc = (tid & 31); cc < D; cc += 32) np1 = fmaf(vw[cc], vw[cc], np1);
+            const float n1 = sqrtf(warp_sum(np1));
             if (n1 > SPAN_ROW_TOL * n0 && n1 > 0.f) {
                 if (tid < D) B0[m * LD + tid] = w1 / n1;
                 ++m;
