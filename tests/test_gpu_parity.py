@@ -195,10 +195,11 @@ def test_tuned_path_rank_deficient_values_with_budget_above_head_dim():
     assert torch.all(outs[0]["delta"].norm(dim=-1) > 1e-6)
 
 
-@pytest.mark.parametrize("T,budget", [(20000, 300), (80000, 200)])
+@pytest.mark.parametrize("T,budget", [(20000, 300), (70000, 250), (80000, 200)])
 def test_long_prompts_take_the_fallback_kernels(T, budget):
-    # 20000 keys: more than the select kernel keeps in shared memory; 80000 keys: more chunks than the
-    # persistent score kernel has blocks, so the shape-generic score kernels run (the Gram pass stays tuned)
+    # 20000 keys: more than the select kernel keeps in shared memory; 70000 keys: one head's team is 137 blocks,
+    # nearly the whole grid of the persistent score kernel; 80000 keys: more chunks than that kernel has blocks,
+    # so the shape-generic score kernels run (the Gram pass stays tuned)
     w = small("long", layers=1, kv_heads=1, G=4, n_obs=8, d=128, dtype="bf16", rank=1, caches=((T, budget),),
               n_outlier=3, n_sink=4, heavy=8, seed=T % 97)
     outs, reps, _ = run_and_check(w)
