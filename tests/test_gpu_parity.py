@@ -172,6 +172,18 @@ def test_tuned_path_ragged_batches_match_oracle_and_generic_path(caches):
     assert any(not r.oracle_skipped for r in reps) or all(c[1] >= 128 for c in caches)
 
 
+def test_tuned_path_with_many_caches_of_different_lengths():
+    # twelve caches in one call: every role of the score kernel walks the per-cache table
+    Ts = [128, 131, 200, 256, 300, 511, 512, 513, 640, 777, 900, 1025]
+    w = small("many", layers=1, kv_heads=2, G=2, n_obs=8, d=128, dtype="bf16", rank=2,
+              caches=tuple((t, 16 + (t % 7)) for t in Ts), n_outlier=3, n_sink=2, seed=5)
+    a, reps, arrays = run_and_check(w)
+    assert all(not r.oracle_skipped for r in reps)
+    b, _, _ = run_and_check(w, arrays=arrays, flags=P.binding.OBF_FLAG_GENERIC_PATH)
+    for x, y in zip(a, b):
+        assert torch.equal(x["K_out"], y["K_out"])
+
+
 def test_tuned_path_rank_deficient_values_with_budget_above_head_dim():
     # head_dim 128, budget 160 >= head_dim, but every selectable value lives in the first 90 channels
     w = small("rd128", d=128, dtype="bf16", rank=3, caches=((700, 160),), heavy=0, kv_heads=2, seed=23)
