@@ -119,6 +119,9 @@ typedef struct {              /* per (layer, KV head) diagnostics (App. K.2 name
     int32_t rho_eff;          /* number of principal directions actually used                       */
     uint32_t status;          /* OBF_DEV_* bits                                                     */
     float revr;               /* sum of the rho_eff kept eigenvalues of R^T R over their total  [REVR]; PCR is 1 - rcr */
+    float pc;                 /* cosine between the sum of the deleted values and the sum of their projections onto
+                                 span(V_keep)  [PC]; 0 when OBF does not run for the head; costs one more pass over V,
+                                 made only when diag_out is given                                        */
 } obf_diag_t;
 
 typedef struct {              /* one agent's prompt cache; T and budget may differ between caches   */

@@ -29,7 +29,7 @@ class Diag(ctypes.Structure):
     _fields_ = [(n, ctypes.c_double) for n in (
         "a_keep", "a_del", "alpha", "vdel_fro2", "r_fro2", "rcr", "rbar_norm",
         "delta_norm", "kth_score", "next_score", "lam_rho", "lam_next", "lam_1")] + [
-        (n, ctypes.c_int32) for n in ("span_rank", "rho_eff", "n_del", "skipped")] + [("revr", ctypes.c_double)]
+        (n, ctypes.c_int32) for n in ("span_rank", "rho_eff", "n_del", "skipped")] + [("revr", ctypes.c_double), ("pc", ctypes.c_double)]
 
     def asdict(self) -> Dict[str, float]:
         return {n: getattr(self, n) for n, _ in self._fields_}

@@ -59,6 +59,8 @@ typedef struct {
     int32_t n_del;       /* number of deleted positions                                     */
     int32_t skipped;     /* 1 if OBF was skipped for this head (footnote to Eq. 7)          */
     double revr;         /* kept share of the residual's squared singular values (REVR, App. K.2) */
+    double pc;           /* cosine between the sum of the deleted values and the sum of their projections
+                            onto span(V_keep) (PC, App. K.2); 0 when OBF does not run          */
 } obf_oracle_diag_t;
 
 /* ------------------------------------------------------------------ */
@@ -413,6 +415,16 @@ static int backfill_given_selection(const float *K, const float *V, const double
         for (int c = 0; c < d; ++c) dg.r_fro2 += r[c] * r[c];
     }
     dg.rcr = dg.r_fro2 / (dg.vdel_fro2 + eps);
+    {   /* PC (App. K.2): CosSim(sum_j V_del[j,:], sum_j V_par[j,:]) with V_par = V_del - R */
+        double ss = 0.0, pp = 0.0, sp = 0.0;
+        for (int c = 0; c < d; ++c) {
+            double sv = 0.0, sr = 0.0;
+            for (int n = 0; n < N; ++n) { sv += (double)V[(size_t)del[n] * d + c]; sr += R[(size_t)n * d + c]; }
+            const double par = sv - sr;
+            ss += sv * sv; pp += par * par; sp += sv * par;
+        }
+        dg.pc = (ss > 0.0 && pp > 0.0) ? sp / (sqrt(ss) * sqrt(pp)) : 0.0;
+    }
 
     /* O8: residual of negligible Frobenius norm -> skip (footnote to Eq. 7) */
     if (dg.r_fro2 <= 1e-12 * dg.vdel_fro2) {

@@ -67,7 +67,7 @@ class ObfDiag(ctypes.Structure):
         "a_keep", "a_del", "alpha", "rcr", "delta_norm", "kth_score", "next_score",
         "lam_1", "lam_rho", "lam_next")] + [
         ("span_rank", ctypes.c_int32), ("rho_eff", ctypes.c_int32), ("status", ctypes.c_uint32),
-        ("revr", ctypes.c_float)]
+        ("revr", ctypes.c_float), ("pc", ctypes.c_float)]
 
 
 DIAG_BYTES = ctypes.sizeof(ObfDiag)

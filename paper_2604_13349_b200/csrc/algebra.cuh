@@ -89,12 +89,12 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
 
     uint32_t status = 0u;
     int m = 0;
-    float rcr = 0.f, lam1 = 0.f, lam_rho = 0.f, lam_next = 0.f, dnorm = 0.f, revr = 0.f;
+    float rcr = 0.f, lam1 = 0.f, lam_rho = 0.f, lam_next = 0.f, dnorm = 0.f, revr = 0.f, pc = 0.f;
     int rho = 0;
     bool done = false;
 
     // ---- 1. k_eff >= d: the span test kernel has already factorised G_keep --
-    if (k >= D && (hflag_in & HFLAG_SPAN_FULL)) { m = D; done = true; status |= OBF_DEV_SKIPPED | OBF_DEV_SPAN_FULL; }
+    if (k >= D && (hflag_in & HFLAG_SPAN_FULL)) { m = D; done = true; pc = 1.f; status |= OBF_DEV_SKIPPED | OBF_DEV_SPAN_FULL; }
 
     // ---- 2. orthonormal basis of span(V_keep), Eq. 2 ------------------------
     if (!done) {
@@ -143,7 +143,7 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
             }
             __syncthreads();
         }
-        if (m >= D) { done = true; status |= OBF_DEV_SKIPPED | OBF_DEV_SPAN_FULL; }
+        if (m >= D) { done = true; pc = 1.f; status |= OBF_DEV_SKIPPED | OBF_DEV_SPAN_FULL; }
     }
 
     if (!done) {
@@ -165,6 +165,19 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
             vu[tid] = s;
         }
         __syncthreads();
+        if (c.diag) {
+            // projection cosine: s = sum of the deleted values, its part inside span(V_keep) is s - P s
+            float sv = 0.f, par = 0.f;
+            if (tid < D) {
+                sv = p.svec[(size_t)g * D + tid];
+                float ps = 0.f;
+                for (int cc = 0; cc < D; ++cc) ps = fmaf(B1[tid * LD + cc], p.svec[(size_t)g * D + cc], ps);
+                par = sv - ps;
+            }
+            const float ss = block_sum<ALG_NT>(sv * sv, red), pp = block_sum<ALG_NT>(par * par, red);
+            const float sp = block_sum<ALG_NT>(sv * par, red);
+            pc = (ss > 0.f && pp > 0.f) ? sp * rsqrtf(ss) * rsqrtf(pp) : 0.f;
+        }
         const float trG = block_sum<ALG_NT>(tid < D ? B2[tid * LD + tid] : 0.f, red);
         // two D x D x D products, a 4 x 8 register tile per thread (rows a0 + 0..3, columns b0 + 32 * 0..7:
         // the lanes of a warp read consecutive columns, and a row's value is a broadcast)
@@ -701,7 +714,7 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
             dg->rcr = rcr; dg->delta_norm = dnorm;
             dg->lam_1 = lam1; dg->lam_rho = lam_rho; dg->lam_next = lam_next;
             dg->span_rank = m; dg->rho_eff = rho; dg->status = status;
-            dg->revr = revr;
+            dg->revr = revr; dg->pc = pc;
         }
     }
 }

@@ -78,6 +78,7 @@ struct CallDev {
     float *gram_k;            // [heads_total, gram_slots, d, d] partial Gram of retained values
     float *uvec;              // [heads_total, gram_slots, u_groups, d] partial sum_j A_j v_j over deleted j
     float *delta;             // [heads_total, d]
+    float *svec;              // [heads_total, d] sum of the deleted value rows (only filled when diagnostics are asked for)
     uint32_t *hflag;          // [heads_total] bit0: delta != 0 -> inject
 };
 

@@ -261,7 +261,7 @@ __global__ void __launch_bounds__(SEL_NT) k_select(const __grid_constant__ CallD
             dg.a_keep = a_keep; dg.a_del = a_del; dg.alpha = a_del / (a_keep + p.eps);
             dg.rcr = 0.f; dg.delta_norm = 0.f; dg.kth_score = tau == 0xFFFFFFFFu ? INFINITY : key_score(tau); dg.next_score = next;
             dg.lam_1 = dg.lam_rho = dg.lam_next = 0.f;
-            dg.span_rank = -1; dg.rho_eff = 0; dg.status = OBF_DEV_SKIPPED; dg.revr = 0.f;
+            dg.span_rank = -1; dg.rho_eff = 0; dg.status = OBF_DEV_SKIPPED; dg.revr = 0.f; dg.pc = 0.f;
             c.diag[lh] = dg;
         }
     }
@@ -455,7 +455,7 @@ __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ Call
                     dg.a_keep = a_keep; dg.a_del = a_del; dg.alpha = a_del / (a_keep + p.eps);
                     dg.rcr = 0.f; dg.delta_norm = 0.f; dg.kth_score = tau == 0xFFFFFFFFu ? INFINITY : key_score(tau); dg.next_score = next;
                     dg.lam_1 = dg.lam_rho = dg.lam_next = 0.f;
-                    dg.span_rank = -1; dg.rho_eff = 0; dg.status = OBF_DEV_SKIPPED; dg.revr = 0.f;
+                    dg.span_rank = -1; dg.rho_eff = 0; dg.status = OBF_DEV_SKIPPED; dg.revr = 0.f; dg.pc = 0.f;
                     c.diag[lh] = dg;
                 }
             }
@@ -473,7 +473,7 @@ __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ Call
             dg.a_keep = a_keep; dg.a_del = a_del; dg.alpha = a_del / (a_keep + p.eps);
             dg.rcr = 0.f; dg.delta_norm = 0.f; dg.kth_score = tau == 0xFFFFFFFFu ? INFINITY : key_score(tau); dg.next_score = next;
             dg.lam_1 = dg.lam_rho = dg.lam_next = 0.f;
-            dg.span_rank = -1; dg.rho_eff = 0; dg.status = OBF_DEV_SKIPPED; dg.revr = 0.f;
+            dg.span_rank = -1; dg.rho_eff = 0; dg.status = OBF_DEV_SKIPPED; dg.revr = 0.f; dg.pc = 0.f;
             c.diag[lh] = dg;
         }
     }
@@ -534,6 +534,35 @@ __global__ void __launch_bounds__(256) k_gather(const __grid_constant__ CallDev 
                 if (WHICH & 1) *reinterpret_cast<uint4 *>(vo + (size_t)r[u] * ROW_BYTES + ch * 16) = vv[u];
             }
         }
+    }
+}
+
+// Diagnostics only (projection cosine): s = sum of the deleted value rows of a head, for heads with a
+// diagnostics record.  grid = (token splits, heads_total), 256 threads = 256 / D row groups x D columns.
+template <typename TIN, int D>
+__global__ void __launch_bounds__(256) k_vsum(const __grid_constant__ CallDev p)
+{
+    __shared__ float part[256];
+    int ci, lh;
+    locate(p, blockIdx.y, ci, lh);
+    const CacheDev &c = p.c[ci];
+    if (!c.diag || c.T <= c.k_eff) return;
+    constexpr int RG = 256 / D > 0 ? 256 / D : 1;         // row groups
+    const int col = threadIdx.x % D, rg = threadIdx.x / D;
+    const int per = (c.T + gridDim.x - 1) / gridDim.x;
+    const int r0 = blockIdx.x * per, r1 = min(c.T, r0 + per);
+    const TIN *V = reinterpret_cast<const TIN *>(c.v) + (size_t)lh * c.T * D;
+    const uint8_t *keep = p.keep + c.tok_off + (size_t)lh * c.T;
+    float acc = 0.f;
+    if (rg < RG)
+        for (int r = r0 + rg; r < r1; r += RG)
+            if (!keep[r]) acc += to_f32(V[(size_t)r * D + col]);
+    part[threadIdx.x] = acc;
+    __syncthreads();
+    if (threadIdx.x < D) {
+        float t = 0.f;
+        for (int g2 = 0; g2 < RG; ++g2) t += part[g2 * D + threadIdx.x];
+        atomicAdd(&p.svec[(size_t)blockIdx.y * D + threadIdx.x], t);
     }
 }
 

@@ -65,7 +65,7 @@ static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; 
 
 struct Layout {
     size_t off_status, off_scores, off_keep, off_stats, off_sums, off_lscores, off_scores2;
-    size_t off_gram_d, off_gram_k, off_uvec, off_delta, off_hflag;
+    size_t off_gram_d, off_gram_k, off_uvec, off_delta, off_hflag, off_svec;
     size_t total;
     int splits;
     int heads_total;
@@ -247,7 +247,7 @@ static void make_layout(const obf_params_t *p, const obf_cache_t *caches, int32_
         L.off_sc_head = o; o = align_up(o + (size_t)L.heads_total * L.sc_qt * 128 * sizeof(unsigned long long), 256);
         L.off_sc_sync = o; o = align_up(o + (size_t)L.heads_total * L.sc_qt * sizeof(uint32_t), 256);
     }
-    L.off_gram_d = L.off_gram_k = L.off_uvec = L.off_delta = L.off_hflag = o;
+    L.off_gram_d = L.off_gram_k = L.off_uvec = L.off_delta = L.off_hflag = L.off_svec = o;
     if (rank > 0) {
         const size_t gsz = (size_t)L.heads_total * L.gram_slots * d * d * sizeof(float);
         L.off_gram_d = o; o = align_up(o + gsz, 256);
@@ -255,6 +255,7 @@ static void make_layout(const obf_params_t *p, const obf_cache_t *caches, int32_
         L.off_uvec = o;   o = align_up(o + (size_t)L.heads_total * L.gram_slots * GT_GROUPS * d * sizeof(float), 256);
         L.off_delta = o;  o = align_up(o + (size_t)L.heads_total * d * sizeof(float), 256);
         L.off_hflag = o;  o = align_up(o + (size_t)L.heads_total * sizeof(uint32_t), 256);
+        L.off_svec = o;   o = align_up(o + (size_t)L.heads_total * d * sizeof(float), 256);
     }
     L.total = o;
 }
@@ -437,6 +438,15 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
             k_gram<TIN, D><<<g5, 256, 0, st>>>(cd);
             mark(st, "k_gram");
         }
+        bool any_diag = false;
+        for (int i = 0; i < cd.n_caches; ++i) any_diag = any_diag || cd.c[i].diag != nullptr;
+        if (any_diag) {
+            // the projection cosine of the diagnostics needs the plain sum of the deleted values: one more pass over V
+            OBF_CUDA_TRY(cudaMemsetAsync(cd.svec, 0, (size_t)heads * D * sizeof(float), st));
+            dim3 gv((T_max + 2047) / 2048, heads);
+            k_vsum<TIN, D><<<gv, 256, 0, st>>>(cd);
+            mark(st, "k_vsum");
+        }
         const size_t sm_span = span_smem_bytes<D>();
         if ((s = set_smem(k_span_test<D>, sm_span)) != OBF_OK) return s;
         if (side) {
@@ -537,6 +547,7 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
     cd.uvec = reinterpret_cast<float *>(ws + L.off_uvec);
     cd.delta = reinterpret_cast<float *>(ws + L.off_delta);
     cd.hflag = reinterpret_cast<uint32_t *>(ws + L.off_hflag);
+    cd.svec = reinterpret_cast<float *>(ws + L.off_svec);
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (!g_keep_status) OBF_CUDA_TRY(cudaMemsetAsync(cd.status, 0, 256, st));     // a slab of a larger job adds to the job's status

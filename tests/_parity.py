@@ -121,6 +121,9 @@ def check_head(dtype: str, K: np.ndarray, V: np.ndarray, Q: np.ndarray, budget: 
         if g_delta is not None and np.linalg.norm(g_delta) == 0:
             assert np.array_equal(g_vbits, in_vbits[g_idx])
         return rep
+    if g_diag is not None and "pc" in dg:
+        # projection cosine of the deleted values (0 when OBF does not run at all)
+        assert abs(g_diag["pc"] - dg["pc"]) <= 2e-3, "%s: PC %.5f vs %.5f" % (name, g_diag["pc"], dg["pc"])
     if dg["skipped"]:
         assert np.array_equal(g_vbits, in_vbits[g_idx]), "%s: V_out must equal V_keep bit for bit" % name
         if g_delta is not None:

@@ -48,6 +48,8 @@ def lib_obf(K, V, Q, budget, rank, eps=1e-12):
     R = Vdel - Vdel @ Pi
     a_del, a_keep = A[~keep].sum(), A[keep].sum()
     out["rcr"] = (R ** 2).sum() / ((Vdel ** 2).sum() + eps)
+    ssum = Vdel.sum(axis=0); psum = ssum @ Pi               # sum of the deleted values and of their projections
+    out["pc"] = float(ssum @ psum / (np.linalg.norm(ssum) * np.linalg.norm(psum)))
     if (R ** 2).sum() <= 1e-12 * (Vdel ** 2).sum():
         return out
     _, s, Vt = np.linalg.svd(R, full_matrices=False)
@@ -284,6 +286,7 @@ def test_obf_matches_lapack_pipeline(seed, T, d, n_q, budget, rank):
     rho = r["diag"]["rho_eff"]
     assert r["diag"]["revr"] == pytest.approx((ref["sing"][:rho] ** 2).sum() / (ref["sing"] ** 2).sum(), rel=1e-9)
     assert r["diag"]["rcr"] == pytest.approx(ref["rcr"], rel=1e-9)
+    assert r["diag"]["pc"] == pytest.approx(ref["pc"], abs=1e-10)             # projection cosine (PC)
     np.testing.assert_allclose(r["proj"], ref["proj"], atol=1e-8)      # sign/rotation free comparison
     np.testing.assert_allclose(r["Delta"], ref["Delta"], atol=1e-9)
     np.testing.assert_allclose(r["delta"], ref["delta"], atol=1e-9)
