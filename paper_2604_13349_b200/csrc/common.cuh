@@ -66,6 +66,8 @@ struct CallDev {
     int32_t layerwise;        // 1: one retained set per layer (masses summed over its KV heads)
     int32_t n_sink;           // protected prefix: the first n_sink positions are retained besides the budget
     int32_t fast_iters;       // > 0: that many Gram subspace iterations instead of the exact eigenvectors
+    int32_t debug_drop_publish;   // test hook: the score kernel never publishes a head's normalisers, so the wait for them runs out
+    unsigned long long wait_limit_ns;   // after this long a device-side wait gives up and reports OBF_DEV_TIMEOUT
     // workspace
     uint32_t *status;
     float *scores;            // [sum heads*T] attention mass (Eq. 1)

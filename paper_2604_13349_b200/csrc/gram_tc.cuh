@@ -112,7 +112,7 @@ __global__ void __launch_bounds__(GT_THREADS, 1) k_gram_tc(const __grid_constant
     __shared__ uint32_t s_tmem, s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    tc::WaitCtx wc{&s_abort, p.status};
+    tc::WaitCtx wc{&s_abort, p.status, p.wait_limit_ns};
 
     if (tid == 0) {
         s_abort = 0u;

@@ -349,7 +349,11 @@ static obf_status_t launch_score_tc(const CallDev &cd, const Layout &L, cudaStre
     const size_t smem = ST_SMEM_BYTES;
     OBF_CUDA_TRY(cudaFuncSetAttribute(k_score_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     OBF_CUDA_TRY(cudaMemsetAsync(cd.sc_head, 0, (L.off_sc_sync - L.off_sc_head) + (size_t)cd.heads_total * L.sc_qt * sizeof(uint32_t), st));
-    k_score_tc<<<L.sc_blocks, ST_THREADS, smem, st>>>(cd, maps);
+    // The blocks of a head's team wait for one another, so the whole grid has to be resident at once: a
+    // cooperative launch starts only when it is (the grid never exceeds one block per multiprocessor).
+    void *args[2] = {const_cast<CallDev *>(&cd), &maps};
+    OBF_CUDA_TRY(cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(k_score_tc), dim3(L.sc_blocks), dim3(ST_THREADS),
+                                             args, smem, st));
     mark(st, "k_score_tc");
     if (L.sc_qt == 2) {
         int T_max = 1;
@@ -539,6 +543,8 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
     cd.layerwise = (p->flags & OBF_FLAG_LAYERWISE) ? 1 : 0;
     cd.n_sink = (int32_t)OBF_FLAG_SINK_OF(p->flags);
     cd.fast_iters = (p->flags & OBF_FLAG_FAST_PATH) ? 3 : 0;
+    cd.wait_limit_ns = tc::WAIT_LIMIT_NS;
+    cd.debug_drop_publish = 0;
     cd.sc_part = reinterpret_cast<float *>(ws + L.off_sc_part);
     cd.sc_head = reinterpret_cast<float *>(ws + L.off_sc_head);
     cd.sc_cnt = reinterpret_cast<uint32_t *>(ws + L.off_sc_sync);

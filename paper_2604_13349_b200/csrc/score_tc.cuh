@@ -15,8 +15,8 @@
 //       (m_t, z_t); the last block of the head to arrive folds all chunks into
 //       M'_t = M_t + log2(Z_t) and publishes that.
 //   pass B (pooling)     S^T = K_tile Q^T with the KEYS on the lanes: a thread owns one
-//       key and sums exp2(s_tj c - M'_t) = softmax_j over its share of the queries;
-//       again nothing crosses lanes.
+//       key and sums exp2(s_tj c - M'_t) = softmax_j over all queries of the tile;
+//       again nothing crosses lanes, and a key's mass is complete in one thread.
 //
 // A head's T keys are cut into chunks of 4 tiles of 128 keys; a head's chunks are worked
 // on by a team of blocks in the same round.  Rounds are dealt as
@@ -30,12 +30,18 @@
 // round ahead; Q of a pass is loaded while the pass before it runs, into the buffer of its
 // kind: one for the statistics passes, one for the pooling passes, which read Q again),
 // warps 1 and 19 MMA issuers, alternate tiles (accumulators in a 4-deep ring of 128 tensor-memory columns),
-// warps 2..17 consumers: warp (quarter, part) reads lanes [32*quarter, +32) and columns
-// [32*part, +32) of every accumulator tile, which frees the tile as soon as the 16 warps
-// have it in registers; warp 18 is the messenger: it publishes the chunk statistics the
-// consumers leave in shared memory, folds a head's chunks when its block is the last to
-// arrive, and then fetches the head's M' for the pooling pass a round later, so that the
-// consumers never wait for global memory.
+// warps 2..17 consumers in four groups of four, group g taking the tiles with index g (mod 4), so
+// that every scheduler holds one warp of each group and the four are at different points of
+// their tiles: a warp owns the 32 tensor-memory lanes of its quarter and walks the 128 columns
+// of its tile in four pieces of 32 (load, wait, exponentials); the tile goes back to the MMA
+// issuers when its last piece is in registers.  A key's pooled mass is complete in one thread.
+// Measured alternatives that were slower: two groups (two warps per scheduler), the load of a
+// piece in flight behind the arithmetic of the piece before it (the unrolled code was slower in
+// every form), a share of the exponentials evaluated as a polynomial on the FMA pipe (the
+// special-function unit is busy about half of the time: it is not what the warps wait for).
+// Warp 18 is the messenger: it publishes the chunk statistics the consumers leave in shared
+// memory, folds a head's chunks when its block is the last to arrive, and then fetches the
+// head's M' for the pooling pass a round later, so that the consumers never wait for global memory.
 #pragma once
 
 #include "tc_common.cuh"
@@ -48,12 +54,13 @@ constexpr int ST_STAGES = 4;                        // K tiles in flight in shar
 constexpr int ST_TBUF = 4;                          // accumulator tiles in tensor memory
 constexpr int ST_LAG = 1;                           // rounds between a chunk's statistics pass and its pooling pass
 constexpr int ST_TILE_BYTES = 128 * 128 * 2;
-constexpr int ST_CONSUMERS = 512;
+constexpr int ST_GROUPS = 4;                        // consumer groups of four warps, one accumulator tile each
+constexpr int ST_CONSUMERS = ST_GROUPS * 128;
 constexpr int ST_THREADS = 64 + ST_CONSUMERS + 64;
 constexpr int ST_MAX_NQ = 256;                      // two query tiles of 128 rows
 constexpr float ST_LOG2E = 1.4426950408889634f;
 constexpr size_t ST_SMEM_BYTES = 1024 + (size_t)2 * ST_TILE_BYTES + (size_t)ST_STAGES * ST_TILE_BYTES +
-                                 (2 * 2 * 4 * 128 + 2 * 128 + 2 * ST_TILES * 4 * 128) * sizeof(float) + 64;
+                                 (2 * 2 * ST_GROUPS * 128 + 2 * 128) * sizeof(float) + 64;
 static_assert(ST_STAGES == ST_TBUF, "a ring stage is released by the accumulator barrier of the same index");
 
 struct ScoreItem {
@@ -143,7 +150,7 @@ __device__ __forceinline__ unsigned long long ld_relaxed_gpu_u64(const unsigned 
     return v;
 }
 
-// Pass A on one thread's 32 logits of a tile: running maximum m (log2 domain) and sum z of
+// Pass A on one thread's 32 logits of a piece: running maximum m (log2 domain) and sum z of
 // exp2(s c - m) of one query.  With MASKED only the first n_valid columns are keys.
 template <bool MASKED>
 __device__ __forceinline__ void stats_update(uint32_t (&rr)[32], int n_valid, float sc, float &m, float &z)
@@ -177,27 +184,40 @@ __device__ __forceinline__ void stats_update(uint32_t (&rr)[32], int n_valid, fl
     }
 }
 
+// Pass B on one thread's 32 logits of a piece: the softmax weights of one key under 32 queries, added up.
+// mp: M'_t of those queries (shared memory, the same address for every lane).
+__device__ __forceinline__ float pool_piece(const uint32_t (&rr)[32], const float *mp, float sc)
+{
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+    for (int e = 0; e < 32; e += 4) {
+        const float4 v = *reinterpret_cast<const float4 *>(mp + e);
+        a0 += ex2_approx(fmaf(__uint_as_float(rr[e]), sc, -v.x));
+        a1 += ex2_approx(fmaf(__uint_as_float(rr[e + 1]), sc, -v.y));
+        a2 += ex2_approx(fmaf(__uint_as_float(rr[e + 2]), sc, -v.z));
+        a3 += ex2_approx(fmaf(__uint_as_float(rr[e + 3]), sc, -v.w));
+    }
+    return (a0 + a1) + (a2 + a3);
+}
+
 __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constant__ CallDev p, const __grid_constant__ TcMaps tm)
 {
     extern __shared__ uint8_t st_smem_raw[];
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(st_smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *q_s = base;                                           // 2 x [128 x 128] bf16: Q of a statistics pass, Q of a pooling pass; two 64-column halves each
     uint8_t *ring = q_s + 2 * ST_TILE_BYTES;                       // ST_STAGES x 32 KiB
-    float *s_m = reinterpret_cast<float *>(ring + ST_STAGES * ST_TILE_BYTES);   // [2][4 parts][128 queries] chunk maxima
-    float *s_z = s_m + 2 * 4 * 128;                                // [2][4 parts][128 queries] chunk sums
-    float *s_mp = s_z + 2 * 4 * 128;                               // [2][128] M'_t of the head being pooled
-    float *s_acc = s_mp + 2 * 128;                                 // [2][ST_TILES][4 parts][128 keys] pooled partial masses of a pass
+    float *s_m = reinterpret_cast<float *>(ring + ST_STAGES * ST_TILE_BYTES);   // [2][groups][128 queries] chunk maxima
+    float *s_z = s_m + 2 * ST_GROUPS * 128;                        // [2][groups][128 queries] chunk sums
+    float *s_mp = s_z + 2 * ST_GROUPS * 128;                       // [2][128] M'_t of the head being pooled
     __shared__ uint64_t bar_q_full[2], bar_q_free[2], bar_full[ST_STAGES];
     __shared__ uint64_t bar_t_full[ST_TBUF], bar_t_empty[ST_TBUF];
-    // pooled partial masses of a pooling pass: written by the four column parts, summed one tile into the next pass
-    __shared__ uint64_t bar_acc_ready[2], bar_acc_free[2];
     __shared__ uint64_t bar_st_ready[2], bar_st_free[2], bar_mp_ready[2], bar_mp_free[2];
     __shared__ ScoreTab s_tab[OBF_MAX_CACHES];
     __shared__ uint32_t s_tmem, s_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int R = p.sc_rounds;
-    tc::WaitCtx wc{&s_abort, p.status};
+    tc::WaitCtx wc{&s_abort, p.status, p.wait_limit_ns};
 
     if (tid == 0) {
         s_abort = 0u;
@@ -205,11 +225,9 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
         for (int s = 0; s < ST_STAGES; ++s) tc::mbar_init(&bar_full[s], 1);
         for (int s = 0; s < ST_TBUF; ++s) {
             tc::mbar_init(&bar_t_full[s], 1);
-            tc::mbar_init(&bar_t_empty[s], ST_CONSUMERS / 32);
+            tc::mbar_init(&bar_t_empty[s], 4);                  // the four warps of the group that owns the tile
         }
         for (int b = 0; b < 2; ++b) {
-            tc::mbar_init(&bar_acc_ready[b], ST_CONSUMERS / 32);
-            tc::mbar_init(&bar_acc_free[b], ST_CONSUMERS / 32);
             tc::mbar_init(&bar_st_ready[b], ST_CONSUMERS / 32);
             tc::mbar_init(&bar_st_free[b], 1);
             tc::mbar_init(&bar_mp_ready[b], 1);
@@ -345,128 +363,90 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
         }
     } else if (warp < 2 + ST_CONSUMERS / 32) {
         // ---------------- consumers ----------------
+        static_assert(ST_TBUF % ST_GROUPS == 0, "an accumulator tile must always belong to the same consumer group");
         const int q = warp & 3;                        // tensor-memory lane quarter this warp may touch
-        const int part = (warp - 2) >> 2;              // columns [32 * part, +32) of every tile; sums tile `part` of a pooling pass
+        const int grp = (warp - 2) >> 2;               // tiles with index == grp (mod ST_GROUPS) are this warp's
         const int row = q * 32 + lane;                 // lane of the accumulator tile: a query (pass A) or a key (pass B)
         const uint32_t tlane = tmem + ((uint32_t)(q * 32) << 16);
         const float sc = ST_LOG2E * rsqrtf(128.0f);
-        uint32_t it = 0, n_a[2] = {0u, 0u}, n_b[2] = {0u, 0u}, n_pool = 0u;
+        uint32_t it = 0, n_a[2] = {0u, 0u}, n_b[2] = {0u, 0u};
 
-        // a pooling pass whose partial masses wait in shared memory for their sum
-        bool pend = false;
-        uint32_t pend_buf = 0u, pend_par = 0u;
-        int pend_T = 0, pend_j = 0, pend_nt = 0;
-        float *pend_dst = nullptr, *pend_out = nullptr;
-        auto finish_pool = [&]() {
-            tc::mbar_wait(&bar_acc_ready[pend_buf], pend_par, wc, 20);
-            float a = 0.f;
-            if (part < pend_nt) {
-                const float *sa = s_acc + ((pend_buf * ST_TILES + part) * 4) * 128 + row;
-                a = (sa[0] + sa[128]) + (sa[256] + sa[384]);
+        // The four 32-column pieces of an accumulator tile, `work(piece, registers)` on each; the tile is handed
+        // back as soon as its last piece is in registers.
+        auto walk_tile = [&](uint32_t ti, auto &&work) {
+            const uint32_t tb = ti % ST_TBUF;
+            tc::mbar_wait(&bar_t_full[tb], (ti / ST_TBUF) & 1u, wc, 20);
+            tc::tc_fence_after();
+            const uint32_t ta = tlane + tb * 128u;
+            uint32_t rr[32];
+#pragma unroll 1
+            for (int pc = 0; pc < 4; ++pc) {
+                tc::tmem_ld32(ta + 32u * pc, rr);
+                tc::tmem_ld_wait();
+                if (pc == 3) {
+                    tc::tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) tc::mbar_arrive(&bar_t_empty[tb]);
+                }
+                work(pc, rr);
             }
-            __syncwarp();
-            if (lane == 0) tc::mbar_arrive(&bar_acc_free[pend_buf]);
-            if (part < pend_nt && pend_j < pend_T) {
-                if (!isfinite(a)) atomicOr(p.status, OBF_DEV_NONFINITE);
-                pend_dst[pend_j] = a;
-                if (pend_out) pend_out[pend_j] = a;
-            }
-            pend = false;
         };
 
         for (int i = 0; i < R + ST_LAG; ++i) {
-            // ======== pass A of round i: maximum and sum per query over columns [32 * part, +32) of the chunk's tiles ========
+            // ======== pass A of round i: maximum and sum per query over the keys of this group's tiles ========
             ScoreItem item;
             if (i < R && score_item(p, s_tab, i, item)) {
                 const int T = s_tab[item.cache].T, buf = i & 1;
                 float m = -INFINITY, z = 0.f;
 #pragma unroll 1
                 for (int t = 0; t < item.nt; ++t) {
-                    // columns [32 * part, +32) of every tile of the chunk; the tile is released as soon as they are in registers
                     const uint32_t ti = it + t;
-                    const int tb = ti % ST_TBUF;
-                    tc::mbar_wait(&bar_t_full[tb], (ti / ST_TBUF) & 1u, wc, 20);
-                    tc::tc_fence_after();
-                    uint32_t rr[32];
-                    tc::tmem_ld32(tlane + (uint32_t)(tb * 128 + part * 32), rr);
-                    tc::tmem_ld_wait();
-                    tc::tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) tc::mbar_arrive(&bar_t_empty[tb]);
-                    const int key0 = item.chunk * ST_CHUNK + t * 128 + part * 32;         // key of column 0 of this block
-                    // two copies of the update: the one that masks missing keys runs for a head's ragged last tile only
-                    if (key0 + 32 > T) stats_update<true>(rr, T - key0, sc, m, z);
-                    else stats_update<false>(rr, 32, sc, m, z);
-                    if (pend) finish_pool();
+                    if ((int)(ti % ST_GROUPS) != grp) continue;
+                    const int key0 = item.chunk * ST_CHUNK + t * 128;                     // key of column 0 of the tile
+                    walk_tile(ti, [&](int pc, uint32_t (&rr)[32]) {
+                        // two copies of the update: the one that masks missing keys runs for a head's ragged last tile only
+                        const int k0 = key0 + 32 * pc;
+                        if (k0 + 32 > T) stats_update<true>(rr, T - k0, sc, m, z);
+                        else stats_update<false>(rr, 32, sc, m, z);
+                    });
                 }
                 it += item.nt;
-                // hand (m, z) of this column part to the messenger
+                // hand (m, z) of this group's tiles to the messenger
                 if (n_a[buf] > 0) tc::mbar_wait(&bar_st_free[buf], (n_a[buf] - 1) & 1u, wc, 20);
-                s_m[(buf * 4 + part) * 128 + row] = m;
-                s_z[(buf * 4 + part) * 128 + row] = z;
+                s_m[(buf * ST_GROUPS + grp) * 128 + row] = m;
+                s_z[(buf * ST_GROUPS + grp) * 128 + row] = z;
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(&bar_st_ready[buf]);
                 ++n_a[buf];
             }
-            // ======== pass B of round i - ST_LAG: pooled mass per key over queries [32 * part, +32) ========
+            // ======== pass B of round i - ST_LAG: pooled mass per key over all queries of the tile ========
             if (i >= ST_LAG && score_item(p, s_tab, i - ST_LAG, item)) {
                 const CacheDev &c = p.c[item.cache];
                 const int T = s_tab[item.cache].T, buf = (i - ST_LAG) & 1;
                 tc::mbar_wait(&bar_mp_ready[buf], n_b[buf] & 1u, wc, 20);
-                float mp[32];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const float4 v = *reinterpret_cast<const float4 *>(s_mp + buf * 128 + part * 32 + e * 4);
-                    mp[4 * e] = v.x; mp[4 * e + 1] = v.y; mp[4 * e + 2] = v.z; mp[4 * e + 3] = v.w;
-                }
-                // this pass's partial masses go to the buffer the pass before the last one used
-                const uint32_t ab = n_pool & 1u, use = n_pool >> 1;
+                const float *mp = s_mp + buf * 128;
+                // with two query tiles per head each writes its own plane; a small kernel adds them up afterwards
+                float *dst = (item.qt ? p.scores2 : p.scores) + c.tok_off + (size_t)item.lh * T;
+                float *out = (c.scores_out && p.sc_qt == 1) ? c.scores_out + (size_t)item.lh * T : nullptr;
 #pragma unroll 1
                 for (int t = 0; t < item.nt; ++t) {
-                    // queries [32 * part, +32) of every tile of the chunk; the tile is released as soon as they are in registers
                     const uint32_t ti = it + t;
-                    const int tb = ti % ST_TBUF;
-                    tc::mbar_wait(&bar_t_full[tb], (ti / ST_TBUF) & 1u, wc, 20);
-                    tc::tc_fence_after();
-                    uint32_t rr[32];
-                    tc::tmem_ld32(tlane + (uint32_t)(tb * 128 + part * 32), rr);
-                    tc::tmem_ld_wait();
-                    tc::tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) tc::mbar_arrive(&bar_t_empty[tb]);
-                    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll
-                    for (int e = 0; e < 32; e += 4) {
-                        a0 += ex2_approx(fmaf(__uint_as_float(rr[e]), sc, -mp[e]));
-                        a1 += ex2_approx(fmaf(__uint_as_float(rr[e + 1]), sc, -mp[e + 1]));
-                        a2 += ex2_approx(fmaf(__uint_as_float(rr[e + 2]), sc, -mp[e + 2]));
-                        a3 += ex2_approx(fmaf(__uint_as_float(rr[e + 3]), sc, -mp[e + 3]));
+                    if ((int)(ti % ST_GROUPS) != grp) continue;
+                    float a = 0.f;
+                    walk_tile(ti, [&](int pc, uint32_t (&rr)[32]) { a += pool_piece(rr, mp + 32 * pc, sc); });
+                    const int j = item.chunk * ST_CHUNK + t * 128 + row;
+                    if (j < T) {
+                        if (!isfinite(a)) atomicOr(p.status, OBF_DEV_NONFINITE);
+                        dst[j] = a;
+                        if (out) out[j] = a;
                     }
-                    if (pend) finish_pool();                       // the pass before this one, one tile late
-                    if (t == 0 && use > 0) tc::mbar_wait(&bar_acc_free[ab], (use - 1) & 1u, wc, 20);
-                    s_acc[((ab * ST_TILES + t) * 4 + part) * 128 + row] = (a0 + a1) + (a2 + a3);
                 }
                 it += item.nt;
                 __syncwarp();
-                if (lane == 0) {
-                    tc::mbar_arrive(&bar_acc_ready[ab]);
-                    tc::mbar_arrive(&bar_mp_free[buf]);
-                }
+                if (lane == 0) tc::mbar_arrive(&bar_mp_free[buf]);
                 ++n_b[buf];
-                ++n_pool;
-                // the four parts' sums of tile `part` become this warp's keys' masses after the next tile
-                pend = true;
-                pend_buf = ab;
-                pend_par = use & 1u;
-                pend_T = T;
-                pend_nt = item.nt;
-                pend_j = item.chunk * ST_CHUNK + part * 128 + row;
-                // with two query tiles per head each writes its own plane; a small kernel adds them up afterwards
-                pend_dst = (item.qt ? p.scores2 : p.scores) + c.tok_off + (size_t)item.lh * T;
-                pend_out = (c.scores_out && p.sc_qt == 1) ? c.scores_out + (size_t)item.lh * T : nullptr;
             }
         }
-        if (pend) finish_pool();
     } else {
         // ---------------- messenger: chunk statistics out, a head's chunks folded by the last block to arrive, M' in ----------------
         uint32_t n_a[2] = {0u, 0u}, n_b[2] = {0u, 0u};
@@ -482,11 +462,13 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 const int t = lane + 32 * k;
-                const float *sm = s_m + buf * 4 * 128 + t, *sz = s_z + buf * 4 * 128 + t;
-                const float M = fmaxf(fmaxf(sm[0], sm[128]), fmaxf(sm[256], sm[384]));
+                const float *sm = s_m + buf * ST_GROUPS * 128 + t, *sz = s_z + buf * ST_GROUPS * 128 + t;
+                float M = sm[0];
+#pragma unroll
+                for (int e = 1; e < ST_GROUPS; ++e) M = fmaxf(M, sm[e * 128]);
                 float Z = 0.f;
 #pragma unroll
-                for (int e = 0; e < 4; ++e)
+                for (int e = 0; e < ST_GROUPS; ++e)
                     if (sm[e * 128] > -INFINITY) Z += sz[e * 128] * ex2_approx(sm[e * 128] - M);
                 if (t < nq) __stcg(&partials[t], make_float2(M, Z));
             }
@@ -500,6 +482,8 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
             last = __shfl_sync(0xffffffffu, last, 0);
             ++n_a[buf];
             if (last) {
+                // every lane reads other blocks' statistics below: each orders its own loads behind lane 0's acquire
+                asm volatile("fence.acq_rel.gpu;" ::: "memory");
                 // this block is the last of its head: fold all chunks, eight chunks of the lane's four queries per sweep
                 // (32 loads in flight: the fold is a few round trips long, whatever the team's size)
                 const float2 *hp = reinterpret_cast<const float2 *>(p.sc_part) + (c.sc_part_off + (size_t)item.lv * team * 128);
@@ -539,7 +523,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                         mp = __int_as_float(0x7fc00000);
                     }
                     // one 64-bit word per query: low = M'_t, high = 1 once it is valid
-                    st_relaxed_gpu_u64(words + t, (1ull << 32) | __float_as_uint(mp));
+                    if (!p.debug_drop_publish) st_relaxed_gpu_u64(words + t, (1ull << 32) | __float_as_uint(mp));
                 }
             }
             // M'_t of this head for the pooling pass one round on; the team has a round to get there
@@ -560,7 +544,7 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                         if (lane + 32 * k < nq && (v[k] >> 32) == 0ull) all = false;
                     // the warp leaves the loop as one: votes, not per-lane exits
                     if (__all_sync(0xffffffffu, all) || __any_sync(0xffffffffu, *(volatile uint32_t *)&s_abort != 0u)) break;
-                    if (__any_sync(0xffffffffu, tc::global_ns() - t0 > tc::WAIT_LIMIT_NS)) {
+                    if (__any_sync(0xffffffffu, tc::global_ns() - t0 > p.wait_limit_ns)) {
                         if (lane == 0) {
                             s_abort = 1u;
                             atomicOr(p.status, OBF_DEV_TIMEOUT);

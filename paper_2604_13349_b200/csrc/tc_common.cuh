@@ -2,7 +2,7 @@
 // waits, TMA tile loads, tensor-memory allocation and access, and tcgen05 matrix
 // multiply-accumulate with shared-memory operand descriptors.
 //
-// Every wait in this file gives up after WAIT_LIMIT_NS: it sets the block's abort
+// Every wait in this file gives up after the call's wait limit (WAIT_LIMIT_NS by default): it sets the block's abort
 // flag and OBF_DEV_TIMEOUT in the device status word and returns, so a wrong
 // handshake can never hang the GPU; the host then sees OBF_ERR_DEVICE_STATUS.
 #pragma once
@@ -14,7 +14,7 @@
 namespace obf {
 namespace tc {
 
-constexpr uint64_t WAIT_LIMIT_NS = 1000000000ull;      // one second per wait
+constexpr uint64_t WAIT_LIMIT_NS = 1000000000ull;      // one second per wait unless the call says otherwise
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -71,10 +71,11 @@ __device__ __forceinline__ bool mbar_test(uint64_t *bar, uint32_t parity)
 struct WaitCtx {
     volatile uint32_t *abort_flag;
     uint32_t *status;
+    uint64_t limit_ns;
 };
 
 // Waits until the phase of `bar` with the given parity has completed.  Returns
-// false (at once if the block already aborted, else after WAIT_LIMIT_NS) when the
+// false (at once if the block already aborted, else after the wait limit) when the
 // wait was abandoned.  A non-zero `sleep_ns` makes a single-thread role (producer,
 // MMA issuer) back off between polls so that it does not take issue slots from
 // the warps that compute.
@@ -90,7 +91,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, const 
             if (sleep_ns) __nanosleep(sleep_ns);
         }
         if (*w.abort_flag) return false;
-        if (global_ns() - t0 > WAIT_LIMIT_NS) {
+        if (global_ns() - t0 > w.limit_ns) {
             *w.abort_flag = 1u;
             atomicOr(w.status, OBF_DEV_TIMEOUT);
             return false;
