@@ -3,7 +3,10 @@
 //
 // Inputs (from the streaming pass): Gram of the deleted values G_del, Gram of the
 // retained values G_keep (only when k_eff >= d), u = sum_del A_j v_j, the demand
-// sums, and the retained rows themselves (read back from v_out).
+// sums, and the retained rows themselves (read back from v_out).  The tuned streaming
+// pass delivers G and u over ALL rows instead (it runs before the selection is known):
+// P G_all P = P G_del P because P annihilates the retained rows; the retained rows'
+// share of u and of the trace of G is subtracted here, while they are read for the basis.
 //
 //   1. k_eff >= d: k_span_test has factorised G_keep (Cholesky).  If every pivot
 //      stayed above 1e-3 of its diagonal entry the retained values span R^d, the
@@ -97,16 +100,33 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
     if (k >= D && (hflag_in & HFLAG_SPAN_FULL)) { m = D; done = true; pc = 1.f; status |= OBF_DEV_SKIPPED | OBF_DEV_SPAN_FULL; }
 
     // ---- 2. orthonormal basis of span(V_keep), Eq. 2 ------------------------
+    float u_keep[U_LEVELS], sq_keep = 0.f;         // retained rows' share of u (channel tid, per mass level) and of tr G
+#pragma unroll
+    for (int l = 0; l < U_LEVELS; ++l) u_keep[l] = 0.f;
     if (!done) {
         const TIN *vk = reinterpret_cast<const TIN *>(c.v_out) + (size_t)lh * k * D;
+        const float *A = p.scores + c.tok_off + (size_t)lh * T;
+        const int32_t *idx = c.idx_out + (size_t)lh * k;
 #pragma unroll 1
         for (int i = 0; i < k && m < D; ++i) {
-            if (tid < D) vw[tid] = to_f32(vk[(size_t)i * D + tid]);
+            if (tid < D) {
+                const float v = to_f32(vk[(size_t)i * D + tid]);
+                vw[tid] = v;
+                if (p.gram_all) {
+                    const float a = A[idx[i]];
+                    const int lev = u_level(a);
+#pragma unroll
+                    for (int l = 0; l < U_LEVELS; ++l)
+                        if (l == lev) u_keep[l] = fmaf(a, v, u_keep[l]);
+                }
+            }
             __syncthreads();
             // the two norms of a row are taken by every warp for itself (same sum, same order): no block reduction
             float np0 = 0.f;
             for (int cc = (tid & 31); cc < D; cc += 32) np0 = fmaf(vw[cc], vw[cc], np0);
-            const float n0 = sqrtf(warp_sum(np0));
+            const float n0sq = warp_sum(np0);
+            sq_keep += n0sq;
+            const float n0 = sqrtf(n0sq);
             for (int pass = 0; pass < 2; ++pass) {
                 {
                     const int j = tid >> 2, part = tid & 3;
@@ -160,8 +180,18 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
             B2[(e / D) * LD + (e % D)] = s;
         }
         if (tid < D) {
+            // per level: what the pass over V added up minus the retained rows' share; smallest masses first
             float s = 0.f;
-            for (int sp = 0; sp < n_del * p.u_groups; ++sp) s += p.uvec[((size_t)g * S * p.u_groups + sp) * D + tid];
+            for (int l = 0; l < p.u_levels; ++l) {
+                float sl = 0.f;
+                for (int sp = 0; sp < n_del; ++sp) sl += p.uvec[(((size_t)g * S + sp) * p.u_levels + l) * D + tid];
+                if (p.gram_all) {
+#pragma unroll
+                    for (int l2 = 0; l2 < U_LEVELS; ++l2)
+                        if (l2 == l) sl -= u_keep[l2];
+                }
+                s += sl;
+            }
             vu[tid] = s;
         }
         __syncthreads();
@@ -178,7 +208,12 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
             const float sp = block_sum<ALG_NT>(sv * par, red);
             pc = (ss > 0.f && pp > 0.f) ? sp * rsqrtf(ss) * rsqrtf(pp) : 0.f;
         }
-        const float trG = block_sum<ALG_NT>(tid < D ? B2[tid * LD + tid] : 0.f, red);
+        // squared Frobenius norm of the deleted values (the denominator of RCR).  As a difference of two fp32 traces
+        // it is resolved down to about 1e-6 of the squared norm of all values: below 1e-5 of it the deleted values
+        // count as negligible beside the retained ones and nothing is injected.
+        const float trAll = block_sum<ALG_NT>(tid < D ? B2[tid * LD + tid] : 0.f, red);
+        const float trG = trAll - (p.gram_all ? sq_keep : 0.f);
+        const bool del_negligible = p.gram_all && !(trG > 1e-5f * trAll);
         // two D x D x D products, a 4 x 8 register tile per thread (rows a0 + 0..3, columns b0 + 32 * 0..7:
         // the lanes of a warp read consecutive columns, and a row's value is a broadcast)
         auto matmul = [&](const float *X, const float *Y, float *Z) {
@@ -230,7 +265,7 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
         for (int e = tid; e < D * D; e += ALG_NT) B1[(e / D) * LD + (e % D)] = (e / D == e % D) ? 1.f : 0.f;
         __syncthreads();
         const float trM = block_sum<ALG_NT>(tid < D ? B2[tid * LD + tid] : 0.f, red);
-        rcr = trM / (trG + p.eps);
+        rcr = del_negligible ? 0.f : trM / (trG + p.eps);
         if (!(rcr >= RCR_SKIP_TOL)) { done = true; status |= OBF_DEV_SKIPPED; }
 
         // ---- 4f. fast path of App. H: C <- orth(C M), a fixed number of times, from the first rows of the identity ----

@@ -24,7 +24,8 @@ struct CacheDev {
     int32_t nsub_keep;        // tuned path: 128-row tiles of V_keep per head (0 when the span test is not needed)
     int32_t pad_;
     size_t tok_off;           // offset of this cache in the per-token workspace arrays (elements)
-    long long sub_base;       // tuned path: index of this cache's first tile in the call-wide tile sequence
+    long long sub_base;       // tuned path: index of this cache's first tile in the tile sequence of the pass over V
+    long long subk_base;      // tuned path: the same in the tile sequence of the retained rows (span test)
     // tuned score kernel: a head's chunks are worked on by a team of slots, heads are dealt in rounds
     int32_t sc_team;          // chunks (= blocks) per head
     int32_t sc_hpr;           // heads per round
@@ -51,9 +52,12 @@ struct CallDev {
     int32_t rank;
     int32_t splits;           // token splits of the Gram pass (shape-generic path)
     int32_t gram_slots;       // partial Gram matrices stored per head (stride of gram_d / gram_k / uvec)
-    int32_t tc_per;           // tuned path: tiles per block of the Gram pass (0: shape-generic path)
-    int32_t u_groups;         // partial u vectors stored per partial Gram matrix (1, tuned Gram pass: 2)
-    long long tc_total_sub;   // tuned path: tiles in the call-wide tile sequence
+    int32_t tc_per;           // tuned path: tiles per block of the pass over V (0: shape-generic path)
+    int32_t tk_per;           // tuned path: tiles per block of the pass over the retained rows
+    long long tc_total_sub;   // tuned path: tiles in the tile sequence of the pass over V
+    long long tk_total_sub;   // tuned path: tiles in the tile sequence of the retained rows
+    int32_t gram_all;         // 1: gram_d and uvec run over all rows of V (tuned path), 0: over the deleted rows only
+    int32_t u_levels;         // partial u vectors per partial Gram matrix: U_LEVELS with gram_all, else 1
     int32_t sc_nq;            // tuned score kernel: query rows of its tiles (0: shape-generic score kernels)
     int32_t sc_subs;          // 128-key tiles per chunk
     int32_t sc_rounds;        // rounds of the persistent score kernel
@@ -76,9 +80,9 @@ struct CallDev {
     uint8_t *keep;            // [sum heads*T] 1 = retained
     float *stats;             // [heads_total, n_q, 2] softmax row max (log2 domain) and normaliser
     float *sums;              // [heads_total, 4] a_keep, a_del, kth, next
-    float *gram_d;            // [heads_total, gram_slots, d, d] partial Gram of deleted values
+    float *gram_d;            // [heads_total, gram_slots, d, d] partial Gram of the deleted (gram_all: of all) values
     float *gram_k;            // [heads_total, gram_slots, d, d] partial Gram of retained values
-    float *uvec;              // [heads_total, gram_slots, u_groups, d] partial sum_j A_j v_j over deleted j
+    float *uvec;              // [heads_total, gram_slots, u_levels, d] partial sum_j A_j v_j over the same rows as gram_d, per mass level
     float *delta;             // [heads_total, d]
     float *svec;              // [heads_total, d] sum of the deleted value rows (only filled when diagnostics are asked for)
     uint32_t *hflag;          // [heads_total] bit0: delta != 0 -> inject
@@ -94,17 +98,28 @@ __device__ __forceinline__ void locate(const CallDev &p, int g, int &ci, int &lh
 }
 
 // How many partial Gram matrices the streaming pass left for one head.
-// kind 0: deleted values (and the u vector), kind 1: retained values.
-// Shape-generic path: one per token split.  Tuned path: the call-wide tile
-// sequence is cut into runs of tc_per tiles, one run per block; a head's tiles
-// of one kind land in consecutive blocks, each of which stores one partial.
+// kind 0: the pass over V (and the u vector), kind 1: retained values.
+// Shape-generic path: one per token split.  Tuned path: the tile sequence of a
+// pass is cut into runs of `per` tiles, one run per block; a head's tiles
+// land in consecutive blocks, each of which stores one partial.
 __device__ __forceinline__ int gram_partial_count(const CallDev &p, const CacheDev &c, int lh, int kind)
 {
     if (p.tc_per == 0) return p.splits;
     const long long len = kind ? c.nsub_keep : c.nsub_del;
     if (len == 0) return 0;
-    const long long start = c.sub_base + (long long)lh * (c.nsub_del + c.nsub_keep) + (kind ? c.nsub_del : 0);
-    return (int)((start + len - 1) / p.tc_per - start / p.tc_per) + 1;
+    const long long per = kind ? p.tk_per : p.tc_per;
+    const long long start = (kind ? c.subk_base : c.sub_base) + (long long)lh * len;
+    return (int)((start + len - 1) / per - start / per) + 1;
+}
+
+// The sum u = sum_j A_j v_j over ALL rows is kept apart by the magnitude of the mass, one partial sum per level
+// (factors of 64 between the levels): the retained rows, whose masses are the largest, are subtracted from it
+// afterwards, and a few large terms must not cost the many small ones their low bits.
+constexpr int U_LEVELS = 5;
+__device__ __forceinline__ int u_level(float a)
+{
+    const int e = (int)((__float_as_uint(a) >> 23) & 0xFFu);       // biased exponent; masses are not negative
+    return e >= 127 ? 4 : e >= 121 ? 3 : e >= 115 ? 2 : e >= 109 ? 1 : 0;
 }
 
 __device__ __forceinline__ float to_f32(float x) { return x; }

@@ -236,7 +236,6 @@ __global__ void __launch_bounds__(SEL_NT) k_select(const __grid_constant__ CallD
         const bool kp = gt || (eq && eq_before < want);
         if (valid) {
             keep[j] = kp ? 1 : 0;
-            if (kp) p.scores[c.tok_off + (size_t)lh * T + j] = -1.0f;   // later passes need the mass of deleted tokens only
             if (kp) {
                 const uint32_t pos = gt_before + min(eq_before, want);
                 if (pos < (uint32_t)k) idx[pos] = j;
@@ -411,7 +410,6 @@ __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ Call
             const float a = j < p.n_sink ? __uint_as_float(A[j]) : key_score(u);     // a protected position's key is not its mass
             keep[j] = kp ? 1 : 0;
             if (kp) {
-                Af[j] = -1.0f;             // later passes need the mass of deleted tokens only
                 const uint32_t pos = gt_before + min(eq_before, want);
                 if (pos < (uint32_t)k) idx[pos] = j;
                 else atomicOr(p.status, OBF_DEV_INTERNAL);
@@ -438,7 +436,6 @@ __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ Call
                 const bool kp = pos != 0xFFFFFFFFu;
                 keep_h[j] = kp ? 1 : 0;
                 if (kp) {
-                    Ah[j] = -1.0f;             // later passes need the mass of deleted tokens only
                     idx_h[pos] = j;
                     sk += a;
                 } else {

@@ -1,26 +1,33 @@
 // Tuned streaming pass of Orthogonal BackFill for bf16 caches with head_dim 128:
-// one pass over V on the tensor cores.
+// one pass over V on the tensor cores that needs no selection result.
 //
-// Per (cache, layer, KV head) it produces what the dense algebra needs:
-//   G_del  = sum over deleted j of v_j v_j^T          (R^T R = P G_del P, Eq. 3 in the Gram form of App. H)
-//   u      = sum over deleted j of A_j v_j            (r_bar = P u / (A_del + eps), Eq. 4)
-//   G_keep = sum over retained j of v_j v_j^T         (only when k_eff >= d: decides whether span(V_keep) = R^d, Eq. 2)
+// With Q an orthonormal basis of the retained values' span and P = I - Q Q^T (Eq. 2-3), every
+// retained row satisfies P v = 0.  Sums over the deleted rows may therefore run over ALL rows:
+//   R^T R = P G_del P = P G_all P,          G_all = sum over all j of v_j v_j^T   (Eq. 3, Gram form of App. H)
+//   r_bar = P u_del / (A_del + eps),        u_del = u_all - sum over retained j of A_j v_j,  u_all = sum_j A_j v_j   (Eq. 4)
+// The pass produces G_all and u_all per (cache, layer, KV head) from V and the attention masses alone; the few
+// retained rows are taken out of u (and out of the trace of G) by the dense algebra, which reads them anyway.
+// It can thus run beside the selection and the gather instead of after them.
 //
-// Work decomposition.  Every head owns nsub_del tiles of 128 tokens of V followed by
-// nsub_keep tiles of 128 rows of the compacted V_keep (read back from v_out).  All
-// tiles of the call form one sequence, cut into gridDim.x runs of tc_per tiles; block b
-// streams run b.  A run crosses head and kind boundaries; each maximal stretch of
-// one (head, kind) inside a run is a segment and yields one partial Gram matrix
-// (and one partial u), stored in slot (b - first block touching that head and kind).
+// A second, small launch of the same kernel (kind 1) builds G_keep = sum of v v^T over the first rows of the
+// compacted V_keep, only when k_eff >= d: it decides whether span(V_keep) = R^d (Eq. 2).
 //
-// Block = 18 warps:
-//   warp 0        TMA producer: 128 x 128 bf16 tiles (two 128-byte-swizzled column halves) into a 6-stage ring
-//   warp 1        issues tcgen05.mma: G (+)= tile^T tile, both operands MN-major views of the same tile,
-//                 accumulators (128 lanes x 128 columns fp32) double-buffered in tensor memory
-//   warps 2..13   fix-up, three groups of four warps taking tiles in turn: zero the retained rows of a
-//                 V tile in shared memory and accumulate u on the CUDA cores; the attention mass of the
-//                 group's next tile (-1 marks a retained token) is fetched while the current one is processed
-//   warps 14..17  epilogue: tensor memory -> partial Gram matrix in the workspace
+// Work decomposition.  Every head owns nsub tiles of 128 tokens (kind 0: ceil(T / 128) tiles of V; kind 1: up to
+// GT_KEEP_TILES_MAX tiles of the head's rows in v_out).  All tiles of a launch form one sequence, cut into
+// gridDim.x runs of `per` tiles; block b streams run b.  A run crosses head boundaries; each maximal stretch of
+// one head inside a run is a segment and yields one partial Gram matrix (and one partial u), stored in slot
+// (b - first block touching that head).
+//
+// Block = 10 warps:
+//   warp 0       TMA producer: 128 x 128 bf16 tiles (two 128-byte-swizzled column halves) into a ring
+//   warp 1       issues tcgen05.mma: G (+)= tile^T tile (both operands MN-major views of the same tile) and
+//                u (+)= tile^T a, a = the tile's 128 masses as three bf16 columns (high, middle and low part of the
+//                fp32 mass: their sum is the mass exactly, and bf16 x bf16 products are exact in fp32), so that the
+//                CUDA cores never read a value tile; the three columns exist once per mass level (common.cuh:
+//                u_level), a token filling those of its own level; accumulators double-buffered in tensor memory
+//   warps 2..5   masses: warp w serves ring stage w; it fetches the 128 masses of its next tile early, splits them
+//                and writes the columns into the stage's mass tile (K-major, 128-byte swizzle)
+//   warps 6..9   epilogue: tensor memory -> partial Gram matrix and partial u in the workspace
 #pragma once
 
 #include "tc_common.cuh"
@@ -28,85 +35,71 @@
 namespace obf {
 
 constexpr int GT_KEEP_TILES_MAX = 2;                // retained-row tiles per head that enter G_keep (span test)
-constexpr int GT_STAGES = 6;
+constexpr int GT_STAGES = 4;
 constexpr int GT_TILE = 128;                       // tokens per tile
 constexpr int GT_TILE_BYTES = GT_TILE * 128 * 2;   // 32 KiB
-constexpr int GT_GROUPS = 3;                       // fix-up groups of four warps, taking tiles in turn
-// A ring stage must always be fixed up by the same group: a thread may wait for a barrier phase only if it
-// also waited for the phase before (waiting on a parity assumes the previous phase is over).
-static_assert(GT_STAGES % GT_GROUPS == 0, "every ring stage must belong to one fix-up group");
-constexpr int GT_FIX_THREADS = 128 * GT_GROUPS;
-constexpr int GT_THREADS = 64 + GT_FIX_THREADS + 128;
-constexpr size_t GT_SMEM_BYTES = 1024 + (size_t)GT_STAGES * GT_TILE_BYTES + GT_GROUPS * 8 * 128 * sizeof(float) +
-                                 GT_GROUPS * 2 * 128 * sizeof(float) + 256;
+constexpr int GT_ATILE_BYTES = 2 * 16 * 128;       // mass tile: [2 token halves][16 rows][64 tokens] bf16, row 3 * level + part
+static_assert(3 * U_LEVELS <= 16, "the mass tile has 16 rows");
+constexpr int GT_THREADS = 64 + 128 + 128;
+constexpr size_t GT_SMEM_BYTES = 1024 + (size_t)GT_STAGES * (GT_TILE_BYTES + GT_ATILE_BYTES) + 64;
+constexpr uint32_t GT_TMEM_COLS = 512;             // 2 x 128 (Gram) + 2 x 16 (u), rounded up to a power of two
+constexpr uint32_t GT_TMEM_U = 256;                // first column of the u accumulators
 
 // Walks the segments of one block's run of tiles.
 struct TileRun {
-    long long pos, end;        // current and one-past-last index in the call-wide tile sequence
-    int ci;
-    __device__ __forceinline__ void init(const CallDev &p, int block)
+    long long pos, end;        // current and one-past-last index in the launch-wide tile sequence
+    int ci, kind, per;
+    __device__ __forceinline__ void init(const CallDev &p, int block, int kind_)
     {
-        pos = (long long)block * p.tc_per;
-        end = pos + p.tc_per;
-        if (end > p.tc_total_sub) end = p.tc_total_sub;
+        kind = kind_;
+        per = kind ? p.tk_per : p.tc_per;
+        const long long total = kind ? p.tk_total_sub : p.tc_total_sub;
+        pos = (long long)block * per;
+        end = pos + per;
+        if (end > total) end = total;
         ci = 0;
     }
-    // Next segment: cache, local head, kind (0 deleted / 1 retained), first tile, tile count, partial slot.
-    __device__ __forceinline__ bool next(const CallDev &p, int &cache, int &lh, int &kind, int &sub0, int &nsub, int &slot)
+    __device__ __forceinline__ long long base_of(const CacheDev &c) const { return kind ? c.subk_base : c.sub_base; }
+    // Next segment: cache, local head, first tile, tile count, partial slot.
+    __device__ __forceinline__ bool next(const CallDev &p, int &cache, int &lh, int &sub0, int &nsub, int &slot)
     {
         if (pos >= end) return false;
-        while (ci + 1 < p.n_caches && pos >= p.c[ci + 1].sub_base) ++ci;
+        while (ci + 1 < p.n_caches && pos >= base_of(p.c[ci + 1])) ++ci;
         const CacheDev &c = p.c[ci];
-        const int per_head = c.nsub_del + c.nsub_keep;
-        const long long rel = pos - c.sub_base;
+        const int per_head = kind ? c.nsub_keep : c.nsub_del;
+        const long long rel = pos - base_of(c);
         lh = (int)(rel / per_head);
-        const int o = (int)(rel - (long long)lh * per_head);
-        kind = o >= c.nsub_del ? 1 : 0;
-        sub0 = kind ? o - c.nsub_del : o;
-        const int left_in_seg = (kind ? c.nsub_keep : c.nsub_del) - sub0;
+        sub0 = (int)(rel - (long long)lh * per_head);
+        const int left_in_seg = per_head - sub0;
         const long long left_in_run = end - pos;
         nsub = left_in_seg < left_in_run ? left_in_seg : (int)left_in_run;
         const long long seg_start = pos - sub0;
-        slot = (int)(pos / p.tc_per - seg_start / p.tc_per);
+        slot = (int)(pos / per - seg_start / per);
         cache = ci;
         pos += nsub;
         return true;
     }
 };
 
-// One tile of a run, with what the fix-up warps need to know about its segment.
-struct TileInfo {
-    int cache, lh, kind, sub, slot;
-    bool first, last;          // first / last tile of its segment within this run
-};
+// Byte offset of element (row n, token k) in a mass tile: two halves of 64 tokens, rows of 128 bytes, the 16-byte
+// chunks of a row permuted by the row number (the 128-byte swizzle the tensor core expects of a K-major operand).
+__device__ __forceinline__ uint32_t gt_atile_off(int n, int k)
+{
+    const int h = k >> 6, kl = k & 63;
+    return (uint32_t)(h * 2048 + n * 128 + ((((kl >> 3) ^ (n & 7))) << 4) + (kl & 7) * 2);
+}
 
-struct TileIter {
-    TileRun run;
-    int cache, lh, kind, sub0, nsub, slot, t;
-    __device__ __forceinline__ void init(const CallDev &p, int block) { run.init(p, block); nsub = 0; t = 0; }
-    __device__ __forceinline__ bool next(const CallDev &p, TileInfo &ti)
-    {
-        if (t >= nsub) {
-            if (!run.next(p, cache, lh, kind, sub0, nsub, slot)) return false;
-            t = 0;
-        }
-        ti.cache = cache; ti.lh = lh; ti.kind = kind; ti.sub = sub0 + t; ti.slot = slot;
-        ti.first = t == 0;
-        ti.last = t == nsub - 1;
-        ++t;
-        return true;
-    }
-};
-
-__global__ void __launch_bounds__(GT_THREADS, 1) k_gram_tc(const __grid_constant__ CallDev p, const __grid_constant__ TcMaps tm)
+// kind 0: G_all and u_all from V; kind 1: G_keep from the compacted retained rows.
+// One block per multiprocessor; the launch bound of three only caps the registers at 64 per thread, so that the
+// blocks of the selection and the gather, which run on a side stream at the same time, find registers beside it.
+__global__ void __launch_bounds__(GT_THREADS, 3) k_gram_tc(const __grid_constant__ CallDev p, const __grid_constant__ TcMaps tm,
+                                                            const int kind)
 {
     constexpr int D = 128;
     extern __shared__ uint8_t gt_smem_raw[];
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(gt_smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *tiles = base;                                                // GT_STAGES x 32 KiB, 1024-byte aligned
-    float *u_red = reinterpret_cast<float *>(tiles + GT_STAGES * GT_TILE_BYTES);   // [GT_GROUPS][8][128]
-    // [GT_GROUPS][2][128] per token of a group's current / next tile: attention mass, -1 for a retained token, 0 beyond T
-    float *s_a = u_red + GT_GROUPS * 8 * 128;
+    uint8_t *atiles = tiles + GT_STAGES * GT_TILE_BYTES;                  // GT_STAGES x 4 KiB, 1024-byte aligned
     __shared__ uint64_t bar_full[GT_STAGES], bar_ready[GT_STAGES], bar_empty[GT_STAGES];
     __shared__ uint64_t bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t s_tmem, s_abort;
@@ -118,13 +111,17 @@ __global__ void __launch_bounds__(GT_THREADS, 1) k_gram_tc(const __grid_constant
         s_abort = 0u;
         for (int s = 0; s < GT_STAGES; ++s) {
             tc::mbar_init(&bar_full[s], 1);
-            tc::mbar_init(&bar_ready[s], 4);
+            tc::mbar_init(&bar_ready[s], 1);
             tc::mbar_init(&bar_empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) { tc::mbar_init(&bar_acc_full[b], 1); tc::mbar_init(&bar_acc_empty[b], 4); }
         tc::mbar_init_fence();
     }
-    if (warp == 1) tc::tmem_alloc(&s_tmem, 256);
+    // the last row of every mass tile stays zero for the whole launch (the others are rewritten per tile)
+    for (int i = tid; i < GT_STAGES * GT_ATILE_BYTES / 16; i += GT_THREADS)
+        reinterpret_cast<uint4 *>(atiles)[i] = make_uint4(0u, 0u, 0u, 0u);
+    tc::fence_async_smem();
+    if (warp == 1) tc::tmem_alloc(&s_tmem, GT_TMEM_COLS);
     tc::tc_fence_before();
     __syncthreads();
     tc::tc_fence_after();
@@ -134,10 +131,10 @@ __global__ void __launch_bounds__(GT_THREADS, 1) k_gram_tc(const __grid_constant
         // ---------------- TMA producer ----------------
         if (lane == 0) {
             TileRun run;
-            run.init(p, blockIdx.x);
-            int cache, lh, kind, sub0, nsub, slot;
+            run.init(p, blockIdx.x, kind);
+            int cache, lh, sub0, nsub, slot;
             uint32_t it = 0;
-            while (run.next(p, cache, lh, kind, sub0, nsub, slot)) {
+            while (run.next(p, cache, lh, sub0, nsub, slot)) {
                 const CUtensorMap *map = kind ? &tm.b[cache] : &tm.a[cache];
                 for (int t = 0; t < nsub; ++t, ++it) {
                     const int s = it % GT_STAGES;
@@ -158,144 +155,152 @@ __global__ void __launch_bounds__(GT_THREADS, 1) k_gram_tc(const __grid_constant
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            constexpr uint32_t IDESC = tc::idesc_bf16(128, 128, 1, 1);
+            constexpr uint32_t IDESC_G = tc::idesc_bf16(128, 128, 1, 1);
+            constexpr uint32_t IDESC_U = tc::idesc_bf16(128, 16, 1, 0);
             TileRun run;
-            run.init(p, blockIdx.x);
-            int cache, lh, kind, sub0, nsub, slot;
+            run.init(p, blockIdx.x, kind);
+            int cache, lh, sub0, nsub, slot;
             uint32_t it = 0, seg = 0;
-            while (run.next(p, cache, lh, kind, sub0, nsub, slot)) {
+            bool dead = false;
+            while (!dead && run.next(p, cache, lh, sub0, nsub, slot)) {
                 const uint32_t buf = seg & 1u;
                 if (!tc::mbar_wait(&bar_acc_empty[buf], ((seg >> 1) & 1u) ^ 1u, wc)) break;
                 tc::tc_fence_after();
-                const uint32_t acc = tmem + buf * 128u;
+                const uint32_t acc = tmem + buf * 128u, acc_u = tmem + GT_TMEM_U + buf * 16u;
                 for (int t = 0; t < nsub; ++t, ++it) {
                     const int s = it % GT_STAGES;
-                    if (!tc::mbar_wait(&bar_ready[s], (it / GT_STAGES) & 1u, wc)) break;
+                    const uint32_t ph = (it / GT_STAGES) & 1u;
+                    if (!tc::mbar_wait(&bar_full[s], ph, wc)) { dead = true; break; }
+                    if (kind == 0 && !tc::mbar_wait(&bar_ready[s], ph, wc)) { dead = true; break; }
                     tc::tc_fence_after();
                     const uint32_t tile = tc::smem_u32(tiles + s * GT_TILE_BYTES);
+                    const uint32_t atile = tc::smem_u32(atiles + s * GT_ATILE_BYTES);
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk) {
                         // 16 tokens per instruction: rows kk*16.. of the tile, both 64-column halves
                         const uint64_t dv = tc::smem_desc_sw128(tile + kk * 2048, GT_TILE_BYTES / 2, 1024);
-                        tc::umma_bf16(acc, dv, dv, IDESC, (t > 0 || kk > 0) ? 1u : 0u);
+                        tc::umma_bf16(acc, dv, dv, IDESC_G, (t > 0 || kk > 0) ? 1u : 0u);
+                        if (kind == 0) {
+                            // the same 16 tokens of the mass tile: 32 bytes along its swizzled rows, second half after 4 steps
+                            const uint64_t da = tc::smem_desc_sw128(atile + (kk >> 2) * 2048 + (kk & 3) * 32, 16, 1024);
+                            tc::umma_bf16(acc_u, dv, da, IDESC_U, (t > 0 || kk > 0) ? 1u : 0u);
+                        }
                     }
                     tc::umma_commit(&bar_empty[s]);
                 }
+                if (dead) break;
                 tc::umma_commit(&bar_acc_full[buf]);
                 ++seg;
                 if (s_abort) break;
             }
         }
-    } else if (warp < 2 + GT_FIX_THREADS / 32) {
-        // ---------------- fix-up: zero retained rows, accumulate u ----------------
-        // GT_GROUPS groups of four warps take the tiles of the run in turn, so that several tiles are
-        // fixed up at the same time; each group keeps its own partial u.
-        const int f = tid - 64;
-        const int grp = f >> 7, fl = f & 127;      // group, thread within the group
-        const int cg = fl & 15, rg = fl >> 4;      // 16-byte column group, row group (8 of them)
-        const uint32_t col_off = (uint32_t)(cg >> 3) * (GT_TILE_BYTES / 2);
-        float *u_red_g = u_red + grp * 8 * 128;
-        const int bar_id = 1 + grp;
-        // attention mass of token fl of a tile as k_select left it: -1 marks a retained token
-        auto fetch = [&](const TileInfo &ti) -> float {
-            if (ti.kind != 0) return 0.f;
-            const CacheDev &c = p.c[ti.cache];
-            const int j = ti.sub * GT_TILE + fl;
-            if (j >= c.T) return 0.f;
-            return __ldg(p.scores + c.tok_off + (size_t)ti.lh * c.T + j);
-        };
-        TileIter iter, ahead;
-        iter.init(p, blockIdx.x);
-        ahead.init(p, blockIdx.x);
-        // the group looks at every tile of the run (to see where segments start and end) but fixes up
-        // only tiles with index == grp (mod GT_GROUPS); the masses of its next tile are requested one tile early
-        TileInfo cur, pre;
-        bool has_cur = iter.next(p, cur);
-        // `ahead` stands on the group's next own tile
-        bool has_pre = true;
-        for (int sk = 0; sk <= grp && has_pre; ++sk) has_pre = ahead.next(p, pre);
-        float a_own = has_pre ? fetch(pre) : 0.f;   // mass for the group's next own tile
-        uint32_t it = 0, n_own = 0;
-        float u[8];
-        float *s_ag = s_a + grp * 2 * 128;
-        while (has_cur) {
-            const bool own = (it % GT_GROUPS) == (uint32_t)grp;
-            if (cur.first) {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) u[e] = 0.f;
-            }
-            if (own) {
-                const int s = it % GT_STAGES;
-                float *sa = s_ag + (n_own & 1u) * 128;
-                sa[fl] = a_own;
-                // the group's next own tile: its masses are in flight while this tile is processed
-                for (int sk = 0; sk < GT_GROUPS && has_pre; ++sk) has_pre = ahead.next(p, pre);
-                if (has_pre) a_own = fetch(pre);
-                tc::mbar_wait(&bar_full[s], (it / GT_STAGES) & 1u, wc);
-                tc::named_barrier(bar_id, 128);        // sa is complete
-                if (cur.kind == 0) {
-                    uint8_t *tile = tiles + s * GT_TILE_BYTES + col_off;
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const int r = rg + 8 * i;
-                        const float a = sa[r];
-                        const bool kept = a < 0.f;
-                        const float am = kept ? 0.f : a;
-                        uint4 *ptr = reinterpret_cast<uint4 *>(tile + r * 128 + (((cg & 7) ^ (r & 7)) << 4));
-                        const uint4 raw = *ptr;
-                        if (kept) *ptr = make_uint4(0u, 0u, 0u, 0u);
-                        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            u[2 * e] = fmaf(am, __uint_as_float(w[e] << 16), u[2 * e]);
-                            u[2 * e + 1] = fmaf(am, __uint_as_float(w[e] & 0xFFFF0000u), u[2 * e + 1]);
-                        }
-                    }
-                    tc::fence_async_smem();
+    } else if (warp < 6) {
+        // ---------------- masses: three bf16 columns per level and tile ----------------
+        // Four warps, each on its own: warp w serves the tiles with index w (mod 4), which are also the tiles of ring
+        // stage w, so that four tiles' masses are under way at once (one tile costs a round trip to the stage's
+        // barrier, the stores and a proxy fence: about as long as the tensor cores need for the tile).
+        static_assert(GT_STAGES == 4, "one mass warp per ring stage");
+        if (kind == 0) {
+            const int mw = warp - 2;
+            TileRun run;
+            run.init(p, blockIdx.x, kind);
+            int cache, lh, sub0, nsub, slot;
+            // position of the walk: tile `t` of the current segment, `it` in the run
+            bool have = run.next(p, cache, lh, sub0, nsub, slot);
+            int t = 0;
+            uint32_t it = 0;
+            // moves the walk to this warp's next tile at or after the current position
+            auto seek = [&]() {
+                while (have && (it & 3u) != (uint32_t)mw) {
+                    ++it;
+                    if (++t >= nsub) { have = run.next(p, cache, lh, sub0, nsub, slot); t = 0; }
                 }
+            };
+            // masses of tokens lane, lane + 32, .. of the tile the walk stands on
+            auto fetch = [&](float (&a)[4]) {
+                const CacheDev &c = p.c[cache];
+                const float *A = p.scores + c.tok_off + (size_t)lh * c.T;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int j = (sub0 + t) * GT_TILE + lane + 32 * e;
+                    a[e] = j < c.T ? __ldg(A + j) : 0.f;
+                }
+            };
+            auto step = [&]() {
+                ++it;
+                if (++t >= nsub) { have = run.next(p, cache, lh, sub0, nsub, slot); t = 0; }
+            };
+            seek();
+            float a_next[4] = {0.f, 0.f, 0.f, 0.f};
+            if (have) fetch(a_next);
+            uint8_t *at = atiles + mw * GT_ATILE_BYTES;
+            const __nv_bfloat16 zero = __float2bfloat16_rn(0.f);
+            while (have) {
+                float a[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) a[e] = a_next[e];
+                const uint32_t ph = (it / GT_STAGES) & 1u;
+                // this warp's next tile: its masses are in flight while the current ones are written
+                step();
+                seek();
+                if (have) fetch(a_next);
+                if (!tc::mbar_wait(&bar_empty[mw], ph ^ 1u, wc)) break;   // the stage's last user is done with its mass tile
+#pragma unroll 1
+                for (int e = 0; e < 4; ++e) {
+                    const int k = lane + 32 * e;
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(a[e]);
+                    const float r1 = a[e] - __bfloat162float(hi);
+                    const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+                    const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+                    const int lev = u_level(a[e]);
+#pragma unroll
+                    for (int l = 0; l < U_LEVELS; ++l) {
+                        const bool mine = l == lev;
+                        *reinterpret_cast<__nv_bfloat16 *>(at + gt_atile_off(3 * l, k)) = mine ? hi : zero;
+                        *reinterpret_cast<__nv_bfloat16 *>(at + gt_atile_off(3 * l + 1, k)) = mine ? mid : zero;
+                        *reinterpret_cast<__nv_bfloat16 *>(at + gt_atile_off(3 * l + 2, k)) = mine ? lo : zero;
+                    }
+                }
+                tc::fence_async_smem();
                 __syncwarp();
-                if (lane == 0) tc::mbar_arrive(&bar_ready[s]);
-                ++n_own;
+                if (lane == 0) tc::mbar_arrive(&bar_ready[mw]);
             }
-            if (cur.kind == 0 && cur.last) {
-                // the group's u over its 8 row groups, in a fixed order
-                const int g = p.c[cur.cache].head_base + cur.lh;
-                tc::named_barrier(bar_id, 128);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) u_red_g[rg * 128 + cg * 8 + e] = u[e];
-                tc::named_barrier(bar_id, 128);
-                float sum = 0.f;
-#pragma unroll
-                for (int r = 0; r < 8; ++r) sum += u_red_g[r * 128 + fl];
-                p.uvec[(((size_t)g * p.gram_slots + cur.slot) * GT_GROUPS + grp) * D + fl] = sum;
-            }
-            has_cur = iter.next(p, cur);
-            ++it;
         }
     } else {
-        // ---------------- epilogue: accumulator -> workspace ----------------
+        // ---------------- epilogue: accumulators -> workspace ----------------
         const int q = warp & 3;                    // lane quarter this warp may read
         const int row = q * 32 + lane;
         TileRun run;
-        run.init(p, blockIdx.x);
-        int cache, lh, kind, sub0, nsub, slot;
+        run.init(p, blockIdx.x, kind);
+        int cache, lh, sub0, nsub, slot;
         uint32_t seg = 0;
-        while (run.next(p, cache, lh, kind, sub0, nsub, slot)) {
+        while (run.next(p, cache, lh, sub0, nsub, slot)) {
             const int g = p.c[cache].head_base + lh;
             const uint32_t buf = seg & 1u;
-            tc::mbar_wait(&bar_acc_full[buf], (seg >> 1) & 1u, wc);
+            if (!tc::mbar_wait(&bar_acc_full[buf], (seg >> 1) & 1u, wc)) break;
             tc::tc_fence_after();
+            const uint32_t tl = tmem + ((uint32_t)(q * 32) << 16);
             float *dst = (kind ? p.gram_k : p.gram_d) + ((size_t)g * p.gram_slots + slot) * D * D + (size_t)row * D;
 #pragma unroll 1
             for (int cb = 0; cb < 4; ++cb) {
                 uint32_t r[32];
-                tc::tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + buf * 128u + cb * 32u, r);
+                tc::tmem_ld32(tl + buf * 128u + cb * 32u, r);
                 tc::tmem_ld_wait();
 #pragma unroll
                 for (int e = 0; e < 8; ++e)
                     *reinterpret_cast<float4 *>(dst + cb * 32 + e * 4) =
                         make_float4(__uint_as_float(r[4 * e]), __uint_as_float(r[4 * e + 1]),
                                     __uint_as_float(r[4 * e + 2]), __uint_as_float(r[4 * e + 3]));
+            }
+            if (kind == 0) {
+                // u of value channel `row`, per mass level: three columns add up the products with the three parts of the masses
+                uint32_t r[32];
+                tc::tmem_ld32(tl + GT_TMEM_U + buf * 16u, r);
+                tc::tmem_ld_wait();
+#pragma unroll
+                for (int l = 0; l < U_LEVELS; ++l)
+                    p.uvec[(((size_t)g * p.gram_slots + slot) * U_LEVELS + l) * D + row] =
+                        (__uint_as_float(r[3 * l]) + __uint_as_float(r[3 * l + 1])) + __uint_as_float(r[3 * l + 2]);
             }
             tc::tc_fence_before();
             __syncwarp();
@@ -306,7 +311,7 @@ __global__ void __launch_bounds__(GT_THREADS, 1) k_gram_tc(const __grid_constant
 
     tc::tc_fence_before();
     __syncthreads();
-    if (warp == 1) tc::tmem_dealloc(tmem, 256);
+    if (warp == 1) tc::tmem_dealloc(tmem, GT_TMEM_COLS);
 }
 
 }  // namespace obf

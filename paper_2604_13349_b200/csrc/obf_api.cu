@@ -74,10 +74,11 @@ struct Layout {
     // tuned bf16 / head_dim 128 path
     bool tuned;
     int gram_slots;                 // partial Gram matrices stored per head
-    int tc_per, tc_blocks;          // tiles per block and blocks of the tensor-core Gram pass
-    long long tc_total_sub;
+    int tc_per, tc_blocks;          // tiles per block and blocks of the tensor-core pass over V
+    int tk_per, tk_blocks;          // the same for the pass over the retained rows (span test)
+    long long tc_total_sub, tk_total_sub;
     int nsub_del[OBF_MAX_CACHES], nsub_keep[OBF_MAX_CACHES];
-    long long sub_base[OBF_MAX_CACHES];
+    long long sub_base[OBF_MAX_CACHES], subk_base[OBF_MAX_CACHES];
     // tensor-core score kernel
     bool sc_on;
     int sc_nq, sc_subs, sc_blocks, sc_rounds, sc_qt;
@@ -168,8 +169,9 @@ static void make_layout(const obf_params_t *p, const obf_cache_t *caches, int32_
     L.tuned = tuned_path_applies(p, caches, n);
     L.gram_slots = L.splits;
     L.tc_per = 0; L.tc_blocks = 0; L.tc_total_sub = 0;
+    L.tk_per = 0; L.tk_blocks = 0; L.tk_total_sub = 0;
     if (L.tuned && rank > 0) {
-        long long total = 0;
+        long long total = 0, total_k = 0;
         for (int i = 0; i < n; ++i) {
             const int T = caches[i].T, ke = k_eff_of(p, caches[i]);
             L.nsub_del[i] = (T + GT_TILE - 1) / GT_TILE;
@@ -179,17 +181,25 @@ static void make_layout(const obf_params_t *p, const obf_cache_t *caches, int32_
             L.nsub_keep[i] = (ke >= d && T > ke) ? (ke + GT_TILE - 1) / GT_TILE : 0;
             if (L.nsub_keep[i] > GT_KEEP_TILES_MAX) L.nsub_keep[i] = GT_KEEP_TILES_MAX;
             L.sub_base[i] = total;
-            total += (long long)hpc * (L.nsub_del[i] + L.nsub_keep[i]);
+            L.subk_base[i] = total_k;
+            total += (long long)hpc * L.nsub_del[i];
+            total_k += (long long)hpc * L.nsub_keep[i];
         }
         const long long sms = sm_count();
-        const long long blocks = total < sms ? total : sms;
+        auto cut = [&](long long tot, int &per, int &blocks) {
+            if (tot == 0) { per = 0; blocks = 0; return; }
+            const long long want = tot < sms ? tot : sms;
+            per = (int)((tot + want - 1) / want);
+            blocks = (int)((tot + per - 1) / per);
+        };
         L.tc_total_sub = total;
-        L.tc_per = (int)((total + blocks - 1) / blocks);
-        L.tc_blocks = (int)((total + L.tc_per - 1) / L.tc_per);
+        L.tk_total_sub = total_k;
+        cut(total, L.tc_per, L.tc_blocks);
+        cut(total_k, L.tk_per, L.tk_blocks);
         int slots = 1;
         for (int i = 0; i < n; ++i) {
             const int a = (L.nsub_del[i] + L.tc_per - 1) / L.tc_per + 1;
-            const int b = L.nsub_keep[i] ? (L.nsub_keep[i] + L.tc_per - 1) / L.tc_per + 1 : 0;
+            const int b = L.nsub_keep[i] ? (L.nsub_keep[i] + L.tk_per - 1) / L.tk_per + 1 : 0;
             if (a > slots) slots = a;
             if (b > slots) slots = b;
         }
@@ -252,7 +262,7 @@ static void make_layout(const obf_params_t *p, const obf_cache_t *caches, int32_
         const size_t gsz = (size_t)L.heads_total * L.gram_slots * d * d * sizeof(float);
         L.off_gram_d = o; o = align_up(o + gsz, 256);
         L.off_gram_k = o; o = align_up(o + gsz, 256);
-        L.off_uvec = o;   o = align_up(o + (size_t)L.heads_total * L.gram_slots * GT_GROUPS * d * sizeof(float), 256);
+        L.off_uvec = o;   o = align_up(o + (size_t)L.heads_total * L.gram_slots * (L.tc_per ? U_LEVELS : 1) * d * sizeof(float), 256);
         L.off_delta = o;  o = align_up(o + (size_t)L.heads_total * d * sizeof(float), 256);
         L.off_hflag = o;  o = align_up(o + (size_t)L.heads_total * sizeof(uint32_t), 256);
         L.off_svec = o;   o = align_up(o + (size_t)L.heads_total * d * sizeof(float), 256);
@@ -275,6 +285,7 @@ template <typename K>
 static obf_status_t set_smem(K kernel, size_t bytes)
 {
     OBF_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+    OBF_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared));
     return OBF_OK;
 }
 
@@ -318,21 +329,27 @@ static obf_status_t encode_rows_map(CUtensorMap *m, const void *ptr, uint64_t ro
     return OBF_OK;
 }
 
-// Streaming pass of OBF on the tensor cores (bf16, head_dim 128).
-static obf_status_t launch_gram_tc(const CallDev &cd, const Layout &L, cudaStream_t st)
+// Streaming passes of OBF on the tensor cores (bf16, head_dim 128).  kind 0: Gram matrix and mass-weighted sum
+// over all rows of V (needs the masses, not the selection); kind 1: Gram matrix of the first retained rows (needs
+// the gathered values).
+static obf_status_t launch_gram_tc(const CallDev &cd, const Layout &L, cudaStream_t st, int kind)
 {
-    static thread_local TcMaps maps;
+    static thread_local TcMaps maps[2];
+    TcMaps &m = maps[kind];
+    const int blocks = kind ? L.tk_blocks : L.tc_blocks;
+    if (blocks == 0) return OBF_OK;
     const uint64_t hpc = (uint64_t)cd.heads_per_cache;
     for (int i = 0; i < cd.n_caches; ++i) {
-        obf_status_t s = encode_rows_map(&maps.a[i], cd.c[i].v, (uint64_t)cd.c[i].T, hpc);
+        obf_status_t s = OBF_OK;
+        if (kind == 0) s = encode_rows_map(&m.a[i], cd.c[i].v, (uint64_t)cd.c[i].T, hpc);
+        else if (L.nsub_keep[i]) s = encode_rows_map(&m.b[i], cd.c[i].v_out, (uint64_t)cd.c[i].k_eff, hpc);
         if (s != OBF_OK) return s;
-        if (L.nsub_keep[i]) {
-            if ((s = encode_rows_map(&maps.b[i], cd.c[i].v_out, (uint64_t)cd.c[i].k_eff, hpc)) != OBF_OK) return s;
-        }
     }
     OBF_CUDA_TRY(cudaFuncSetAttribute(k_gram_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GT_SMEM_BYTES));
-    k_gram_tc<<<L.tc_blocks, GT_THREADS, GT_SMEM_BYTES, st>>>(cd, maps);
-    mark(st, "k_gram_tc");
+    // the whole shared-memory capacity, so that the side stream's blocks find room beside this kernel's
+    OBF_CUDA_TRY(cudaFuncSetAttribute(k_gram_tc, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared));
+    k_gram_tc<<<blocks, GT_THREADS, GT_SMEM_BYTES, st>>>(cd, m, kind);
+    mark(st, kind ? "k_gram_tc_keep" : "k_gram_tc");
     return OBF_OK;
 }
 
@@ -383,20 +400,31 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
         k_score_pool<TIN, D><<<g2, SC_NT, sm_sc, st>>>(cd);
         mark(st, "k_score_pool");
     }
+    // The tuned pass over V needs the masses but not the selection (it sums over all rows, gram_tc.cuh): it runs
+    // on the caller's stream while selection and gather run on a side stream of the library.  (Not while
+    // profiling per launch, where every kernel is timed alone.)
+    const bool tuned_obf = cd.rank > 0 && L.tc_per > 0;
+    SideStream *side = (tuned_obf && !g_prof.active) ? side_stream() : nullptr;
+    cudaStream_t sel = side ? side->stream : st;       // stream of selection and gather
+    if (side) {
+        OBF_CUDA_TRY(cudaEventRecord(side->fork, st));
+        OBF_CUDA_TRY(cudaStreamWaitEvent(side->stream, side->fork, 0));
+        if ((s = launch_gram_tc(cd, L, st, 0)) != OBF_OK) return s;
+    }
     if (cd.layerwise) {
         // masses of a layer's KV heads added up, then every head's block selects on its layer's sums
         const int n_layers = heads / cd.kv_heads;
         const size_t sm_sel = (size_t)T_max * sizeof(uint32_t);
         dim3 gl((T_max + 255) / 256, n_layers);
-        k_layer_sum<<<gl, 256, 0, st>>>(cd);
-        mark(st, "k_layer_sum");
+        k_layer_sum<<<gl, 256, 0, sel>>>(cd);
+        mark(sel, "k_layer_sum");
         const int sms = sm_count();
         if (heads > 2 * sms && heads <= 4 * sms) {
             if ((s = set_smem(k_select_smem<512, true>, sm_sel)) != OBF_OK) return s;
-            k_select_smem<512, true><<<heads, 512, sm_sel, st>>>(cd);
+            k_select_smem<512, true><<<heads, 512, sm_sel, sel>>>(cd);
         } else {
             if ((s = set_smem(k_select_smem<1024, true>, sm_sel)) != OBF_OK) return s;
-            k_select_smem<1024, true><<<heads, 1024, sm_sel, st>>>(cd);
+            k_select_smem<1024, true><<<heads, 1024, sm_sel, sel>>>(cd);
         }
     } else if (T_max <= SEL_SMEM_MAX_T) {
         const size_t sm_sel = (size_t)T_max * sizeof(uint32_t);
@@ -405,38 +433,28 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
         const int sms = sm_count();
         if (heads > 2 * sms && heads <= 4 * sms) {
             if ((s = set_smem(k_select_smem<512>, sm_sel)) != OBF_OK) return s;
-            k_select_smem<512><<<heads, 512, sm_sel, st>>>(cd);
+            k_select_smem<512><<<heads, 512, sm_sel, sel>>>(cd);
         } else {
             if ((s = set_smem(k_select_smem<1024>, sm_sel)) != OBF_OK) return s;
-            k_select_smem<1024><<<heads, 1024, sm_sel, st>>>(cd);
+            k_select_smem<1024><<<heads, 1024, sm_sel, sel>>>(cd);
         }
     } else {
-        k_select<<<heads, SEL_NT, 0, st>>>(cd);
+        k_select<<<heads, SEL_NT, 0, sel>>>(cd);
     }
-    mark(st, "k_select");
+    mark(sel, "k_select");
     dim3 g4((k_max + GATHER_ROWS - 1) / GATHER_ROWS, heads);
-    // With OBF to follow, only the values are needed by the later kernels: the keys are copied on a side stream
-    // beside the span test and the dense algebra, which leave the memory system idle.  (Not while profiling per
-    // launch, where every kernel is timed alone.)
-    SideStream *side = (cd.rank > 0 && !g_prof.active) ? side_stream() : nullptr;
+    k_gather<D * (int)sizeof(TIN)><<<g4, 256, 0, sel>>>(cd);
+    mark(sel, "k_gather");
     if (side) {
-        k_gather<D * (int)sizeof(TIN), 1><<<g4, 256, 0, st>>>(cd);
-        mark(st, "k_gather");
-    } else {
-        k_gather<D * (int)sizeof(TIN)><<<g4, 256, 0, st>>>(cd);
-        mark(st, "k_gather");
+        OBF_CUDA_TRY(cudaEventRecord(side->join, side->stream));
+        OBF_CUDA_TRY(cudaStreamWaitEvent(st, side->join, 0));
     }
     if (cd.rank > 0) {
         const size_t sm_alg = algebra_smem_bytes<D>();
         if ((s = set_smem(k_obf_algebra<TIN, D>, sm_alg)) != OBF_OK) return s;
-        if constexpr (sizeof(TIN) == 2 && D == 128) {
-            if (L.tuned) {
-                if ((s = launch_gram_tc(cd, L, st)) != OBF_OK) return s;
-            } else {
-                dim3 g5(cd.splits, heads);
-                k_gram<TIN, D><<<g5, 256, 0, st>>>(cd);
-                mark(st, "k_gram");
-            }
+        if (tuned_obf) {
+            if (!side && (s = launch_gram_tc(cd, L, st, 0)) != OBF_OK) return s;
+            if ((s = launch_gram_tc(cd, L, st, 1)) != OBF_OK) return s;
         } else {
             dim3 g5(cd.splits, heads);
             k_gram<TIN, D><<<g5, 256, 0, st>>>(cd);
@@ -453,19 +471,10 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
         }
         const size_t sm_span = span_smem_bytes<D>();
         if ((s = set_smem(k_span_test<D>, sm_span)) != OBF_OK) return s;
-        if (side) {
-            // fork: the key copy starts when the streaming pass is over (it would only share HBM with it)
-            OBF_CUDA_TRY(cudaEventRecord(side->fork, st));
-            OBF_CUDA_TRY(cudaStreamWaitEvent(side->stream, side->fork, 0));
-            k_gather<D * (int)sizeof(TIN), 2><<<g4, 256, 0, side->stream>>>(cd);
-            ++g_last_launches;
-            OBF_CUDA_TRY(cudaEventRecord(side->join, side->stream));
-        }
         k_span_test<D><<<heads, ST_NT, sm_span, st>>>(cd);
         mark(st, "k_span_test");
         k_obf_algebra<TIN, D><<<heads, ALG_NT, sm_alg, st>>>(cd);
         mark(st, "k_obf_algebra");
-        if (side) OBF_CUDA_TRY(cudaStreamWaitEvent(st, side->join, 0));      // join: the call ends when both streams have
     }
     OBF_CUDA_TRY(cudaGetLastError());
     return OBF_OK;
@@ -508,6 +517,7 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
         c.nsub_del = L.tc_per ? L.nsub_del[i] : 0;
         c.nsub_keep = L.tc_per ? L.nsub_keep[i] : 0;
         c.sub_base = L.tc_per ? L.sub_base[i] : 0;
+        c.subk_base = L.tc_per ? L.subk_base[i] : 0;
         c.sc_team = L.sc_on ? L.sc_team[i] : 0;
         c.sc_hpr = L.sc_on ? L.sc_hpr[i] : 0;
         c.sc_round_base = L.sc_on ? L.sc_round_base[i] : 0;
@@ -524,8 +534,11 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
     cd.splits = L.splits;
     cd.gram_slots = L.gram_slots;
     cd.tc_per = L.tc_per;
-    cd.u_groups = L.tc_per ? GT_GROUPS : 1;
+    cd.tk_per = L.tk_per;
+    cd.gram_all = L.tc_per ? 1 : 0;
+    cd.u_levels = L.tc_per ? U_LEVELS : 1;
     cd.tc_total_sub = L.tc_total_sub;
+    cd.tk_total_sub = L.tk_total_sub;
     cd.sc_nq = L.sc_on ? L.sc_nq : 0;
     cd.sc_qt = L.sc_on ? L.sc_qt : 1;
     cd.sc_subs = L.sc_subs;

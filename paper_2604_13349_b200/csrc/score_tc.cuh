@@ -206,8 +206,8 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(st_smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *q_s = base;                                           // 2 x [128 x 128] bf16: Q of a statistics pass, Q of a pooling pass; two 64-column halves each
     uint8_t *ring = q_s + 2 * ST_TILE_BYTES;                       // ST_STAGES x 32 KiB
-    float *s_m = reinterpret_cast<float *>(ring + ST_STAGES * ST_TILE_BYTES);   // [2][groups][128 queries] chunk maxima
-    float *s_z = s_m + 2 * ST_GROUPS * 128;                        // [2][groups][128 queries] chunk sums
+    float *s_m = reinterpret_cast<float *>(ring + ST_STAGES * ST_TILE_BYTES);   // [2][tile of the chunk][128 queries] tile maxima
+    float *s_z = s_m + 2 * ST_GROUPS * 128;                        // [2][tile of the chunk][128 queries] tile sums
     float *s_mp = s_z + 2 * ST_GROUPS * 128;                       // [2][128] M'_t of the head being pooled
     __shared__ uint64_t bar_q_full[2], bar_q_free[2], bar_full[ST_STAGES];
     __shared__ uint64_t bar_t_full[ST_TBUF], bar_t_empty[ST_TBUF];
@@ -397,11 +397,15 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
             ScoreItem item;
             if (i < R && score_item(p, s_tab, i, item)) {
                 const int T = s_tab[item.cache].T, buf = i & 1;
+                // a chunk has at most as many tiles as there are groups: this group meets at most one of them
+                static_assert(ST_GROUPS == ST_TILES, "one tile of a chunk per consumer group");
                 float m = -INFINITY, z = 0.f;
+                int my_t = -1;
 #pragma unroll 1
                 for (int t = 0; t < item.nt; ++t) {
                     const uint32_t ti = it + t;
                     if ((int)(ti % ST_GROUPS) != grp) continue;
+                    my_t = t;
                     const int key0 = item.chunk * ST_CHUNK + t * 128;                     // key of column 0 of the tile
                     walk_tile(ti, [&](int pc, uint32_t (&rr)[32]) {
                         // two copies of the update: the one that masks missing keys runs for a head's ragged last tile only
@@ -411,10 +415,13 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                     });
                 }
                 it += item.nt;
-                // hand (m, z) of this group's tiles to the messenger
+                // hand (m, z) of the tile to the messenger, filed under the tile's place in the chunk: the messenger
+                // merges a chunk's tiles in that order whichever groups worked on them
                 if (n_a[buf] > 0) tc::mbar_wait(&bar_st_free[buf], (n_a[buf] - 1) & 1u, wc, 20);
-                s_m[(buf * ST_GROUPS + grp) * 128 + row] = m;
-                s_z[(buf * ST_GROUPS + grp) * 128 + row] = z;
+                if (my_t >= 0) {
+                    s_m[(buf * ST_TILES + my_t) * 128 + row] = m;
+                    s_z[(buf * ST_TILES + my_t) * 128 + row] = z;
+                }
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(&bar_st_ready[buf]);
                 ++n_a[buf];
@@ -462,13 +469,11 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 const int t = lane + 32 * k;
-                const float *sm = s_m + buf * ST_GROUPS * 128 + t, *sz = s_z + buf * ST_GROUPS * 128 + t;
+                const float *sm = s_m + buf * ST_TILES * 128 + t, *sz = s_z + buf * ST_TILES * 128 + t;
                 float M = sm[0];
-#pragma unroll
-                for (int e = 1; e < ST_GROUPS; ++e) M = fmaxf(M, sm[e * 128]);
+                for (int e = 1; e < item.nt; ++e) M = fmaxf(M, sm[e * 128]);
                 float Z = 0.f;
-#pragma unroll
-                for (int e = 0; e < ST_GROUPS; ++e)
+                for (int e = 0; e < item.nt; ++e)
                     if (sm[e * 128] > -INFINITY) Z += sz[e * 128] * ex2_approx(sm[e * 128] - M);
                 if (t < nq) __stcg(&partials[t], make_float2(M, Z));
             }

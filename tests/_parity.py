@@ -146,7 +146,10 @@ def check_head(dtype: str, K: np.ndarray, V: np.ndarray, Q: np.ndarray, budget: 
         gd = g_delta.astype(np.float64)
         if np.linalg.norm(gd) > 0:
             assert np.abs(Vk @ gd).max() / (np.linalg.norm(Vk, 2) * np.linalg.norm(gd)) <= 1e-4
-            assert np.linalg.norm(gd) <= scale * (1 + 1e-3)
+            # The tuned path sums A_j v_j over all rows and takes the retained rows out afterwards, which leaves
+            # delta an absolute error of a few fp32 ulps of the largest retained value (measured: 1.1e-8 of its
+            # norm); it shows only where A_del / A_keep is so small that delta itself is of that size.
+            assert np.linalg.norm(gd) <= scale * (1 + 1e-3) + 2.0 ** -22 * np.linalg.norm(Vk, axis=1).max()
     if g_diag is not None and "revr" in dg:
         # kept share of the residual's squared singular values: a ratio of well-conditioned eigenvalue sums
         assert abs(g_diag["revr"] - dg["revr"]) <= 1e-4, "%s: REVR %.6f vs %.6f" % (name, g_diag["revr"], dg["revr"])

@@ -330,9 +330,10 @@ def test_host_entry_point_pipelines_slabs_of_layers_for_ragged_batches(layers):
         assert torch.equal(h["oK"].view(torch.int16), outs[ci]["K_out"].cpu().view(torch.int16))
         assert torch.allclose(h["oV"].float(), outs[ci]["V_out"].cpu().float(), rtol=1e-2, atol=1e-5)
         assert torch.equal(h["oS"], outs[ci]["scores"].cpu())
-        # the streaming pass cuts its tile sequence by the size of the call, so a slab adds its partial Gram
-        # matrices up in another order than the whole call: delta agrees to fp32 rounding, not bit for bit
-        assert torch.allclose(h["oD"], outs[ci]["delta"].cpu(), rtol=1e-4, atol=1e-6)
+        # the streaming pass cuts its tile sequence by the size of the call, so a slab adds its partial sums
+        # up in another order than the whole call: delta agrees to fp32 rounding of the largest terms of those
+        # sums (2^-22 of a value row's norm, about 15 here), not bit for bit
+        assert torch.allclose(h["oD"], outs[ci]["delta"].cpu(), rtol=1e-4, atol=4e-6)
 
 
 # ---------------------------------------------------------------------------
