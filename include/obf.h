@@ -93,6 +93,14 @@ typedef enum { OBF_F32 = 0, OBF_BF16 = 1 } obf_dtype_t;
                                       candidates of the selection, so k_eff = min(n, T) + min(budget, T - min(n, T));
                                       size the outputs with that k_eff                                            */
 #define OBF_FLAG_SINK_OF(flags) (((flags) >> 8) & 0xFFu)
+#define OBF_FLAG_TEST_WAIT_EXPIRES 0x10000u
+                                   /* test hook for the bounded device-side waits of the tuned score kernel: no block
+                                      publishes a head's softmax normalisers and the wait limit drops from one second to
+                                      20 ms, so every wait for them runs out, the kernels return by themselves, the
+                                      status word carries OBF_DEV_TIMEOUT and the outputs hold valid positions but no
+                                      meaningful selection.  Accepted only for at most 4 (layer, KV head) pairs in all,
+                                      every T <= 2048, on the tuned bf16 / head_dim 128 path; else
+                                      OBF_ERR_INVALID_ARG                                                         */
 
 #define OBF_MAX_CACHES 32          /* caches per call                                              */
 #define OBF_MAX_T (1 << 20)        /* prompt positions per cache                                   */
@@ -150,9 +158,20 @@ obf_status_t obf_workspace_bytes(const obf_params_t *params, const obf_cache_t *
  * are host structs (copied before return); `workspace` is device memory of at
  * least obf_workspace_bytes(), 256-byte aligned, private to this call until
  * the enqueued work completes; `stream` is a cudaStream_t passed as void*.
- * With rank > 0 the copy of the retained keys runs on a stream of the library
- * (created on first use per host thread and device) that forks from and joins
- * `stream` inside the call: everything the call does is ordered on `stream`.
+ * With rank > 0 on the tuned path the selection and the gather run on a stream
+ * of the library (created on first use per host thread and device) that forks
+ * from and joins `stream` inside the call, beside the pass over V: everything
+ * the call does is ordered on `stream`.
+ *
+ * Calls that overlap on one device (different streams or host threads, each
+ * with its own workspace) are legal but do not speed each other up: the tuned
+ * score kernel's blocks wait for one another, so it is launched cooperatively
+ * and starts only when the whole grid (one block per multiprocessor) can be
+ * resident; until then it waits for whatever else holds the multiprocessors.
+ * Every device-side wait is bounded (one second): if one ever runs out the
+ * kernels return by themselves, the status word carries OBF_DEV_TIMEOUT (see
+ * obf_last_device_status) and the outputs hold valid positions but no
+ * meaningful selection.
  */
 obf_status_t obf_compress(const obf_params_t *params, const obf_cache_t *caches, int32_t n_caches,
                           void *workspace, size_t workspace_bytes, void *stream);
@@ -232,7 +251,8 @@ const char *obf_phase_name(int32_t phase);
  * - Calls no cudaMalloc, cudaFree or any other allocating routine.
  * - The first call on each device resolves the array's device address
  *   (cudaGetSymbolAddress, with that device current); make that first call
- *   before starting any stream capture on the device.
+ *   before starting any stream capture on the device.  Host threads may make
+ *   their first calls at the same time (the address is kept in an atomic).
  * - All calls on one device share the one array and it keeps whatever the
  *   previous call left; the call clears the part that has to start at zero
  *   (the status word) and overwrites the rest before reading it.  Two calls

@@ -35,6 +35,7 @@ OBF_DEV_SPAN_FULL = 0x200
 OBF_FLAG_GENERIC_PATH = 0x1
 OBF_FLAG_LAYERWISE = 0x2        # one retained set per layer (masses summed over its KV heads)
 OBF_FLAG_FAST_PATH = 0x4        # three Gram subspace iterations instead of the exact eigenvectors
+OBF_FLAG_TEST_WAIT_EXPIRES = 0x10000   # test hook: the score kernel's wait for a head's normalisers runs out
 
 
 def OBF_FLAG_SINK(n: int) -> int:

@@ -1,5 +1,6 @@
 // Host side of the C ABI declared in include/obf.h: argument validation,
 // workspace layout, kernel dispatch.  Allocates no device memory.
+#include <atomic>
 #include <cstdio>
 #include <cstring>
 
@@ -500,6 +501,12 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
     make_layout(p, caches, n, rank, L);
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < L.total)
         return OBF_ERR_WORKSPACE;
+    if (p->flags & OBF_FLAG_TEST_WAIT_EXPIRES) {
+        // the test hook is for tiny calls on the tuned score kernel only
+        if (!L.sc_on || L.heads_total > 4) return OBF_ERR_INVALID_ARG;
+        for (int i = 0; i < n; ++i)
+            if (caches[i].T > 2048) return OBF_ERR_INVALID_ARG;
+    }
 
     CallDev cd;
     std::memset(&cd, 0, sizeof(cd));
@@ -558,6 +565,10 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
     cd.fast_iters = (p->flags & OBF_FLAG_FAST_PATH) ? 3 : 0;
     cd.wait_limit_ns = tc::WAIT_LIMIT_NS;
     cd.debug_drop_publish = 0;
+    if (p->flags & OBF_FLAG_TEST_WAIT_EXPIRES) {
+        cd.wait_limit_ns = 20000000ull;
+        cd.debug_drop_publish = 1;
+    }
     cd.sc_part = reinterpret_cast<float *>(ws + L.off_sc_part);
     cd.sc_head = reinterpret_cast<float *>(ws + L.off_sc_head);
     cd.sc_cnt = reinterpret_cast<uint32_t *>(ws + L.off_sc_sync);
@@ -842,23 +853,23 @@ namespace {
 static __device__ __align__(256) unsigned char g_static_scratch[OBF_STATIC_SCRATCH_BYTES];
 
 constexpr int kMaxDevices = 64;
-void *g_static_scratch_addr[kMaxDevices];       // device address of the array, per device ordinal
-bool g_static_scratch_ready[kMaxDevices];
+// Device address of the array, per device ordinal; null until resolved.  Host threads that make their first call
+// on a device at the same time may each resolve it: they store the same value, and the atomic makes that well defined.
+std::atomic<void *> g_static_scratch_addr[kMaxDevices];
 
-// Device address of the scratch array on the current device; resolved once per device.
+// Device address of the scratch array on the current device; resolved on the first call per device.
 obf_status_t static_scratch_ptr(void **out)
 {
     int dev = -1;
     OBF_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices) return OBF_ERR_UNSUPPORTED;
-    if (!g_static_scratch_ready[dev]) {
-        void *ptr = nullptr;
+    void *ptr = g_static_scratch_addr[dev].load(std::memory_order_acquire);
+    if (!ptr) {
         OBF_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
         if (!ptr) return OBF_ERR_CUDA;
-        g_static_scratch_addr[dev] = ptr;
-        g_static_scratch_ready[dev] = true;
+        g_static_scratch_addr[dev].store(ptr, std::memory_order_release);
     }
-    *out = g_static_scratch_addr[dev];
+    *out = ptr;
     return OBF_OK;
 }
 

@@ -207,6 +207,51 @@ def test_tuned_path_rank_deficient_values_with_budget_above_head_dim():
     assert torch.all(outs[0]["delta"].norm(dim=-1) > 1e-6)
 
 
+def _subspace_case(full_later: bool):
+    """T = 2000, budget 400 >= head_dim.  Positions below 1500 hold values confined to the first 100 channels, so
+    the first 256 retained rows (the subset the span test factorises) have rank 100.  full_later: the values at
+    positions >= 1500 fill all 128 channels, else they are confined too and only a few unselectable tokens carry
+    the other channels."""
+    w = small("subspace", d=128, dtype="bf16", rank=3, caches=((2000, 400),), heavy=0, kv_heads=2, seed=29)
+    arrays = [synth.gen_cache(w, 0)]
+    a = arrays[0]
+    K = par.f32_view(a["K"], "bf16").copy(); V = par.f32_view(a["V"], "bf16").copy()
+    Qv = par.f32_view(a["Q"], "bf16").reshape(1, 2, w.n_q, 128)
+    g = np.random.default_rng(8)
+    V[:, :, :1500, 100:] = 0.0
+    if not full_later:
+        V[:, :, 1500:, 100:] = 0.0
+        for h in range(2):
+            qm = Qv[0, h].mean(axis=0)
+            odd = g.choice(2000, 60, replace=False)
+            K[0, h, odd] = -1.5 * qm / np.linalg.norm(qm) * np.linalg.norm(K[0, h, odd], axis=1, keepdims=True)
+            V[0, h, odd, 100:] = g.standard_normal((60, 28)).astype(np.float32)
+    a["K"], a["V"] = synth.to_bf16_bits(K), synth.to_bf16_bits(V)
+    outs, reps, _ = run_and_check(w, arrays=arrays)
+    idx = outs[0]["idx"].cpu().numpy()
+    for h in range(2):
+        assert (idx[0, h] < 1500).sum() >= 256 and (idx[0, h] >= 1500).sum() >= 40    # the construction holds
+    return outs, reps
+
+
+def test_span_subset_deficient_but_all_retained_rows_span_everything():
+    # the Cholesky test on the first 256 retained rows fails; Gram-Schmidt over all 400 must reach rank 128: delta = 0
+    outs, reps = _subspace_case(full_later=True)
+    diags = P.parse_diag(outs[0]["diag"])
+    assert all(dg["span_rank"] == 128 for dg in diags)
+    assert all(r.oracle_skipped for r in reps)               # run_and_check has compared V_out bit for bit
+    assert torch.all(outs[0]["delta"] == 0)
+
+
+def test_span_subset_deficient_and_all_retained_rows_deficient_too():
+    outs, reps = _subspace_case(full_later=False)
+    diags = P.parse_diag(outs[0]["diag"])
+    assert all(dg["span_rank"] == 100 for dg in diags)
+    assert all(not r.oracle_skipped for r in reps)
+    assert torch.all(outs[0]["delta"][..., :100].abs() < 1e-4)
+    assert torch.all(outs[0]["delta"].norm(dim=-1) > 1e-6)
+
+
 @pytest.mark.parametrize("T,budget", [(20000, 300), (70000, 250), (80000, 200)])
 def test_long_prompts_take_the_fallback_kernels(T, budget):
     # 20000 keys: more than the select kernel keeps in shared memory; 70000 keys: one head's team is 137 blocks,
@@ -282,6 +327,28 @@ def test_non_finite_inputs_set_the_status_word_and_stay_in_bounds():
     assert len(set(idx.tolist())) == 10 and idx.min() >= 0 and idx.max() < 120
 
 
+def test_a_device_side_wait_that_runs_out_reports_a_timeout_and_the_kernels_return():
+    # nothing publishes the head's softmax normalisers and the wait limit is 20 ms: the score kernel's wait runs out
+    w = small("expire", layers=1, kv_heads=2, G=2, n_obs=8, d=128, dtype="bf16", rank=2, caches=((700, 40),), seed=13)
+    arrays = [synth.gen_cache(w, 0)]
+    outs, dev, st = par.run_gpu(w, arrays, flags=P.binding.OBF_FLAG_TEST_WAIT_EXPIRES)
+    assert st & P.binding.OBF_DEV_TIMEOUT
+    idx = outs[0]["idx"].cpu().numpy()
+    assert idx.min() >= 0 and idx.max() < 700               # whatever was selected lies inside the cache
+    assert np.all(np.diff(idx, axis=-1) > 0)
+    # the workspace, the streams and the device are as usable as before
+    ws = outs[0]["workspace"]
+    good = P.compress_caches(par.params_for(w), dev, want_scores=True, workspace=ws)
+    torch.cuda.synchronize()
+    assert P.obf_last_device_status(ws) & 0xFF == 0
+    reps = par.check_cache(w, 0, arrays[0], good[0], all_heads(w))
+    assert all(not r.oracle_skipped for r in reps)
+    # the hook is refused outside its small shapes
+    big = small("expire_big", layers=3, kv_heads=2, G=2, n_obs=8, d=128, dtype="bf16", caches=((700, 40),))
+    with pytest.raises(Exception):
+        par.run_gpu(big, [synth.gen_cache(big, 0)], flags=P.binding.OBF_FLAG_TEST_WAIT_EXPIRES)
+
+
 def test_host_entry_point_matches_the_device_entry_point():
     w = synth.workload("c1")
     arrays = [synth.gen_cache(w, 0)]
@@ -337,45 +404,62 @@ def test_host_entry_point_pipelines_slabs_of_layers_for_ragged_batches(layers):
 
 
 # ---------------------------------------------------------------------------
-# benchmark configurations at full size, in the benchmark's launch configuration,
-# checked on sampled heads that the oracle computes one by one
+# benchmark configurations at full size: every head of every cache against one oracle run per cache, and the
+# call shape the benchmark times (no optional outputs) bit for bit against the call with all outputs
 # ---------------------------------------------------------------------------
 @pytest.fixture(scope="module")
 def c4_arrays():
     return [synth.gen_cache(synth.workload("c4"), 0)]
 
 
-def test_c3_full_size_sampled_heads():
-    w = synth.workload("c3")
-    run_and_check(w, heads=[(0, 0), (17, 3), (35, 7)])
+def run_whole(wname, arrays=None, evict=False, flags=0, layerwise=False):
+    w = synth.workload(wname)
+    arrays = arrays or [synth.gen_cache(w, ci) for ci in range(len(w.caches))]
+    outs, dev, st = par.run_gpu(w, arrays, evict=evict, flags=flags)
+    assert st & 0xFF == 0, "device status %#x" % st
+    # what the benchmark times: the same call without diagnostics, masses and delta
+    bare, _, st2 = par.run_gpu(w, arrays, evict=evict, flags=flags, want_scores=False, dev=dev,
+                               want_delta=False, want_diag=False)
+    assert st2 & 0xFF == 0
+    for x, y in zip(outs, bare):
+        assert torch.equal(x["idx"], y["idx"]), "retained positions depend on the optional outputs"
+        assert torch.equal(x["K_out"].view(torch.int16), y["K_out"].view(torch.int16))
+        assert torch.equal(x["V_out"].view(torch.int16), y["V_out"].view(torch.int16))
+    del bare
+    total = {}
+    for ci in range(len(w.caches)):
+        st_ci = par.check_cache_whole(w, ci, arrays[ci], outs[ci], rank=0 if evict else None, layerwise=layerwise)
+        for k, v in st_ci.items():
+            total[k] = total.get(k, 0) + v
+    print("\n[%s whole] %s" % (wname, total))
+    assert total["heads"] == len(w.caches) * w.layers * w.kv_heads
+    return total
 
 
-def test_c4_full_size_rank4_sampled_heads(c4_arrays):
-    run_and_check(synth.workload("c4"), heads=[(0, 0), (21, 5), (39, 7)], arrays=c4_arrays)
+def test_c3_full_size_every_head():
+    run_whole("c3")
 
 
-def test_c4_full_size_evict_only_sampled_heads(c4_arrays):
-    run_and_check(synth.workload("c4_evict"), evict=True, heads=[(3, 1), (39, 6)], arrays=c4_arrays)
+def test_c4_full_size_rank4_every_head(c4_arrays):
+    run_whole("c4", arrays=c4_arrays)
 
 
-def test_c4_full_size_layerwise_sampled_layers(c4_arrays):
-    w = synth.workload("c4_layer")
-    outs, _, st = par.run_gpu(w, c4_arrays, flags=P.binding.OBF_FLAG_LAYERWISE)
-    assert st & 0xFF == 0
-    reps = par.check_cache_layerwise(w, 0, c4_arrays[0], outs[0], [0, 39])
-    print("\n[c4_layer] %s" % par.summarize(reps))
+def test_c4_full_size_evict_only_every_head(c4_arrays):
+    run_whole("c4_evict", arrays=c4_arrays, evict=True)
 
 
-def test_c5_ragged_relay_batch_sampled_heads():
-    w = synth.workload("c5")
-    run_and_check(w, heads=[(0, 0), (35, 7)])
+def test_c4_full_size_layerwise_every_layer(c4_arrays):
+    run_whole("c4_layer", arrays=c4_arrays, flags=P.binding.OBF_FLAG_LAYERWISE, layerwise=True)
 
 
-def test_paper_regime_budget_32_sampled_heads():
+def test_c5_ragged_relay_batch_every_head_of_every_cache():
+    run_whole("c5")
+
+
+def test_paper_regime_budget_32_every_head():
     # kv_budget = 32 < head_dim with 40 latent steps: OBF's dense algebra runs for every head
-    w = synth.workload("pa")
-    outs, reps, _ = run_and_check(w, heads=[(0, 0), (9, 4), (35, 7)])
-    assert all(not r.oracle_skipped for r in reps)
+    total = run_whole("pa")
+    assert total["backfilled"] == total["heads"]
 
 
 # ---------------------------------------------------------------------------

@@ -6,7 +6,8 @@ afford an allocation's device-wide synchronisation) pass only inputs and
 outputs; the scratch is a fixed array inside the library.  The test calls it
 through the C ABI twice in a row, on different inputs, and requires the very
 same outputs as evict_only with a caller-provided workspace: retained positions
-and compacted K/V bit for bit (the parity tests' bar for eviction-only results).
+and compacted K/V bit for bit (the parity tests' bar for eviction-only results),
+and holds them against the CPU oracle's eviction-only result as well.
 The second call finds the first call's leftovers in the shared array and must
 not be affected by them.  Runs last so that a failure here cannot hide another
 test's result.
@@ -52,15 +53,25 @@ def test_static_scratch_entry_point_matches_evict_only_on_two_calls_in_a_row(nam
         ref = _reference(w, arrays)
         dev, outs, caches = _device_caches(w, arrays)
         params = par.params_for(w)
-        before = torch.cuda.memory_allocated()
+        P.evict_only_static(params, caches)                # the first call on a device resolves the array's address
+        torch.cuda.synchronize()
+        for o in outs:
+            o["idx"].fill_(-1); o["K_out"].zero_(); o["V_out"].zero_()
+        torch.cuda.synchronize()
+        before, before_free = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
         P.evict_only_static(params, caches)
         torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated() == before     # nothing was allocated through torch either
+        assert torch.cuda.memory_allocated() == before     # nothing was allocated through torch
+        assert torch.cuda.mem_get_info()[0] == before_free  # nor behind its back: the driver's free memory is unchanged
         assert P.obf_static_scratch_status() & 0xFF == 0
         for o, r in zip(outs, ref):
             assert torch.equal(o["idx"], r["idx"])
             assert torch.equal(o["K_out"], r["K_out"])
             assert torch.equal(o["V_out"], r["V_out"])
+        # and against the oracle's eviction-only result: retained positions (bit-exact outside the tie band) and
+        # bit-exact copies of the retained rows, every head
+        stats = par.check_cache_whole(w, 0, arrays[0], outs[0], rank=0, name="static " + name)
+        assert stats["heads"] == w.layers * w.kv_heads
 
 
 def test_static_scratch_entry_point_rejects_shapes_beyond_its_array(capfd):
