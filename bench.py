@@ -9,6 +9,12 @@ algorithmic bytes (K, V and queries read once; compacted K, V and the index list
 written once) over the device time of the step.  With N > 1 every rank runs an
 independent replica of the workload on its own GPU (the path has no exchange
 step) and the aggregate is reported.  Prints ONE JSON line on rank 0.
+
+Timing: a batch is exactly --steps calls between two CUDA events on the launching stream, bracketed by a
+barrier and a device synchronisation, max over ranks.  Batches are repeated until at least MIN_TIMED_S seconds
+of device time have been measured; `ms_per_step` is the median batch, `best_ms_per_step` the fastest one, and
+the SM clock is sampled all the while (`clocks`), so that `ms_per_step_x_sm_ghz` (time x median clock = kilo-cycles
+per step) can be compared between runs made at different clocks.
 """
 from __future__ import annotations
 
@@ -28,6 +34,8 @@ sys.path.insert(0, ROOT)
 
 METRIC = "prompt_kv_gbs_compressed"
 UNIT = "GB/s"
+MIN_TIMED_S = 2.0          # device time measured per workload (the bench workload; 0.5 s for the side workloads)
+MAX_BATCHES = 400
 
 
 def load_peaks():
@@ -74,7 +82,10 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        inside = [r for t, r in self.rows if t0 - 0.05 <= t <= t1 + 0.15] or [r for _, r in self.rows]
+        inside = [r for t, r in self.rows if t0 <= t <= t1 + 0.1]
+        outside_only = not inside
+        if outside_only:
+            inside = [r for _, r in self.rows]
         sm, mx, reasons = [], [], set()
         for r in inside:
             p = [x.strip() for x in r.split(",")]
@@ -87,8 +98,9 @@ class ClockSampler:
             for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_min_mhz": min(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons), "samples": len(sm),
+                "samples_outside_timed_region": outside_only}
 
 
 def cpu_baseline(w, arrays0, seconds_target: float = 15.0):
@@ -154,6 +166,173 @@ def run_reference(args):
     return 0
 
 
+# fp32 work of the dense algebra per (layer, KV head) whose retained values do not span R^d, as the kernel
+# formulates it (Eq. 2-6): twice-iterated Gram-Schmidt over the k retained rows, P = I - Q^T Q, the two products of
+# M = P G P, the Householder reduction of M to tridiagonal form and the way back for rank + 1 vectors.
+def algebra_flops(d: int, k: int, rank: int) -> float:
+    m = min(k, d)
+    gram_schmidt = 2 * 2 * (2.0 * d) * sum(min(i, d) for i in range(k))     # two passes of dot + update against i rows
+    projector = 2.0 * m * d * d
+    products = 2 * 2.0 * d ** 3
+    tridiagonal = 4.0 / 3.0 * d ** 3 * 2                                     # both triangles are updated
+    back = (rank + 1) * 2 * 2.0 * d * d
+    return gram_schmidt + projector + products + tridiagonal + back
+
+
+def kernel_source_stamp() -> str:
+    """Hash of the CUDA sources: an ncu traffic figure is only quoted for the sources it was captured on."""
+    import hashlib
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2604_13349_b200", "csrc")
+    for f in sorted(os.listdir(csrc)):
+        if f.endswith((".cu", ".cuh")):
+            with open(os.path.join(csrc, f), "rb") as fh:
+                h.update(fh.read())
+    return h.hexdigest()[:12]
+
+
+def measured_traffic(kernel: str, workload: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one launch, from profiles/dram_traffic.txt
+    ("kernel workload bytes stamp"); None when the kernels have changed since the capture."""
+    tpath = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    if not os.path.exists(tpath):
+        return None
+    stamp = kernel_source_stamp()
+    with open(tpath) as f:
+        for ln in f:
+            parts = ln.split("#")[0].split()
+            if len(parts) == 4 and parts[0] == kernel and parts[1] == workload and parts[3] == stamp:
+                return int(parts[2])
+    return None
+
+
+class Bench:
+    """One workload resident on the device: inputs, outputs, workspace, and the timed loops over it."""
+
+    def __init__(self, name: str):
+        import torch
+        import paper_2604_13349_b200 as P
+        from paper_2604_13349_b200 import synth
+        self.torch, self.P = torch, P
+        w = self.w = synth.workload(name)
+        self.params = P.make_params(w.layers, w.kv_heads, w.q_heads, w.head.head_dim, w.n_obs, w.rank,
+                                    P.OBF_F32 if w.dtype == "f32" else P.OBF_BF16, 1e-12,
+                                    (P.binding.OBF_FLAG_LAYERWISE if w.layerwise else 0)
+                                    | (P.binding.OBF_FLAG_FAST_PATH if w.fast_path else 0))
+        self.tdt = torch.float32 if w.dtype == "f32" else torch.bfloat16
+        self.host_arrays = [synth.gen_cache(w, ci) for ci in range(len(w.caches))]
+        self.dev_in, self.caches, self.outs = [], [], []
+        for ci, a in enumerate(self.host_arrays):
+            K, V, Q = self.as_t(a["K"]).cuda(), self.as_t(a["V"]).cuda(), self.as_t(a["Q"]).cuda()
+            T, budget = w.caches[ci].T, w.caches[ci].budget
+            ke = min(budget, T)
+            o = {"K_out": torch.empty((w.layers, w.kv_heads, ke, w.head.head_dim), dtype=self.tdt, device="cuda"),
+                 "V_out": torch.empty((w.layers, w.kv_heads, ke, w.head.head_dim), dtype=self.tdt, device="cuda"),
+                 "idx": torch.empty((w.layers, w.kv_heads, ke), dtype=torch.int32, device="cuda")}
+            q8 = None
+            if w.int8_out:
+                o["K_q8"] = torch.empty((w.layers, w.kv_heads, ke, w.head.head_dim), dtype=torch.int8, device="cuda")
+                o["V_q8"] = torch.empty_like(o["K_q8"])
+                o["K_scale"] = torch.empty((w.layers, w.kv_heads, ke), dtype=torch.float32, device="cuda")
+                o["V_scale"] = torch.empty_like(o["K_scale"])
+                q8 = (o["K_q8"], o["V_q8"], o["K_scale"], o["V_scale"])
+            self.dev_in.append((K, V, Q)); self.outs.append(o)
+            self.caches.append(P.make_cache(K, V, Q, T, budget, o["K_out"], o["V_out"], o["idx"], q8=q8))
+        self.ws = torch.empty(P.obf_workspace_bytes(self.params, self.caches), dtype=torch.uint8, device="cuda")
+        self.stream = torch.cuda.current_stream()
+        e, d, hpc = w.elem_bytes, w.head.head_dim, w.layers * w.kv_heads
+        self.kv_bytes = sum(hpc * c.T * d * e for c in w.caches)
+        self.q_bytes = len(w.caches) * hpc * w.n_q * d * e
+        self.out_bytes = sum(hpc * min(c.budget, c.T) * (2 * d * e + 4) for c in w.caches)
+        self.score_bytes = sum(hpc * c.T * 4 for c in w.caches)            # the mass array A (fp32)
+
+    def as_t(self, a):
+        t = self.torch.from_numpy(a.view(np.int16) if self.w.dtype == "bf16" else a)
+        return t.view(self.torch.bfloat16) if self.w.dtype == "bf16" else t
+
+    def step(self):
+        self.P.obf_compress(self.params, self.caches, self.ws, stream=self.stream)
+
+    def warm(self, n: int) -> int:
+        for _ in range(n):
+            self.step()
+        launches = self.P.obf_last_launch_count()
+        self.torch.cuda.synchronize()
+        status = self.P.obf_last_device_status(self.ws)
+        if status & 0xFF:
+            raise SystemExit("device status %#x after warm-up" % status)
+        return launches
+
+    def time_batches(self, steps: int, min_seconds: float, dist):
+        """Batches of exactly `steps` calls, each between two events on the launching stream and bracketed by a
+        barrier and a synchronisation (max over ranks), until min_seconds of device time are measured.
+        Returns the per-step times of the batches in ms."""
+        torch = self.torch
+        per_step, total_ms = [], 0.0
+        while (total_ms < min_seconds * 1e3 or len(per_step) < 5) and len(per_step) < MAX_BATCHES:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            dist.barrier()
+            torch.cuda.synchronize()
+            e0.record(self.stream)
+            for _ in range(steps):
+                self.step()
+            e1.record(self.stream)
+            torch.cuda.synchronize()
+            dist.barrier()
+            ms = dist.max_over_ranks(e0.elapsed_time(e1))
+            per_step.append(ms / steps)
+            total_ms += ms
+        return per_step
+
+    def phases(self, n_prof: int = 5):
+        """Per-kernel device times of one step (events between launches, on the same stream)."""
+        acc = {}
+        for _ in range(n_prof):
+            for name, ms in self.P.obf_compress_profiled(self.params, self.caches, self.ws, stream=self.stream):
+                acc[name] = acc.get(name, 0.0) + ms / n_prof
+        return acc
+
+    def roofline(self, phase_acc, ms_per_step: float, sm_mhz):
+        """Roofline of the dominant kernel: HBM for the streaming kernels, the fp32 pipes for the dense algebra."""
+        w = self.w
+        dom = max(phase_acc, key=phase_acc.get)
+        peak, peak_kind = load_peaks()
+        step_bytes = w.algorithmic_bytes()
+        kv, q, sc, ob = self.kv_bytes, self.q_bytes, self.score_bytes, self.out_bytes
+        # algorithmic bytes of a launch: what that step of the path must move
+        kernel_bytes = {"k_score_stats": kv + q, "k_score_pool": kv + q + sc,
+                        "k_score_tc": kv + q + sc,                          # K and Q read once, A written
+                        "k_gram": kv, "k_gram_tc": kv + sc,                 # V and A read once
+                        "k_gather": 2 * ob, "k_select": sc}.get(dom)
+        common = {"kernel": dom, "kernel_ms": phase_acc[dom],
+                  "whole_step_frac": (step_bytes / (ms_per_step * 1e-3) / 1e9) / peak,
+                  "whole_step_peak": peak, "whole_step_peak_kind": peak_kind,
+                  "phases_ms": {k: round(v, 4) for k, v in phase_acc.items()}}
+        if kernel_bytes is None:
+            # the dense algebra (and the span test): no HBM traffic to speak of, fp32 arithmetic in shared memory.
+            # Peak: 148 SMs x 128 FMA lanes x 2 flop x SM clock.
+            hpc = w.layers * w.kv_heads
+            flops = sum(hpc * algebra_flops(w.head.head_dim, min(c.budget, c.T), w.rank)
+                        for c in w.caches if min(c.budget, c.T) < w.head.head_dim)
+            clock = sm_mhz or 1965.0
+            alu_peak = 148 * 128 * 2 * clock * 1e6 / 1e12
+            ach = flops / (phase_acc[dom] * 1e-3) / 1e12
+            return dict(common, bound="alu", achieved=ach, peak=alu_peak, unit="TFLOP/s", frac=ach / alu_peak,
+                        peak_kind="derived: 148 SMs x 128 fp32 FMA lanes x 2 x %.0f MHz" % clock, traffic=None,
+                        algorithmic_flops_per_launch=flops)
+        achieved = kernel_bytes / (phase_acc[dom] * 1e-3) / 1e9
+        r = dict(common, bound="hbm", achieved=achieved, peak=peak, unit="GB/s", frac=achieved / peak,
+                 peak_kind=peak_kind, traffic=measured_traffic(dom, w.name), algorithmic_bytes_per_launch=kernel_bytes)
+        if dom == "k_score_tc":
+            # the attention-mass kernel evaluates 2 exponentials per (query, key): a second ceiling beside HBM is
+            # the special-function unit (16 results per clock and SM)
+            n_exp = 2.0 * sum(w.layers * w.kv_heads * c.T * w.n_q for c in w.caches)
+            sfu_peak = 16 * 148 * (sm_mhz or 1965.0) * 1e6 / 1e9
+            r["sfu"] = {"unit": "Gexp/s", "achieved": n_exp / (phase_acc[dom] * 1e-3) / 1e9, "peak": sfu_peak,
+                        "frac": n_exp / (phase_acc[dom] * 1e-3) / 1e9 / sfu_peak}
+        return r
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -163,6 +342,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--also", default="c4_evict,pa", help="workloads reported beside the bench workload at 1 GPU ('' for none)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
@@ -170,7 +350,7 @@ def main():
 
     import torch
     import paper_2604_13349_b200 as P
-    from paper_2604_13349_b200 import dist, synth
+    from paper_2604_13349_b200 import dist
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -182,106 +362,31 @@ def main():
         dist.init("nccl")
     P.load()
 
-    w = synth.workload(args.workload)
-    params = P.make_params(w.layers, w.kv_heads, w.q_heads, w.head.head_dim, w.n_obs, w.rank,
-                           P.OBF_F32 if w.dtype == "f32" else P.OBF_BF16, 1e-12,
-                           (P.binding.OBF_FLAG_LAYERWISE if w.layerwise else 0)
-                           | (P.binding.OBF_FLAG_FAST_PATH if w.fast_path else 0))
-    tdt = torch.float32 if w.dtype == "f32" else torch.bfloat16
-
-    def as_t(a):
-        t = torch.from_numpy(a.view(np.int16) if w.dtype == "bf16" else a)
-        return t.view(torch.bfloat16) if w.dtype == "bf16" else t
-
-    host_arrays = [synth.gen_cache(w, ci) for ci in range(len(w.caches))]
-    dev_in, caches, outs = [], [], []
-    for ci, a in enumerate(host_arrays):
-        K, V, Q = as_t(a["K"]).cuda(), as_t(a["V"]).cuda(), as_t(a["Q"]).cuda()
-        T, budget = w.caches[ci].T, w.caches[ci].budget
-        ke = min(budget, T)
-        o = {"K_out": torch.empty((w.layers, w.kv_heads, ke, w.head.head_dim), dtype=tdt, device="cuda"),
-             "V_out": torch.empty((w.layers, w.kv_heads, ke, w.head.head_dim), dtype=tdt, device="cuda"),
-             "idx": torch.empty((w.layers, w.kv_heads, ke), dtype=torch.int32, device="cuda")}
-        dev_in.append((K, V, Q)); outs.append(o)
-        caches.append(P.make_cache(K, V, Q, T, budget, o["K_out"], o["V_out"], o["idx"]))
-    ws = torch.empty(P.obf_workspace_bytes(params, caches), dtype=torch.uint8, device="cuda")
-    stream = torch.cuda.current_stream()
+    b = Bench(args.workload)
+    w = b.w
+    d = w.head.head_dim
     step_bytes = w.algorithmic_bytes()
-
-    for _ in range(args.warmup):
-        P.obf_compress(params, caches, ws, stream=stream)
-    launches_per_step = P.obf_last_launch_count()
-    torch.cuda.synchronize()
-    status = P.obf_last_device_status(ws)
-    if status & 0xFF:
-        raise SystemExit("device status %#x after warm-up" % status)
+    launches_per_step = b.warm(args.warmup)
 
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
         time.sleep(0.25)
-    dist.barrier()
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_wall0 = time.time()
-    e0.record(stream)
-    for _ in range(args.steps):
-        P.obf_compress(params, caches, ws, stream=stream)
-    e1.record(stream)
-    torch.cuda.synchronize()
+    per_step = b.time_batches(args.steps, MIN_TIMED_S, dist)
     t_wall1 = time.time()
-    dist.barrier()
-    ms_total = dist.max_over_ranks(e0.elapsed_time(e1))
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
-    ms_per_step = ms_total / args.steps
+    ms_per_step = statistics.median(per_step)
     total_bytes = dist.sum_over_ranks(float(step_bytes))
     value = total_bytes / (ms_per_step * 1e-3) / 1e9
     tokens_per_s = dist.sum_over_ranks(float(w.tokens())) / (ms_per_step * 1e-3)
 
-    # per-kernel device times of one step (events between launches, on the same stream)
-    phase_acc = {}
-    n_prof = 5
-    for _ in range(n_prof):
-        for name, ms in P.obf_compress_profiled(params, caches, ws, stream=stream):
-            phase_acc[name] = phase_acc.get(name, 0.0) + ms / n_prof
-    dom = max(phase_acc, key=phase_acc.get)
-    peak, peak_kind = load_peaks()
-    # algorithmic bytes of the dominant kernel's launch: what that step of the path must move
-    e = w.elem_bytes
-    d = w.head.head_dim
-    hpc = w.layers * w.kv_heads
-    kv_bytes = sum(hpc * c.T * d * e for c in w.caches)
-    q_bytes = len(w.caches) * hpc * w.n_q * d * e
-    out_bytes = sum(hpc * min(c.budget, c.T) * (2 * d * e + 4) for c in w.caches)
-    score_bytes = sum(hpc * c.T * 4 for c in w.caches)                 # the mass array A (fp32)
-    kernel_bytes = {"k_score_stats": kv_bytes + q_bytes, "k_score_pool": kv_bytes + q_bytes + score_bytes,
-                    "k_score_tc": kv_bytes + q_bytes + score_bytes,     # K and Q read once, A written
-                    "k_gram": kv_bytes, "k_gram_tc": kv_bytes,          # V read once
-                    "k_gather": 2 * out_bytes, "k_select": score_bytes,
-                    "k_span_test": 0, "k_obf_algebra": 0}.get(dom, step_bytes)
-    achieved = kernel_bytes / (phase_acc[dom] * 1e-3) / 1e9
-    traffic = None
-    # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu summaries ("kernel workload bytes")
-    tpath = os.path.join(ROOT, "profiles", "dram_traffic.txt")
-    if os.path.exists(tpath):
-        with open(tpath) as f:
-            for ln in f:
-                parts = ln.split("#")[0].split()
-                if len(parts) == 3 and parts[0] == dom and parts[1] == w.name:
-                    traffic = int(parts[2])
-    # the attention-mass kernel evaluates 2 exponentials per (query, key): its own ceiling is the
-    # special-function unit (16 results per clock and SM), not HBM
-    n_exp = 2.0 * sum(hpc * c.T * w.n_q for c in w.caches)
-    sm_clock = (clocks or {}).get("sm_mhz") or 1965.0
-    sfu_peak = 16 * 148 * sm_clock * 1e6 / 1e9
-    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_kind": peak_kind, "traffic": traffic,
-                "kernel_ms": phase_acc[dom], "algorithmic_bytes_per_launch": kernel_bytes,
-                "whole_step_frac": (step_bytes / (ms_per_step * 1e-3) / 1e9) / peak,
-                "phases_ms": {k: round(v, 4) for k, v in phase_acc.items()}}
-    if dom == "k_score_tc":
-        roofline["sfu"] = {"unit": "Gexp/s", "achieved": n_exp / (phase_acc[dom] * 1e-3) / 1e9, "peak": sfu_peak,
-                           "frac": n_exp / (phase_acc[dom] * 1e-3) / 1e9 / sfu_peak}
+    phase_acc = b.phases()
+    sm_mhz = (clocks or {}).get("sm_mhz")
+    roofline = b.roofline(phase_acc, ms_per_step, sm_mhz)
+    kv_bytes, q_bytes, out_bytes = b.kv_bytes, b.q_bytes, b.out_bytes
+    host_arrays, outs, params, tdt, stream = b.host_arrays, b.outs, b.params, b.tdt, b.stream
+    as_t = b.as_t
 
     # end to end through the host entry point: pinned host buffers, copies inside the timed region
     e2e = None
@@ -317,10 +422,32 @@ def main():
     if rank == 0 and not args.no_cpu_baseline:
         cpu = cpu_baseline(w, host_arrays[0])
 
+    # Beside the bench workload: the same shapes in eviction-only mode (isolates the cost of OBF) and the paper's
+    # own regime (budget 32 < head_dim, where the back-fill is not zero and the dense algebra runs for every head;
+    # on c2-c5 the retained values span R^d and delta = 0).  1 GPU only.
+    others = {}
+    if world == 1 and args.also:
+        del b
+        torch.cuda.empty_cache()
+        for name in [n for n in args.also.split(",") if n and n != w.name]:
+            ob = Bench(name)
+            ob.warm(args.warmup)
+            ps = ob.time_batches(args.steps, 0.5, dist)
+            ms = statistics.median(ps)
+            others[name] = {"ms_per_step": ms, "best_ms_per_step": min(ps), "batches": len(ps),
+                            "value": ob.w.algorithmic_bytes() / (ms * 1e-3) / 1e9, "unit": UNIT,
+                            "relay_tokens_per_s": ob.w.tokens() / (ms * 1e-3),
+                            "roofline": ob.roofline(ob.phases(), ms, sm_mhz)}
+            del ob
+            torch.cuda.empty_cache()
+
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "best_ms_per_step": min(per_step),
+            "batches": len(per_step), "timed_region_s": sum(per_step) * args.steps * 1e-3,
+            "ms_per_step_x_sm_ghz": ms_per_step * sm_mhz * 1e-3 if sm_mhz else None,
+            "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": w.name, "layers": w.layers, "kv_heads": w.kv_heads, "q_heads": w.q_heads,
                        "head_dim": d, "n_obs": w.n_obs, "rank": w.rank, "selector": "layerwise" if w.layerwise else "headwise",
@@ -330,7 +457,8 @@ def main():
             "relay_tokens_per_s": tokens_per_s,
             "algorithmic_bytes_per_step": step_bytes,
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
-            "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+            "gpu_launches": launches_per_step * args.steps * len(per_step), "gpu_launches_per_step": launches_per_step,
+            "clocks": clocks, "other_workloads": others,
         }
         print(json.dumps(line))
     dist.finish()

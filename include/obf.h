@@ -142,6 +142,21 @@ typedef struct {              /* one agent's prompt cache; T and budget may diff
     obf_diag_t *diag_out;     /* optional [layers, kv_heads], or NULL                               */
     float *scores_out;        /* optional [layers, kv_heads, T] attention mass A (Eq. 1), or NULL   */
     float *delta_out;         /* optional [layers, kv_heads, head_dim] injected vector (Eq. 6), or NULL */
+    const float *lse_extra;   /* optional device [layers, q_heads, n_obs] fp32, or NULL: per observation query the
+                                 natural log of the sum of exp(q.k / sqrt(d)) over the keys OUTSIDE the prompt that the
+                                 model's softmax also ran over (earlier agents' relay, the latent positions before it:
+                                 Section 3.1 defines the weights of Eq. 1 as a softmax over the whole cache, App. L.1
+                                 restates it over the prompt).  Those keys take their share of every row's
+                                 normaliser, so a row's weights over the prompt add up to less than one.  NULL or
+                                 minus infinity: softmax over the prompt keys alone                          */
+    /* Optional int8 copy of the compacted relay (post-hoc quantisation stacked on the compression, App. E, Table 7;
+       the paper fixes no quantiser: symmetric, one fp32 scale per retained row, scale = max|x| / 127, code =
+       round-half-even(x / scale), a row of zeros has scale 0).  All four NULL, or all four device pointers:
+       k_q8_out, v_q8_out int8 [layers, kv_heads, k_eff, head_dim]; k_scale_out, v_scale_out fp32
+       [layers, kv_heads, k_eff].  The codes are taken from k_out / v_out as the call leaves them (v_out after the
+       injection of Eq. 7), which are still written.                                                           */
+    int8_t *k_q8_out, *v_q8_out;
+    float *k_scale_out, *v_scale_out;
 } obf_cache_t;
 
 /*

@@ -58,6 +58,8 @@ def lib():
         ci = ctypes.c_int
         _lib.obf_oracle_scores.argtypes = [fp, fp, ci, ci, ci, dp]
         _lib.obf_oracle_scores.restype = None
+        _lib.obf_oracle_scores_ext.argtypes = [fp, fp, fp, ci, ci, ci, dp]
+        _lib.obf_oracle_scores_ext.restype = None
         _lib.obf_oracle_topk.argtypes = [dp, ci, ci, ip, dp, dp]
         _lib.obf_oracle_topk.restype = ci
         _lib.obf_oracle_topk_sink.argtypes = [dp, ci, ci, ci, ip, dp, dp]
@@ -73,6 +75,8 @@ def lib():
         _lib.obf_oracle_head_sink.restype = ci
         _lib.obf_oracle_head_ex.argtypes = _lib.obf_oracle_head.argtypes + [ci, ci]
         _lib.obf_oracle_head_ex.restype = ci
+        _lib.obf_oracle_head_lse.argtypes = [fp, fp, fp, fp] + _lib.obf_oracle_head.argtypes[3:] + [ci, ci]
+        _lib.obf_oracle_head_lse.restype = ci
         _lib.obf_oracle_compress.argtypes = [fp, fp, fp, ci, ci, ci, ci, ci, ci, ci, ci,
                                              ctypes.c_double, ip, dp, dp, dp, ctypes.POINTER(Diag), ci]
         _lib.obf_oracle_compress.restype = ci
@@ -81,6 +85,8 @@ def lib():
         _lib.obf_oracle_layer.restype = ci
         _lib.obf_oracle_compress_layerwise.argtypes = _lib.obf_oracle_compress.argtypes
         _lib.obf_oracle_compress_layerwise.restype = ci
+        _lib.obf_oracle_quantize_rows.argtypes = [fp, ci, ci, ctypes.POINTER(ctypes.c_int8), fp]
+        _lib.obf_oracle_quantize_rows.restype = None
         _lib.obf_oracle_num_threads.argtypes = []
         _lib.obf_oracle_num_threads.restype = ci
     return _lib
@@ -102,13 +108,22 @@ def num_threads() -> int:
     return int(lib().obf_oracle_num_threads())
 
 
-def scores(K, Q) -> np.ndarray:
-    """Attention mass A[T] of one KV head (Eq. 1); K [T,d], Q [n_q,d]."""
+def scores(K, Q, lse_extra=None) -> np.ndarray:
+    """Attention mass A[T] of one KV head (Eq. 1); K [T,d], Q [n_q,d].
+
+    lse_extra [n_q] (optional): log-sum-exp of each query row's logits over the keys outside the prompt; they
+    take their share of the softmax normaliser."""
     K, Q = _f32(K), _f32(Q)
     T, d = K.shape
     A = np.empty(T, dtype=np.float64)
-    lib().obf_oracle_scores(_p(K, ctypes.c_float), _p(Q, ctypes.c_float), T, d, Q.shape[0],
-                            _p(A, ctypes.c_double))
+    if lse_extra is None:
+        lib().obf_oracle_scores(_p(K, ctypes.c_float), _p(Q, ctypes.c_float), T, d, Q.shape[0],
+                                _p(A, ctypes.c_double))
+    else:
+        le = _f32(lse_extra)
+        assert le.shape == (Q.shape[0],)
+        lib().obf_oracle_scores_ext(_p(K, ctypes.c_float), _p(Q, ctypes.c_float), _p(le, ctypes.c_float), T, d,
+                                    Q.shape[0], _p(A, ctypes.c_double))
     return A
 
 
@@ -152,12 +167,13 @@ def sym_eig(S):
 
 
 def head(K, V, Q, budget: int, rank: int, eps: float = 1e-12, n_sink: int = 0,
-         fast_iters: int = 0) -> Dict[str, object]:
+         fast_iters: int = 0, lse_extra=None) -> Dict[str, object]:
     """Algorithm 2 (headwise) + Algorithm 3 on one (layer, KV head).
 
     K, V [T,d]; Q [n_q,d] (float32 values; bf16 inputs up-cast exactly).
     fast_iters > 0: the subspace comes from that many Gram subspace iterations (App. H) started at the first
     rows of the identity, instead of the exact eigenvectors.
+    lse_extra [n_q] (optional): out-of-prompt softmax mass per query row, see scores().
     Returns idx, K_out, V_out (float64), A, delta, rbar, Delta, eigvals, proj, diag.
     """
     K, V, Q = _f32(K), _f32(V), _f32(Q)
@@ -171,8 +187,10 @@ def head(K, V, Q, budget: int, rank: int, eps: float = 1e-12, n_sink: int = 0,
     proj = np.empty((d, d))
     dg = Diag()
     cd = ctypes.c_double
-    k2 = lib().obf_oracle_head_ex(
-        _p(K, ctypes.c_float), _p(V, ctypes.c_float), _p(Q, ctypes.c_float),
+    le = None if lse_extra is None else _f32(lse_extra)
+    assert le is None or le.shape == (Q.shape[0],)
+    k2 = lib().obf_oracle_head_lse(
+        _p(K, ctypes.c_float), _p(V, ctypes.c_float), _p(Q, ctypes.c_float), _p(le, ctypes.c_float),
         T, d, Q.shape[0], budget, rank, eps,
         _p(idx, ctypes.c_int32), _p(K_out, cd), _p(V_out, cd), _p(A, cd), _p(delta, cd),
         _p(rbar, cd), _p(Delta, cd), _p(eig, cd), _p(proj, cd), ctypes.byref(dg), n_sink, fast_iters)
@@ -206,6 +224,18 @@ def layer(K, V, Q, budget: int, rank: int, eps: float = 1e-12, n_sink: int = 0) 
     assert k2 == k
     return {"idx": idx[:, :k].copy(), "K_out": K_out[:, :k], "V_out": V_out[:, :k], "S": S, "A": A,
             "delta": delta, "diag": [diags[h].asdict() for h in range(H)]}
+
+
+def quantize_rows(X):
+    """Post-hoc int8 quantisation of compacted rows (App. E): X [..., d] float32 -> (codes int8 [..., d], scales
+    float32 [...]), one symmetric absmax scale per row."""
+    X = _f32(X)
+    d = X.shape[-1]
+    rows = X.size // d
+    codes = np.empty(X.shape, dtype=np.int8)
+    scales = np.empty(X.shape[:-1], dtype=np.float32)
+    lib().obf_oracle_quantize_rows(_p(X, ctypes.c_float), rows, d, _p(codes, ctypes.c_int8), _p(scales, ctypes.c_float))
+    return codes, scales
 
 
 def compress(K, V, Q, q_heads: int, n_obs: int, budget: int, rank: int,

@@ -13,7 +13,10 @@
  *
  * Pin status (see tests, all CPU-only):
  *   scores      pinned: row-sum invariant, equal-key closed form, T=2 sigmoid
- *               closed form, library softmax, permutation equivariance
+ *               closed form, library softmax, permutation equivariance;
+ *               with out-of-prompt mass: minus infinity gives the plain masses,
+ *               an appended key whose mass is dropped gives the same masses,
+ *               library log-sum-exp
  *   top-k       pinned: brute-force full sort on tiny inputs, library stable
  *               argsort, planted exact ties
  *   sink prefix pinned: protected positions always retained, the rest equals
@@ -28,6 +31,9 @@
  *               form, codimension-1 closed form, hand-worked planted example
  *   scaling     pinned: single-query identity from the error-bound appendix,
  *               hand-worked planted example
+ *   int8 relay  pinned: round-trip error at most half a step per element, the
+ *               largest element of a row maps to +-127, library rounding
+ *               (numpy rint in float32), zero rows
  * No function here is "parity unpinned".
  */
 #include <math.h>
@@ -72,14 +78,22 @@ typedef struct {
  * KV head (Eq. 1's sum extended over the GQA group).  Softmax runs over the T
  * prompt keys only, natural exponential, maximum subtracted first.
  */
-void obf_oracle_scores(const float *K, const float *Q, int T, int d, int n_q, double *A)
+/*
+ * lse_extra (may be NULL): per query row t the natural logarithm of the sum of exp(logit) over the keys
+ * OUTSIDE the prompt that the model's softmax also ran over (Section 3.1: the attention weights are a softmax
+ * over the whole cache; the prompt is one part of it).  The normaliser then is the prompt's sum plus
+ * exp(lse_extra[t]), so a row's weights over the prompt add up to less than one.  NULL or minus infinity:
+ * the softmax over the prompt keys alone (App. L.1).
+ */
+void obf_oracle_scores_ext(const float *K, const float *Q, const float *lse_extra, int T, int d, int n_q, double *A)
 {
     double *s = (double *)malloc((size_t)T * sizeof(double));
     const double scale = 1.0 / sqrt((double)d);
     for (int j = 0; j < T; ++j) A[j] = 0.0;
     for (int t = 0; t < n_q; ++t) {
         const float *q = Q + (size_t)t * d;
-        double mx = -INFINITY;
+        const double extra = lse_extra ? (double)lse_extra[t] : -INFINITY;
+        double mx = extra;
         for (int j = 0; j < T; ++j) {
             const float *k = K + (size_t)j * d;
             double acc = 0.0;
@@ -87,11 +101,16 @@ void obf_oracle_scores(const float *K, const float *Q, int T, int d, int n_q, do
             s[j] = acc * scale;
             if (s[j] > mx) mx = s[j];
         }
-        double Z = 0.0;
+        double Z = extra > -INFINITY ? exp(extra - mx) : 0.0;
         for (int j = 0; j < T; ++j) { s[j] = exp(s[j] - mx); Z += s[j]; }
         for (int j = 0; j < T; ++j) A[j] += s[j] / Z;
     }
     free(s);
+}
+
+void obf_oracle_scores(const float *K, const float *Q, int T, int d, int n_q, double *A)
+{
+    obf_oracle_scores_ext(K, Q, NULL, T, d, n_q, A);
 }
 
 /* ------------------------------------------------------------------ */
@@ -309,15 +328,32 @@ int obf_oracle_head_sink(const float *K, const float *V, const float *Q,
 
 /* fast_iters > 0: the principal subspace comes from that many steps of the Gram subspace iteration of App. H
  * instead of the exact eigen-decomposition (see backfill_given_selection). */
+int obf_oracle_head_lse(const float *K, const float *V, const float *Q, const float *lse_extra,
+                        int T, int d, int n_q, int budget, int rank, double eps,
+                        int32_t *idx, double *K_out, double *V_out,
+                        double *A_out, double *delta_out, double *rbar_out, double *Delta_out,
+                        double *eigvals_out, double *proj_out, obf_oracle_diag_t *diag, int n_sink, int fast_iters);
+
 int obf_oracle_head_ex(const float *K, const float *V, const float *Q,
                        int T, int d, int n_q, int budget, int rank, double eps,
                        int32_t *idx, double *K_out, double *V_out,
                        double *A_out, double *delta_out, double *rbar_out, double *Delta_out,
                        double *eigvals_out, double *proj_out, obf_oracle_diag_t *diag, int n_sink, int fast_iters)
 {
+    return obf_oracle_head_lse(K, V, Q, NULL, T, d, n_q, budget, rank, eps, idx, K_out, V_out, A_out, delta_out,
+                               rbar_out, Delta_out, eigvals_out, proj_out, diag, n_sink, fast_iters);
+}
+
+/* lse_extra: out-of-prompt softmax mass per query row (see obf_oracle_scores_ext), or NULL. */
+int obf_oracle_head_lse(const float *K, const float *V, const float *Q, const float *lse_extra,
+                        int T, int d, int n_q, int budget, int rank, double eps,
+                        int32_t *idx, double *K_out, double *V_out,
+                        double *A_out, double *delta_out, double *rbar_out, double *Delta_out,
+                        double *eigvals_out, double *proj_out, obf_oracle_diag_t *diag, int n_sink, int fast_iters)
+{
     /* O1: attention mass */
     double *A = (double *)malloc((size_t)T * sizeof(double));
-    obf_oracle_scores(K, Q, T, d, n_q, A);
+    obf_oracle_scores_ext(K, Q, lse_extra, T, d, n_q, A);
     if (A_out) memcpy(A_out, A, (size_t)T * sizeof(double));
 
     /* O2: headwise TopK_B, ascending index list */
@@ -650,6 +686,35 @@ int obf_oracle_compress_layerwise(const float *K, const float *V, const float *Q
                          delta_out ? delta_out + lh * d : NULL, diag_out ? diag_out + lh : NULL, n_sink);
     }
     return k;
+}
+
+/* ------------------------------------------------------------------ */
+/* Post-hoc int8 quantisation of the compacted relay (App. E)          */
+/* ------------------------------------------------------------------ */
+/*
+ * The paper stacks int8 quantisation on the compressed relay (App. E, Table 7) without fixing the quantiser.
+ * Reading taken: symmetric, one fp32 scale per row (one retained position of one KV head),
+ *   scale = max_c |x_c| / 127,   code_c = round-half-even(x_c / scale) in [-127, 127],   x_c ~ code_c * scale;
+ * a row of zeros gets scale 0 and codes 0.  With head_dim 128 a row shrinks from 256 to 132 bytes, the factor
+ * 1.94 by which Table 7's ratio grows from 4.6 to 9.0.  The decision of a code is taken in float32 (the
+ * precision of the scale that is stored), on both sides.
+ * X [rows, d] float32 (bf16 values up-cast exactly); codes [rows, d]; scales [rows].
+ */
+void obf_oracle_quantize_rows(const float *X, int rows, int d, int8_t *codes, float *scales)
+{
+    for (int r = 0; r < rows; ++r) {
+        const float *x = X + (size_t)r * d;
+        float amax = 0.0f;
+        for (int c = 0; c < d; ++c) { const float a = fabsf(x[c]); if (a > amax) amax = a; }
+        const float scale = amax / 127.0f;
+        scales[r] = scale;
+        for (int c = 0; c < d; ++c) {
+            float q = scale > 0.0f ? rintf(x[c] / scale) : 0.0f;
+            if (q > 127.0f) q = 127.0f;
+            if (q < -127.0f) q = -127.0f;
+            codes[(size_t)r * d + c] = (int8_t)q;
+        }
+    }
 }
 
 int obf_oracle_num_threads(void)

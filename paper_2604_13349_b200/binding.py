@@ -79,7 +79,9 @@ class ObfCache(ctypes.Structure):
     _fields_ = [("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("q_obs", ctypes.c_void_p),
                 ("T", ctypes.c_int32), ("budget", ctypes.c_int32),
                 ("k_out", ctypes.c_void_p), ("v_out", ctypes.c_void_p), ("idx_out", ctypes.c_void_p),
-                ("diag_out", ctypes.c_void_p), ("scores_out", ctypes.c_void_p), ("delta_out", ctypes.c_void_p)]
+                ("diag_out", ctypes.c_void_p), ("scores_out", ctypes.c_void_p), ("delta_out", ctypes.c_void_p),
+                ("lse_extra", ctypes.c_void_p), ("k_q8_out", ctypes.c_void_p), ("v_q8_out", ctypes.c_void_p),
+                ("k_scale_out", ctypes.c_void_p), ("v_scale_out", ctypes.c_void_p)]
 
 
 class ObfError(RuntimeError):
@@ -152,10 +154,13 @@ def _ptr(t) -> Optional[int]:
 
 
 def make_cache(k, v, q_obs, T: int, budget: int, k_out, v_out, idx_out, diag_out=None,
-               scores_out=None, delta_out=None) -> ObfCache:
-    """Tensors (device or, for the host entry point, pinned/pageable CPU) or raw addresses."""
+               scores_out=None, delta_out=None, lse_extra=None, q8=None) -> ObfCache:
+    """Tensors (device or, for the host entry point, pinned/pageable CPU) or raw addresses.
+    q8: (k_q8_out, v_q8_out, k_scale_out, v_scale_out) for the int8 copy of the relay, or None."""
+    q8 = q8 or (None, None, None, None)
     return ObfCache(_ptr(k), _ptr(v), _ptr(q_obs), int(T), int(budget), _ptr(k_out), _ptr(v_out),
-                    _ptr(idx_out), _ptr(diag_out), _ptr(scores_out), _ptr(delta_out))
+                    _ptr(idx_out), _ptr(diag_out), _ptr(scores_out), _ptr(delta_out), _ptr(lse_extra),
+                    _ptr(q8[0]), _ptr(q8[1]), _ptr(q8[2]), _ptr(q8[3]))
 
 
 def _carray(caches: Sequence[ObfCache]):
@@ -270,11 +275,13 @@ def parse_diag(diag_bytes: torch.Tensor) -> List[Dict[str, float]]:
 
 def compress_caches(params: ObfParams, caches_in: Sequence[Dict[str, object]], *, evict: bool = False,
                     want_scores: bool = False, want_delta: bool = True, want_diag: bool = True,
+                    want_int8: bool = False,
                     stream=None, workspace: Optional[torch.Tensor] = None) -> List[Dict[str, object]]:
     """Compress a batch of device caches.
 
     ``caches_in``: dicts with device tensors ``K, V [layers, kv_heads, T, d]``,
-    ``Q [layers, q_heads, n_obs, d]`` and an int ``budget``.  Returns one dict per
+    ``Q [layers, q_heads, n_obs, d]``, an int ``budget`` and optionally ``lse_extra [layers, q_heads, n_obs]``
+    (fp32, the out-of-prompt softmax mass per observation query).  Returns one dict per
     cache with ``K_out, V_out, idx`` (and ``scores``, ``delta``, ``diag`` bytes when asked).
     """
     dt = _torch_dtype(params.dtype)
@@ -297,9 +304,16 @@ def compress_caches(params: ObfParams, caches_in: Sequence[Dict[str, object]], *
             "delta": torch.zeros((params.layers, params.kv_heads, params.head_dim), dtype=torch.float32,
                                  device=dev) if want_delta else None,
         }
+        q8 = None
+        if want_int8:
+            o["K_q8"] = torch.empty((params.layers, params.kv_heads, ke, params.head_dim), dtype=torch.int8, device=dev)
+            o["V_q8"] = torch.empty_like(o["K_q8"])
+            o["K_scale"] = torch.empty((params.layers, params.kv_heads, ke), dtype=torch.float32, device=dev)
+            o["V_scale"] = torch.empty_like(o["K_scale"])
+            q8 = (o["K_q8"], o["V_q8"], o["K_scale"], o["V_scale"])
         outs.append(o)
         cs.append(make_cache(K, V, Q, T, ci["budget"], o["K_out"], o["V_out"], o["idx"], o["diag"],
-                             o["scores"], o["delta"]))
+                             o["scores"], o["delta"], ci.get("lse_extra"), q8))
     nb = obf_workspace_bytes(params, cs)
     if workspace is None or workspace.numel() * workspace.element_size() < nb:
         workspace = torch.empty(nb, dtype=torch.uint8, device=caches_in[0]["K"].device)

@@ -18,6 +18,9 @@ struct CacheDev {
     obf_diag_t *diag;
     float *scores_out;
     float *delta_out;
+    const float *lse_extra;   // out-of-prompt softmax mass per query row (natural log), or null
+    int8_t *k_q8, *v_q8;      // optional int8 copy of the compacted relay, with one scale per row
+    float *k_scale, *v_scale;
     int32_t T, k_eff;
     int32_t head_base;        // global id of this cache's first (layer, kv head)
     int32_t nsub_del;         // tuned path: 128-token tiles of V per head (ceil(T / 128))
@@ -207,6 +210,18 @@ __device__ __forceinline__ float block_max(float v, float *red)
     t = red[0];
     __syncthreads();
     return t;
+}
+
+// Folds the out-of-prompt softmax mass of a query row (natural log of the sum of exp(logit) over the keys outside
+// the prompt) into the row's running maximum m (log2 domain) and normaliser z = sum_j 2^(x_j - m).
+__device__ __forceinline__ void fold_lse_extra(float lse_natural, float &m, float &z)
+{
+    const float L = lse_natural * 1.4426950408889634f;
+    if (L > -INFINITY) {
+        const float mn = fmaxf(m, L);
+        z = (m > -INFINITY ? z * exp2f(m - mn) : 0.f) + exp2f(L - mn);
+        m = mn;
+    }
 }
 
 // Order-preserving map from a float's bits to an unsigned key (larger float -> larger key).

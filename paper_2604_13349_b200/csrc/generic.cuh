@@ -92,6 +92,7 @@ __global__ void __launch_bounds__(SC_NT) k_score_stats(const __grid_constant__ C
         for (int i = 0; i < 4; ++i) {
             const int row = q0 + ty + 16 * i;
             if (row < n_q) {
+                if (c.lse_extra) fold_lse_extra(c.lse_extra[(size_t)lh * n_q + row], m[i], Z[i]);
                 float *st = p.stats + ((size_t)blockIdx.y * n_q + row) * 2;
                 st[0] = m[i];
                 st[1] = Z[i];
@@ -532,6 +533,62 @@ __global__ void __launch_bounds__(256) k_gather(const __grid_constant__ CallDev 
             }
         }
     }
+}
+
+// Post-hoc int8 quantisation of the compacted relay (App. E): a warp per retained row of K_out and of V_out,
+// symmetric with one fp32 scale per row, scale = max|x| / 127, code = round-half-even(x / scale).
+// A warp takes QR_ROWS rows of both arrays at once (all loads in flight before the first reduction).
+// grid = (ceil(k_eff_max / (8 * QR_ROWS)), heads_total), 256 threads.
+constexpr int QR_ROWS = 4;
+
+template <typename TIN, int D>
+__global__ void __launch_bounds__(256) k_quantize_rows(const __grid_constant__ CallDev p)
+{
+    int ci, lh;
+    locate(p, blockIdx.y, ci, lh);
+    const CacheDev &c = p.c[ci];
+    if (!c.k_q8) return;
+    const int r0 = (blockIdx.x * 8 + (threadIdx.x >> 5)) * QR_ROWS, lane = threadIdx.x & 31;
+    if (r0 >= c.k_eff) return;
+    constexpr int PER = D / 32;                                        // consecutive elements per lane
+    const size_t row0 = (size_t)lh * c.k_eff + r0;
+    float x[2][QR_ROWS][PER];
+#pragma unroll
+    for (int which = 0; which < 2; ++which)
+#pragma unroll
+        for (int i = 0; i < QR_ROWS; ++i) {
+            const TIN *src = reinterpret_cast<const TIN *>(which ? c.v_out : c.k_out) + (row0 + i) * D + lane * PER;
+#pragma unroll
+            for (int e = 0; e < PER; ++e) x[which][i][e] = r0 + i < c.k_eff ? to_f32(src[e]) : 0.f;
+        }
+#pragma unroll
+    for (int which = 0; which < 2; ++which)
+#pragma unroll
+        for (int i = 0; i < QR_ROWS; ++i) {
+            if (r0 + i >= c.k_eff) break;
+            float amax = 0.f;
+#pragma unroll
+            for (int e = 0; e < PER; ++e) amax = fmaxf(amax, fabsf(x[which][i][e]));
+            amax = warp_max(amax);
+            const float scale = amax / 127.0f;
+            int8_t q[PER];
+#pragma unroll
+            for (int e = 0; e < PER; ++e) {
+                float v = scale > 0.f ? rintf(x[which][i][e] / scale) : 0.f;
+                v = fminf(fmaxf(v, -127.f), 127.f);
+                q[e] = (int8_t)v;
+            }
+            int8_t *dst = (which ? c.v_q8 : c.k_q8) + (row0 + i) * D + lane * PER;
+            if constexpr (PER == 4) {
+                // one 4-byte store per lane (the arrays are 4-byte aligned: validated on the host)
+                *reinterpret_cast<uint32_t *>(dst) = (uint32_t)(uint8_t)q[0] | ((uint32_t)(uint8_t)q[1] << 8) |
+                                                     ((uint32_t)(uint8_t)q[2] << 16) | ((uint32_t)(uint8_t)q[3] << 24);
+            } else {
+#pragma unroll
+                for (int e = 0; e < PER; ++e) dst[e] = q[e];
+            }
+            if (lane == 0) (which ? c.v_scale : c.k_scale)[row0 + i] = scale;
+        }
 }
 
 // Diagnostics only (projection cosine): s = sum of the deleted value rows of a head, for heads with a

@@ -477,6 +477,13 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
         k_obf_algebra<TIN, D><<<heads, ALG_NT, sm_alg, st>>>(cd);
         mark(st, "k_obf_algebra");
     }
+    bool any_q8 = false;
+    for (int i = 0; i < cd.n_caches; ++i) any_q8 = any_q8 || cd.c[i].k_q8 != nullptr;
+    if (any_q8) {
+        dim3 gq((k_max + 8 * QR_ROWS - 1) / (8 * QR_ROWS), heads);
+        k_quantize_rows<TIN, D><<<gq, 256, 0, st>>>(cd);
+        mark(st, "k_quantize_rows");
+    }
     OBF_CUDA_TRY(cudaGetLastError());
     return OBF_OK;
 }
@@ -496,6 +503,13 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
         if (c.diag_out && (reinterpret_cast<uintptr_t>(c.diag_out) & 3u)) return OBF_ERR_INVALID_ARG;
         if (c.scores_out && (reinterpret_cast<uintptr_t>(c.scores_out) & 3u)) return OBF_ERR_INVALID_ARG;
         if (c.delta_out && (reinterpret_cast<uintptr_t>(c.delta_out) & 3u)) return OBF_ERR_INVALID_ARG;
+        if (c.lse_extra && (reinterpret_cast<uintptr_t>(c.lse_extra) & 3u)) return OBF_ERR_INVALID_ARG;
+        // the int8 copy of the relay: all four arrays or none
+        const int n_q8 = (c.k_q8_out != nullptr) + (c.v_q8_out != nullptr) + (c.k_scale_out != nullptr) + (c.v_scale_out != nullptr);
+        if (n_q8 != 0 && n_q8 != 4) return OBF_ERR_INVALID_ARG;
+        if (n_q8 && ((reinterpret_cast<uintptr_t>(c.k_scale_out) & 3u) || (reinterpret_cast<uintptr_t>(c.v_scale_out) & 3u) ||
+                     (reinterpret_cast<uintptr_t>(c.k_q8_out) & 3u) || (reinterpret_cast<uintptr_t>(c.v_q8_out) & 3u)))
+            return OBF_ERR_INVALID_ARG;
     }
     Layout L;
     make_layout(p, caches, n, rank, L);
@@ -517,6 +531,9 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
         c.k = caches[i].k; c.v = caches[i].v; c.q = caches[i].q_obs;
         c.k_out = caches[i].k_out; c.v_out = caches[i].v_out; c.idx_out = caches[i].idx_out;
         c.diag = caches[i].diag_out; c.scores_out = caches[i].scores_out; c.delta_out = caches[i].delta_out;
+        c.lse_extra = caches[i].lse_extra;
+        c.k_q8 = caches[i].k_q8_out; c.v_q8 = caches[i].v_q8_out;
+        c.k_scale = caches[i].k_scale_out; c.v_scale = caches[i].v_scale_out;
         c.T = caches[i].T;
         c.k_eff = k_eff_of(p, caches[i]);
         c.head_base = i * hpc;
@@ -626,7 +643,7 @@ obf_status_t evict_only(const obf_params_t *params, const obf_cache_t *caches, i
 struct HostArena {
     size_t k[OBF_MAX_CACHES], v[OBF_MAX_CACHES], q[OBF_MAX_CACHES];
     size_t k_out[OBF_MAX_CACHES], v_out[OBF_MAX_CACHES], idx[OBF_MAX_CACHES];
-    size_t diag[OBF_MAX_CACHES], scores[OBF_MAX_CACHES], delta[OBF_MAX_CACHES];
+    size_t diag[OBF_MAX_CACHES], scores[OBF_MAX_CACHES], delta[OBF_MAX_CACHES], lse[OBF_MAX_CACHES];
     size_t ws, ws_bytes, total;
 };
 
@@ -646,6 +663,7 @@ static void host_arena_layout(const obf_params_t *p, const obf_cache_t *caches, 
         H.diag[i] = o; o = align_up(o + hpc * sizeof(obf_diag_t), 256);
         H.scores[i] = o; if (caches[i].scores_out) o = align_up(o + hpc * T * 4, 256);
         H.delta[i] = o; o = align_up(o + hpc * d * 4, 256);
+        H.lse[i] = o; if (caches[i].lse_extra) o = align_up(o + (size_t)p->layers * p->q_heads * p->n_obs * 4, 256);
     }
     Layout L;
     make_layout(p, caches, n, p->rank, L);
@@ -705,6 +723,7 @@ obf_status_t obf_compress_host(const obf_params_t *params, const obf_cache_t *ca
     for (int i = 0; i < n_caches; ++i) {
         const obf_cache_t &c = caches[i];
         if (!c.k || !c.v || !c.q_obs || !c.k_out || !c.v_out || !c.idx_out) return OBF_ERR_INVALID_ARG;
+        if (c.k_q8_out || c.v_q8_out || c.k_scale_out || c.v_scale_out) return OBF_ERR_UNSUPPORTED;   // device entry points only
     }
     HostArena H;
     host_arena_layout(params, caches, n_caches, H);
@@ -739,6 +758,11 @@ obf_status_t obf_compress_host(const obf_params_t *params, const obf_cache_t *ca
             dev[i].diag_out = c.diag_out ? reinterpret_cast<obf_diag_t *>(base + H.diag[i]) + l0 * H_kv : nullptr;
             dev[i].scores_out = c.scores_out ? reinterpret_cast<float *>(base + H.scores[i]) + l0 * H_kv * T : nullptr;
             dev[i].delta_out = c.delta_out ? reinterpret_cast<float *>(base + H.delta[i]) + l0 * H_kv * d : nullptr;
+            const size_t lse_l = (size_t)params->q_heads * params->n_obs;
+            dev[i].lse_extra = c.lse_extra ? reinterpret_cast<const float *>(base + H.lse[i]) + l0 * lse_l : nullptr;
+            if (c.lse_extra)
+                OBF_CUDA_TRY(cudaMemcpyAsync(const_cast<float *>(dev[i].lse_extra), c.lse_extra + l0 * lse_l,
+                                             nl * lse_l * sizeof(float), cudaMemcpyHostToDevice, hp->cin));
             OBF_CUDA_TRY(cudaMemcpyAsync(const_cast<void *>(dev[i].k), static_cast<const char *>(c.k) + l0 * kv_l, nl * kv_l,
                                          cudaMemcpyHostToDevice, hp->cin));
             OBF_CUDA_TRY(cudaMemcpyAsync(const_cast<void *>(dev[i].v), static_cast<const char *>(c.v) + l0 * kv_l, nl * kv_l,

@@ -522,6 +522,8 @@ __global__ void __launch_bounds__(ST_THREADS, 1) k_score_tc(const __grid_constan
                 for (int k = 0; k < 4; ++k) {
                     const int t = lane + 32 * k;
                     if (t >= nq) continue;
+                    // the keys outside the prompt take their share of the normaliser
+                    if (c.lse_extra) fold_lse_extra(c.lse_extra[(size_t)item.lh * p.n_q + 128 * item.qt + t], M[k], Z[k]);
                     float mp = M[k] + lg2_approx(Z[k]);
                     if (!(Z[k] > 0.f) || !isfinite(mp)) {
                         atomicOr(p.status, OBF_DEV_NONFINITE);

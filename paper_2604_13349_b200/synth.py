@@ -103,6 +103,7 @@ class Workload:
     caches: Tuple[CacheSpec, ...]
     layerwise: bool = False       # layerwise selector: one retained set per layer
     fast_path: bool = False       # three Gram subspace iterations instead of the exact eigenvectors
+    int8_out: bool = False        # the relay leaves as int8 codes with one fp32 scale per row (App. E)
 
     @property
     def G(self) -> int:
@@ -117,13 +118,15 @@ class Workload:
         return 4 if self.dtype == "f32" else 2
 
     def algorithmic_bytes(self) -> int:
-        """K, V and queries read once; compacted K, V and the index list written once."""
+        """K, V and queries read once; compacted K, V and the index list written once (with int8_out the relay
+        that leaves is the int8 codes and their scales: d + 4 bytes per row instead of d * elem_bytes)."""
         d, e = self.head.head_dim, self.elem_bytes
+        row = (d + 4) if self.int8_out else d * e
         total = 0
         for c in self.caches:
             ke = k_eff(c.budget, c.T)
             heads = self.layers * self.kv_heads
-            total += heads * (2 * c.T * d * e + self.n_q * d * e + 2 * ke * d * e + 4 * ke)
+            total += heads * (2 * c.T * d * e + self.n_q * d * e + 2 * ke * row + 4 * ke)
         return total
 
     def tokens(self) -> int:
@@ -237,6 +240,8 @@ def _make_workloads() -> Dict[str, Workload]:
     out["c4_evict"] = dataclasses.replace(out["c4"], name="c4_evict", rank=0)
     # the layerwise selector with the rank the paper pairs it with (L-OBF, pca_rank 4)
     out["c4_layer"] = dataclasses.replace(out["c4"], name="c4_layer", layerwise=True)
+    # L-OBF + int8 (App. E, Table 7): the layerwise relay leaves as int8 codes
+    out["c4_int8"] = dataclasses.replace(out["c4"], name="c4_int8", layerwise=True, int8_out=True)
     Ts = _ragged_T(4, 4)
     out["c5"] = Workload(
         name="c5", seed=4, layers=36, kv_heads=8, q_heads=32, n_obs=32, rank=2, dtype="bf16",

@@ -97,9 +97,12 @@ def check_head(dtype: str, K: np.ndarray, V: np.ndarray, Q: np.ndarray, budget: 
     # -- a1: attention mass ------------------------------------------------
     if g_scores is not None:
         err = np.abs(g_scores.astype(np.float64) - A)
-        rep.score_err = float((err / (1e-6 + 5e-5 * A)).max())
+        # measured over the whole suite: at most 0.045 of the former bound 1e-6 + 5e-5 A; the bound below is 5 times tighter
+        rep.score_err = float((err / (2e-7 + 1e-5 * A)).max())
         assert rep.score_err <= 1.0, "%s: attention mass off by %.3g x tolerance" % (name, rep.score_err)
-        assert abs(float(g_scores.astype(np.float64).sum()) - Q.shape[0]) <= 1e-3 * Q.shape[0]
+        # every softmax row adds up to one (less the share of the keys outside the prompt, where those are given)
+        assert abs(float(g_scores.astype(np.float64).sum()) - float(A.sum())) <= 1e-3 * Q.shape[0]
+        assert A.sum() <= Q.shape[0] * (1 + 1e-12)
 
     # -- a2: retained positions -----------------------------------------------
     assert g_idx.shape == (k,)

@@ -600,6 +600,89 @@ def test_sink_prefix_is_retained_besides_the_budget(dtype, d, caches, layerwise)
     print("\n[sink] %s" % par.summarize(reps))
 
 
+# ---------------------------------------------------------------------------
+# out-of-prompt softmax mass: the keys outside the prompt take their share of every row's normaliser
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype,d,G,n_obs,caches,flags", [
+    ("f32", 64, 2, 5, ((200, 12), (90, 9)), 0),
+    ("bf16", 128, 2, 9, ((300, 20), (777, 100), (1100, 32)), 0),                 # tuned score kernel, several chunks per head
+    ("bf16", 128, 5, 32, ((640, 24),), 0),                                       # two query tiles per head
+    ("bf16", 128, 2, 9, ((300, 20),), P.binding.OBF_FLAG_GENERIC_PATH)])
+def test_out_of_prompt_softmax_mass(dtype, d, G, n_obs, caches, flags):
+    w = small("lse", layers=2, kv_heads=2, G=G, n_obs=n_obs, d=d, dtype=dtype, rank=2, caches=caches, seed=71 + G)
+    arrays = [synth.gen_cache(w, ci) for ci in range(len(w.caches))]
+    g = np.random.default_rng(17)
+    params = par.params_for(w, flags=flags)
+    dev, lses = [], []
+    from scipy.special import logsumexp
+    for ci, a in enumerate(arrays):
+        # around each row's own log-sum-exp over the prompt: between "nearly nothing outside the prompt" and
+        # "most of the mass outside it"; one row without any
+        Kf = par.f32_view(a["K"], dtype).astype(np.float64)
+        Qf = par.f32_view(a["Q"], dtype).astype(np.float64).reshape(w.layers, w.kv_heads, w.n_q, d)
+        own = logsumexp(np.einsum("lhqd,lhtd->lhqt", Qf, Kf) / np.sqrt(d), axis=-1)
+        le = (own + g.standard_normal(own.shape) * 3).astype(np.float32).reshape(w.layers, w.q_heads, w.n_obs)
+        le[0, 0, 0] = -np.inf
+        lses.append(le)
+        dev.append({"K": par.to_device(a["K"], dtype), "V": par.to_device(a["V"], dtype), "Q": par.to_device(a["Q"], dtype),
+                    "budget": w.caches[ci].budget, "lse_extra": torch.from_numpy(le).cuda()})
+    outs = P.compress_caches(params, dev, want_scores=True)
+    torch.cuda.synchronize()
+    assert P.obf_last_device_status(outs[0]["workspace"]) & 0xFF == 0
+    bits = np.int16 if dtype == "bf16" else np.int32
+    reps = []
+    for ci, a in enumerate(arrays):
+        Qv = par.f32_view(a["Q"], dtype).reshape(w.layers, w.kv_heads, w.n_q, d)
+        le = lses[ci].reshape(w.layers, w.kv_heads, w.n_q)
+        diags = P.parse_diag(outs[ci]["diag"])
+        for l, h in all_heads(w):
+            K, V = par.f32_view(a["K"][l, h], dtype), par.f32_view(a["V"][l, h], dtype)
+            ref = oracle.head(K, V, Qv[l, h], w.caches[ci].budget, w.rank, lse_extra=le[l, h])
+            assert ref["A"].sum() < w.n_q * 0.999                   # the outside keys did take mass
+            out = outs[ci]
+            reps.append(par.check_head(
+                dtype, K, V, Qv[l, h], w.caches[ci].budget, w.rank, out["idx"][l, h].cpu().numpy(),
+                par.out_bits(out["K_out"][l, h]), par.out_bits(out["V_out"][l, h]), par.out_to_f32(out["V_out"][l, h]),
+                out["scores"][l, h].cpu().numpy(), out["delta"][l, h].cpu().numpy(), diags[l * w.kv_heads + h],
+                a["K"][l, h].view(bits), a["V"][l, h].view(bits), name="lse cache %d layer %d head %d" % (ci, l, h), ref=ref))
+    print("\n[lse_extra] %s" % par.summarize(reps))
+
+
+# ---------------------------------------------------------------------------
+# int8 copy of the compacted relay (post-hoc quantisation stacked on the compression, App. E)
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype,d,caches,flags", [
+    ("f32", 64, ((200, 12), (90, 90)), 0),
+    ("bf16", 128, ((300, 20), (777, 140)), 0),
+    ("bf16", 128, ((512, 28),), P.binding.OBF_FLAG_LAYERWISE)])
+def test_int8_copy_of_the_relay(dtype, d, caches, flags):
+    w = small("q8", layers=2, kv_heads=2, G=2, n_obs=6, d=d, dtype=dtype, rank=2, caches=caches, seed=83)
+    arrays = [synth.gen_cache(w, ci) for ci in range(len(w.caches))]
+    outs, _, st = par.run_gpu(w, arrays, flags=flags, want_int8=True)
+    assert st & 0xFF == 0
+    plain, _, _ = par.run_gpu(w, arrays, flags=flags)
+    injected = 0
+    for ci, a in enumerate(arrays):
+        o = outs[ci]
+        # the usual outputs do not depend on the int8 copy being asked for
+        for key in ("idx", "K_out", "V_out"):
+            assert torch.equal(o[key], plain[ci][key]), key
+        Kf, Vf = o["K_out"].float().cpu().numpy(), o["V_out"].float().cpu().numpy()
+        for name, X in (("K", Kf), ("V", Vf)):
+            codes, scales = oracle.quantize_rows(X)                     # the oracle's quantiser on the relay as it left
+            assert np.array_equal(o[name + "_q8"].cpu().numpy(), codes), "%s codes differ" % name
+            assert np.array_equal(o[name + "_scale"].cpu().numpy(), scales), "%s scales differ" % name
+            back = codes.astype(np.float64) * scales.astype(np.float64)[..., None]
+            assert np.all(np.abs(back - X) <= 0.5 * scales[..., None] * (1 + 1e-6))
+        # the keys are exact copies of the inputs: their codes are those of the oracle's own gather
+        idx = o["idx"].cpu().numpy()
+        Kin = par.f32_view(a["K"], dtype)
+        for l, h in all_heads(w):
+            assert np.array_equal(o["K_q8"][l, h].cpu().numpy(), oracle.quantize_rows(Kin[l, h][idx[l, h]])[0])
+        injected += int((o["delta"].abs().sum(dim=-1) > 0).sum())
+    assert injected > 0                                                 # some values were quantised after an injection
+
+
 def test_sink_prefix_longer_than_the_prompt_keeps_everything():
     w = small("sink_all", d=64, dtype="f32", rank=1, caches=((6, 3),), heavy=0)
     arrays = [synth.gen_cache(w, 0)]

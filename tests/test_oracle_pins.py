@@ -128,6 +128,43 @@ def test_scores_permutation_equivariance():
     np.testing.assert_allclose(oracle.scores(K, Q[pq]), A, rtol=1e-13)
 
 
+# out-of-prompt softmax mass (Section 3.1: the attention weights are a softmax over the whole cache)
+def test_scores_with_no_out_of_prompt_mass_are_the_plain_scores():
+    K, _, Q = rand_head(7, 90, 16, 5)
+    A = oracle.scores(K, Q)
+    assert np.array_equal(oracle.scores(K, Q, np.full(5, -np.inf, np.float32)), A)
+    np.testing.assert_allclose(oracle.scores(K, Q, np.full(5, -200.0, np.float32)), A, rtol=1e-13)
+
+
+@pytest.mark.parametrize("seed", range(3))
+def test_scores_with_out_of_prompt_mass_equal_an_appended_key_that_is_dropped(seed):
+    # one more key behind the prompt, whose logit per query IS that query's out-of-prompt log-sum-exp
+    K, _, Q = rand_head(seed, 70, 16, 6, heavy=3)
+    extra = np.random.default_rng(seed).standard_normal(16).astype(np.float32) * 2
+    lse = ((Q.astype(np.float64) @ extra.astype(np.float64)) / 4.0).astype(np.float32)     # 1 / sqrt(16)
+    # the logits of the appended key as the oracle would see them: recompute from the float32 lse for equality
+    full = oracle.scores(np.vstack([K, extra[None]]), Q)
+    part = oracle.scores(K, Q, lse)
+    np.testing.assert_allclose(part, full[:70], rtol=1e-6)          # lse is rounded to float32: 6e-8 in the logit
+    assert part.sum() < 6.0
+    np.testing.assert_allclose(part.sum() + full[70], 6.0, rtol=1e-6)
+
+
+def test_scores_with_out_of_prompt_mass_match_library_logsumexp():
+    from scipy.special import logsumexp
+    K, _, Q = rand_head(11, 120, 32, 7, heavy=4)
+    lse = np.linspace(-3.0, 9.0, 7).astype(np.float32)
+    S = (Q.astype(np.float64) @ K.astype(np.float64).T) / math.sqrt(32)
+    denom = logsumexp(np.concatenate([S, lse.astype(np.float64)[:, None]], axis=1), axis=1)
+    ref = np.exp(S - denom[:, None]).sum(axis=0)
+    np.testing.assert_allclose(oracle.scores(K, Q, lse), ref, rtol=1e-12)
+    # and through the whole head: the selection runs on these masses
+    _, V, _ = rand_head(12, 120, 32, 7)
+    h = oracle.head(K, V, Q, 10, 1, lse_extra=lse)
+    np.testing.assert_allclose(h["A"], ref, rtol=1e-12)
+    assert np.array_equal(h["idx"], np.sort(np.argsort(-ref, kind="stable")[:10]))
+
+
 # --------------------------------------------------------------------------
 # top-k (Section 4.3.2, ties to the lowest index, ascending output)
 # --------------------------------------------------------------------------
@@ -598,3 +635,35 @@ def test_fast_path_reaches_the_exact_subspace_when_the_spectrum_has_a_gap():
                                atol=1e-9 * np.abs(exact["delta"]).max())
     assert np.linalg.norm(oracle.head(K, V, Q, 4, 2, fast_iters=1)["delta"] - exact["delta"]) > \
         np.linalg.norm(fast["delta"] - exact["delta"])
+
+
+# --------------------------------------------------------------------------
+# post-hoc int8 quantisation of the compacted relay (App. E)
+# --------------------------------------------------------------------------
+def test_int8_rows_round_trip_within_half_a_step_and_use_the_full_range():
+    g = np.random.default_rng(3)
+    X = (g.standard_normal((37, 128)) * g.uniform(0.01, 30, (37, 1))).astype(np.float32)
+    codes, scales = oracle.quantize_rows(X)
+    assert codes.dtype == np.int8 and scales.dtype == np.float32
+    back = codes.astype(np.float64) * scales.astype(np.float64)[:, None]
+    assert np.all(np.abs(back - X) <= 0.5 * scales[:, None] * (1 + 1e-6))
+    assert np.all(np.abs(codes).max(axis=1) == 127)                      # the largest element of a row sits at the end of the range
+    assert np.all(np.sign(codes[np.arange(37), np.abs(X).argmax(axis=1)]) == np.sign(X[np.arange(37), np.abs(X).argmax(axis=1)]))
+    np.testing.assert_allclose(scales, np.abs(X).max(axis=1) / 127.0, rtol=1e-6)
+
+
+def test_int8_rows_match_a_library_statement_and_handle_zero_rows():
+    g = np.random.default_rng(4)
+    X = g.standard_normal((5, 3, 64)).astype(np.float32)
+    X[2, 1] = 0.0
+    X[0, 0, :4] = [0.5, 1.5, 2.5, -2.5]                                   # halves: the rounding rule shows
+    X[0, 0, 4:] = 0.0
+    X[0, 0, 5] = 127.0                                                    # scale exactly 1
+    codes, scales = oracle.quantize_rows(X)
+    sc = (np.abs(X).max(axis=-1) / np.float32(127.0)).astype(np.float32)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        ref = np.where(sc[..., None] > 0, np.rint((X / sc[..., None]).astype(np.float32)), 0.0)
+    assert np.array_equal(codes, np.clip(ref, -127, 127).astype(np.int8))
+    assert np.array_equal(scales, sc)
+    assert scales[2, 1] == 0 and not codes[2, 1].any()
+    assert codes[0, 0, :4].tolist() == [0, 2, 2, -2]                      # ties go to the even code
