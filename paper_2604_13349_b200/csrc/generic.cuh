@@ -541,6 +541,22 @@ __global__ void __launch_bounds__(256) k_gather(const __grid_constant__ CallDev 
 // grid = (ceil(k_eff_max / (8 * QR_ROWS)), heads_total), 256 threads.
 constexpr int QR_ROWS = 4;
 
+// PER consecutive elements (2 or 4) as floats, one vector load.
+template <typename TIN, int PER>
+__device__ __forceinline__ void load_run_f32(const TIN *src, float (&x)[PER])
+{
+    if constexpr (sizeof(TIN) == 4) {
+        if constexpr (PER == 4) { const float4 v = *reinterpret_cast<const float4 *>(src); x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w; }
+        else { const float2 v = *reinterpret_cast<const float2 *>(src); x[0] = v.x; x[1] = v.y; }
+    } else {
+        uint32_t w[PER / 2];
+        if constexpr (PER == 4) { const uint2 v = *reinterpret_cast<const uint2 *>(src); w[0] = v.x; w[1] = v.y; }
+        else w[0] = *reinterpret_cast<const uint32_t *>(src);
+#pragma unroll
+        for (int e = 0; e < PER / 2; ++e) { x[2 * e] = __uint_as_float(w[e] << 16); x[2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u); }
+    }
+}
+
 template <typename TIN, int D>
 __global__ void __launch_bounds__(256) k_quantize_rows(const __grid_constant__ CallDev p)
 {
@@ -558,8 +574,11 @@ __global__ void __launch_bounds__(256) k_quantize_rows(const __grid_constant__ C
 #pragma unroll
         for (int i = 0; i < QR_ROWS; ++i) {
             const TIN *src = reinterpret_cast<const TIN *>(which ? c.v_out : c.k_out) + (row0 + i) * D + lane * PER;
+            if (r0 + i < c.k_eff) load_run_f32<TIN, PER>(src, x[which][i]);
+            else {
 #pragma unroll
-            for (int e = 0; e < PER; ++e) x[which][i][e] = r0 + i < c.k_eff ? to_f32(src[e]) : 0.f;
+                for (int e = 0; e < PER; ++e) x[which][i][e] = 0.f;
+            }
         }
 #pragma unroll
     for (int which = 0; which < 2; ++which)

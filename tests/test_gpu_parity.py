@@ -673,7 +673,8 @@ def test_int8_copy_of_the_relay(dtype, d, caches, flags):
             assert np.array_equal(o[name + "_q8"].cpu().numpy(), codes), "%s codes differ" % name
             assert np.array_equal(o[name + "_scale"].cpu().numpy(), scales), "%s scales differ" % name
             back = codes.astype(np.float64) * scales.astype(np.float64)[..., None]
-            assert np.all(np.abs(back - X) <= 0.5 * scales[..., None] * (1 + 1e-6))
+            # x / scale is rounded to fp32 before the rounding to a code: 127 * 2^-24 of a step on top of half a step
+            assert np.all(np.abs(back - X) <= 0.5 * scales[..., None] * (1 + 2.0 ** -15))
         # the keys are exact copies of the inputs: their codes are those of the oracle's own gather
         idx = o["idx"].cpu().numpy()
         Kin = par.f32_view(a["K"], dtype)
