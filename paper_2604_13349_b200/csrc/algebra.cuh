@@ -14,8 +14,10 @@
 //   2. Otherwise: orthonormal basis Q of span(V_keep) (Eq. 2) by twice-iterated
 //      Gram-Schmidt over the retained rows; a row adds a direction when what is
 //      left of it exceeds 1e-4 of its own norm.
-//   3. P = I - Q^T Q,  M = P G_del P = R^T R  (Eq. 3 in Gram form, App. H),
-//      r_bar = P u / (A_del + eps)  (Eq. 4).
+//   3. M = P G P = R^T R with P = I - Q^T Q (Eq. 3 in Gram form, App. H), formed without P as two rank-m
+//      updates with the m basis rows in Q: X <- X - Q^T (Q X) from the left, then the same from the right
+//      (8 m d^2 flops instead of the 4 d^3 of two full products),
+//      r_bar = P u / (A_del + eps) = (u - Q^T (Q u)) / (A_del + eps)  (Eq. 4).
 //   4. C = eigenvectors of the `rank` largest eigenvalues of M above 1e-5 of the
 //      largest.  For rank <= ALG_TRI_MAX_RANK: Householder reduction of M to
 //      tridiagonal form, the rank + 1 largest eigenvalues by bisection on Sturm
@@ -23,8 +25,13 @@
 //      the largest eigenvalue are kept orthogonal during the iteration), mapped
 //      back through the reflectors.  For larger ranks: full eigen-decomposition by
 //      parallel-order Jacobi rotations run to convergence.
-//   5. Delta = C^T C r_bar (Eq. 5), delta = A_del / (A_keep + eps) * Delta (Eq. 6),
+//   5. Delta = C^T C r_bar (Eq. 5), delta = A_del / (A_keep + eps) * Delta (Eq. 6), projected once more off the
+//      basis rows (the subtractions that form M leave rounding noise of the size of G's largest entries),
 //      V_out = V_keep + delta on the head's retained rows (Eq. 7).
+//
+// Shared memory: M (d x d) plus a region sized by the number of basis rows any head of the call can have
+// (min(k_eff, d)): with budgets below d two blocks share a multiprocessor, which is what the latency-bound
+// steps of the eigen-solver need.
 #pragma once
 
 #include "common.cuh"
@@ -57,20 +64,50 @@ __device__ __forceinline__ int sturm_count(const float *a, const float *b, float
     return cnt;
 }
 
+// Floats of the eigen-solver's workspace: tridiagonal form (diagonal, off-diagonal, eigenvalues, rank + 1 vectors
+// with five factor arrays each), or the d x d eigenvector matrix of the Jacobi route, or two row blocks of the
+// fixed-iteration route.
 template <int D>
-constexpr size_t algebra_smem_bytes() { return (size_t)(3 * D * (D + 1) + 6 * D + 64) * sizeof(float) + 2 * D * sizeof(int); }
+__host__ __device__ constexpr int algebra_eig_floats(int rank, int fast_iters)
+{
+    const int ne = (rank < D ? rank : D) + 1;
+    const int tri = 2 * D + 16 + ne * D + ne * 5 * D;
+    const int jac = D * (D + 1);
+    const int fast = 2 * (rank < D ? rank : D) * (D + 1);
+    return fast_iters > 0 ? fast : (rank <= ALG_TRI_MAX_RANK ? tri : jac);
+}
+
+// mcap: basis rows any head of the call can have, min(largest k_eff, D).
+template <int D>
+__host__ __device__ constexpr int algebra_region_floats(int mcap, int rank, int fast_iters)
+{
+    const int thin = mcap * (D + 1);                                // Q X of a projection
+    const int eig = algebra_eig_floats<D>(rank, fast_iters);
+    return mcap * (D + 1) + (thin > eig ? thin : eig);
+}
+
+template <int D>
+inline size_t algebra_smem_bytes(int mcap, int rank, int fast_iters)
+{
+    return (size_t)(D * (D + 1) + 6 * D + 64 + algebra_region_floats<D>(mcap, rank, fast_iters)) * sizeof(float) +
+           2 * D * sizeof(int);
+}
 
 template <typename TIN, int D>
-__global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ CallDev p)
+__global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant__ CallDev p)
 {
     constexpr int LD = D + 1;
     extern __shared__ float sm[];
-    float *B0 = sm, *B1 = B0 + D * LD, *B2 = B1 + D * LD;
+    const int mcap = p.alg_rows;                   // basis rows any head of this call can have
+    float *B2 = sm;                                // d x d: G, then M, then the reflectors in M's dead columns
     float *vw = B2 + D * LD, *vc = vw + D, *vu = vc + D, *vl = vu + D, *vcs = vl + D;  // vcs: 2*D/2 floats (c,s)
     float *red = vcs + D;                          // 32 floats
     float *misc = red + 32;                        // 32 floats
     int *ipq = reinterpret_cast<int *>(misc + 32); // D ints: pairs (p,q); then D ints: selected eigen-columns
     int *isel = ipq + D;
+    float *Qb = reinterpret_cast<float *>(isel + D);   // basis rows of span(V_keep), mcap x LD; stays to the end
+    float *Bm = Qb + mcap * LD;                    // Q X (m x d) of the two projections; the eigen-solvers reuse this
+    float *WS = Bm;                                // workspace of the eigen-solvers
 
     const int g = blockIdx.x, tid = threadIdx.x;
     int ci, lh;
@@ -107,13 +144,22 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
         const TIN *vk = reinterpret_cast<const TIN *>(c.v_out) + (size_t)lh * k * D;
         const float *A = p.scores + c.tok_off + (size_t)lh * T;
         const int32_t *idx = c.idx_out + (size_t)lh * k;
+        // the next row and its mass are asked for while the current row is worked on
+        float v_next = 0.f, a_next = 0.f;
+        if (tid < D && k > 0) {
+            v_next = to_f32(vk[tid]);
+            if (p.gram_all) a_next = A[idx[0]];
+        }
 #pragma unroll 1
         for (int i = 0; i < k && m < D; ++i) {
             if (tid < D) {
-                const float v = to_f32(vk[(size_t)i * D + tid]);
+                const float v = v_next, a = a_next;
+                if (i + 1 < k) {
+                    v_next = to_f32(vk[(size_t)(i + 1) * D + tid]);
+                    if (p.gram_all) a_next = A[idx[i + 1]];
+                }
                 vw[tid] = v;
                 if (p.gram_all) {
-                    const float a = A[idx[i]];
                     const int lev = u_level(a);
 #pragma unroll
                     for (int l = 0; l < U_LEVELS; ++l)
@@ -132,7 +178,7 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
                     const int j = tid >> 2, part = tid & 3;
                     float s = 0.f;
                     if (j < m) {
-                        const float *qj = B0 + j * LD + part * (D / 4);
+                        const float *qj = Qb + j * LD + part * (D / 4);
                         const float *ww = vw + part * (D / 4);
 #pragma unroll 8
                         for (int e = 0; e < D / 4; ++e) s = fmaf(qj[e], ww[e], s);
@@ -146,7 +192,7 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
                     const int cc = tid >> 2, part = tid & 3;
                     float s = 0.f;
                     if (cc < D)
-                        for (int j = part; j < m; j += 4) s = fmaf(vc[j], B0[j * LD + cc], s);
+                        for (int j = part; j < m; j += 4) s = fmaf(vc[j], Qb[j * LD + cc], s);
                     s += __shfl_xor_sync(0xffffffffu, s, 1);
                     s += __shfl_xor_sync(0xffffffffu, s, 2);
                     if (part == 0 && cc < D) vw[cc] -= s;
@@ -158,22 +204,18 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
             for (int cc = (tid & 31); cc < D; cc += 32) np1 = fmaf(vw[cc], vw[cc], np1);
             const float n1 = sqrtf(warp_sum(np1));
             if (n1 > SPAN_ROW_TOL * n0 && n1 > 0.f) {
-                if (tid < D) B0[m * LD + tid] = w1 / n1;
+                // a head can only have more basis rows than the call's layout holds if they reach d (span full)
+                if (m < mcap && tid < D) Qb[m * LD + tid] = w1 / n1;
                 ++m;
             }
             __syncthreads();
         }
         if (m >= D) { done = true; pc = 1.f; status |= OBF_DEV_SKIPPED | OBF_DEV_SPAN_FULL; }
+        else if (m > mcap) { done = true; status |= OBF_DEV_INTERNAL | OBF_DEV_SKIPPED; }   // cannot happen: m <= min(k, d)
     }
 
     if (!done) {
-        // ---- 3. P = I - Q^T Q; M = P G_del P; r_bar --------------------------
-        for (int e = tid; e < D * D; e += ALG_NT) {
-            const int a = e / D, b = e % D;
-            float s = 0.f;
-            for (int j = 0; j < m; ++j) s = fmaf(B0[j * LD + a], B0[j * LD + b], s);
-            B1[a * LD + b] = (a == b ? 1.f : 0.f) - s;
-        }
+        // ---- 3. G, u; M = P G P and r_bar without forming P -----------------------
         for (int e = tid; e < D * D; e += ALG_NT) {
             float s = 0.f;
             for (int sp = 0; sp < n_del; ++sp) s += p.gram_d[((size_t)g * S + sp) * D * D + e];
@@ -193,17 +235,40 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
                 s += sl;
             }
             vu[tid] = s;
+            if (c.diag) vw[tid] = p.svec[(size_t)g * D + tid];
         }
         __syncthreads();
+        // x -> P x = x - Q^T (Q x) for the vector in `x` (d floats in shared memory), in place; vc is scratch
+        auto project = [&](float *x) {
+            {
+                const int j = tid >> 2, part = tid & 3;
+                float sacc = 0.f;
+                if (j < m) {
+                    const float *qj = Qb + j * LD + part * (D / 4);
+#pragma unroll 8
+                    for (int e = 0; e < D / 4; ++e) sacc = fmaf(qj[e], x[part * (D / 4) + e], sacc);
+                }
+                sacc += __shfl_xor_sync(0xffffffffu, sacc, 1);
+                sacc += __shfl_xor_sync(0xffffffffu, sacc, 2);
+                if (part == 0 && j < m) vc[j] = sacc;
+            }
+            __syncthreads();
+            {
+                const int cc = tid >> 2, part = tid & 3;
+                float sacc = 0.f;
+                if (cc < D)
+                    for (int j = part; j < m; j += 4) sacc = fmaf(vc[j], Qb[j * LD + cc], sacc);
+                sacc += __shfl_xor_sync(0xffffffffu, sacc, 1);
+                sacc += __shfl_xor_sync(0xffffffffu, sacc, 2);
+                if (part == 0 && cc < D) x[cc] -= sacc;
+            }
+            __syncthreads();
+        };
         if (c.diag) {
             // projection cosine: s = sum of the deleted values, its part inside span(V_keep) is s - P s
-            float sv = 0.f, par = 0.f;
-            if (tid < D) {
-                sv = p.svec[(size_t)g * D + tid];
-                float ps = 0.f;
-                for (int cc = 0; cc < D; ++cc) ps = fmaf(B1[tid * LD + cc], p.svec[(size_t)g * D + cc], ps);
-                par = sv - ps;
-            }
+            const float sv = tid < D ? vw[tid] : 0.f;
+            project(vw);
+            const float par = tid < D ? sv - vw[tid] : 0.f;
             const float ss = block_sum<ALG_NT>(sv * sv, red), pp = block_sum<ALG_NT>(par * par, red);
             const float sp = block_sum<ALG_NT>(sv * par, red);
             pc = (ss > 0.f && pp > 0.f) ? sp * rsqrtf(ss) * rsqrtf(pp) : 0.f;
@@ -214,65 +279,105 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
         const float trAll = block_sum<ALG_NT>(tid < D ? B2[tid * LD + tid] : 0.f, red);
         const float trG = trAll - (p.gram_all ? sq_keep : 0.f);
         const bool del_negligible = p.gram_all && !(trG > 1e-5f * trAll);
-        // two D x D x D products, a 4 x 8 register tile per thread (rows a0 + 0..3, columns b0 + 32 * 0..7:
-        // the lanes of a warp read consecutive columns, and a row's value is a broadcast)
-        auto matmul = [&](const float *X, const float *Y, float *Z) {
-            constexpr int TILES_B = D / 8 < 32 ? D / 8 : 32;      // threads across the columns
-            constexpr int NB = D / TILES_B;                       // columns per thread
-            for (int t = tid; t < (D / 4) * TILES_B; t += ALG_NT) {
-                const int a0 = (t / TILES_B) * 4, b0 = t % TILES_B;
-                float acc[4][NB];
+        // M = (I - Q^T Q) G (I - Q^T Q) as two rank-m updates: B = Q X (m x d), X -= Q^T B, first on X = G from the
+        // left, then on the transposed problem from the right (X is symmetric up to rounding, so "B = Q X^T")
+        for (int side = 0; side < 2; ++side) {
+            // B[j][c] = sum_a Q[j][a] X[a][c] (left) or sum_a Q[j][a] X[c][a] (right): a 1 x 4 register tile per thread
+            for (int t = tid; t < m * (D / 4); t += ALG_NT) {
+                const int j = t / (D / 4), c0 = (t % (D / 4)) * 4;
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                const float *qj = Qb + j * LD;
+                if (side == 0) {
+#pragma unroll 4
+                    for (int a = 0; a < D; ++a) {
+                        const float qv = qj[a];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) acc[e] = fmaf(qv, B2[a * LD + c0 + e], acc[e]);
+                    }
+                } else {
+#pragma unroll 4
+                    for (int a = 0; a < D; ++a) {
+                        const float qv = qj[a];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) acc[e] = fmaf(qv, B2[(c0 + e) * LD + a], acc[e]);
+                    }
+                }
+#pragma unroll
+                for (int e = 0; e < 4; ++e) Bm[j * LD + c0 + e] = acc[e];
+            }
+            __syncthreads();
+            // left: X[a][c] -= sum_j Q[j][a] B[j][c];  right: X[a][c] -= sum_j B[j][a] Q[j][c].  4 x 4 tile per thread
+            const float *Lf = side == 0 ? Qb : Bm, *Rf = side == 0 ? Bm : Qb;
+            for (int t = tid; t < (D / 4) * (D / 4); t += ALG_NT) {
+                const int a0 = (t / (D / 4)) * 4, c0 = (t % (D / 4)) * 4;
+                float acc[4][4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
 #pragma unroll
-                    for (int j = 0; j < NB; ++j) acc[i][j] = 0.f;
-#pragma unroll 4
-                for (int cc = 0; cc < D; ++cc) {
-                    float x[4], y[NB];
+                    for (int e = 0; e < 4; ++e) acc[i][e] = 0.f;
+                for (int j = 0; j < m; ++j) {
+                    float l[4], r[4];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) x[i] = X[(a0 + i) * LD + cc];
-#pragma unroll
-                    for (int j = 0; j < NB; ++j) y[j] = Y[cc * LD + b0 + j * TILES_B];
+                    for (int i = 0; i < 4; ++i) { l[i] = Lf[j * LD + a0 + i]; r[i] = Rf[j * LD + c0 + i]; }
 #pragma unroll
                     for (int i = 0; i < 4; ++i)
 #pragma unroll
-                        for (int j = 0; j < NB; ++j) acc[i][j] = fmaf(x[i], y[j], acc[i][j]);
+                        for (int e = 0; e < 4; ++e) acc[i][e] = fmaf(l[i], r[e], acc[i][e]);
                 }
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
 #pragma unroll
-                    for (int j = 0; j < NB; ++j) Z[(a0 + i) * LD + b0 + j * TILES_B] = acc[i][j];
+                    for (int e = 0; e < 4; ++e) B2[(a0 + i) * LD + c0 + e] -= acc[i][e];
             }
-        };
-        matmul(B2, B1, B0);                                     // W = G_del P  -> B0
-        __syncthreads();
-        matmul(B1, B0, B2);                                     // M = P W -> B2
-        if (tid < D) {                                          // r_bar = P u / (A_del + eps)
-            float s = 0.f;
-            for (int cc = 0; cc < D; ++cc) s = fmaf(B1[tid * LD + cc], vu[cc], s);
-            vc[tid] = s / (a_del + p.eps);
+            __syncthreads();
         }
-        __syncthreads();
-        if (tid < D) vu[tid] = vc[tid];
         for (int e = tid; e < D * D; e += ALG_NT) {            // symmetrise
-            const int a = e / D, b = e % D;
-            if (a < b) {
-                const float s = 0.5f * (B2[a * LD + b] + B2[b * LD + a]);
-                B2[a * LD + b] = s;
-                B2[b * LD + a] = s;
+            const int a = e / D, bb = e % D;
+            if (a < bb) {
+                const float sy = 0.5f * (B2[a * LD + bb] + B2[bb * LD + a]);
+                B2[a * LD + bb] = sy;
+                B2[bb * LD + a] = sy;
             }
         }
-        for (int e = tid; e < D * D; e += ALG_NT) B1[(e / D) * LD + (e % D)] = (e / D == e % D) ? 1.f : 0.f;
+        // r_bar = P u / (A_del + eps)
+        project(vu);
+        if (tid < D) vu[tid] = vu[tid] / (a_del + p.eps);
         __syncthreads();
         const float trM = block_sum<ALG_NT>(tid < D ? B2[tid * LD + tid] : 0.f, red);
         rcr = del_negligible ? 0.f : trM / (trG + p.eps);
         if (!(rcr >= RCR_SKIP_TOL)) { done = true; status |= OBF_DEV_SKIPPED; }
 
+        // delta, projected once more off the basis rows, published and injected (Eq. 5-7): dl = this thread's channel
+        auto finish_delta = [&](float dl) {
+            if (tid < D) vw[tid] = dl;
+            __syncthreads();
+            project(vw);
+            dl = tid < D ? vw[tid] : 0.f;
+            const float dn2 = block_sum<ALG_NT>(dl * dl, red);
+            dnorm = sqrtf(dn2);
+            if (!isfinite(dn2)) { status |= OBF_DEV_NONFINITE | OBF_DEV_SKIPPED; dnorm = 0.f; }
+            else if (rho == 0 || dn2 == 0.f) status |= OBF_DEV_SKIPPED;
+            else {
+                if (tid < D) {
+                    p.delta[(size_t)g * D + tid] = dl;
+                    if (c.delta_out) c.delta_out[(size_t)lh * D + tid] = dl;
+                }
+                if (tid == 0) p.hflag[g] = HFLAG_INJECT;
+                // Eq. 7: V_out = V_keep + delta on every retained row; the fp32 sum is rounded once
+                TIN *rows = reinterpret_cast<TIN *>(c.v_out) + (size_t)lh * k * D;
+                for (int e = tid; e < k * D; e += ALG_NT) {
+                    const float sum = to_f32(rows[e]) + vw[e % D];
+                    if constexpr (sizeof(TIN) == 4) rows[e] = sum;
+                    else rows[e] = __float2bfloat16_rn(sum);
+                }
+            }
+        };
+
         // ---- 4f. fast path of App. H: C <- orth(C M), a fixed number of times, from the first rows of the identity ----
         if (!done && p.fast_iters > 0) {
             const int lane = tid & 31, warp = tid >> 5;
             int rho_f = min(min(p.rank, D), D - m);               // rank(R) <= d - m
-            float *C = B0, *Y = B1;                                // rows of length D (stride LD)
+            float *C = WS, *Y = WS + min(p.rank, D) * LD;         // row blocks of length D (stride LD)
             for (int e = tid; e < rho_f * D; e += ALG_NT) C[(e / D) * LD + (e % D)] = (e / D == e % D) ? 1.f : 0.f;
             __syncthreads();
 #pragma unroll 1
@@ -346,25 +451,8 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
                 for (int t = 0; t < rho; ++t) sacc = fmaf(vc[t], C[t * LD + tid], sacc);
                 dl = alpha * sacc;
             }
-            const float dn2 = block_sum<ALG_NT>(dl * dl, red);
-            dnorm = sqrtf(dn2);
-            if (!isfinite(dn2)) { status |= OBF_DEV_NONFINITE | OBF_DEV_SKIPPED; dnorm = 0.f; }
-            else if (rho == 0 || dn2 == 0.f) status |= OBF_DEV_SKIPPED;
-            else {
-                if (tid < D) {
-                    p.delta[(size_t)g * D + tid] = dl;
-                    if (c.delta_out) c.delta_out[(size_t)lh * D + tid] = dl;
-                    vw[tid] = dl;
-                }
-                if (tid == 0) p.hflag[g] = HFLAG_INJECT;
-                __syncthreads();
-                TIN *rows = reinterpret_cast<TIN *>(c.v_out) + (size_t)lh * k * D;
-                for (int e = tid; e < k * D; e += ALG_NT) {        // Eq. 7, the fp32 sum rounded once
-                    const float sum = to_f32(rows[e]) + vw[e % D];
-                    if constexpr (sizeof(TIN) == 4) rows[e] = sum;
-                    else rows[e] = __float2bfloat16_rn(sum);
-                }
-            }
+            __syncthreads();                                        // vc is scratch of the projection that follows
+            finish_delta(dl);
             done = true;
         }
 
@@ -372,11 +460,12 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
         if (!done && p.rank <= ALG_TRI_MAX_RANK) {
             const int lane = tid & 31, warp = tid >> 5;
             const int ne = min(min(p.rank, D) + 1, D);             // eigenpairs computed: the wanted ones and the next
-            float *ta = B0, *tb = B0 + D;                          // diagonal, off-diagonal (tb[i] couples i and i + 1)
-            float *tlam = tb + D;                                  // ALG_TRI_NE eigenvalues, largest first
-            float *tz = tlam + 16;                                 // [ALG_TRI_NE][D] eigenvectors
-            float *twk = tz + ALG_TRI_NE * D;                      // [ALG_TRI_NE][5][D] factors of T - lambda I
-            // Householder reduction: reflector k (a unit vector, row k of B1) zeroes column k below the sub-diagonal
+            float *ta = WS, *tb = WS + D;                          // diagonal, off-diagonal (tb[i] couples i and i + 1)
+            float *tlam = tb + D;                                  // ne <= ALG_TRI_NE eigenvalues, largest first (16 floats)
+            float *tz = tlam + 16;                                 // [ne][D] eigenvectors
+            float *twk = tz + ne * D;                              // [ne][5][D] factors of T - lambda I
+            // Householder reduction: reflector k (a unit vector) zeroes column k below the sub-diagonal.  During its step it
+            // sits in vl; afterwards in the part of column k of M that the step has just emptied (rows k + 1 .. d - 1)
             const float tiny2 = 1e-20f * trM * trM;
             // Three block barriers per column: the two reductions of a step (column norm, v . pvec) are taken by
             // every warp for itself rather than by the block, and w = pvec - (v . pvec) v is formed on the fly.
@@ -395,12 +484,14 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
                 if (tid < D) {
                     float v = 0.f;
                     if (!skip && tid > k) v = (tid == k + 1 ? x0 - al : B2[tid * LD + k]) * rsqrtf(vn2);
-                    B1[k * LD + tid] = v;
+                    vl[tid] = v;
                 }
                 if (tid == 0) { ta[k] = B2[k * LD + k]; tb[k] = skip ? x0 : al; }
                 __syncthreads();
-                if (skip) continue;
-                const float *v = B1 + k * LD;
+                // every warp has read column k by now: it takes the reflector (zeros when there is none)
+                if (tid > k && tid < D) B2[tid * LD + k] = vl[tid];
+                if (skip) { __syncthreads(); continue; }
+                const float *v = vl;
                 {                                                   // pvec = 2 M v on the trailing block -> vc
                     float acc[RPW];
 #pragma unroll
@@ -466,7 +557,6 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
                 ta[D - 2] = B2[(D - 2) * LD + D - 2]; tb[D - 2] = B2[(D - 1) * LD + D - 2];
                 ta[D - 1] = B2[(D - 1) * LD + D - 1]; tb[D - 1] = 0.f;
             }
-            if (tid < D) B1[(D - 2) * LD + tid] = 0.f;              // no reflector for the last two columns
             __syncthreads();
             // bounds of the spectrum (Gershgorin) and the pivot floor of the Sturm counts
             float gl = INFINITY, gh = -INFINITY, b2 = 0.f;
@@ -573,11 +663,11 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
                 float *y = tz + warp * D;
 #pragma unroll 1
                 for (int k = D - 3; k >= 0; --k) {
-                    const float *v = B1 + k * LD;
+                    // reflector k: column k of B2 below the diagonal
                     float dsum = 0.f;
-                    for (int cc = lane; cc < D; cc += 32) dsum = fmaf(v[cc], y[cc], dsum);
+                    for (int cc = k + 1 + lane; cc < D; cc += 32) dsum = fmaf(B2[cc * LD + k], y[cc], dsum);
                     dsum = 2.f * warp_sum(dsum);
-                    for (int cc = lane; cc < D; cc += 32) y[cc] -= dsum * v[cc];
+                    for (int cc = k + 1 + lane; cc < D; cc += 32) y[cc] -= dsum * B2[cc * LD + k];
                     __syncwarp();
                 }
             }
@@ -601,31 +691,16 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
                 for (int t = 0; t < rho; ++t) sacc = fmaf(vc[t], tz[t * D + tid], sacc);
                 dl = alpha * sacc;
             }
-            const float dn2 = block_sum<ALG_NT>(dl * dl, red);
-            dnorm = sqrtf(dn2);
-            if (!isfinite(dn2)) { status |= OBF_DEV_NONFINITE | OBF_DEV_SKIPPED; dnorm = 0.f; }
-            else if (rho == 0 || dn2 == 0.f) status |= OBF_DEV_SKIPPED;
-            else {
-                if (tid < D) {
-                    p.delta[(size_t)g * D + tid] = dl;
-                    if (c.delta_out) c.delta_out[(size_t)lh * D + tid] = dl;
-                    vw[tid] = dl;
-                }
-                if (tid == 0) p.hflag[g] = HFLAG_INJECT;
-                __syncthreads();
-                // Eq. 7: V_out = V_keep + delta on every retained row; the fp32 sum is rounded once
-                TIN *rows = reinterpret_cast<TIN *>(c.v_out) + (size_t)lh * k * D;
-                for (int e = tid; e < k * D; e += ALG_NT) {
-                    const float sum = to_f32(rows[e]) + vw[e % D];
-                    if constexpr (sizeof(TIN) == 4) rows[e] = sum;
-                    else rows[e] = __float2bfloat16_rn(sum);
-                }
-            }
+            __syncthreads();                                        // vc is scratch of the projection that follows
+            finish_delta(dl);
             done = true;
         }
 
-        // ---- 4b. Jacobi eigen-decomposition of M (B2), eigenvectors in B1 -----
+        // ---- 4b. Jacobi eigen-decomposition of M (B2), eigenvectors in U (workspace) -----
         if (!done) {
+            float *U = WS;                                          // d x d, starts as the identity
+            for (int e = tid; e < D * D; e += ALG_NT) U[(e / D) * LD + (e % D)] = (e / D == e % D) ? 1.f : 0.f;
+            __syncthreads();
             // rotations below the fp32 noise level of the largest eigenvalue never settle: stop there
             const float floor_abs = 2e-7f * block_max<ALG_NT>(tid < D ? B2[tid * LD + tid] : 0.f, red);
             bool converged = false;
@@ -661,9 +736,9 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
                             const float mp = B2[i * LD + pp], mq = B2[i * LD + qq];
                             B2[i * LD + pp] = cs * mp - sn * mq;
                             B2[i * LD + qq] = sn * mp + cs * mq;
-                            const float up = B1[i * LD + pp], uq = B1[i * LD + qq];
-                            B1[i * LD + pp] = cs * up - sn * uq;
-                            B1[i * LD + qq] = sn * up + cs * uq;
+                            const float up = U[i * LD + pp], uq = U[i * LD + qq];
+                            U[i * LD + pp] = cs * up - sn * uq;
+                            U[i * LD + qq] = sn * up + cs * uq;
                         }
                     }
                     __syncthreads();
@@ -709,36 +784,18 @@ __global__ void __launch_bounds__(ALG_NT) k_obf_algebra(const __grid_constant__ 
             if (tid < rho) {
                 const int col = isel[tid];
                 float s = 0.f;
-                for (int cc = 0; cc < D; ++cc) s = fmaf(B1[cc * LD + col], vu[cc], s);
+                for (int cc = 0; cc < D; ++cc) s = fmaf(U[cc * LD + col], vu[cc], s);
                 vc[tid] = s;
             }
             __syncthreads();
             float dl = 0.f;
             if (tid < D) {
                 float s = 0.f;
-                for (int t = 0; t < rho; ++t) s = fmaf(vc[t], B1[tid * LD + isel[t]], s);
+                for (int t = 0; t < rho; ++t) s = fmaf(vc[t], U[tid * LD + isel[t]], s);
                 dl = alpha * s;
             }
-            const float dn2 = block_sum<ALG_NT>(dl * dl, red);
-            dnorm = sqrtf(dn2);
-            if (!isfinite(dn2)) { status |= OBF_DEV_NONFINITE | OBF_DEV_SKIPPED; dnorm = 0.f; }
-            else if (rho == 0 || dn2 == 0.f) status |= OBF_DEV_SKIPPED;
-            else {
-                if (tid < D) {
-                    p.delta[(size_t)g * D + tid] = dl;
-                    if (c.delta_out) c.delta_out[(size_t)lh * D + tid] = dl;
-                    vw[tid] = dl;
-                }
-                if (tid == 0) p.hflag[g] = HFLAG_INJECT;
-                __syncthreads();
-                // Eq. 7: V_out = V_keep + delta on every retained row; the fp32 sum is rounded once
-                TIN *rows = reinterpret_cast<TIN *>(c.v_out) + (size_t)lh * k * D;
-                for (int e = tid; e < k * D; e += ALG_NT) {
-                    const float sum = to_f32(rows[e]) + vw[e % D];
-                    if constexpr (sizeof(TIN) == 4) rows[e] = sum;
-                    else rows[e] = __float2bfloat16_rn(sum);
-                }
-            }
+            __syncthreads();                                        // vc is scratch of the projection that follows
+            finish_delta(dl);
         }
     }
 

@@ -61,6 +61,7 @@ struct CallDev {
     long long tk_total_sub;   // tuned path: tiles in the tile sequence of the retained rows
     int32_t gram_all;         // 1: gram_d and uvec run over all rows of V (tuned path), 0: over the deleted rows only
     int32_t u_levels;         // partial u vectors per partial Gram matrix: U_LEVELS with gram_all, else 1
+    int32_t alg_rows;         // dense algebra: basis rows any head of the call can have, min(largest k_eff, d)
     int32_t sc_nq;            // tuned score kernel: query rows of its tiles (0: shape-generic score kernels)
     int32_t sc_subs;          // 128-key tiles per chunk
     int32_t sc_rounds;        // rounds of the persistent score kernel

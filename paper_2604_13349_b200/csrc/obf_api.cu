@@ -451,7 +451,7 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
         OBF_CUDA_TRY(cudaStreamWaitEvent(st, side->join, 0));
     }
     if (cd.rank > 0) {
-        const size_t sm_alg = algebra_smem_bytes<D>();
+        const size_t sm_alg = algebra_smem_bytes<D>(cd.alg_rows, cd.rank, cd.fast_iters);
         if ((s = set_smem(k_obf_algebra<TIN, D>, sm_alg)) != OBF_OK) return s;
         if (tuned_obf) {
             if (!side && (s = launch_gram_tc(cd, L, st, 0)) != OBF_OK) return s;
@@ -580,6 +580,7 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
     cd.layerwise = (p->flags & OBF_FLAG_LAYERWISE) ? 1 : 0;
     cd.n_sink = (int32_t)OBF_FLAG_SINK_OF(p->flags);
     cd.fast_iters = (p->flags & OBF_FLAG_FAST_PATH) ? 3 : 0;
+    cd.alg_rows = k_max < p->head_dim ? k_max : p->head_dim;
     cd.wait_limit_ns = tc::WAIT_LIMIT_NS;
     cd.debug_drop_publish = 0;
     if (p->flags & OBF_FLAG_TEST_WAIT_EXPIRES) {
