@@ -342,7 +342,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--also", default="c4_evict,pa", help="workloads reported beside the bench workload at 1 GPU ('' for none)")
+    ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_S,
+                    help="device time to measure before stopping (at least 5 batches are always timed)")
+    ap.add_argument("--also", default="c4_evict,pa", help="workloads reported beside the bench workload at 1 GPU ('none' for none)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
@@ -373,7 +375,7 @@ def main():
         sampler.start()
         time.sleep(0.25)
     t_wall0 = time.time()
-    per_step = b.time_batches(args.steps, MIN_TIMED_S, dist)
+    per_step = b.time_batches(args.steps, args.min_seconds, dist)
     t_wall1 = time.time()
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
     ms_per_step = statistics.median(per_step)
@@ -429,10 +431,10 @@ def main():
     if world == 1 and args.also:
         del b
         torch.cuda.empty_cache()
-        for name in [n for n in args.also.split(",") if n and n != w.name]:
+        for name in [n for n in args.also.split(",") if n and n != "none" and n != w.name]:
             ob = Bench(name)
             ob.warm(args.warmup)
-            ps = ob.time_batches(args.steps, 0.5, dist)
+            ps = ob.time_batches(args.steps, min(0.5, args.min_seconds), dist)
             ms = statistics.median(ps)
             others[name] = {"ms_per_step": ms, "best_ms_per_step": min(ps), "batches": len(ps),
                             "value": ob.w.algorithmic_bytes() / (ms * 1e-3) / 1e9, "unit": UNIT,
