@@ -20,13 +20,14 @@
 //
 // Block = 10 warps:
 //   warp 0       TMA producer: 128 x 128 bf16 tiles (two 128-byte-swizzled column halves) into a ring
-//   warp 1       issues tcgen05.mma: G (+)= tile^T tile (both operands MN-major views of the same tile) and
-//                u (+)= tile^T a, a = the tile's 128 masses as three bf16 columns (high, middle and low part of the
-//                fp32 mass: their sum is the mass exactly, and bf16 x bf16 products are exact in fp32), so that the
-//                CUDA cores never read a value tile; the three columns exist once per mass level (common.cuh:
-//                u_level), a token filling those of its own level; accumulators double-buffered in tensor memory
-//   warps 2..5   masses: warp w serves ring stage w; it fetches the 128 masses of its next tile early, splits them
-//                and writes the columns into the stage's mass tile (K-major, 128-byte swizzle)
+//   warp 1       issues tcgen05.mma: [G | u] (+)= tile^T [tile | a] in ONE instruction per 16 tokens (N = 144): the
+//                B operand is the value tile followed, as a third 64-column block of the same MN-major layout, by
+//                the tile's 128 masses as bf16 columns: high, middle and low part of the fp32 mass (their sum is
+//                the mass exactly, and bf16 x bf16 products are exact in fp32), so that the CUDA cores never read
+//                a value tile; the three columns exist once per mass level (common.cuh: u_level), a token filling
+//                those of its own level; accumulators double-buffered in tensor memory
+//   warps 2..4   masses: warp w serves ring stage w; it fetches the 128 masses of its next tile early, splits them
+//                and writes the columns into the stage's mass block (rows of 128 bytes, 128-byte swizzle)
 //   warps 6..9   epilogue: tensor memory -> partial Gram matrix and partial u in the workspace
 #pragma once
 
@@ -35,15 +36,17 @@
 namespace obf {
 
 constexpr int GT_KEEP_TILES_MAX = 2;                // retained-row tiles per head that enter G_keep (span test)
-constexpr int GT_STAGES = 4;
+constexpr int GT_STAGES = 3;
 constexpr int GT_TILE = 128;                       // tokens per tile
 constexpr int GT_TILE_BYTES = GT_TILE * 128 * 2;   // 32 KiB
-constexpr int GT_ATILE_BYTES = 2 * 16 * 128;       // mass tile: [2 token halves][16 rows][64 tokens] bf16, row 3 * level + part
-static_assert(3 * U_LEVELS <= 16, "the mass tile has 16 rows");
+constexpr int GT_ABLOCK_BYTES = GT_TILE * 128;     // mass block: [128 tokens][64 columns] bf16 like a column block of the tile; columns 3 * level + part in use
+constexpr int GT_STAGE_BYTES = GT_TILE_BYTES + GT_ABLOCK_BYTES;   // the mass block sits right behind its value tile
+constexpr int GT_NU = 16;                          // columns of the mass block that enter the MMA
+static_assert(3 * U_LEVELS <= GT_NU, "the mass columns must fit the MMA's extra columns");
 constexpr int GT_THREADS = 64 + 128 + 128;
-constexpr size_t GT_SMEM_BYTES = 1024 + (size_t)GT_STAGES * (GT_TILE_BYTES + GT_ATILE_BYTES) + 64;
-constexpr uint32_t GT_TMEM_COLS = 512;             // 2 x 128 (Gram) + 2 x 16 (u), rounded up to a power of two
-constexpr uint32_t GT_TMEM_U = 256;                // first column of the u accumulators
+constexpr size_t GT_SMEM_BYTES = 1024 + (size_t)GT_STAGES * GT_STAGE_BYTES + 64;
+constexpr uint32_t GT_TMEM_COLS = 512;             // 2 accumulators of 128 + 16 columns at a stride of 256
+constexpr uint32_t GT_TMEM_STRIDE = 256;
 
 // Walks the segments of one block's run of tiles.
 struct TileRun {
@@ -81,14 +84,6 @@ struct TileRun {
     }
 };
 
-// Byte offset of element (row n, token k) in a mass tile: two halves of 64 tokens, rows of 128 bytes, the 16-byte
-// chunks of a row permuted by the row number (the 128-byte swizzle the tensor core expects of a K-major operand).
-__device__ __forceinline__ uint32_t gt_atile_off(int n, int k)
-{
-    const int h = k >> 6, kl = k & 63;
-    return (uint32_t)(h * 2048 + n * 128 + ((((kl >> 3) ^ (n & 7))) << 4) + (kl & 7) * 2);
-}
-
 // kind 0: G_all and u_all from V; kind 1: G_keep from the compacted retained rows.
 // One block per multiprocessor; the launch bound of three only caps the registers at 64 per thread, so that the
 // blocks of the selection and the gather, which run on a side stream at the same time, find registers beside it.
@@ -98,8 +93,7 @@ __global__ void __launch_bounds__(GT_THREADS, 3) k_gram_tc(const __grid_constant
     constexpr int D = 128;
     extern __shared__ uint8_t gt_smem_raw[];
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(gt_smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t *tiles = base;                                                // GT_STAGES x 32 KiB, 1024-byte aligned
-    uint8_t *atiles = tiles + GT_STAGES * GT_TILE_BYTES;                  // GT_STAGES x 4 KiB, 1024-byte aligned
+    uint8_t *tiles = base;                                                // GT_STAGES x (32 KiB tile + 16 KiB mass block), 1024-byte aligned
     __shared__ uint64_t bar_full[GT_STAGES], bar_ready[GT_STAGES], bar_empty[GT_STAGES];
     __shared__ uint64_t bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t s_tmem, s_abort;
@@ -117,10 +111,6 @@ __global__ void __launch_bounds__(GT_THREADS, 3) k_gram_tc(const __grid_constant
         for (int b = 0; b < 2; ++b) { tc::mbar_init(&bar_acc_full[b], 1); tc::mbar_init(&bar_acc_empty[b], 4); }
         tc::mbar_init_fence();
     }
-    // the last row of every mass tile stays zero for the whole launch (the others are rewritten per tile)
-    for (int i = tid; i < GT_STAGES * GT_ATILE_BYTES / 16; i += GT_THREADS)
-        reinterpret_cast<uint4 *>(atiles)[i] = make_uint4(0u, 0u, 0u, 0u);
-    tc::fence_async_smem();
     if (warp == 1) tc::tmem_alloc(&s_tmem, GT_TMEM_COLS);
     tc::tc_fence_before();
     __syncthreads();
@@ -141,7 +131,7 @@ __global__ void __launch_bounds__(GT_THREADS, 3) k_gram_tc(const __grid_constant
                     const uint32_t ph = (it / GT_STAGES) & 1u;
                     if (!tc::mbar_wait(&bar_empty[s], ph ^ 1u, wc)) break;
                     tc::mbar_expect_tx(&bar_full[s], GT_TILE_BYTES);
-                    const uint32_t dst = tc::smem_u32(tiles + s * GT_TILE_BYTES);
+                    const uint32_t dst = tc::smem_u32(tiles + s * GT_STAGE_BYTES);
                     tc::tma_load_3d(dst, map, &bar_full[s], 0, (sub0 + t) * GT_TILE, lh);
                     tc::tma_load_3d(dst + GT_TILE_BYTES / 2, map, &bar_full[s], 64, (sub0 + t) * GT_TILE, lh);
                 }
@@ -156,7 +146,8 @@ __global__ void __launch_bounds__(GT_THREADS, 3) k_gram_tc(const __grid_constant
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
             constexpr uint32_t IDESC_G = tc::idesc_bf16(128, 128, 1, 1);
-            constexpr uint32_t IDESC_U = tc::idesc_bf16(128, 16, 1, 0);
+            constexpr uint32_t IDESC_GU = tc::idesc_bf16(128, 128 + GT_NU, 1, 1);
+            const uint32_t idesc = kind == 0 ? IDESC_GU : IDESC_G;
             TileRun run;
             run.init(p, blockIdx.x, kind);
             int cache, lh, sub0, nsub, slot;
@@ -166,25 +157,20 @@ __global__ void __launch_bounds__(GT_THREADS, 3) k_gram_tc(const __grid_constant
                 const uint32_t buf = seg & 1u;
                 if (!tc::mbar_wait(&bar_acc_empty[buf], ((seg >> 1) & 1u) ^ 1u, wc)) break;
                 tc::tc_fence_after();
-                const uint32_t acc = tmem + buf * 128u, acc_u = tmem + GT_TMEM_U + buf * 16u;
+                const uint32_t acc = tmem + buf * GT_TMEM_STRIDE;
                 for (int t = 0; t < nsub; ++t, ++it) {
                     const int s = it % GT_STAGES;
                     const uint32_t ph = (it / GT_STAGES) & 1u;
                     if (!tc::mbar_wait(&bar_full[s], ph, wc)) { dead = true; break; }
                     if (kind == 0 && !tc::mbar_wait(&bar_ready[s], ph, wc)) { dead = true; break; }
                     tc::tc_fence_after();
-                    const uint32_t tile = tc::smem_u32(tiles + s * GT_TILE_BYTES);
-                    const uint32_t atile = tc::smem_u32(atiles + s * GT_ATILE_BYTES);
+                    const uint32_t tile = tc::smem_u32(tiles + s * GT_STAGE_BYTES);
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk) {
-                        // 16 tokens per instruction: rows kk*16.. of the tile, both 64-column halves
+                        // 16 tokens per instruction: rows kk*16.. of the tile; the column blocks of 64 follow one another
+                        // at 16 KiB: two of the value tile and, for the B operand of the pass over V, the mass block
                         const uint64_t dv = tc::smem_desc_sw128(tile + kk * 2048, GT_TILE_BYTES / 2, 1024);
-                        tc::umma_bf16(acc, dv, dv, IDESC_G, (t > 0 || kk > 0) ? 1u : 0u);
-                        if (kind == 0) {
-                            // the same 16 tokens of the mass tile: 32 bytes along its swizzled rows, second half after 4 steps
-                            const uint64_t da = tc::smem_desc_sw128(atile + (kk >> 2) * 2048 + (kk & 3) * 32, 16, 1024);
-                            tc::umma_bf16(acc_u, dv, da, IDESC_U, (t > 0 || kk > 0) ? 1u : 0u);
-                        }
+                        tc::umma_bf16(acc, dv, dv, idesc, (t > 0 || kk > 0) ? 1u : 0u);
                     }
                     tc::umma_commit(&bar_empty[s]);
                 }
@@ -196,12 +182,11 @@ __global__ void __launch_bounds__(GT_THREADS, 3) k_gram_tc(const __grid_constant
         }
     } else if (warp < 6) {
         // ---------------- masses: three bf16 columns per level and tile ----------------
-        // Four warps, each on its own: warp w serves the tiles with index w (mod 4), which are also the tiles of ring
-        // stage w, so that four tiles' masses are under way at once (one tile costs a round trip to the stage's
-        // barrier, the stores and a proxy fence: about as long as the tensor cores need for the tile).
-        static_assert(GT_STAGES == 4, "one mass warp per ring stage");
-        if (kind == 0) {
-            const int mw = warp - 2;
+        // One warp per ring stage, each on its own: warp w serves the tiles with index w (mod GT_STAGES), so that the
+        // masses of several tiles are under way at once (one tile costs a round trip to the stage's barrier, the
+        // stores and a proxy fence).
+        const int mw = warp - 2;
+        if (kind == 0 && mw < GT_STAGES) {
             TileRun run;
             run.init(p, blockIdx.x, kind);
             int cache, lh, sub0, nsub, slot;
@@ -209,12 +194,13 @@ __global__ void __launch_bounds__(GT_THREADS, 3) k_gram_tc(const __grid_constant
             bool have = run.next(p, cache, lh, sub0, nsub, slot);
             int t = 0;
             uint32_t it = 0;
+            auto step = [&]() {
+                ++it;
+                if (++t >= nsub) { have = run.next(p, cache, lh, sub0, nsub, slot); t = 0; }
+            };
             // moves the walk to this warp's next tile at or after the current position
             auto seek = [&]() {
-                while (have && (it & 3u) != (uint32_t)mw) {
-                    ++it;
-                    if (++t >= nsub) { have = run.next(p, cache, lh, sub0, nsub, slot); t = 0; }
-                }
+                while (have && (it % GT_STAGES) != (uint32_t)mw) step();
             };
             // masses of tokens lane, lane + 32, .. of the tile the walk stands on
             auto fetch = [&](float (&a)[4]) {
@@ -226,15 +212,10 @@ __global__ void __launch_bounds__(GT_THREADS, 3) k_gram_tc(const __grid_constant
                     a[e] = j < c.T ? __ldg(A + j) : 0.f;
                 }
             };
-            auto step = [&]() {
-                ++it;
-                if (++t >= nsub) { have = run.next(p, cache, lh, sub0, nsub, slot); t = 0; }
-            };
             seek();
             float a_next[4] = {0.f, 0.f, 0.f, 0.f};
             if (have) fetch(a_next);
-            uint8_t *at = atiles + mw * GT_ATILE_BYTES;
-            const __nv_bfloat16 zero = __float2bfloat16_rn(0.f);
+            uint8_t *ab = tiles + mw * GT_STAGE_BYTES + GT_TILE_BYTES;     // this stage's mass block
             while (have) {
                 float a[4];
 #pragma unroll
@@ -244,22 +225,30 @@ __global__ void __launch_bounds__(GT_THREADS, 3) k_gram_tc(const __grid_constant
                 step();
                 seek();
                 if (have) fetch(a_next);
-                if (!tc::mbar_wait(&bar_empty[mw], ph ^ 1u, wc)) break;   // the stage's last user is done with its mass tile
-#pragma unroll 1
+                if (!tc::mbar_wait(&bar_empty[mw], ph ^ 1u, wc)) break;   // the stage's last user is done with its mass block
+#pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     const int k = lane + 32 * e;
                     const __nv_bfloat16 hi = __float2bfloat16_rn(a[e]);
                     const float r1 = a[e] - __bfloat162float(hi);
                     const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
                     const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+                    const uint32_t part[3] = {(uint32_t)__bfloat16_as_ushort(hi), (uint32_t)__bfloat16_as_ushort(mid),
+                                              (uint32_t)__bfloat16_as_ushort(lo)};
                     const int lev = u_level(a[e]);
+                    // columns 0..15 of the token's row: column 3 * lev + i holds part i, the others zero
+                    uint32_t w[8];
 #pragma unroll
-                    for (int l = 0; l < U_LEVELS; ++l) {
-                        const bool mine = l == lev;
-                        *reinterpret_cast<__nv_bfloat16 *>(at + gt_atile_off(3 * l, k)) = mine ? hi : zero;
-                        *reinterpret_cast<__nv_bfloat16 *>(at + gt_atile_off(3 * l + 1, k)) = mine ? mid : zero;
-                        *reinterpret_cast<__nv_bfloat16 *>(at + gt_atile_off(3 * l + 2, k)) = mine ? lo : zero;
+                    for (int n2 = 0; n2 < 8; ++n2) {
+                        const int n0 = 2 * n2, n1 = 2 * n2 + 1;
+                        const uint32_t v0 = (n0 / 3 == lev && n0 < 3 * U_LEVELS) ? part[n0 % 3] : 0u;
+                        const uint32_t v1 = (n1 / 3 == lev && n1 < 3 * U_LEVELS) ? part[n1 % 3] : 0u;
+                        w[n2] = v0 | (v1 << 16);
                     }
+                    // the two 16-byte chunks of columns 0..7 and 8..15 sit at chunk (0 or 1) XOR (token mod 8) of the row
+                    uint8_t *rowp = ab + k * 128;
+                    *reinterpret_cast<uint4 *>(rowp + ((0 ^ (k & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    *reinterpret_cast<uint4 *>(rowp + ((1 ^ (k & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
                 }
                 tc::fence_async_smem();
                 __syncwarp();
@@ -284,7 +273,7 @@ __global__ void __launch_bounds__(GT_THREADS, 3) k_gram_tc(const __grid_constant
 #pragma unroll 1
             for (int cb = 0; cb < 4; ++cb) {
                 uint32_t r[32];
-                tc::tmem_ld32(tl + buf * 128u + cb * 32u, r);
+                tc::tmem_ld32(tl + buf * GT_TMEM_STRIDE + cb * 32u, r);
                 tc::tmem_ld_wait();
 #pragma unroll
                 for (int e = 0; e < 8; ++e)
@@ -295,7 +284,7 @@ __global__ void __launch_bounds__(GT_THREADS, 3) k_gram_tc(const __grid_constant
             if (kind == 0) {
                 // u of value channel `row`, per mass level: three columns add up the products with the three parts of the masses
                 uint32_t r[32];
-                tc::tmem_ld32(tl + GT_TMEM_U + buf * 16u, r);
+                tc::tmem_ld32(tl + buf * GT_TMEM_STRIDE + 128u, r);
                 tc::tmem_ld_wait();
 #pragma unroll
                 for (int l = 0; l < U_LEVELS; ++l)

@@ -31,7 +31,7 @@ static thread_local int g_phase_count = 0;
 // of the fork and the join.  Created on first use; no device memory is involved.
 struct SideStream {
     cudaStream_t stream = nullptr;
-    cudaEvent_t fork = nullptr, join = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr, join_keys = nullptr;
     int device = -1;
 };
 
@@ -44,7 +44,8 @@ static SideStream *side_stream()
     if (s.device != dev) {
         if (cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) != cudaSuccess ||
             cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) != cudaSuccess ||
-            cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) != cudaSuccess) {
+            cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&s.join_keys, cudaEventDisableTiming) != cudaSuccess) {
             cudaGetLastError();
             return nullptr;
         }
@@ -444,11 +445,19 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
     }
     mark(sel, "k_select");
     dim3 g4((k_max + GATHER_ROWS - 1) / GATHER_ROWS, heads);
-    k_gather<D * (int)sizeof(TIN)><<<g4, 256, 0, sel>>>(cd);
-    mark(sel, "k_gather");
     if (side) {
+        // the values first: the rest of the call needs them; the keys are needed by nothing that follows and are
+        // copied while the span test and the dense algebra leave the memory system idle
+        k_gather<D * (int)sizeof(TIN), 1><<<g4, 256, 0, sel>>>(cd);
+        mark(sel, "k_gather");
         OBF_CUDA_TRY(cudaEventRecord(side->join, side->stream));
+        k_gather<D * (int)sizeof(TIN), 2><<<g4, 256, 0, sel>>>(cd);
+        ++g_last_launches;
+        OBF_CUDA_TRY(cudaEventRecord(side->join_keys, side->stream));
         OBF_CUDA_TRY(cudaStreamWaitEvent(st, side->join, 0));
+    } else {
+        k_gather<D * (int)sizeof(TIN)><<<g4, 256, 0, sel>>>(cd);
+        mark(sel, "k_gather");
     }
     if (cd.rank > 0) {
         const size_t sm_alg = algebra_smem_bytes<D>(cd.alg_rows, cd.rank, cd.fast_iters);
@@ -477,6 +486,7 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
         k_obf_algebra<TIN, D><<<heads, ALG_NT, sm_alg, st>>>(cd);
         mark(st, "k_obf_algebra");
     }
+    if (side) OBF_CUDA_TRY(cudaStreamWaitEvent(st, side->join_keys, 0));   // the call ends when both streams have
     bool any_q8 = false;
     for (int i = 0; i < cd.n_caches; ++i) any_q8 = any_q8 || cd.c[i].k_q8 != nullptr;
     if (any_q8) {
