@@ -31,7 +31,7 @@ static thread_local int g_phase_count = 0;
 // of the fork and the join.  Created on first use; no device memory is involved.
 struct SideStream {
     cudaStream_t stream = nullptr;
-    cudaEvent_t fork = nullptr, join = nullptr, join_keys = nullptr;
+    cudaEvent_t fork = nullptr, pass_done = nullptr, join = nullptr, join_keys = nullptr;
     int device = -1;
 };
 
@@ -44,6 +44,7 @@ static SideStream *side_stream()
     if (s.device != dev) {
         if (cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) != cudaSuccess ||
             cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&s.pass_done, cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&s.join_keys, cudaEventDisableTiming) != cudaSuccess) {
             cudaGetLastError();
@@ -412,6 +413,7 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
         OBF_CUDA_TRY(cudaEventRecord(side->fork, st));
         OBF_CUDA_TRY(cudaStreamWaitEvent(side->stream, side->fork, 0));
         if ((s = launch_gram_tc(cd, L, st, 0)) != OBF_OK) return s;
+        OBF_CUDA_TRY(cudaEventRecord(side->pass_done, st));
     }
     if (cd.layerwise) {
         // masses of a layer's KV heads added up, then every head's block selects on its layer's sums
@@ -447,10 +449,12 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
     dim3 g4((k_max + GATHER_ROWS - 1) / GATHER_ROWS, heads);
     if (side) {
         // the values first: the rest of the call needs them; the keys are needed by nothing that follows and are
-        // copied while the span test and the dense algebra leave the memory system idle
+        // copied once the pass over V is over (it is bound by HBM), while the span test and the dense algebra
+        // leave the memory system idle
         k_gather<D * (int)sizeof(TIN), 1><<<g4, 256, 0, sel>>>(cd);
         mark(sel, "k_gather");
         OBF_CUDA_TRY(cudaEventRecord(side->join, side->stream));
+        OBF_CUDA_TRY(cudaStreamWaitEvent(side->stream, side->pass_done, 0));
         k_gather<D * (int)sizeof(TIN), 2><<<g4, 256, 0, sel>>>(cd);
         ++g_last_launches;
         OBF_CUDA_TRY(cudaEventRecord(side->join_keys, side->stream));
