@@ -85,6 +85,8 @@ def lib():
         _lib.obf_oracle_layer.restype = ci
         _lib.obf_oracle_compress_layerwise.argtypes = _lib.obf_oracle_compress.argtypes
         _lib.obf_oracle_compress_layerwise.restype = ci
+        _lib.obf_oracle_backfill.argtypes = [fp, fp, dp, ci, ci, ci, ci, ctypes.c_double, ip, dp, dp, dp, ctypes.POINTER(Diag)]
+        _lib.obf_oracle_backfill.restype = ci
         _lib.obf_oracle_quantize_rows.argtypes = [fp, ci, ci, ctypes.POINTER(ctypes.c_int8), fp]
         _lib.obf_oracle_quantize_rows.restype = None
         _lib.obf_oracle_num_threads.argtypes = []
@@ -224,6 +226,20 @@ def layer(K, V, Q, budget: int, rank: int, eps: float = 1e-12, n_sink: int = 0) 
     assert k2 == k
     return {"idx": idx[:, :k].copy(), "K_out": K_out[:, :k], "V_out": V_out[:, :k], "S": S, "A": A,
             "delta": delta, "diag": [diags[h].asdict() for h in range(H)]}
+
+
+def backfill(K, V, A, idx, rank: int, eps: float = 1e-12) -> Dict[str, object]:
+    """Algorithm 3 on one (layer, KV head) for given masses A [T] and given ascending retained positions idx."""
+    K, V, A = _f32(K), _f32(V), _f64(A)
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    T, d = K.shape
+    k = idx.shape[0]
+    K_out = np.zeros((max(k, 1), d)); V_out = np.zeros((max(k, 1), d)); delta = np.zeros(d)
+    dg = Diag()
+    cd = ctypes.c_double
+    lib().obf_oracle_backfill(_p(K, ctypes.c_float), _p(V, ctypes.c_float), _p(A, cd), T, d, k, rank, eps,
+                              _p(idx, ctypes.c_int32), _p(K_out, cd), _p(V_out, cd), _p(delta, cd), ctypes.byref(dg))
+    return {"idx": idx, "K_out": K_out[:k], "V_out": V_out[:k], "A": A, "delta": delta, "diag": dg.asdict()}
 
 
 def quantize_rows(X):

@@ -688,6 +688,18 @@ int obf_oracle_compress_layerwise(const float *K, const float *V, const float *Q
     return k;
 }
 
+/*
+ * Algorithm 3 for a retained set chosen elsewhere: masses A [T] and k ascending positions idx are given (the
+ * last step of Algorithm 2 and everything after it).  For checking a result whose positions differ from this
+ * oracle's inside the tie band: the back-fill is then compared on the positions that were actually retained.
+ */
+int obf_oracle_backfill(const float *K, const float *V, const double *A, int T, int d, int k, int rank, double eps,
+                        const int32_t *idx, double *K_out, double *V_out, double *delta_out, obf_oracle_diag_t *diag)
+{
+    return backfill_given_selection(K, V, A, T, d, k, rank, eps, idx, 0.0, -1.0, K_out, V_out, delta_out,
+                                    NULL, NULL, NULL, NULL, diag, 0);
+}
+
 /* ------------------------------------------------------------------ */
 /* Post-hoc int8 quantisation of the compacted relay (App. E)          */
 /* ------------------------------------------------------------------ */

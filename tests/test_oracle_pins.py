@@ -668,3 +668,17 @@ def test_int8_rows_match_a_library_statement_and_handle_zero_rows():
     assert np.array_equal(scales, sc)
     assert scales[2, 1] == 0 and not codes[2, 1].any()
     assert codes[0, 0, :4].tolist() == [0, 2, 2, -2]                      # ties go to the even code
+
+
+def test_backfill_for_given_positions_is_the_head_result_on_its_own_positions():
+    K, V, Q = rand_head(21, 90, 32, 6, heavy=3)
+    h = oracle.head(K, V, Q, 12, 2)
+    b = oracle.backfill(K, V, h["A"], h["idx"], 2)
+    np.testing.assert_array_equal(b["V_out"], h["V_out"])
+    np.testing.assert_array_equal(b["delta"], h["delta"])
+    # another retained set: the last position swapped for a deleted one; the gather follows it
+    idx2 = np.sort(np.append(h["idx"][:-1], np.setdiff1d(np.arange(90), h["idx"])[0])).astype(np.int32)
+    b2 = oracle.backfill(K, V, h["A"], idx2, 2)
+    np.testing.assert_array_equal(b2["K_out"], K[idx2].astype(np.float64))
+    Vk = V[idx2].astype(np.float64)
+    assert np.abs(Vk @ b2["delta"]).max() <= 1e-10 * np.linalg.norm(Vk, 2) * max(np.linalg.norm(b2["delta"]), 1e-300)
