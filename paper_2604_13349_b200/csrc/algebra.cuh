@@ -114,7 +114,7 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
     locate(p, g, ci, lh);
     const CacheDev &c = p.c[ci];
     const int T = c.T, k = c.k_eff, S = p.gram_slots;
-    const int n_del = gram_partial_count(p, c, lh, 0), n_keep = gram_partial_count(p, c, lh, 1);
+    const int n_del = gram_partial_count(p, c, lh);
     const float a_keep = p.sums[(size_t)g * 4], a_del = p.sums[(size_t)g * 4 + 1];
     const float alpha = a_del / (a_keep + p.eps);
 

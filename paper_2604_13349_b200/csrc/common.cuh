@@ -24,11 +24,10 @@ struct CacheDev {
     int32_t T, k_eff;
     int32_t head_base;        // global id of this cache's first (layer, kv head)
     int32_t nsub_del;         // tuned path: 128-token tiles of V per head (ceil(T / 128))
-    int32_t nsub_keep;        // tuned path: 128-row tiles of V_keep per head (0 when the span test is not needed)
+    int32_t pad0_;
     int32_t pad_;
     size_t tok_off;           // offset of this cache in the per-token workspace arrays (elements)
     long long sub_base;       // tuned path: index of this cache's first tile in the tile sequence of the pass over V
-    long long subk_base;      // tuned path: the same in the tile sequence of the retained rows (span test)
     // tuned score kernel: a head's chunks are worked on by a team of slots, heads are dealt in rounds
     int32_t sc_team;          // chunks (= blocks) per head
     int32_t sc_hpr;           // heads per round
@@ -38,7 +37,7 @@ struct CacheDev {
 };
 
 // Tensor maps of a tuned-path kernel, two per cache, passed as a kernel parameter
-// (score kernel: a = K, b = Q; Gram kernel: a = V, b = compacted V_keep).
+// (score kernel: a = K, b = Q; Gram kernel: a = V).
 struct TcMaps {
     CUtensorMap a[OBF_MAX_CACHES];
     CUtensorMap b[OBF_MAX_CACHES];
@@ -56,9 +55,8 @@ struct CallDev {
     int32_t splits;           // token splits of the Gram pass (shape-generic path)
     int32_t gram_slots;       // partial Gram matrices stored per head (stride of gram_d / gram_k / uvec)
     int32_t tc_per;           // tuned path: tiles per block of the pass over V (0: shape-generic path)
-    int32_t tk_per;           // tuned path: tiles per block of the pass over the retained rows
+    int32_t pad1_;
     long long tc_total_sub;   // tuned path: tiles in the tile sequence of the pass over V
-    long long tk_total_sub;   // tuned path: tiles in the tile sequence of the retained rows
     int32_t gram_all;         // 1: gram_d and uvec run over all rows of V (tuned path), 0: over the deleted rows only
     int32_t u_levels;         // partial u vectors per partial Gram matrix: U_LEVELS with gram_all, else 1
     int32_t alg_rows;         // dense algebra: basis rows any head of the call can have, min(largest k_eff, d)
@@ -85,7 +83,7 @@ struct CallDev {
     float *stats;             // [heads_total, n_q, 2] softmax row max (log2 domain) and normaliser
     float *sums;              // [heads_total, 4] a_keep, a_del, kth, next
     float *gram_d;            // [heads_total, gram_slots, d, d] partial Gram of the deleted (gram_all: of all) values
-    float *gram_k;            // [heads_total, gram_slots, d, d] partial Gram of retained values
+    float *gram_k;            // [heads_total, gram_slots, d, d] partial Gram of retained values (shape-generic path only)
     float *uvec;              // [heads_total, gram_slots, u_levels, d] partial sum_j A_j v_j over the same rows as gram_d, per mass level
     float *delta;             // [heads_total, d]
     float *svec;              // [heads_total, d] sum of the deleted value rows (only filled when diagnostics are asked for)
@@ -101,19 +99,16 @@ __device__ __forceinline__ void locate(const CallDev &p, int g, int &ci, int &lh
     lh = g - p.c[ci].head_base;
 }
 
-// How many partial Gram matrices the streaming pass left for one head.
-// kind 0: the pass over V (and the u vector), kind 1: retained values.
-// Shape-generic path: one per token split.  Tuned path: the tile sequence of a
-// pass is cut into runs of `per` tiles, one run per block; a head's tiles
-// land in consecutive blocks, each of which stores one partial.
-__device__ __forceinline__ int gram_partial_count(const CallDev &p, const CacheDev &c, int lh, int kind)
+// How many partial Gram matrices (and u vectors) the streaming pass left for one head.
+// Shape-generic path: one per token split (for the deleted and for the retained rows alike).  Tuned path: the
+// tile sequence of the pass over V is cut into runs of tc_per tiles, one run per block; a head's tiles land in
+// consecutive blocks, each of which stores one partial.
+__device__ __forceinline__ int gram_partial_count(const CallDev &p, const CacheDev &c, int lh)
 {
     if (p.tc_per == 0) return p.splits;
-    const long long len = kind ? c.nsub_keep : c.nsub_del;
-    if (len == 0) return 0;
-    const long long per = kind ? p.tk_per : p.tc_per;
-    const long long start = (kind ? c.subk_base : c.sub_base) + (long long)lh * len;
-    return (int)((start + len - 1) / per - start / per) + 1;
+    const long long len = c.nsub_del;
+    const long long start = c.sub_base + (long long)lh * len;
+    return (int)((start + len - 1) / p.tc_per - start / p.tc_per) + 1;
 }
 
 // The sum u = sum_j A_j v_j over ALL rows is kept apart by the magnitude of the mass, one partial sum per level

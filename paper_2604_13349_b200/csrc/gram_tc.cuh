@@ -9,11 +9,9 @@
 // retained rows are taken out of u (and out of the trace of G) by the dense algebra, which reads them anyway.
 // It can thus run beside the selection and the gather instead of after them.
 //
-// A second, small launch of the same kernel (kind 1) builds G_keep = sum of v v^T over the first rows of the
-// compacted V_keep, only when k_eff >= d: it decides whether span(V_keep) = R^d (Eq. 2).
+// (Whether span(V_keep) = R^d, Eq. 2, is decided by k_span_test from the gathered rows themselves.)
 //
-// Work decomposition.  Every head owns nsub tiles of 128 tokens (kind 0: ceil(T / 128) tiles of V; kind 1: up to
-// GT_KEEP_TILES_MAX tiles of the head's rows in v_out).  All tiles of a launch form one sequence, cut into
+// Work decomposition.  Every head owns ceil(T / 128) tiles of 128 tokens of V.  All tiles of a launch form one sequence, cut into
 // gridDim.x runs of `per` tiles; block b streams run b.  A run crosses head boundaries; each maximal stretch of
 // one head inside a run is a segment and yields one partial Gram matrix (and one partial u), stored in slot
 // (b - first block touching that head).
@@ -35,7 +33,6 @@
 
 namespace obf {
 
-constexpr int GT_KEEP_TILES_MAX = 2;                // retained-row tiles per head that enter G_keep (span test)
 constexpr int GT_STAGES = 3;
 constexpr int GT_TILE = 128;                       // tokens per tile
 constexpr int GT_TILE_BYTES = GT_TILE * 128 * 2;   // 32 KiB
@@ -51,25 +48,24 @@ constexpr uint32_t GT_TMEM_STRIDE = 256;
 // Walks the segments of one block's run of tiles.
 struct TileRun {
     long long pos, end;        // current and one-past-last index in the launch-wide tile sequence
-    int ci, kind, per;
-    __device__ __forceinline__ void init(const CallDev &p, int block, int kind_)
+    int ci, per;
+    __device__ __forceinline__ void init(const CallDev &p, int block)
     {
-        kind = kind_;
-        per = kind ? p.tk_per : p.tc_per;
-        const long long total = kind ? p.tk_total_sub : p.tc_total_sub;
+        per = p.tc_per;
+        const long long total = p.tc_total_sub;
         pos = (long long)block * per;
         end = pos + per;
         if (end > total) end = total;
         ci = 0;
     }
-    __device__ __forceinline__ long long base_of(const CacheDev &c) const { return kind ? c.subk_base : c.sub_base; }
+    __device__ __forceinline__ long long base_of(const CacheDev &c) const { return c.sub_base; }
     // Next segment: cache, local head, first tile, tile count, partial slot.
     __device__ __forceinline__ bool next(const CallDev &p, int &cache, int &lh, int &sub0, int &nsub, int &slot)
     {
         if (pos >= end) return false;
         while (ci + 1 < p.n_caches && pos >= base_of(p.c[ci + 1])) ++ci;
         const CacheDev &c = p.c[ci];
-        const int per_head = kind ? c.nsub_keep : c.nsub_del;
+        const int per_head = c.nsub_del;
         const long long rel = pos - base_of(c);
         lh = (int)(rel / per_head);
         sub0 = (int)(rel - (long long)lh * per_head);
@@ -84,11 +80,10 @@ struct TileRun {
     }
 };
 
-// kind 0: G_all and u_all from V; kind 1: G_keep from the compacted retained rows.
+// G_all and u_all from V.
 // One block per multiprocessor; the launch bound of three only caps the registers at 64 per thread, so that the
 // blocks of the selection and the gather, which run on a side stream at the same time, find registers beside it.
-__global__ void __launch_bounds__(GT_THREADS, 3) k_gram_tc(const __grid_constant__ CallDev p, const __grid_constant__ TcMaps tm,
-                                                            const int kind)
+__global__ void __launch_bounds__(GT_THREADS, 3) k_gram_tc(const __grid_constant__ CallDev p, const __grid_constant__ TcMaps tm)
 {
     constexpr int D = 128;
     extern __shared__ uint8_t gt_smem_raw[];
@@ -121,11 +116,11 @@ __global__ void __launch_bounds__(GT_THREADS, 3) k_gram_tc(const __grid_constant
         // ---------------- TMA producer ----------------
         if (lane == 0) {
             TileRun run;
-            run.init(p, blockIdx.x, kind);
+            run.init(p, blockIdx.x);
             int cache, lh, sub0, nsub, slot;
             uint32_t it = 0;
             while (run.next(p, cache, lh, sub0, nsub, slot)) {
-                const CUtensorMap *map = kind ? &tm.b[cache] : &tm.a[cache];
+                const CUtensorMap *map = &tm.a[cache];
                 for (int t = 0; t < nsub; ++t, ++it) {
                     const int s = it % GT_STAGES;
                     const uint32_t ph = (it / GT_STAGES) & 1u;
@@ -145,11 +140,9 @@ __global__ void __launch_bounds__(GT_THREADS, 3) k_gram_tc(const __grid_constant
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            constexpr uint32_t IDESC_G = tc::idesc_bf16(128, 128, 1, 1);
-            constexpr uint32_t IDESC_GU = tc::idesc_bf16(128, 128 + GT_NU, 1, 1);
-            const uint32_t idesc = kind == 0 ? IDESC_GU : IDESC_G;
+            constexpr uint32_t idesc = tc::idesc_bf16(128, 128 + GT_NU, 1, 1);
             TileRun run;
-            run.init(p, blockIdx.x, kind);
+            run.init(p, blockIdx.x);
             int cache, lh, sub0, nsub, slot;
             uint32_t it = 0, seg = 0;
             bool dead = false;
@@ -162,13 +155,13 @@ __global__ void __launch_bounds__(GT_THREADS, 3) k_gram_tc(const __grid_constant
                     const int s = it % GT_STAGES;
                     const uint32_t ph = (it / GT_STAGES) & 1u;
                     if (!tc::mbar_wait(&bar_full[s], ph, wc)) { dead = true; break; }
-                    if (kind == 0 && !tc::mbar_wait(&bar_ready[s], ph, wc)) { dead = true; break; }
+                    if (!tc::mbar_wait(&bar_ready[s], ph, wc)) { dead = true; break; }
                     tc::tc_fence_after();
                     const uint32_t tile = tc::smem_u32(tiles + s * GT_STAGE_BYTES);
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk) {
                         // 16 tokens per instruction: rows kk*16.. of the tile; the column blocks of 64 follow one another
-                        // at 16 KiB: two of the value tile and, for the B operand of the pass over V, the mass block
+                        // at 16 KiB: two of the value tile and, for the B operand, the mass block
                         const uint64_t dv = tc::smem_desc_sw128(tile + kk * 2048, GT_TILE_BYTES / 2, 1024);
                         tc::umma_bf16(acc, dv, dv, idesc, (t > 0 || kk > 0) ? 1u : 0u);
                     }
@@ -186,9 +179,9 @@ __global__ void __launch_bounds__(GT_THREADS, 3) k_gram_tc(const __grid_constant
         // masses of several tiles are under way at once (one tile costs a round trip to the stage's barrier, the
         // stores and a proxy fence).
         const int mw = warp - 2;
-        if (kind == 0 && mw < GT_STAGES) {
+        if (mw < GT_STAGES) {
             TileRun run;
-            run.init(p, blockIdx.x, kind);
+            run.init(p, blockIdx.x);
             int cache, lh, sub0, nsub, slot;
             // position of the walk: tile `t` of the current segment, `it` in the run
             bool have = run.next(p, cache, lh, sub0, nsub, slot);
@@ -260,7 +253,7 @@ __global__ void __launch_bounds__(GT_THREADS, 3) k_gram_tc(const __grid_constant
         const int q = warp & 3;                    // lane quarter this warp may read
         const int row = q * 32 + lane;
         TileRun run;
-        run.init(p, blockIdx.x, kind);
+        run.init(p, blockIdx.x);
         int cache, lh, sub0, nsub, slot;
         uint32_t seg = 0;
         while (run.next(p, cache, lh, sub0, nsub, slot)) {
@@ -269,7 +262,7 @@ __global__ void __launch_bounds__(GT_THREADS, 3) k_gram_tc(const __grid_constant
             if (!tc::mbar_wait(&bar_acc_full[buf], (seg >> 1) & 1u, wc)) break;
             tc::tc_fence_after();
             const uint32_t tl = tmem + ((uint32_t)(q * 32) << 16);
-            float *dst = (kind ? p.gram_k : p.gram_d) + ((size_t)g * p.gram_slots + slot) * D * D + (size_t)row * D;
+            float *dst = p.gram_d + ((size_t)g * p.gram_slots + slot) * D * D + (size_t)row * D;
 #pragma unroll 1
             for (int cb = 0; cb < 4; ++cb) {
                 uint32_t r[32];
@@ -281,7 +274,7 @@ __global__ void __launch_bounds__(GT_THREADS, 3) k_gram_tc(const __grid_constant
                         make_float4(__uint_as_float(r[4 * e]), __uint_as_float(r[4 * e + 1]),
                                     __uint_as_float(r[4 * e + 2]), __uint_as_float(r[4 * e + 3]));
             }
-            if (kind == 0) {
+            {
                 // u of value channel `row`, per mass level: three columns add up the products with the three parts of the masses
                 uint32_t r[32];
                 tc::tmem_ld32(tl + buf * GT_TMEM_STRIDE + 128u, r);

@@ -78,10 +78,9 @@ struct Layout {
     bool tuned;
     int gram_slots;                 // partial Gram matrices stored per head
     int tc_per, tc_blocks;          // tiles per block and blocks of the tensor-core pass over V
-    int tk_per, tk_blocks;          // the same for the pass over the retained rows (span test)
-    long long tc_total_sub, tk_total_sub;
-    int nsub_del[OBF_MAX_CACHES], nsub_keep[OBF_MAX_CACHES];
-    long long sub_base[OBF_MAX_CACHES], subk_base[OBF_MAX_CACHES];
+    long long tc_total_sub;
+    int nsub_del[OBF_MAX_CACHES];
+    long long sub_base[OBF_MAX_CACHES];
     // tensor-core score kernel
     bool sc_on;
     int sc_nq, sc_subs, sc_blocks, sc_rounds, sc_qt;
@@ -172,39 +171,22 @@ static void make_layout(const obf_params_t *p, const obf_cache_t *caches, int32_
     L.tuned = tuned_path_applies(p, caches, n);
     L.gram_slots = L.splits;
     L.tc_per = 0; L.tc_blocks = 0; L.tc_total_sub = 0;
-    L.tk_per = 0; L.tk_blocks = 0; L.tk_total_sub = 0;
     if (L.tuned && rank > 0) {
-        long long total = 0, total_k = 0;
+        long long total = 0;
         for (int i = 0; i < n; ++i) {
-            const int T = caches[i].T, ke = k_eff_of(p, caches[i]);
-            L.nsub_del[i] = (T + GT_TILE - 1) / GT_TILE;
-            // The span test only has to certify span(V_keep) = R^d, and any subset of the retained rows that spans
-            // R^d does: the first two tiles (256 rows >= head_dim) are enough.  A head whose subset fails the test
-            // goes through the full Gram-Schmidt basis over all its retained rows, like every head with k < d.
-            L.nsub_keep[i] = (ke >= d && T > ke) ? (ke + GT_TILE - 1) / GT_TILE : 0;
-            if (L.nsub_keep[i] > GT_KEEP_TILES_MAX) L.nsub_keep[i] = GT_KEEP_TILES_MAX;
+            L.nsub_del[i] = (caches[i].T + GT_TILE - 1) / GT_TILE;
             L.sub_base[i] = total;
-            L.subk_base[i] = total_k;
             total += (long long)hpc * L.nsub_del[i];
-            total_k += (long long)hpc * L.nsub_keep[i];
         }
         const long long sms = sm_count();
-        auto cut = [&](long long tot, int &per, int &blocks) {
-            if (tot == 0) { per = 0; blocks = 0; return; }
-            const long long want = tot < sms ? tot : sms;
-            per = (int)((tot + want - 1) / want);
-            blocks = (int)((tot + per - 1) / per);
-        };
+        const long long want = total < sms ? total : sms;
         L.tc_total_sub = total;
-        L.tk_total_sub = total_k;
-        cut(total, L.tc_per, L.tc_blocks);
-        cut(total_k, L.tk_per, L.tk_blocks);
+        L.tc_per = (int)((total + want - 1) / want);
+        L.tc_blocks = (int)((total + L.tc_per - 1) / L.tc_per);
         int slots = 1;
         for (int i = 0; i < n; ++i) {
             const int a = (L.nsub_del[i] + L.tc_per - 1) / L.tc_per + 1;
-            const int b = L.nsub_keep[i] ? (L.nsub_keep[i] + L.tk_per - 1) / L.tk_per + 1 : 0;
             if (a > slots) slots = a;
-            if (b > slots) slots = b;
         }
         L.gram_slots = slots;
     }
@@ -264,7 +246,7 @@ static void make_layout(const obf_params_t *p, const obf_cache_t *caches, int32_
     if (rank > 0) {
         const size_t gsz = (size_t)L.heads_total * L.gram_slots * d * d * sizeof(float);
         L.off_gram_d = o; o = align_up(o + gsz, 256);
-        L.off_gram_k = o; o = align_up(o + gsz, 256);
+        L.off_gram_k = o; if (!L.tc_per) o = align_up(o + gsz, 256);   // the tuned path forms G_keep inside the span test
         L.off_uvec = o;   o = align_up(o + (size_t)L.heads_total * L.gram_slots * (L.tc_per ? U_LEVELS : 1) * d * sizeof(float), 256);
         L.off_delta = o;  o = align_up(o + (size_t)L.heads_total * d * sizeof(float), 256);
         L.off_hflag = o;  o = align_up(o + (size_t)L.heads_total * sizeof(uint32_t), 256);
@@ -332,27 +314,22 @@ static obf_status_t encode_rows_map(CUtensorMap *m, const void *ptr, uint64_t ro
     return OBF_OK;
 }
 
-// Streaming passes of OBF on the tensor cores (bf16, head_dim 128).  kind 0: Gram matrix and mass-weighted sum
-// over all rows of V (needs the masses, not the selection); kind 1: Gram matrix of the first retained rows (needs
-// the gathered values).
-static obf_status_t launch_gram_tc(const CallDev &cd, const Layout &L, cudaStream_t st, int kind)
+// Streaming pass of OBF on the tensor cores (bf16, head_dim 128): Gram matrix and mass-weighted sum over all rows
+// of V (needs the masses, not the selection).
+static obf_status_t launch_gram_tc(const CallDev &cd, const Layout &L, cudaStream_t st)
 {
-    static thread_local TcMaps maps[2];
-    TcMaps &m = maps[kind];
-    const int blocks = kind ? L.tk_blocks : L.tc_blocks;
-    if (blocks == 0) return OBF_OK;
+    static thread_local TcMaps m;
+    if (L.tc_blocks == 0) return OBF_OK;
     const uint64_t hpc = (uint64_t)cd.heads_per_cache;
     for (int i = 0; i < cd.n_caches; ++i) {
-        obf_status_t s = OBF_OK;
-        if (kind == 0) s = encode_rows_map(&m.a[i], cd.c[i].v, (uint64_t)cd.c[i].T, hpc);
-        else if (L.nsub_keep[i]) s = encode_rows_map(&m.b[i], cd.c[i].v_out, (uint64_t)cd.c[i].k_eff, hpc);
+        const obf_status_t s = encode_rows_map(&m.a[i], cd.c[i].v, (uint64_t)cd.c[i].T, hpc);
         if (s != OBF_OK) return s;
     }
     OBF_CUDA_TRY(cudaFuncSetAttribute(k_gram_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GT_SMEM_BYTES));
     // the whole shared-memory capacity, so that the side stream's blocks find room beside this kernel's
     OBF_CUDA_TRY(cudaFuncSetAttribute(k_gram_tc, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared));
-    k_gram_tc<<<blocks, GT_THREADS, GT_SMEM_BYTES, st>>>(cd, m, kind);
-    mark(st, kind ? "k_gram_tc_keep" : "k_gram_tc");
+    k_gram_tc<<<L.tc_blocks, GT_THREADS, GT_SMEM_BYTES, st>>>(cd, m);
+    mark(st, "k_gram_tc");
     return OBF_OK;
 }
 
@@ -412,7 +389,7 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
     if (side) {
         OBF_CUDA_TRY(cudaEventRecord(side->fork, st));
         OBF_CUDA_TRY(cudaStreamWaitEvent(side->stream, side->fork, 0));
-        if ((s = launch_gram_tc(cd, L, st, 0)) != OBF_OK) return s;
+        if ((s = launch_gram_tc(cd, L, st)) != OBF_OK) return s;
         OBF_CUDA_TRY(cudaEventRecord(side->pass_done, st));
     }
     if (cd.layerwise) {
@@ -467,8 +444,7 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
         const size_t sm_alg = algebra_smem_bytes<D>(cd.alg_rows, cd.rank, cd.fast_iters);
         if ((s = set_smem(k_obf_algebra<TIN, D>, sm_alg)) != OBF_OK) return s;
         if (tuned_obf) {
-            if (!side && (s = launch_gram_tc(cd, L, st, 0)) != OBF_OK) return s;
-            if ((s = launch_gram_tc(cd, L, st, 1)) != OBF_OK) return s;
+            if (!side && (s = launch_gram_tc(cd, L, st)) != OBF_OK) return s;
         } else {
             dim3 g5(cd.splits, heads);
             k_gram<TIN, D><<<g5, 256, 0, st>>>(cd);
@@ -484,8 +460,19 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
             mark(st, "k_vsum");
         }
         const size_t sm_span = span_smem_bytes<D>();
-        if ((s = set_smem(k_span_test<D>, sm_span)) != OBF_OK) return s;
-        k_span_test<D><<<heads, ST_NT, sm_span, st>>>(cd);
+        if constexpr (sizeof(TIN) == 2 && D == 128) {
+            if (tuned_obf) {
+                // the tuned path forms G_keep inside the span test, from the gathered rows
+                if ((s = set_smem(k_span_test<D, true>, sm_span)) != OBF_OK) return s;
+                k_span_test<D, true><<<heads, ST_NT, sm_span, st>>>(cd);
+            } else {
+                if ((s = set_smem(k_span_test<D>, sm_span)) != OBF_OK) return s;
+                k_span_test<D><<<heads, ST_NT, sm_span, st>>>(cd);
+            }
+        } else {
+            if ((s = set_smem(k_span_test<D>, sm_span)) != OBF_OK) return s;
+            k_span_test<D><<<heads, ST_NT, sm_span, st>>>(cd);
+        }
         mark(st, "k_span_test");
         k_obf_algebra<TIN, D><<<heads, ALG_NT, sm_alg, st>>>(cd);
         mark(st, "k_obf_algebra");
@@ -553,9 +540,7 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
         c.head_base = i * hpc;
         c.tok_off = L.tok_off[i];
         c.nsub_del = L.tc_per ? L.nsub_del[i] : 0;
-        c.nsub_keep = L.tc_per ? L.nsub_keep[i] : 0;
         c.sub_base = L.tc_per ? L.sub_base[i] : 0;
-        c.subk_base = L.tc_per ? L.subk_base[i] : 0;
         c.sc_team = L.sc_on ? L.sc_team[i] : 0;
         c.sc_hpr = L.sc_on ? L.sc_hpr[i] : 0;
         c.sc_round_base = L.sc_on ? L.sc_round_base[i] : 0;
@@ -572,11 +557,9 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
     cd.splits = L.splits;
     cd.gram_slots = L.gram_slots;
     cd.tc_per = L.tc_per;
-    cd.tk_per = L.tk_per;
     cd.gram_all = L.tc_per ? 1 : 0;
     cd.u_levels = L.tc_per ? U_LEVELS : 1;
     cd.tc_total_sub = L.tc_total_sub;
-    cd.tk_total_sub = L.tk_total_sub;
     cd.sc_nq = L.sc_on ? L.sc_nq : 0;
     cd.sc_qt = L.sc_on ? L.sc_qt : 1;
     cd.sc_subs = L.sc_subs;

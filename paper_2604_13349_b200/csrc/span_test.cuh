@@ -11,6 +11,10 @@
 // below it by one thread per row, the lower triangle of the trailing matrix by
 // 8x4 register tiles.
 // Result: bit 1 of hflag[head].
+//
+// FROM_ROWS (tuned path: bf16, head_dim 128): G_keep is not read from the workspace but formed here from the
+// first 256 gathered rows of the head (any subset of the retained rows that spans R^d certifies the test), with
+// warp-level mma (bf16 products are exact, fp32 accumulation) while the rows sit in the memory the matrix then takes.
 #pragma once
 
 #include "common.cuh"
@@ -25,7 +29,9 @@ constexpr uint32_t HFLAG_SPAN_FULL = 2u;   // span(V_keep) = R^d
 template <int D>
 constexpr size_t span_smem_bytes() { return (size_t)(D * (D + 1) + 32 * 33 + 32 + D + 64 + 256 + 3) * sizeof(float); }
 
-template <int D>
+constexpr int SPAN_ROWS = 256;          // retained rows that enter G_keep with FROM_ROWS
+
+template <int D, bool FROM_ROWS = false>
 __global__ void __launch_bounds__(ST_NT, 3) k_span_test(const __grid_constant__ CallDev p)
 {
     constexpr int LD = D + 1, NB = 32, L11_LD = NB + 1;
@@ -47,32 +53,113 @@ __global__ void __launch_bounds__(ST_NT, 3) k_span_test(const __grid_constant__ 
         if (tid == 0) p.hflag[g] = 0u;
         return;
     }
-    const int n_part = gram_partial_count(p, c, lh, 1);
-    const float *parts = p.gram_k + (size_t)g * p.gram_slots * D * D;
-    for (int e0 = tid; e0 < D * D / 4; e0 += 4 * ST_NT) {
-        float4 acc[4];
+    if constexpr (FROM_ROWS) {
+        static_assert(D == 128, "the row-based Gram matrix is written for head_dim 128");
+        static_assert(SPAN_ROWS * D * 2 <= D * (D + 1) * 4, "the rows are staged in the matrix's memory");
+        // X: the first rows of the head's compacted values, [SPAN_ROWS][128] bf16, rows past the end zero; the
+        // 16-byte chunks of a row are permuted by the row number so that 8 x 8 matrix loads hit distinct banks
+        uint8_t *X = reinterpret_cast<uint8_t *>(A);
+        const int n_rows = c.k_eff < SPAN_ROWS ? c.k_eff : SPAN_ROWS;
+        const uint4 *src = reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(c.v_out) + (size_t)lh * c.k_eff * D);
+        // eight 16-byte loads in flight per thread
+#pragma unroll 1
+        for (int i0 = tid; i0 < SPAN_ROWS * 16; i0 += 8 * ST_NT) {
+            uint4 v[8];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int sp = 0; sp < n_part; ++sp) {
-            float4 v[4];
+            for (int u = 0; u < 8; ++u) {
+                const int i = i0 + u * ST_NT, r = i >> 4, ch = i & 15;
+                v[u] = r < n_rows ? __ldg(src + (size_t)r * 16 + ch) : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = i0 + u * ST_NT, r = i >> 4, ch = i & 15;
+                *reinterpret_cast<uint4 *>(X + r * 256 + (((ch & 8) | ((ch ^ r) & 7)) << 4)) = v[u];
+            }
+        }
+        __syncthreads();
+        // G = X^T X: warp w owns rows [16 w, 16 w + 16) of G, in two halves of 64 columns (m16n8k16, A = X^T and
+        // B = X both read with transposing 8 x 8 loads from the row-major X)
+        const uint32_t xbase = (uint32_t)__cvta_generic_to_shared(X);
+        const int mi = lane >> 3, rr = lane & 7;
+        float acc[2][8][4];
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) acc[hf][nt][e] = 0.f;
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+#pragma unroll 1
+            for (int k0 = 0; k0 < SPAN_ROWS; k0 += 16) {
+                uint32_t a[4];
+                {
+                    // matrices: (tokens k0.., dims i0..), (tokens k0.., dims i0 + 8..), (tokens k0 + 8.., dims i0..), (k0 + 8.., i0 + 8..)
+                    const int tok = k0 + (mi >> 1) * 8 + rr, chn = (16 * warp + (mi & 1) * 8) >> 3;
+                    const uint32_t addr = xbase + tok * 256 + (((chn & 8) | ((chn ^ tok) & 7)) << 4);
+                    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                                 : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3]) : "r"(addr));
+                }
+#pragma unroll
+                for (int np = 0; np < 4; ++np) {
+                    // two 8-column tiles at once: (tokens k0.., dims n0..), (k0 + 8.., n0..), (k0.., n0 + 8..), (k0 + 8.., n0 + 8..)
+                    const int n0 = hf * 64 + np * 16;
+                    if (n0 > 16 * warp) continue;              // right of the diagonal: only the lower triangle is ever read
+                    const int tok = k0 + (mi & 1) * 8 + rr, chn = (n0 + (mi >> 1) * 8) >> 3;
+                    const uint32_t addr = xbase + tok * 256 + (((chn & 8) | ((chn ^ tok) & 7)) << 4);
+                    uint32_t b[4];
+                    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                                 : "=r"(b[0]), "=r"(b[1]), "=r"(b[2]), "=r"(b[3]) : "r"(addr));
+#pragma unroll
+                    for (int t2 = 0; t2 < 2; ++t2) {
+                        float *d4 = acc[hf][2 * np + t2];
+                        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                     : "+f"(d4[0]), "+f"(d4[1]), "+f"(d4[2]), "+f"(d4[3])
+                                     : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[2 * t2]), "r"(b[2 * t2 + 1]));
+                    }
+                }
+            }
+        }
+        __syncthreads();                                   // every warp is done reading X: the matrix takes its place
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) {
+                const int row = 16 * warp + (lane >> 2), col = hf * 64 + nt * 8 + 2 * (lane & 3);
+                if (hf * 64 + (nt >> 1) * 16 > 16 * warp) continue;
+                A[row * LD + col] = acc[hf][nt][0];
+                A[row * LD + col + 1] = acc[hf][nt][1];
+                A[(row + 8) * LD + col] = acc[hf][nt][2];
+                A[(row + 8) * LD + col + 1] = acc[hf][nt][3];
+            }
+    } else {
+        const int n_part = gram_partial_count(p, c, lh);           // shape-generic path: one per token split
+        const float *parts = p.gram_k + (size_t)g * p.gram_slots * D * D;
+        for (int e0 = tid; e0 < D * D / 4; e0 += 4 * ST_NT) {
+            float4 acc[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int sp = 0; sp < n_part; ++sp) {
+                float4 v[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int e4 = e0 + u * ST_NT;
+                    // only the lower triangle is ever read: skip the 4-element groups right of the diagonal
+                    const bool lower = e4 < D * D / 4 && (e4 * 4) % D <= (e4 * 4) / D;
+                    v[u] = lower ? *reinterpret_cast<const float4 *>(parts + (size_t)sp * D * D + e4 * 4)
+                                 : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) { acc[u].x += v[u].x; acc[u].y += v[u].y; acc[u].z += v[u].z; acc[u].w += v[u].w; }
+            }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const int e4 = e0 + u * ST_NT;
-                // only the lower triangle is ever read: skip the 4-element groups right of the diagonal
-                const bool lower = e4 < D * D / 4 && (e4 * 4) % D <= (e4 * 4) / D;
-                v[u] = lower ? *reinterpret_cast<const float4 *>(parts + (size_t)sp * D * D + e4 * 4)
-                             : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) { acc[u].x += v[u].x; acc[u].y += v[u].y; acc[u].z += v[u].z; acc[u].w += v[u].w; }
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int e4 = e0 + u * ST_NT;
-            if (e4 < D * D / 4) {
-                const int r = (e4 * 4) / D, cc = (e4 * 4) % D;
-                float *o = A + r * LD + cc;
-                o[0] = acc[u].x; o[1] = acc[u].y; o[2] = acc[u].z; o[3] = acc[u].w;
+                if (e4 < D * D / 4) {
+                    const int r = (e4 * 4) / D, cc = (e4 * 4) % D;
+                    float *o = A + r * LD + cc;
+                    o[0] = acc[u].x; o[1] = acc[u].y; o[2] = acc[u].z; o[3] = acc[u].w;
+                }
             }
         }
     }
