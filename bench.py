@@ -218,7 +218,8 @@ class Bench:
         self.params = P.make_params(w.layers, w.kv_heads, w.q_heads, w.head.head_dim, w.n_obs, w.rank,
                                     P.OBF_F32 if w.dtype == "f32" else P.OBF_BF16, 1e-12,
                                     (P.binding.OBF_FLAG_LAYERWISE if w.layerwise else 0)
-                                    | (P.binding.OBF_FLAG_FAST_PATH if w.fast_path else 0))
+                                    | (P.binding.OBF_FLAG_FAST_PATH if w.fast_path else 0)
+                                    | (P.binding.OBF_FLAG_MERGE if w.merge else 0))
         self.tdt = torch.float32 if w.dtype == "f32" else torch.bfloat16
         self.host_arrays = [synth.gen_cache(w, ci) for ci in range(len(w.caches))]
         self.dev_in, self.caches, self.outs = [], [], []

@@ -86,6 +86,15 @@ typedef enum { OBF_F32 = 0, OBF_BF16 = 1 } obf_dtype_t;
                                       the identity (the paper leaves the start open), instead of the exact
                                       eigenvectors: an approximation whose error depends on the residual's spectrum.
                                       diag: lam_1 / lam_rho are Rayleigh quotients, lam_next is 0                  */
+#define OBF_FLAG_ATTN_INJECT  0x8u /* Attn-inject (App. D.2, alternative designs): the vector delta of Eq. 6 is added in
+                                      proportion to each retained position's attention mass instead of uniformly,
+                                      V*_t = V_t + k_eff * A_t / (A_keep + eps) * delta (the shares average one).
+                                      delta_out and the diagnostics are those of the uniform injection             */
+#define OBF_FLAG_MERGE        0x10u /* cache-merging baseline instead of Orthogonal BackFill (App. E, the comparison
+                                      method): after selection and gather every deleted position is routed to the
+                                      retained position with the most similar key (cosine; ties: lowest position) and
+                                      V*_t = V_t + sum over the j routed to t of A_j / (A_t + eps) V_j.  params->rank is
+                                      ignored; delta_out stays zero                                                */
 #define OBF_FLAG_SINK(n) (((uint32_t)(n) & 0xFFu) << 8)
                                    /* protected sink prefix (App. F of the paper: the compressors protect the first s
                                       indices of the cache; the eligible set of Section 3.2 leaves the sink out): the
@@ -157,6 +166,8 @@ typedef struct {              /* one agent's prompt cache; T and budget may diff
        injection of Eq. 7), which are still written.                                                           */
     int8_t *k_q8_out, *v_q8_out;
     float *k_scale_out, *v_scale_out;
+    int32_t *assign_out;      /* optional device [layers, kv_heads, T], or NULL; with OBF_FLAG_MERGE: the slot
+                                 (0 .. k_eff-1) every deleted position was routed to, -1 for retained positions   */
 } obf_cache_t;
 
 /*

@@ -87,6 +87,12 @@ def lib():
         _lib.obf_oracle_compress_layerwise.restype = ci
         _lib.obf_oracle_backfill.argtypes = [fp, fp, dp, ci, ci, ci, ci, ctypes.c_double, ip, dp, dp, dp, ctypes.POINTER(Diag)]
         _lib.obf_oracle_backfill.restype = ci
+        _lib.obf_oracle_merge_head.argtypes = [fp, fp, fp, ci, ci, ci, ci, ctypes.c_double, ci, ip, dp, dp, dp, ip, dp]
+        _lib.obf_oracle_merge_head.restype = ci
+        _lib.obf_oracle_merge_given.argtypes = [fp, dp, ip, ci, ip, ci, ci, ctypes.c_double, dp]
+        _lib.obf_oracle_merge_given.restype = None
+        _lib.obf_oracle_attn_inject.argtypes = [fp, dp, ip, ci, ci, dp, ctypes.c_double, dp]
+        _lib.obf_oracle_attn_inject.restype = None
         _lib.obf_oracle_quantize_rows.argtypes = [fp, ci, ci, ctypes.POINTER(ctypes.c_int8), fp]
         _lib.obf_oracle_quantize_rows.restype = None
         _lib.obf_oracle_num_threads.argtypes = []
@@ -240,6 +246,46 @@ def backfill(K, V, A, idx, rank: int, eps: float = 1e-12) -> Dict[str, object]:
     lib().obf_oracle_backfill(_p(K, ctypes.c_float), _p(V, ctypes.c_float), _p(A, cd), T, d, k, rank, eps,
                               _p(idx, ctypes.c_int32), _p(K_out, cd), _p(V_out, cd), _p(delta, cd), ctypes.byref(dg))
     return {"idx": idx, "K_out": K_out[:k], "V_out": V_out[:k], "A": A, "delta": delta, "diag": dg.asdict()}
+
+
+def merge_head(K, V, Q, budget: int, eps: float = 1e-12, n_sink: int = 0) -> Dict[str, object]:
+    """Cache-merging baseline (App. E) on one (layer, KV head): select, route every deleted position to the
+    retained position with the most similar key (cosine), add its value in, weighted by A_j / (A_t + eps).
+    Returns idx, K_out, V_out, A, assign [T] (-1 for retained positions), margin [T]."""
+    K, V, Q = _f32(K), _f32(V), _f32(Q)
+    T, d = K.shape
+    k = k_eff(T, budget, n_sink)
+    idx = np.empty(max(k, 1), dtype=np.int32)
+    K_out = np.zeros((max(k, 1), d)); V_out = np.zeros((max(k, 1), d))
+    A = np.empty(T); assign = np.empty(T, dtype=np.int32); margin = np.empty(T)
+    cd = ctypes.c_double
+    k2 = lib().obf_oracle_merge_head(_p(K, ctypes.c_float), _p(V, ctypes.c_float), _p(Q, ctypes.c_float), T, d, Q.shape[0],
+                                     budget, eps, n_sink, _p(idx, ctypes.c_int32), _p(K_out, cd), _p(V_out, cd), _p(A, cd),
+                                     _p(assign, ctypes.c_int32), _p(margin, cd))
+    assert k2 == k
+    return {"idx": idx[:k].copy(), "K_out": K_out[:k], "V_out": V_out[:k], "A": A, "assign": assign, "margin": margin}
+
+
+def merge_given(V, A, idx, assign, eps: float = 1e-12) -> np.ndarray:
+    """Step (iii) of the cache-merging baseline for a given routing."""
+    V, A = _f32(V), _f64(A)
+    idx = np.ascontiguousarray(idx, dtype=np.int32); assign = np.ascontiguousarray(assign, dtype=np.int32)
+    T, d = V.shape
+    out = np.zeros((max(len(idx), 1), d))
+    lib().obf_oracle_merge_given(_p(V, ctypes.c_float), _p(A, ctypes.c_double), _p(idx, ctypes.c_int32), len(idx),
+                                 _p(assign, ctypes.c_int32), T, d, eps, _p(out, ctypes.c_double))
+    return out[:len(idx)]
+
+
+def attn_inject(V, A, idx, delta, eps: float = 1e-12) -> np.ndarray:
+    """Attn-inject (App. D.2): V_out [k, d] = V[idx] + k * A[idx] / (sum A[idx] + eps) * delta."""
+    V, A, delta = _f32(V), _f64(A), _f64(delta)
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    k, d = idx.shape[0], V.shape[1]
+    out = np.zeros((max(k, 1), d))
+    lib().obf_oracle_attn_inject(_p(V, ctypes.c_float), _p(A, ctypes.c_double), _p(idx, ctypes.c_int32), k, d,
+                                 _p(delta, ctypes.c_double), eps, _p(out, ctypes.c_double))
+    return out[:k]
 
 
 def quantize_rows(X):

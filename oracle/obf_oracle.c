@@ -31,6 +31,11 @@
  *               form, codimension-1 closed form, hand-worked planted example
  *   scaling     pinned: single-query identity from the error-bound appendix,
  *               hand-worked planted example
+ *   merging     pinned: library cosine / argmax statement (numpy), every deleted
+ *               position routed exactly once, mass-weighted value sums conserved,
+ *               a duplicate of a retained key is routed to it
+ *   attn-inject pinned: equal masses give the uniform injection, the shares add up
+ *               to the number of retained positions, library statement
  *   int8 relay  pinned: round-trip error at most half a step per element, the
  *               largest element of a row maps to +-127, library rounding
  *               (numpy rint in float32), zero rows
@@ -698,6 +703,97 @@ int obf_oracle_backfill(const float *K, const float *V, const double *A, int T, 
 {
     return backfill_given_selection(K, V, A, T, d, k, rank, eps, idx, 0.0, -1.0, K_out, V_out, delta_out,
                                     NULL, NULL, NULL, NULL, diag, 0);
+}
+
+/*
+ * Attn-inject (App. D.2, alternative designs): the back-fill vector delta of Eq. 6 is not added uniformly but in
+ * proportion to each retained position's attention mass,
+ *   V*_t = V_t + B * w_t * delta,   w_t = A_t / (sum over retained s of A_s + eps),   B = number of retained positions,
+ * so that the shares average one.  V [T, d], A [T], idx [k] ascending, delta [d] (the vector obf_oracle_head returns);
+ * V_out [k, d].
+ */
+void obf_oracle_attn_inject(const float *V, const double *A, const int32_t *idx, int k, int d, const double *delta,
+                            double eps, double *V_out)
+{
+    double a_keep = 0.0;
+    for (int r = 0; r < k; ++r) a_keep += A[idx[r]];
+    for (int r = 0; r < k; ++r) {
+        const double w = (double)k * A[idx[r]] / (a_keep + eps);
+        for (int c = 0; c < d; ++c) V_out[(size_t)r * d + c] = (double)V[(size_t)idx[r] * d + c] + w * delta[c];
+    }
+}
+
+/* ------------------------------------------------------------------ */
+/* Cache-merging baseline (App. E)                                      */
+/* ------------------------------------------------------------------ */
+/*
+ * The comparison method of App. E on one (layer, KV head): (i) the same attention selector picks the retained
+ * positions; (ii) every deleted position j is routed to the retained position whose key has the largest cosine
+ * similarity with K_j (ties: the lowest position; a key of zero norm has similarity 0 with everything);
+ * (iii) V*_t = V_t + sum over the j routed to t of A_j / (A_t + eps) * V_j; keys unchanged.
+ * Outputs: idx [k], K_out, V_out [k, d], A_out [T] (may be NULL), assign [T] (slot 0..k-1 a deleted position is
+ * routed to, -1 for retained positions; may be NULL), margin [T] (best minus second-best similarity of a deleted
+ * position, +inf with a single retained position or for retained positions; may be NULL).  Returns k.
+ */
+int obf_oracle_merge_head(const float *K, const float *V, const float *Q, int T, int d, int n_q, int budget, double eps,
+                          int n_sink, int32_t *idx, double *K_out, double *V_out, double *A_out, int32_t *assign,
+                          double *margin)
+{
+    double *A = (double *)malloc((size_t)T * sizeof(double));
+    obf_oracle_scores(K, Q, T, d, n_q, A);
+    if (A_out) memcpy(A_out, A, (size_t)T * sizeof(double));
+    double kth = 0.0, next = -1.0;
+    const int k = obf_oracle_topk_sink(A, T, budget, n_sink, idx, &kth, &next);
+    char *keep = (char *)calloc((size_t)T, 1);
+    double *norm = (double *)malloc((size_t)T * sizeof(double));
+    for (int j = 0; j < T; ++j) {
+        double s = 0.0;
+        for (int c = 0; c < d; ++c) s += (double)K[(size_t)j * d + c] * (double)K[(size_t)j * d + c];
+        norm[j] = sqrt(s);
+    }
+    for (int r = 0; r < k; ++r) {
+        keep[idx[r]] = 1;
+        for (int c = 0; c < d; ++c) {
+            K_out[(size_t)r * d + c] = (double)K[(size_t)idx[r] * d + c];
+            V_out[(size_t)r * d + c] = (double)V[(size_t)idx[r] * d + c];
+        }
+    }
+    for (int j = 0; j < T; ++j) {
+        if (assign) assign[j] = -1;
+        if (margin) margin[j] = INFINITY;
+        if (keep[j]) continue;
+        int best_r = 0;
+        double best = -INFINITY, second = -INFINITY;
+        for (int r = 0; r < k; ++r) {
+            const int t = idx[r];
+            double dot = 0.0;
+            for (int c = 0; c < d; ++c) dot += (double)K[(size_t)j * d + c] * (double)K[(size_t)t * d + c];
+            const double den = norm[j] * norm[t];
+            const double cs = den > 0.0 ? dot / den : 0.0;
+            if (cs > best) { second = best; best = cs; best_r = r; }
+            else if (cs > second) second = cs;
+        }
+        if (assign) assign[j] = best_r;
+        if (margin) margin[j] = k > 1 ? best - second : INFINITY;
+        const double w = A[j] / (A[idx[best_r]] + eps);
+        for (int c = 0; c < d; ++c) V_out[(size_t)best_r * d + c] += w * (double)V[(size_t)j * d + c];
+    }
+    free(norm); free(keep); free(A);
+    return k;
+}
+
+/* Step (iii) alone for a given routing (assign as above): for checking a result whose routing differs from this
+ * oracle's where two similarities are closer than the arithmetic can tell apart. */
+void obf_oracle_merge_given(const float *V, const double *A, const int32_t *idx, int k, const int32_t *assign,
+                            int T, int d, double eps, double *V_out)
+{
+    for (int r = 0; r < k; ++r)
+        for (int c = 0; c < d; ++c) V_out[(size_t)r * d + c] = (double)V[(size_t)idx[r] * d + c];
+    for (int j = 0; j < T; ++j) {
+        if (assign[j] < 0) continue;
+        const double w = A[j] / (A[idx[assign[j]]] + eps);
+        for (int c = 0; c < d; ++c) V_out[(size_t)assign[j] * d + c] += w * (double)V[(size_t)j * d + c];
+    }
 }
 
 /* ------------------------------------------------------------------ */

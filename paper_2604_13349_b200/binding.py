@@ -35,6 +35,8 @@ OBF_DEV_SPAN_FULL = 0x200
 OBF_FLAG_GENERIC_PATH = 0x1
 OBF_FLAG_LAYERWISE = 0x2        # one retained set per layer (masses summed over its KV heads)
 OBF_FLAG_FAST_PATH = 0x4        # three Gram subspace iterations instead of the exact eigenvectors
+OBF_FLAG_ATTN_INJECT = 0x8      # the back-fill shared out by attention mass instead of uniformly (App. D.2)
+OBF_FLAG_MERGE = 0x10           # cache-merging baseline instead of Orthogonal BackFill (App. E)
 OBF_FLAG_TEST_WAIT_EXPIRES = 0x10000   # test hook: the score kernel's wait for a head's normalisers runs out
 
 
@@ -81,7 +83,7 @@ class ObfCache(ctypes.Structure):
                 ("k_out", ctypes.c_void_p), ("v_out", ctypes.c_void_p), ("idx_out", ctypes.c_void_p),
                 ("diag_out", ctypes.c_void_p), ("scores_out", ctypes.c_void_p), ("delta_out", ctypes.c_void_p),
                 ("lse_extra", ctypes.c_void_p), ("k_q8_out", ctypes.c_void_p), ("v_q8_out", ctypes.c_void_p),
-                ("k_scale_out", ctypes.c_void_p), ("v_scale_out", ctypes.c_void_p)]
+                ("k_scale_out", ctypes.c_void_p), ("v_scale_out", ctypes.c_void_p), ("assign_out", ctypes.c_void_p)]
 
 
 class ObfError(RuntimeError):
@@ -154,13 +156,13 @@ def _ptr(t) -> Optional[int]:
 
 
 def make_cache(k, v, q_obs, T: int, budget: int, k_out, v_out, idx_out, diag_out=None,
-               scores_out=None, delta_out=None, lse_extra=None, q8=None) -> ObfCache:
+               scores_out=None, delta_out=None, lse_extra=None, q8=None, assign_out=None) -> ObfCache:
     """Tensors (device or, for the host entry point, pinned/pageable CPU) or raw addresses.
     q8: (k_q8_out, v_q8_out, k_scale_out, v_scale_out) for the int8 copy of the relay, or None."""
     q8 = q8 or (None, None, None, None)
     return ObfCache(_ptr(k), _ptr(v), _ptr(q_obs), int(T), int(budget), _ptr(k_out), _ptr(v_out),
                     _ptr(idx_out), _ptr(diag_out), _ptr(scores_out), _ptr(delta_out), _ptr(lse_extra),
-                    _ptr(q8[0]), _ptr(q8[1]), _ptr(q8[2]), _ptr(q8[3]))
+                    _ptr(q8[0]), _ptr(q8[1]), _ptr(q8[2]), _ptr(q8[3]), _ptr(assign_out))
 
 
 def _carray(caches: Sequence[ObfCache]):
@@ -275,7 +277,7 @@ def parse_diag(diag_bytes: torch.Tensor) -> List[Dict[str, float]]:
 
 def compress_caches(params: ObfParams, caches_in: Sequence[Dict[str, object]], *, evict: bool = False,
                     want_scores: bool = False, want_delta: bool = True, want_diag: bool = True,
-                    want_int8: bool = False,
+                    want_int8: bool = False, want_assign: bool = False,
                     stream=None, workspace: Optional[torch.Tensor] = None) -> List[Dict[str, object]]:
     """Compress a batch of device caches.
 
@@ -311,9 +313,10 @@ def compress_caches(params: ObfParams, caches_in: Sequence[Dict[str, object]], *
             o["K_scale"] = torch.empty((params.layers, params.kv_heads, ke), dtype=torch.float32, device=dev)
             o["V_scale"] = torch.empty_like(o["K_scale"])
             q8 = (o["K_q8"], o["V_q8"], o["K_scale"], o["V_scale"])
+        o["assign"] = torch.empty((params.layers, params.kv_heads, T), dtype=torch.int32, device=dev) if want_assign else None
         outs.append(o)
         cs.append(make_cache(K, V, Q, T, ci["budget"], o["K_out"], o["V_out"], o["idx"], o["diag"],
-                             o["scores"], o["delta"], ci.get("lse_extra"), q8))
+                             o["scores"], o["delta"], ci.get("lse_extra"), q8, o["assign"]))
     nb = obf_workspace_bytes(params, cs)
     if workspace is None or workspace.numel() * workspace.element_size() < nb:
         workspace = torch.empty(nb, dtype=torch.uint8, device=caches_in[0]["K"].device)

@@ -363,10 +363,15 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
                     if (c.delta_out) c.delta_out[(size_t)lh * D + tid] = dl;
                 }
                 if (tid == 0) p.hflag[g] = HFLAG_INJECT;
-                // Eq. 7: V_out = V_keep + delta on every retained row; the fp32 sum is rounded once
+                // Eq. 7: V_out = V_keep + delta on every retained row; the fp32 sum is rounded once.  Attn-inject
+                // (App. D.2): row t takes k * A_t / (A_keep + eps) times delta instead
                 TIN *rows = reinterpret_cast<TIN *>(c.v_out) + (size_t)lh * k * D;
+                const float *Am = p.scores + c.tok_off + (size_t)lh * T;
+                const int32_t *ix = c.idx_out + (size_t)lh * k;
+                const float share = (float)k / (a_keep + p.eps);
                 for (int e = tid; e < k * D; e += ALG_NT) {
-                    const float sum = to_f32(rows[e]) + vw[e % D];
+                    const float wgt = p.attn_inject ? share * Am[ix[e / D]] : 1.f;
+                    const float sum = fmaf(wgt, vw[e % D], to_f32(rows[e]));
                     if constexpr (sizeof(TIN) == 4) rows[e] = sum;
                     else rows[e] = __float2bfloat16_rn(sum);
                 }

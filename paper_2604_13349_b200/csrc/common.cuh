@@ -21,6 +21,7 @@ struct CacheDev {
     const float *lse_extra;   // out-of-prompt softmax mass per query row (natural log), or null
     int8_t *k_q8, *v_q8;      // optional int8 copy of the compacted relay, with one scale per row
     float *k_scale, *v_scale;
+    int32_t *assign_out;      // optional: routing of the cache-merging baseline
     int32_t T, k_eff;
     int32_t head_base;        // global id of this cache's first (layer, kv head)
     int32_t nsub_del;         // tuned path: 128-token tiles of V per head (ceil(T / 128))
@@ -72,6 +73,8 @@ struct CallDev {
     int32_t layerwise;        // 1: one retained set per layer (masses summed over its KV heads)
     int32_t n_sink;           // protected prefix: the first n_sink positions are retained besides the budget
     int32_t fast_iters;       // > 0: that many Gram subspace iterations instead of the exact eigenvectors
+    int32_t merge;            // 1: cache-merging baseline after the gather (App. E)
+    int32_t attn_inject;      // 1: delta is added in proportion to the retained positions' masses (App. D.2)
     int32_t debug_drop_publish;   // test hook: the score kernel never publishes a head's normalisers, so the wait for them runs out
     unsigned long long wait_limit_ns;   // after this long a device-side wait gives up and reports OBF_DEV_TIMEOUT
     // workspace
@@ -80,6 +83,7 @@ struct CallDev {
     float *scores2;           // tuned score kernel with two query tiles: masses of the second tile, added into `scores` afterwards
     float *lscores;           // layerwise selector: [sum layers*T] masses summed over a layer's KV heads (cache offset tok_off / kv_heads)
     uint8_t *keep;            // [sum heads*T] 1 = retained
+    int32_t *assign;          // [sum heads*T] cache-merging baseline: slot a deleted position is routed to, -1 = retained
     float *stats;             // [heads_total, n_q, 2] softmax row max (log2 domain) and normaliser
     float *sums;              // [heads_total, 4] a_keep, a_del, kth, next
     float *gram_d;            // [heads_total, gram_slots, d, d] partial Gram of the deleted (gram_all: of all) values

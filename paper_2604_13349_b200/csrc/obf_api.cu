@@ -8,6 +8,7 @@
 #include "common.cuh"
 #include "generic.cuh"
 #include "gram_tc.cuh"
+#include "merge.cuh"
 #include "score_tc.cuh"
 #include "span_test.cuh"
 
@@ -68,7 +69,7 @@ static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; 
 
 struct Layout {
     size_t off_status, off_scores, off_keep, off_stats, off_sums, off_lscores, off_scores2;
-    size_t off_gram_d, off_gram_k, off_uvec, off_delta, off_hflag, off_svec;
+    size_t off_gram_d, off_gram_k, off_uvec, off_delta, off_hflag, off_svec, off_assign;
     size_t total;
     int splits;
     int heads_total;
@@ -252,6 +253,8 @@ static void make_layout(const obf_params_t *p, const obf_cache_t *caches, int32_
         L.off_hflag = o;  o = align_up(o + (size_t)L.heads_total * sizeof(uint32_t), 256);
         L.off_svec = o;   o = align_up(o + (size_t)L.heads_total * d * sizeof(float), 256);
     }
+    L.off_assign = o;
+    if (p->flags & OBF_FLAG_MERGE) o = align_up(o + tok * sizeof(int32_t), 256);
     L.total = o;
 }
 
@@ -478,6 +481,17 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
         mark(st, "k_obf_algebra");
     }
     if (side) OBF_CUDA_TRY(cudaStreamWaitEvent(st, side->join_keys, 0));   // the call ends when both streams have
+    if (cd.merge) {
+        // cache-merging baseline (App. E): route the deleted positions, then add their values into the retained rows
+        const size_t sm_mg = merge_smem_bytes<D>();
+        if ((s = set_smem(k_merge_assign<TIN, D>, sm_mg)) != OBF_OK) return s;
+        dim3 ga((T_max + MG_TILE - 1) / MG_TILE, heads);
+        k_merge_assign<TIN, D><<<ga, 256, sm_mg, st>>>(cd);
+        mark(st, "k_merge_assign");
+        dim3 gm((k_max + 7) / 8, heads);
+        k_merge_apply<TIN, D><<<gm, 256, 0, st>>>(cd);
+        mark(st, "k_merge_apply");
+    }
     bool any_q8 = false;
     for (int i = 0; i < cd.n_caches; ++i) any_q8 = any_q8 || cd.c[i].k_q8 != nullptr;
     if (any_q8) {
@@ -535,6 +549,7 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
         c.lse_extra = caches[i].lse_extra;
         c.k_q8 = caches[i].k_q8_out; c.v_q8 = caches[i].v_q8_out;
         c.k_scale = caches[i].k_scale_out; c.v_scale = caches[i].v_scale_out;
+        c.assign_out = caches[i].assign_out;
         c.T = caches[i].T;
         c.k_eff = k_eff_of(p, caches[i]);
         c.head_base = i * hpc;
@@ -577,6 +592,7 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
     cd.layerwise = (p->flags & OBF_FLAG_LAYERWISE) ? 1 : 0;
     cd.n_sink = (int32_t)OBF_FLAG_SINK_OF(p->flags);
     cd.fast_iters = (p->flags & OBF_FLAG_FAST_PATH) ? 3 : 0;
+    cd.attn_inject = (p->flags & OBF_FLAG_ATTN_INJECT) ? 1 : 0;
     cd.alg_rows = k_max < p->head_dim ? k_max : p->head_dim;
     cd.wait_limit_ns = tc::WAIT_LIMIT_NS;
     cd.debug_drop_publish = 0;
@@ -593,6 +609,8 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
     cd.delta = reinterpret_cast<float *>(ws + L.off_delta);
     cd.hflag = reinterpret_cast<uint32_t *>(ws + L.off_hflag);
     cd.svec = reinterpret_cast<float *>(ws + L.off_svec);
+    cd.assign = reinterpret_cast<int32_t *>(ws + L.off_assign);
+    cd.merge = (p->flags & OBF_FLAG_MERGE) ? 1 : 0;
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (!g_keep_status) OBF_CUDA_TRY(cudaMemsetAsync(cd.status, 0, 256, st));     // a slab of a larger job adds to the job's status
@@ -619,7 +637,7 @@ obf_status_t obf_workspace_bytes(const obf_params_t *params, const obf_cache_t *
     obf_status_t s = validate_shapes(params, caches, n_caches, params ? params->rank : 0);
     if (s != OBF_OK) return s;
     Layout L;
-    make_layout(params, caches, n_caches, params->rank, L);
+    make_layout(params, caches, n_caches, (params->flags & OBF_FLAG_MERGE) ? 0 : params->rank, L);
     *bytes = L.total;
     return OBF_OK;
 }
@@ -628,14 +646,17 @@ obf_status_t obf_compress(const obf_params_t *params, const obf_cache_t *caches,
                           void *workspace, size_t workspace_bytes, void *stream)
 {
     if (!params) return OBF_ERR_INVALID_ARG;
-    return run(params, caches, n_caches, params->rank, workspace, workspace_bytes, stream);
+    const int rank = (params->flags & OBF_FLAG_MERGE) ? 0 : params->rank;     // the merging baseline replaces the back-fill
+    return run(params, caches, n_caches, rank, workspace, workspace_bytes, stream);
 }
 
 obf_status_t evict_only(const obf_params_t *params, const obf_cache_t *caches, int32_t n_caches,
                         void *workspace, size_t workspace_bytes, void *stream)
 {
     if (!params) return OBF_ERR_INVALID_ARG;
-    return run(params, caches, n_caches, 0, workspace, workspace_bytes, stream);
+    obf_params_t pe = *params;
+    pe.flags &= ~(uint32_t)OBF_FLAG_MERGE;                 // eviction only: nothing is merged either
+    return run(&pe, caches, n_caches, 0, workspace, workspace_bytes, stream);
 }
 
 struct HostArena {
@@ -721,7 +742,7 @@ obf_status_t obf_compress_host(const obf_params_t *params, const obf_cache_t *ca
     for (int i = 0; i < n_caches; ++i) {
         const obf_cache_t &c = caches[i];
         if (!c.k || !c.v || !c.q_obs || !c.k_out || !c.v_out || !c.idx_out) return OBF_ERR_INVALID_ARG;
-        if (c.k_q8_out || c.v_q8_out || c.k_scale_out || c.v_scale_out) return OBF_ERR_UNSUPPORTED;   // device entry points only
+        if (c.k_q8_out || c.v_q8_out || c.k_scale_out || c.v_scale_out || c.assign_out) return OBF_ERR_UNSUPPORTED;   // device entry points only
     }
     HostArena H;
     host_arena_layout(params, caches, n_caches, H);
@@ -771,7 +792,7 @@ obf_status_t obf_compress_host(const obf_params_t *params, const obf_cache_t *ca
         OBF_CUDA_TRY(cudaEventRecord(hp->in_done[sl], hp->cin));
         OBF_CUDA_TRY(cudaStreamWaitEvent(st, hp->in_done[sl], 0));
         g_keep_status = sl > 0;
-        s = run(&ps, dev, n_caches, ps.rank, base + H.ws, H.ws_bytes, stream);
+        s = run(&ps, dev, n_caches, (ps.flags & OBF_FLAG_MERGE) ? 0 : ps.rank, base + H.ws, H.ws_bytes, stream);
         g_keep_status = false;
         if (s != OBF_OK) { cudaStreamSynchronize(hp->cin); cudaStreamSynchronize(st); cudaStreamSynchronize(hp->cout); return s; }
         OBF_CUDA_TRY(cudaEventRecord(hp->comp_done[sl], st));
@@ -902,6 +923,9 @@ extern "C" obf_status_t evict_only_static(const obf_params_t *params, const obf_
 {
     obf_status_t s = validate_shapes(params, caches, n_caches, 0);
     if (s != OBF_OK) return s;
+    obf_params_t pe = *params;
+    pe.flags &= ~(uint32_t)OBF_FLAG_MERGE;                 // eviction only: nothing is merged either
+    params = &pe;
     Layout L;
     make_layout(params, caches, n_caches, 0, L);
     if (L.total > (size_t)OBF_STATIC_SCRATCH_BYTES) {

@@ -104,6 +104,7 @@ class Workload:
     layerwise: bool = False       # layerwise selector: one retained set per layer
     fast_path: bool = False       # three Gram subspace iterations instead of the exact eigenvectors
     int8_out: bool = False        # the relay leaves as int8 codes with one fp32 scale per row (App. E)
+    merge: bool = False           # cache-merging baseline instead of Orthogonal BackFill (App. E)
 
     @property
     def G(self) -> int:
@@ -257,6 +258,8 @@ def _make_workloads() -> Dict[str, Workload]:
         head=hs_paper, caches=(CacheSpec(T=2048, budget=32),))
     # the paper's own approximation of the subspace (App. H), on the paper-regime shape
     out["pa_fast"] = dataclasses.replace(out["pa"], name="pa_fast", fast_path=True)
+    # the cache-merging comparison method on the paper-regime shape
+    out["pa_merge"] = dataclasses.replace(out["pa"], name="pa_merge", merge=True)
     return out
 
 

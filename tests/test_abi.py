@@ -35,7 +35,7 @@ def test_header_functions_are_all_exported(lib):
 def test_struct_sizes_match_the_header():
     assert ctypes.sizeof(binding.ObfParams) == 36
     assert ctypes.sizeof(binding.ObfDiag) == 60
-    assert ctypes.sizeof(binding.ObfCache) == 120
+    assert ctypes.sizeof(binding.ObfCache) == 128
 
 
 def test_status_strings(lib):

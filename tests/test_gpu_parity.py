@@ -649,6 +649,111 @@ def test_out_of_prompt_softmax_mass(dtype, d, G, n_obs, caches, flags):
 
 
 # ---------------------------------------------------------------------------
+# Attn-inject (App. D.2): the back-fill shared out by attention mass
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype,d,caches", [("f32", 64, ((200, 12), (90, 9))), ("bf16", 128, ((300, 20), (1024, 32)))])
+def test_attn_inject_shares_the_backfill_by_attention_mass(dtype, d, caches):
+    w = small("attn", layers=2, kv_heads=2, G=2, n_obs=6, d=d, dtype=dtype, rank=2, caches=caches, seed=97)
+    arrays = [synth.gen_cache(w, ci) for ci in range(len(w.caches))]
+    outs, _, st = par.run_gpu(w, arrays, flags=P.binding.OBF_FLAG_ATTN_INJECT)
+    assert st & 0xFF == 0
+    plain, _, _ = par.run_gpu(w, arrays)
+    checked = 0
+    for ci, a in enumerate(arrays):
+        o = outs[ci]
+        # selection, keys and delta itself are those of the uniform injection
+        assert torch.equal(o["idx"], plain[ci]["idx"]) and torch.equal(o["K_out"], plain[ci]["K_out"])
+        assert torch.equal(o["delta"], plain[ci]["delta"])
+        Qv = par.f32_view(a["Q"], dtype).reshape(w.layers, w.kv_heads, w.n_q, d)
+        for l, h in all_heads(w):
+            K, V = par.f32_view(a["K"][l, h], dtype), par.f32_view(a["V"][l, h], dtype)
+            ref = oracle.head(K, V, Qv[l, h], w.caches[ci].budget, w.rank)
+            idx = o["idx"][l, h].cpu().numpy()
+            if not np.array_equal(idx, ref["idx"]) or ref["diag"]["skipped"]:
+                continue
+            dg = ref["diag"]
+            gap = (dg["lam_rho"] - dg["lam_next"]) / dg["lam_1"]
+            if gap < 1e-3:
+                continue
+            expect = oracle.attn_inject(V, ref["A"], idx, ref["delta"])
+            share = len(idx) * ref["A"][idx] / (ref["A"][idx].sum() + 1e-12)
+            dtol = max(2e-5 if dtype == "f32" else 2e-4, 200.0 * par.U32 / gap * dg["alpha"] * dg["rbar_norm"])
+            # the tolerance on delta times the row's share (plus the share's own error: masses to 1e-5), and half a
+            # bf16 ulp of the result on the bf16 path
+            bound = share[:, None] * (dtol + 2e-5 * np.abs(ref["delta"])[None, :]) + 1e-6
+            if dtype == "bf16":
+                bound = bound + 2.0 ** -8 * 1.01 * np.abs(expect)
+            err = np.abs(par.out_to_f32(o["V_out"][l, h]).astype(np.float64) - expect)
+            assert np.all(err <= bound), "cache %d layer %d head %d: max err %.3g" % (ci, l, h, err.max())
+            assert not np.allclose(share, 1.0)                      # the shares do differ from the uniform ones
+            checked += 1
+    assert checked >= 4
+
+
+# ---------------------------------------------------------------------------
+# cache-merging baseline (App. E): deleted values merged into the retained position with the most similar key
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype,d,caches,flags", [
+    ("f32", 64, ((200, 12), (90, 9), (70, 70)), 0),
+    ("bf16", 128, ((300, 20), (1024, 32), (700, 150)), 0),
+    ("bf16", 128, ((512, 28),), P.binding.OBF_FLAG_LAYERWISE)])
+def test_cache_merging_baseline(dtype, d, caches, flags):
+    w = small("merge", layers=2, kv_heads=2, G=2, n_obs=6, d=d, dtype=dtype, rank=2, caches=caches, seed=101)
+    arrays = [synth.gen_cache(w, ci) for ci in range(len(w.caches))]
+    outs, _, st = par.run_gpu(w, arrays, flags=flags | P.binding.OBF_FLAG_MERGE, want_assign=True)
+    assert st & 0xFF == 0
+    ev, _, _ = par.run_gpu(w, arrays, evict=True, flags=flags)
+    bits = np.int16 if dtype == "bf16" else np.int32
+    near_ties = flips = 0
+    for ci, a in enumerate(arrays):
+        o = outs[ci]
+        assert torch.equal(o["idx"], ev[ci]["idx"]) and torch.equal(o["K_out"], ev[ci]["K_out"])    # selection and keys: plain eviction
+        assert torch.all(o["delta"] == 0)
+        Qv = par.f32_view(a["Q"], dtype).reshape(w.layers, w.kv_heads, w.n_q, d)
+        for l in range(w.layers):
+            lay = None
+            if flags & P.binding.OBF_FLAG_LAYERWISE:
+                lay = oracle.layer(par.f32_view(a["K"][l], dtype), par.f32_view(a["V"][l], dtype), Qv[l], w.caches[ci].budget, 0)
+            for h in range(w.kv_heads):
+                K, V = par.f32_view(a["K"][l, h], dtype), par.f32_view(a["V"][l, h], dtype)
+                ref = oracle.merge_head(K, V, Qv[l, h], w.caches[ci].budget)
+                idx = o["idx"][l, h].cpu().numpy()
+                g_assign = o["assign"][l, h].cpu().numpy()
+                if lay is not None:
+                    assert np.array_equal(idx, lay["idx"][h])
+                elif not np.array_equal(idx, ref["idx"]):
+                    continue                                        # a tie inside the selection band
+                T = K.shape[0]
+                keep = np.zeros(T, bool); keep[idx] = True
+                assert np.all(g_assign[keep] == -1) and np.all((g_assign[~keep] >= 0) & (g_assign[~keep] < len(idx)))
+                A = lay["A"][h] if lay is not None else ref["A"]
+                if lay is None:
+                    # routing: equal to the oracle's wherever the two best similarities are further apart than fp32
+                    # can blur (1e-5); elsewhere the GPU's choice must be one of the near-best
+                    clear = ref["margin"] > 1e-5
+                    assert np.array_equal(g_assign[clear & ~keep], ref["assign"][clear & ~keep])
+                    near_ties += int((~clear & ~keep).sum())
+                    flips += int((g_assign != ref["assign"]).sum())
+                    Kd = K.astype(np.float64); Kn = Kd / np.maximum(np.linalg.norm(Kd, axis=1, keepdims=True), 1e-300)
+                    for j in np.flatnonzero(g_assign != ref["assign"]):
+                        cs = Kn[idx] @ Kn[j]
+                        assert cs[g_assign[j]] >= cs.max() - 1e-5
+                # merged values: the oracle's step (iii) on the routing the GPU took
+                expect = oracle.merge_given(V, A, idx, g_assign)
+                absum = np.abs(V[idx].astype(np.float64))
+                for j in np.flatnonzero(~keep):
+                    absum[g_assign[j]] += A[j] / (A[idx[g_assign[j]]] + 1e-12) * np.abs(V[j].astype(np.float64))
+                # fp32 accumulation of the weighted sum (weights carry the masses' 1e-5) and one rounding of the result
+                bound = 4e-5 * absum + 1e-6
+                if dtype == "bf16":
+                    bound = bound + 2.0 ** -8 * 1.01 * np.abs(expect)
+                err = np.abs(par.out_to_f32(o["V_out"][l, h]).astype(np.float64) - expect)
+                assert np.all(err <= bound), "cache %d layer %d head %d: merged values off by %.3g" % (ci, l, h, err.max())
+                assert np.array_equal(par.out_bits(o["K_out"][l, h]), a["K"][l, h].view(bits)[idx])
+    print("\n[merge] near-tie routings %d, of which the GPU chose another near-best slot %d" % (near_ties, flips))
+
+
+# ---------------------------------------------------------------------------
 # int8 copy of the compacted relay (post-hoc quantisation stacked on the compression, App. E)
 # ---------------------------------------------------------------------------
 @pytest.mark.parametrize("dtype,d,caches,flags", [

@@ -682,3 +682,66 @@ def test_backfill_for_given_positions_is_the_head_result_on_its_own_positions():
     np.testing.assert_array_equal(b2["K_out"], K[idx2].astype(np.float64))
     Vk = V[idx2].astype(np.float64)
     assert np.abs(Vk @ b2["delta"]).max() <= 1e-10 * np.linalg.norm(Vk, 2) * max(np.linalg.norm(b2["delta"]), 1e-300)
+
+
+# --------------------------------------------------------------------------
+# Attn-inject (App. D.2): the back-fill shared out by attention mass
+# --------------------------------------------------------------------------
+def test_attn_inject_shares_add_up_and_equal_masses_give_the_uniform_injection():
+    g = np.random.default_rng(6)
+    V = g.standard_normal((40, 16)).astype(np.float32)
+    delta = g.standard_normal(16)
+    idx = np.array([1, 5, 6, 20, 33], np.int32)
+    A = g.uniform(0.1, 2.0, 40)
+    out = oracle.attn_inject(V, A, idx, delta)
+    ref = V[idx].astype(np.float64) + (5 * A[idx] / (A[idx].sum() + 1e-12))[:, None] * delta[None, :]
+    np.testing.assert_allclose(out, ref, rtol=1e-14, atol=1e-15)
+    # the shares average one: the mean injected vector is delta
+    np.testing.assert_allclose((out - V[idx]).mean(axis=0), delta, rtol=1e-10)
+    A[idx] = 0.7
+    np.testing.assert_allclose(oracle.attn_inject(V, A, idx, delta), V[idx] + delta[None, :], rtol=1e-11, atol=1e-12)
+
+
+# --------------------------------------------------------------------------
+# cache-merging baseline (App. E)
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("seed", range(3))
+def test_merge_matches_a_library_statement(seed):
+    K, V, Q = rand_head(30 + seed, 120, 32, 6, heavy=3)
+    m = oracle.merge_head(K, V, Q, 9)
+    A = oracle.scores(K, Q)
+    idx = oracle.topk(A, 9)[0]
+    assert np.array_equal(m["idx"], idx)
+    Kd = K.astype(np.float64)
+    Kn = Kd / np.linalg.norm(Kd, axis=1, keepdims=True)
+    cos = Kn @ Kn[idx].T                                              # [T, k]
+    route = cos.argmax(axis=1)
+    dele = np.setdiff1d(np.arange(120), idx)
+    assert np.array_equal(m["assign"][dele], route[dele]) and np.all(m["assign"][idx] == -1)
+    srt = np.sort(cos[dele], axis=1)
+    np.testing.assert_allclose(m["margin"][dele], srt[:, -1] - srt[:, -2], atol=1e-14)
+    ref = V[idx].astype(np.float64).copy()
+    for j in dele:
+        ref[route[j]] += A[j] / (A[idx[route[j]]] + 1e-12) * V[j].astype(np.float64)
+    np.testing.assert_allclose(m["V_out"], ref, rtol=1e-12, atol=1e-13)
+    assert np.array_equal(m["K_out"], K[idx].astype(np.float64))
+    np.testing.assert_allclose(oracle.merge_given(V, A, idx, m["assign"]), m["V_out"], rtol=1e-13, atol=1e-14)
+
+
+def test_merge_conserves_the_mass_weighted_values_and_routes_a_duplicate_to_its_twin():
+    K, V, Q = rand_head(41, 80, 16, 5, heavy=2)
+    m0 = oracle.merge_head(K, V, Q, 7)
+    j = int(np.setdiff1d(np.arange(80), m0["idx"])[3])
+    t = int(m0["idx"][2])
+    K[j] = 3.0 * K[t]                                                # same direction as a retained key
+    m = oracle.merge_head(K, V, Q, 7)
+    if j not in m["idx"] and t in m["idx"]:
+        assert m["idx"][m["assign"][j]] == t
+    # sum over retained t of A_t V*_t = sum over all positions of A_j V_j (eps aside): nothing is dropped
+    A, idx = m["A"], m["idx"]
+    lhs = (A[idx][:, None] * m["V_out"]).sum(axis=0)
+    rhs = (A[:, None] * V.astype(np.float64)).sum(axis=0)
+    np.testing.assert_allclose(lhs, rhs, rtol=1e-9, atol=1e-9)
+    # budget >= T: nothing to merge
+    full = oracle.merge_head(K, V, Q, 80)
+    assert np.array_equal(full["V_out"], V.astype(np.float64)) and np.all(full["assign"] == -1)
