@@ -313,8 +313,12 @@ class Bench:
             # the dense algebra (and the span test): no HBM traffic to speak of, fp32 arithmetic in shared memory.
             # Peak: 148 SMs x 128 FMA lanes x 2 flop x SM clock.
             hpc = w.layers * w.kv_heads
-            flops = sum(hpc * algebra_flops(w.head.head_dim, min(c.budget, c.T), w.rank)
-                        for c in w.caches if min(c.budget, c.T) < w.head.head_dim)
+            if dom.startswith("k_merge"):
+                # cache-merging baseline: the similarities of every position with every retained key
+                flops = sum(hpc * 2.0 * c.T * min(c.budget, c.T) * w.head.head_dim for c in w.caches)
+            else:
+                flops = sum(hpc * algebra_flops(w.head.head_dim, min(c.budget, c.T), w.rank)
+                            for c in w.caches if min(c.budget, c.T) < w.head.head_dim)
             clock = sm_mhz or 1965.0
             alu_peak = 148 * 128 * 2 * clock * 1e6 / 1e12
             ach = flops / (phase_acc[dom] * 1e-3) / 1e12

@@ -630,6 +630,9 @@ using namespace obf;
 
 extern "C" {
 
+// The rank a call runs with: the cache-merging baseline replaces the back-fill.
+static inline int effective_rank(const obf_params_t *p) { return (p->flags & OBF_FLAG_MERGE) ? 0 : p->rank; }
+
 obf_status_t obf_workspace_bytes(const obf_params_t *params, const obf_cache_t *caches, int32_t n_caches,
                                  size_t *bytes)
 {
@@ -637,7 +640,7 @@ obf_status_t obf_workspace_bytes(const obf_params_t *params, const obf_cache_t *
     obf_status_t s = validate_shapes(params, caches, n_caches, params ? params->rank : 0);
     if (s != OBF_OK) return s;
     Layout L;
-    make_layout(params, caches, n_caches, (params->flags & OBF_FLAG_MERGE) ? 0 : params->rank, L);
+    make_layout(params, caches, n_caches, effective_rank(params), L);
     *bytes = L.total;
     return OBF_OK;
 }
@@ -646,8 +649,7 @@ obf_status_t obf_compress(const obf_params_t *params, const obf_cache_t *caches,
                           void *workspace, size_t workspace_bytes, void *stream)
 {
     if (!params) return OBF_ERR_INVALID_ARG;
-    const int rank = (params->flags & OBF_FLAG_MERGE) ? 0 : params->rank;     // the merging baseline replaces the back-fill
-    return run(params, caches, n_caches, rank, workspace, workspace_bytes, stream);
+    return run(params, caches, n_caches, effective_rank(params), workspace, workspace_bytes, stream);
 }
 
 obf_status_t evict_only(const obf_params_t *params, const obf_cache_t *caches, int32_t n_caches,
@@ -685,7 +687,7 @@ static void host_arena_layout(const obf_params_t *p, const obf_cache_t *caches, 
         H.lse[i] = o; if (caches[i].lse_extra) o = align_up(o + (size_t)p->layers * p->q_heads * p->n_obs * 4, 256);
     }
     Layout L;
-    make_layout(p, caches, n, p->rank, L);
+    make_layout(p, caches, n, effective_rank(p), L);
     H.ws = o; H.ws_bytes = L.total; o += L.total;
     H.total = o;
 }
@@ -792,7 +794,7 @@ obf_status_t obf_compress_host(const obf_params_t *params, const obf_cache_t *ca
         OBF_CUDA_TRY(cudaEventRecord(hp->in_done[sl], hp->cin));
         OBF_CUDA_TRY(cudaStreamWaitEvent(st, hp->in_done[sl], 0));
         g_keep_status = sl > 0;
-        s = run(&ps, dev, n_caches, (ps.flags & OBF_FLAG_MERGE) ? 0 : ps.rank, base + H.ws, H.ws_bytes, stream);
+        s = run(&ps, dev, n_caches, effective_rank(&ps), base + H.ws, H.ws_bytes, stream);
         g_keep_status = false;
         if (s != OBF_OK) { cudaStreamSynchronize(hp->cin); cudaStreamSynchronize(st); cudaStreamSynchronize(hp->cout); return s; }
         OBF_CUDA_TRY(cudaEventRecord(hp->comp_done[sl], st));
@@ -840,14 +842,14 @@ obf_status_t obf_compress_profiled(const obf_params_t *params, const obf_cache_t
     for (int i = 0; i <= OBF_MAX_PHASES; ++i) OBF_CUDA_TRY(cudaEventCreate(&g_prof.ev[i]));
     // One untimed pass first: while the device works on it the host enqueues the timed pass, so that
     // the events of the timed pass are not separated by host-side launch latency.
-    obf_status_t s = run(params, caches, n_caches, params->rank, workspace, workspace_bytes, stream);
+    obf_status_t s = run(params, caches, n_caches, effective_rank(params), workspace, workspace_bytes, stream);
     if (s != OBF_OK) {
         for (int i = 0; i <= OBF_MAX_PHASES; ++i) cudaEventDestroy(g_prof.ev[i]);
         return s;
     }
     g_prof.n = 0;
     g_prof.active = true;
-    s = run(params, caches, n_caches, params->rank, workspace, workspace_bytes, stream);
+    s = run(params, caches, n_caches, effective_rank(params), workspace, workspace_bytes, stream);
     g_prof.active = false;
     cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
     *n_phases = 0;
