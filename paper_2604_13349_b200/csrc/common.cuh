@@ -65,8 +65,9 @@ struct CallDev {
     int32_t sc_subs;          // 128-key tiles per chunk
     int32_t sc_rounds;        // rounds of the persistent score kernel
     int32_t sc_qt;            // tuned score kernel: 128-row query tiles per head (1 or 2)
-    float *sc_part;           // per (head, chunk, even / odd tiles, query of 128): maximum and normaliser over those keys
-    uint32_t *sc_cnt;         // per (head, query tile): statistics warps of the head's team that have written their pairs
+    float *sc_part;           // per (head, chunk, query of 128): chunk maximum and normaliser
+    float *sc_head;           // per (head, query of 128): one 64-bit word, low = M + log2(Z) over all keys, high = 1 when valid
+    uint32_t *sc_cnt;         // per head: chunks that have published
     float eps;
     int32_t kv_heads;         // KV heads per layer
     int32_t layerwise;        // 1: one retained set per layer (masses summed over its KV heads)
@@ -74,7 +75,7 @@ struct CallDev {
     int32_t fast_iters;       // > 0: that many Gram subspace iterations instead of the exact eigenvectors
     int32_t merge;            // 1: cache-merging baseline after the gather (App. E)
     int32_t attn_inject;      // 1: delta is added in proportion to the retained positions' masses (App. D.2)
-    int32_t debug_drop_publish;   // test hook: the score kernel's statistics warps never count themselves in, so the wait for a head's team runs out
+    int32_t debug_drop_publish;   // test hook: the score kernel never publishes a head's normalisers, so the wait for them runs out
     unsigned long long wait_limit_ns;   // after this long a device-side wait gives up and reports OBF_DEV_TIMEOUT
     // workspace
     uint32_t *status;

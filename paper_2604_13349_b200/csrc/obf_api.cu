@@ -87,7 +87,7 @@ struct Layout {
     int sc_nq, sc_subs, sc_blocks, sc_rounds, sc_qt;
     int sc_team[OBF_MAX_CACHES], sc_hpr[OBF_MAX_CACHES], sc_round_base[OBF_MAX_CACHES];
     size_t sc_part_off[OBF_MAX_CACHES], sc_part_pairs;
-    size_t off_sc_part, off_sc_sync;
+    size_t off_sc_part, off_sc_head, off_sc_sync;
 };
 
 // Streaming multiprocessors of the current device (148 on a B200 when no device can be asked).
@@ -220,7 +220,7 @@ static void make_layout(const obf_params_t *p, const obf_cache_t *caches, int32_
             L.sc_round_base[i] = rounds;
             rounds += (hpc + L.sc_hpr[i] - 1) / L.sc_hpr[i];
             L.sc_part_off[i] = pairs;
-            pairs += (size_t)hpc * L.sc_team[i] * ST_PART * 128;
+            pairs += (size_t)hpc * L.sc_team[i] * 128;
         }
         L.sc_on = fits;
         L.sc_rounds = rounds;
@@ -236,10 +236,11 @@ static void make_layout(const obf_params_t *p, const obf_cache_t *caches, int32_
     if (L.sc_on && L.sc_qt == 2) o = align_up(o + tok * sizeof(float), 256);
     L.off_lscores = o;
     if (p->flags & OBF_FLAG_LAYERWISE) o = align_up(o + tok / p->kv_heads * sizeof(float), 256);
-    L.off_sc_part = L.off_sc_sync = o;
+    L.off_sc_part = L.off_sc_head = L.off_sc_sync = o;
     if (L.sc_on) {
         L.off_sc_part = o; o = align_up(o + L.sc_part_pairs * 2 * sizeof(float), 256);
-        // cleared before every launch
+        // sc_head and sc_cnt are cleared together before every launch
+        L.off_sc_head = o; o = align_up(o + (size_t)L.heads_total * L.sc_qt * 128 * sizeof(unsigned long long), 256);
         L.off_sc_sync = o; o = align_up(o + (size_t)L.heads_total * L.sc_qt * sizeof(uint32_t), 256);
     }
     L.off_gram_d = L.off_gram_k = L.off_uvec = L.off_delta = L.off_hflag = L.off_svec = o;
@@ -347,7 +348,7 @@ static obf_status_t launch_score_tc(const CallDev &cd, const Layout &L, cudaStre
     }
     const size_t smem = ST_SMEM_BYTES;
     OBF_CUDA_TRY(cudaFuncSetAttribute(k_score_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    OBF_CUDA_TRY(cudaMemsetAsync(cd.sc_cnt, 0, (size_t)cd.heads_total * L.sc_qt * sizeof(uint32_t), st));
+    OBF_CUDA_TRY(cudaMemsetAsync(cd.sc_head, 0, (L.off_sc_sync - L.off_sc_head) + (size_t)cd.heads_total * L.sc_qt * sizeof(uint32_t), st));
     // The blocks of a head's team wait for one another, so the whole grid has to be resident at once: a
     // cooperative launch starts only when it is (the grid never exceeds one block per multiprocessor).
     void *args[2] = {const_cast<CallDev *>(&cd), &maps};
@@ -600,6 +601,7 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
         cd.debug_drop_publish = 1;
     }
     cd.sc_part = reinterpret_cast<float *>(ws + L.off_sc_part);
+    cd.sc_head = reinterpret_cast<float *>(ws + L.off_sc_head);
     cd.sc_cnt = reinterpret_cast<uint32_t *>(ws + L.off_sc_sync);
     cd.gram_d = reinterpret_cast<float *>(ws + L.off_gram_d);
     cd.gram_k = reinterpret_cast<float *>(ws + L.off_gram_k);
