@@ -58,7 +58,8 @@ __device__ __forceinline__ int sturm_count(const float *a, const float *b, float
 #pragma unroll 4
     for (int i = 1; i < D; ++i) {
         if (fabsf(q) < pivmin) q = -pivmin;
-        q = a[i] - x - b[i - 1] * b[i - 1] / q;
+        // the quotient need not be rounded correctly: an error of a few ulp moves the count's switching point by as much
+        q = a[i] - x - __fdividef(b[i - 1] * b[i - 1], q);
         cnt += q < 0.f ? 1 : 0;
     }
     return cnt;
@@ -129,6 +130,38 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
 
     uint32_t status = 0u;
     int m = 0;
+    // c = Q x (vc) and x -= Q^T c for a vector x of d floats in shared memory: four threads per basis row / per
+    // channel.  The thread's share of the row is cut so that the 32 lanes of a warp meet 32 different banks (rows are
+    // d + 1 floats apart: lanes of neighbouring rows are one bank apart, the four threads of a row eight).
+    auto q_dot = [&](const float *x, int rows) {
+        const int j = tid >> 2, part = tid & 3;
+        float sacc = 0.f;
+        if (j < rows) {
+            const float *qj = Qb + j * LD;
+#pragma unroll 8
+            for (int e = 0; e < D / 4; ++e) {
+                const int cc = ((e >> 3) << 5) + part * 8 + (e & 7);
+                sacc = fmaf(qj[cc], x[cc], sacc);
+            }
+        }
+        sacc += __shfl_xor_sync(0xffffffffu, sacc, 1);
+        sacc += __shfl_xor_sync(0xffffffffu, sacc, 2);
+        if (part == 0 && j < rows) vc[j] = sacc;
+    };
+    auto q_minus = [&](float *x, int rows) {
+        const int cc = tid >> 2, part = tid & 3;
+        float sacc = 0.f;
+        if (cc < D) {
+            const int n_e = ((rows + 31) >> 5) << 3;
+            for (int e = 0; e < n_e; ++e) {
+                const int j = ((e >> 3) << 5) + part * 8 + (e & 7);
+                if (j < rows) sacc = fmaf(vc[j], Qb[j * LD + cc], sacc);
+            }
+        }
+        sacc += __shfl_xor_sync(0xffffffffu, sacc, 1);
+        sacc += __shfl_xor_sync(0xffffffffu, sacc, 2);
+        if (part == 0 && cc < D) x[cc] -= sacc;
+    };
     float rcr = 0.f, lam1 = 0.f, lam_rho = 0.f, lam_next = 0.f, dnorm = 0.f, revr = 0.f, pc = 0.f;
     int rho = 0;
     bool done = false;
@@ -174,29 +207,9 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
             sq_keep += n0sq;
             const float n0 = sqrtf(n0sq);
             for (int pass = 0; pass < 2; ++pass) {
-                {
-                    const int j = tid >> 2, part = tid & 3;
-                    float s = 0.f;
-                    if (j < m) {
-                        const float *qj = Qb + j * LD + part * (D / 4);
-                        const float *ww = vw + part * (D / 4);
-#pragma unroll 8
-                        for (int e = 0; e < D / 4; ++e) s = fmaf(qj[e], ww[e], s);
-                    }
-                    s += __shfl_xor_sync(0xffffffffu, s, 1);
-                    s += __shfl_xor_sync(0xffffffffu, s, 2);
-                    if (part == 0 && j < m) vc[j] = s;
-                }
+                q_dot(vw, m);
                 __syncthreads();
-                {
-                    const int cc = tid >> 2, part = tid & 3;
-                    float s = 0.f;
-                    if (cc < D)
-                        for (int j = part; j < m; j += 4) s = fmaf(vc[j], Qb[j * LD + cc], s);
-                    s += __shfl_xor_sync(0xffffffffu, s, 1);
-                    s += __shfl_xor_sync(0xffffffffu, s, 2);
-                    if (part == 0 && cc < D) vw[cc] -= s;
-                }
+                q_minus(vw, m);
                 __syncthreads();
             }
             const float w1 = tid < D ? vw[tid] : 0.f;
@@ -240,28 +253,9 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
         __syncthreads();
         // x -> P x = x - Q^T (Q x) for the vector in `x` (d floats in shared memory), in place; vc is scratch
         auto project = [&](float *x) {
-            {
-                const int j = tid >> 2, part = tid & 3;
-                float sacc = 0.f;
-                if (j < m) {
-                    const float *qj = Qb + j * LD + part * (D / 4);
-#pragma unroll 8
-                    for (int e = 0; e < D / 4; ++e) sacc = fmaf(qj[e], x[part * (D / 4) + e], sacc);
-                }
-                sacc += __shfl_xor_sync(0xffffffffu, sacc, 1);
-                sacc += __shfl_xor_sync(0xffffffffu, sacc, 2);
-                if (part == 0 && j < m) vc[j] = sacc;
-            }
+            q_dot(x, m);
             __syncthreads();
-            {
-                const int cc = tid >> 2, part = tid & 3;
-                float sacc = 0.f;
-                if (cc < D)
-                    for (int j = part; j < m; j += 4) sacc = fmaf(vc[j], Qb[j * LD + cc], sacc);
-                sacc += __shfl_xor_sync(0xffffffffu, sacc, 1);
-                sacc += __shfl_xor_sync(0xffffffffu, sacc, 2);
-                if (part == 0 && cc < D) x[cc] -= sacc;
-            }
+            q_minus(x, m);
             __syncthreads();
         };
         if (c.diag) {
@@ -282,9 +276,10 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
         // M = (I - Q^T Q) G (I - Q^T Q) as two rank-m updates: B = Q X (m x d), X -= Q^T B, first on X = G from the
         // left, then on the transposed problem from the right (X is symmetric up to rounding, so "B = Q X^T")
         for (int side = 0; side < 2; ++side) {
-            // B[j][c] = sum_a Q[j][a] X[a][c] (left) or sum_a Q[j][a] X[c][a] (right): a 1 x 4 register tile per thread
+            // B[j][c] = sum_a Q[j][a] X[a][c] (left) or sum_a Q[j][a] X[c][a] (right): a 1 x 4 register tile per thread,
+            // its four columns d / 4 apart so that the lanes of a warp read neighbouring banks
             for (int t = tid; t < m * (D / 4); t += ALG_NT) {
-                const int j = t / (D / 4), c0 = (t % (D / 4)) * 4;
+                const int j = t / (D / 4), c0 = t % (D / 4);
                 float acc[4] = {0.f, 0.f, 0.f, 0.f};
                 const float *qj = Qb + j * LD;
                 if (side == 0) {
@@ -292,24 +287,24 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
                     for (int a = 0; a < D; ++a) {
                         const float qv = qj[a];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) acc[e] = fmaf(qv, B2[a * LD + c0 + e], acc[e]);
+                        for (int e = 0; e < 4; ++e) acc[e] = fmaf(qv, B2[a * LD + c0 + e * (D / 4)], acc[e]);
                     }
                 } else {
 #pragma unroll 4
                     for (int a = 0; a < D; ++a) {
                         const float qv = qj[a];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) acc[e] = fmaf(qv, B2[(c0 + e) * LD + a], acc[e]);
+                        for (int e = 0; e < 4; ++e) acc[e] = fmaf(qv, B2[(c0 + e * (D / 4)) * LD + a], acc[e]);
                     }
                 }
 #pragma unroll
-                for (int e = 0; e < 4; ++e) Bm[j * LD + c0 + e] = acc[e];
+                for (int e = 0; e < 4; ++e) Bm[j * LD + c0 + e * (D / 4)] = acc[e];
             }
             __syncthreads();
             // left: X[a][c] -= sum_j Q[j][a] B[j][c];  right: X[a][c] -= sum_j B[j][a] Q[j][c].  4 x 4 tile per thread
             const float *Lf = side == 0 ? Qb : Bm, *Rf = side == 0 ? Bm : Qb;
             for (int t = tid; t < (D / 4) * (D / 4); t += ALG_NT) {
-                const int a0 = (t / (D / 4)) * 4, c0 = (t % (D / 4)) * 4;
+                const int a0 = (t / (D / 4)) * 4, c0 = t % (D / 4);       // rows a0 .. a0 + 3, columns c0 + e d / 4
                 float acc[4][4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
@@ -318,7 +313,7 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
                 for (int j = 0; j < m; ++j) {
                     float l[4], r[4];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) { l[i] = Lf[j * LD + a0 + i]; r[i] = Rf[j * LD + c0 + i]; }
+                    for (int i = 0; i < 4; ++i) { l[i] = Lf[j * LD + a0 + i]; r[i] = Rf[j * LD + c0 + i * (D / 4)]; }
 #pragma unroll
                     for (int i = 0; i < 4; ++i)
 #pragma unroll
@@ -327,7 +322,7 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) B2[(a0 + i) * LD + c0 + e] -= acc[i][e];
+                    for (int e = 0; e < 4; ++e) B2[(a0 + i) * LD + c0 + e * (D / 4)] -= acc[i][e];
             }
             __syncthreads();
         }
@@ -470,98 +465,121 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
             float *tz = tlam + 16;                                 // [ne][D] eigenvectors
             float *twk = tz + ne * D;                              // [ne][5][D] factors of T - lambda I
             // Householder reduction: reflector k (a unit vector) zeroes column k below the sub-diagonal.  During its step it
-            // sits in vl; afterwards in the part of column k of M that the step has just emptied (rows k + 1 .. d - 1)
+            // sits in one of two vectors (vl, vcs); afterwards in the part of column k of M that the step has emptied
+            // (rows k + 1 .. d - 1).
+            //
+            // Two block barriers per column.  Step k:
+            //   B  p = 2 M v_k on the trailing block (rows and columns > k), four threads per row;
+            //   C  kk = v_k . p and w = p - kk v_k (every warp for itself), then
+            //      - row k + 1 as the update M - v w^T - w v^T leaves it, formed by every warp for itself from the old row:
+            //        its first entry is the next diagonal entry, the rest gives reflector k + 1 (norm, sign) at once, so
+            //        no barrier stands between the update and the next reflector;
+            //      - the update itself on rows and columns > k + 1 (row and column k + 1 are dead from here on; column
+            //        k + 1 takes its reflector a step later);
+            //      - reflector k into column k.
+            // The loop starts at k = -1 with v = 0: that step only forms reflector 0 from row 0.
             const float tiny2 = 1e-20f * trM * trM;
-            // Three block barriers per column: the two reductions of a step (column norm, v . pvec) are taken by
-            // every warp for itself rather than by the block, and w = pvec - (v . pvec) v is formed on the fly.
             constexpr int RPW = (D + ALG_NT / 32 - 1) / (ALG_NT / 32);   // rows a warp handles per sweep
+            constexpr int CPL = (D + 31) / 32;                           // columns per lane
+            if (tid < D) { vl[tid] = 0.f; vcs[tid] = 0.f; vc[tid] = 0.f; }
+            __syncthreads();
 #pragma unroll 1
-            for (int k = 0; k < D - 2; ++k) {
-                float part = 0.f;
-                for (int i = k + 2 + lane; i < D; i += 32) { const float x = B2[i * LD + k]; part = fmaf(x, x, part); }
-                const float below2 = warp_sum(part);               // squares below the sub-diagonal entry
-                const float x0 = B2[(k + 1) * LD + k];
+            for (int k = -1; k < D - 2; ++k) {
+                const float *v = (k & 1) ? vl : vcs;                // v_k; v_{k+1} goes to the other vector
+                float *vnext = (k & 1) ? vcs : vl;
+                if (k >= 0) {                                       // B: p = 2 M v on the trailing block -> vc
+                    const int j = tid >> 2, part = tid & 3;
+                    const bool on = j > k && j < D;
+                    float s0 = 0.f, s1 = 0.f;
+                    if (on) {
+                        const float *row = B2 + j * LD;
+                        // columns from the 32-column group of k + 1 on (v is zero up to k); the four threads of a row
+                        // take eight columns of a group each, which keeps the lanes of a warp on different banks
+#pragma unroll 4
+                        for (int e = ((k + 1) >> 5) << 3; e < D / 4; e += 2) {
+                            const int c0 = ((e >> 3) << 5) + part * 8 + (e & 7);
+                            s0 = fmaf(row[c0], v[c0], s0);
+                            s1 = fmaf(row[c0 + 1], v[c0 + 1], s1);
+                        }
+                    }
+                    float sacc = s0 + s1;
+                    sacc += __shfl_xor_sync(0xffffffffu, sacc, 1);
+                    sacc += __shfl_xor_sync(0xffffffffu, sacc, 2);
+                    if (on && part == 0) vc[j] = 2.f * sacc;
+                    __syncthreads();
+                }
+                // C
+                float kpart = 0.f;
+                for (int cc = k + 1 + lane; cc < D; cc += 32) kpart = fmaf(v[cc], vc[cc], kpart);
+                const float kk = warp_sum(kpart);                   // v . p, the same sum in every warp
+                float vj[CPL], wj[CPL], xj[CPL];
+                const float vr = v[k + 1], wr = vc[k + 1] - kk * vr;     // entries k + 1 of v and w
+                float part2 = 0.f;
+#pragma unroll
+                for (int cI = 0; cI < CPL; ++cI) {
+                    const int j = k + 1 + lane + 32 * cI;
+                    vj[cI] = j < D ? v[j] : 0.f;
+                    wj[cI] = j < D ? vc[j] - kk * vj[cI] : 0.f;
+                    // row k + 1 after the update (the same expression as the update below)
+                    xj[cI] = j < D ? B2[(k + 1) * LD + j] - (vr * wj[cI] + wr * vj[cI]) : 0.f;
+                    if (j >= k + 3) part2 = fmaf(xj[cI], xj[cI], part2);
+                }
+                const float below2 = warp_sum(part2);              // squares right of the super-diagonal entry
+                const float dg = __shfl_sync(0xffffffffu, xj[0], 0);    // entry (k + 1, k + 1)
+                const float x0 = __shfl_sync(0xffffffffu, xj[0], 1);    // entry (k + 1, k + 2)
                 const float nrm2 = below2 + x0 * x0;
                 const float nrm = sqrtf(nrm2);
                 const float al = x0 >= 0.f ? -nrm : nrm;
                 const float vn2 = 2.f * nrm * (nrm + fabsf(x0));   // |x - al e_0|^2
-                const bool skip = !(below2 > tiny2) || !(vn2 > 0.f);   // nothing below the sub-diagonal
-                if (tid < D) {
-                    float v = 0.f;
-                    if (!skip && tid > k) v = (tid == k + 1 ? x0 - al : B2[tid * LD + k]) * rsqrtf(vn2);
-                    vl[tid] = v;
-                }
-                if (tid == 0) { ta[k] = B2[k * LD + k]; tb[k] = skip ? x0 : al; }
-                __syncthreads();
-                // every warp has read column k by now: it takes the reflector (zeros when there is none)
-                if (tid > k && tid < D) B2[tid * LD + k] = vl[tid];
-                if (skip) { __syncthreads(); continue; }
-                const float *v = vl;
-                {                                                   // pvec = 2 M v on the trailing block -> vc
-                    float acc[RPW];
-#pragma unroll
-                    for (int r = 0; r < RPW; ++r) acc[r] = 0.f;
-                    // rows of this warp inside the trailing block (the same for all its lanes: real branches below)
-                    const int nr = (D - (k + 1 + warp) + ALG_NT / 32 - 1) / (ALG_NT / 32);
-                    for (int cc = k + 1 + lane; cc < D; cc += 32) {
-                        const float vcc = v[cc];
-#pragma unroll
-                        for (int r = 0; r < RPW; ++r) {
-                            if (r >= nr) break;
-                            acc[r] = fmaf(B2[(k + 1 + warp + r * (ALG_NT / 32)) * LD + cc], vcc, acc[r]);
-                        }
-                    }
-#pragma unroll
-                    for (int r = 0; r < RPW; ++r) {
-                        if (r >= nr) break;
-#pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) acc[r] += __shfl_xor_sync(0xffffffffu, acc[r], o);
-                        if (lane == 0) vc[k + 1 + warp + r * (ALG_NT / 32)] = 2.f * acc[r];
-                    }
-                }
-                __syncthreads();
-                float kpart = 0.f;
-                for (int cc = k + 1 + lane; cc < D; cc += 32) kpart = fmaf(v[cc], vc[cc], kpart);
-                const float kk = warp_sum(kpart);                   // v . pvec, the same sum in every warp
-                // M <- H M H = M - v w^T - w v^T with w = pvec - kk v, on the trailing block
-                // (all loads of a thread's elements are issued before the first store: the loop bodies are short)
-                {
-                    constexpr int CPL = (D + 31) / 32;             // columns per lane
-                    float vj[CPL], wj[CPL];
+                const bool skip = !(below2 > tiny2) || !(vn2 > 0.f);   // nothing beyond the super-diagonal
+                if (warp == 0) {
+                    const float rs = skip ? 0.f : rsqrtf(vn2);
 #pragma unroll
                     for (int cI = 0; cI < CPL; ++cI) {
                         const int j = k + 1 + lane + 32 * cI;
-                        vj[cI] = j < D ? v[j] : 0.f;
-                        wj[cI] = j < D ? vc[j] - kk * vj[cI] : 0.f;
+                        if (j < D) vnext[j] = j == k + 1 ? 0.f : (j == k + 2 ? x0 - al : xj[cI]) * rs;
                     }
-                    const int nr = (D - (k + 1 + warp) + ALG_NT / 32 - 1) / (ALG_NT / 32);   // rows of this warp in the block
-                    const int nc = (D - (k + 1) + 31) / 32;                                  // 32-column groups in the block
+                    if (lane == 0) {
+                        if (k >= 0) vnext[k] = 0.f;
+                        ta[k + 1] = dg;
+                        tb[k + 1] = skip ? x0 : al;
+                    }
+                }
+                if (k >= 0) {
+                    // M <- H M H = M - v w^T - w v^T on rows and columns > k + 1; a warp's rows are read before the first
+                    // is written back (the compiler cannot tell that they do not overlap), four at a time
 #pragma unroll
-                    for (int r = 0; r < RPW; ++r) {
-                        if (r >= nr) break;
-                        const int i = k + 1 + warp + r * (ALG_NT / 32);
-                        const float vi = v[i], wi = vc[i] - kk * vi;
-                        float m_[CPL];
+                    for (int r0 = 0; r0 < RPW; r0 += 4) {
+                        float m_[4][CPL], vi[4], wi[4];
 #pragma unroll
-                        for (int cI = 0; cI < CPL; ++cI) {
-                            if (cI >= nc) break;
-                            const int j = k + 1 + lane + 32 * cI;
-                            m_[cI] = j < D ? B2[i * LD + j] : 0.f;
+                        for (int r = 0; r < 4; ++r) {
+                            const int i = k + 2 + warp + (r0 + r) * (ALG_NT / 32);
+                            const bool on = r0 + r < RPW && i < D;
+                            vi[r] = on ? v[i] : 0.f;
+                            wi[r] = on ? vc[i] - kk * vi[r] : 0.f;
+#pragma unroll
+                            for (int cI = 0; cI < CPL; ++cI) {
+                                const int j = k + 1 + lane + 32 * cI;
+                                m_[r][cI] = (on && j < D) ? B2[i * LD + j] : 0.f;
+                            }
                         }
 #pragma unroll
-                        for (int cI = 0; cI < CPL; ++cI) {
-                            if (cI >= nc) break;
-                            const int j = k + 1 + lane + 32 * cI;
-                            if (j < D) B2[i * LD + j] = m_[cI] - (vi * wj[cI] + wi * vj[cI]);
+                        for (int r = 0; r < 4; ++r) {
+                            const int i = k + 2 + warp + (r0 + r) * (ALG_NT / 32);
+                            const bool on = r0 + r < RPW && i < D;
+#pragma unroll
+                            for (int cI = 0; cI < CPL; ++cI) {
+                                const int j = k + 1 + lane + 32 * cI;
+                                if (on && j > k + 1 && j < D) B2[i * LD + j] = m_[r][cI] - (vi[r] * wj[cI] + wi[r] * vj[cI]);
+                            }
                         }
                     }
+                    // reflector k into the column it has emptied
+                    if (tid > k && tid < D) B2[tid * LD + k] = v[tid];
                 }
                 __syncthreads();
             }
-            if (tid == 0) {
-                ta[D - 2] = B2[(D - 2) * LD + D - 2]; tb[D - 2] = B2[(D - 1) * LD + D - 2];
-                ta[D - 1] = B2[(D - 1) * LD + D - 1]; tb[D - 1] = 0.f;
-            }
+            if (tid == 0) { ta[D - 1] = B2[(D - 1) * LD + D - 1]; tb[D - 1] = 0.f; }
             __syncthreads();
             // bounds of the spectrum (Gershgorin) and the pivot floor of the Sturm counts
             float gl = INFINITY, gh = -INFINITY, b2 = 0.f;
@@ -596,23 +614,34 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
                 float *dd = twk + (warp * 5) * D, *dl = dd + D, *du = dl + D, *du2 = du + D, *pv = du2 + D;
                 const float pert = 4e-7f * fmaxf(fabsf(g_hi), fabsf(g_lo)) + 1e-30f;
                 for (int i = 0; i < D; ++i) { dd[i] = ta[i] - lam; dl[i] = tb[i]; du[i] = tb[i]; du2[i] = 0.f; }
+                // the running pivot and the entry above the next one travel in registers: a step of the chain is a
+                // reciprocal and two multiply-adds, not a round trip through shared memory
+                float di = dd[0], ui = du[0];
                 for (int i = 0; i < D - 1; ++i) {
-                    if (fabsf(dd[i]) >= fabsf(dl[i])) {
-                        if (dd[i] == 0.f) dd[i] = pert;
-                        const float f = dl[i] / dd[i];
-                        dl[i] = f; dd[i + 1] -= f * du[i]; pv[i] = 0.f;
+                    const float li = dl[i];
+                    float dn = dd[i + 1], un = i < D - 2 ? du[i + 1] : 0.f;
+                    if (fabsf(di) >= fabsf(li)) {
+                        if (di == 0.f) di = pert;
+                        const float f = __fdividef(li, di);
+                        dd[i] = di; dl[i] = f; pv[i] = 0.f;
+                        dn -= f * ui;
                     } else {
-                        const float f = dd[i] / dl[i];
-                        dd[i] = dl[i]; dl[i] = f;
-                        const float t = du[i];
-                        du[i] = dd[i + 1]; dd[i + 1] = t - f * dd[i + 1];
-                        if (i < D - 2) { du2[i] = du[i + 1]; du[i + 1] = -f * du[i + 1]; }
+                        const float f = __fdividef(di, li);
+                        dd[i] = li; dl[i] = f; du[i] = dn;
+                        dn = ui - f * dn;
+                        if (i < D - 2) { du2[i] = un; un = -f * un; }
                         pv[i] = 1.f;
                     }
+                    di = dn; ui = un;
+                    if (i < D - 2) du[i + 1] = un;
                 }
-                if (dd[D - 1] == 0.f) dd[D - 1] = pert;
-                for (int i = 0; i < D; ++i)
-                    if (fabsf(dd[i]) < pert) dd[i] = dd[i] < 0.f ? -pert : pert;
+                dd[D - 1] = di == 0.f ? pert : di;
+                // the solves multiply by the pivots' reciprocals
+                for (int i = 0; i < D; ++i) {
+                    float dv = dd[i];
+                    if (fabsf(dv) < pert) dv = dv < 0.f ? -pert : pert;
+                    dd[i] = 1.f / dv;
+                }
             }
             if (warp < ne) {
                 float *y = tz + warp * D;
@@ -624,20 +653,36 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
             __syncthreads();
 #pragma unroll 1
             for (int itn = 0; itn < 3; ++itn) {
-                if (warp < ne && lane == 0) {
+                if (warp < ne) {
                     float *y = tz + warp * D;
-                    const float *dd = twk + (warp * 5) * D, *dl = dd + D, *du = dl + D, *du2 = du + D, *pv = du2 + D;
-                    for (int i = 0; i < D - 1; ++i) {
-                        if (pv[i] == 0.f) y[i + 1] -= dl[i] * y[i];
-                        else { const float t = y[i]; y[i] = y[i + 1]; y[i + 1] = t - dl[i] * y[i]; }
+                    if (lane == 0) {
+                        // dd holds the reciprocals of the pivots; the value a step hands to the next stays in a register
+                        const float *dd = twk + (warp * 5) * D, *dl = dd + D, *du = dl + D, *du2 = du + D, *pv = du2 + D;
+                        float yi = y[0];
+                        for (int i = 0; i < D - 1; ++i) {
+                            const float yn = y[i + 1];
+                            if (pv[i] == 0.f) { y[i] = yi; yi = yn - dl[i] * yi; }
+                            else { y[i] = yn; yi = yi - dl[i] * yn; }
+                        }
+                        float y1 = yi * dd[D - 1];                               // y[i + 1]
+                        y[D - 1] = y1;
+                        float y0 = (y[D - 2] - du[D - 2] * y1) * dd[D - 2];      // y[i]
+                        y[D - 2] = y0;
+                        for (int i = D - 3; i >= 0; --i) {
+                            const float t = (y[i] - du[i] * y0 - du2[i] * y1) * dd[i];
+                            y[i] = t;
+                            y1 = y0;
+                            y0 = t;
+                        }
                     }
-                    y[D - 1] /= dd[D - 1];
-                    y[D - 2] = (y[D - 2] - du[D - 2] * y[D - 1]) / dd[D - 2];
-                    for (int i = D - 3; i >= 0; --i) y[i] = (y[i] - du[i] * y[i + 1] - du2[i] * y[i + 2]) / dd[i];
+                    __syncwarp();
+                    // scaled to largest entry 1 by the whole warp
                     float mx = 0.f;
-                    for (int i = 0; i < D; ++i) mx = fmaxf(mx, fabsf(y[i]));
+                    for (int i = lane; i < D; i += 32) mx = fmaxf(mx, fabsf(y[i]));
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
                     const float sc1 = mx > 0.f ? 1.f / mx : 1.f;
-                    for (int i = 0; i < D; ++i) y[i] *= sc1;
+                    for (int i = lane; i < D; i += 32) y[i] *= sc1;
                 }
                 __syncthreads();
                 if (warp == 0) {
