@@ -479,7 +479,7 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
             //      - reflector k into column k.
             // The loop starts at k = -1 with v = 0: that step only forms reflector 0 from row 0.
             const float tiny2 = 1e-20f * trM * trM;
-            constexpr int RPW = (D + ALG_NT / 32 - 1) / (ALG_NT / 32);   // rows a warp handles per sweep
+            constexpr int RPW = (D + ALG_NT / 32 - 2) / (ALG_NT / 32 - 1);   // rows a warp of the update handles
             constexpr int CPL = (D + 31) / 32;                           // columns per lane
             if (tid < D) { vl[tid] = 0.f; vcs[tid] = 0.f; vc[tid] = 0.f; }
             __syncthreads();
@@ -512,27 +512,33 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
                 float kpart = 0.f;
                 for (int cc = k + 1 + lane; cc < D; cc += 32) kpart = fmaf(v[cc], vc[cc], kpart);
                 const float kk = warp_sum(kpart);                   // v . p, the same sum in every warp
-                float vj[CPL], wj[CPL], xj[CPL];
-                const float vr = v[k + 1], wr = vc[k + 1] - kk * vr;     // entries k + 1 of v and w
-                float part2 = 0.f;
+                float vj[CPL], wj[CPL];
 #pragma unroll
                 for (int cI = 0; cI < CPL; ++cI) {
                     const int j = k + 1 + lane + 32 * cI;
                     vj[cI] = j < D ? v[j] : 0.f;
                     wj[cI] = j < D ? vc[j] - kk * vj[cI] : 0.f;
-                    // row k + 1 after the update (the same expression as the update below)
-                    xj[cI] = j < D ? B2[(k + 1) * LD + j] - (vr * wj[cI] + wr * vj[cI]) : 0.f;
-                    if (j >= k + 3) part2 = fmaf(xj[cI], xj[cI], part2);
                 }
-                const float below2 = warp_sum(part2);              // squares right of the super-diagonal entry
-                const float dg = __shfl_sync(0xffffffffu, xj[0], 0);    // entry (k + 1, k + 1)
-                const float x0 = __shfl_sync(0xffffffffu, xj[0], 1);    // entry (k + 1, k + 2)
-                const float nrm2 = below2 + x0 * x0;
-                const float nrm = sqrtf(nrm2);
-                const float al = x0 >= 0.f ? -nrm : nrm;
-                const float vn2 = 2.f * nrm * (nrm + fabsf(x0));   // |x - al e_0|^2
-                const bool skip = !(below2 > tiny2) || !(vn2 > 0.f);   // nothing beyond the super-diagonal
                 if (warp == 0) {
+                    // warp 0 forms reflector k + 1; the other warps share the update
+                    float xj[CPL];
+                    const float vr = v[k + 1], wr = vc[k + 1] - kk * vr;     // entries k + 1 of v and w
+                    float part2 = 0.f;
+#pragma unroll
+                    for (int cI = 0; cI < CPL; ++cI) {
+                        const int j = k + 1 + lane + 32 * cI;
+                        // row k + 1 after the update (the same expression as the update below)
+                        xj[cI] = j < D ? B2[(k + 1) * LD + j] - (vr * wj[cI] + wr * vj[cI]) : 0.f;
+                        if (j >= k + 3) part2 = fmaf(xj[cI], xj[cI], part2);
+                    }
+                    const float below2 = warp_sum(part2);              // squares right of the super-diagonal entry
+                    const float dg = __shfl_sync(0xffffffffu, xj[0], 0);    // entry (k + 1, k + 1)
+                    const float x0 = __shfl_sync(0xffffffffu, xj[0], 1);    // entry (k + 1, k + 2)
+                    const float nrm2 = below2 + x0 * x0;
+                    const float nrm = sqrtf(nrm2);
+                    const float al = x0 >= 0.f ? -nrm : nrm;
+                    const float vn2 = 2.f * nrm * (nrm + fabsf(x0));   // |x - al e_0|^2
+                    const bool skip = !(below2 > tiny2) || !(vn2 > 0.f);   // nothing beyond the super-diagonal
                     const float rs = skip ? 0.f : rsqrtf(vn2);
 #pragma unroll
                     for (int cI = 0; cI < CPL; ++cI) {
@@ -545,7 +551,7 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
                         tb[k + 1] = skip ? x0 : al;
                     }
                 }
-                if (k >= 0) {
+                if (k >= 0 && warp > 0) {
                     // M <- H M H = M - v w^T - w v^T on rows and columns > k + 1; a warp's rows are read before the first
                     // is written back (the compiler cannot tell that they do not overlap), four at a time
 #pragma unroll
@@ -553,7 +559,7 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
                         float m_[4][CPL], vi[4], wi[4];
 #pragma unroll
                         for (int r = 0; r < 4; ++r) {
-                            const int i = k + 2 + warp + (r0 + r) * (ALG_NT / 32);
+                            const int i = k + 2 + (warp - 1) + (r0 + r) * (ALG_NT / 32 - 1);
                             const bool on = r0 + r < RPW && i < D;
                             vi[r] = on ? v[i] : 0.f;
                             wi[r] = on ? vc[i] - kk * vi[r] : 0.f;
@@ -565,7 +571,7 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
                         }
 #pragma unroll
                         for (int r = 0; r < 4; ++r) {
-                            const int i = k + 2 + warp + (r0 + r) * (ALG_NT / 32);
+                            const int i = k + 2 + (warp - 1) + (r0 + r) * (ALG_NT / 32 - 1);
                             const bool on = r0 + r < RPW && i < D;
 #pragma unroll
                             for (int cI = 0; cI < CPL; ++cI) {
@@ -574,9 +580,9 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
                             }
                         }
                     }
-                    // reflector k into the column it has emptied
-                    if (tid > k && tid < D) B2[tid * LD + k] = v[tid];
                 }
+                // reflector k into the column it has emptied
+                if (k >= 0 && tid > k && tid < D) B2[tid * LD + k] = v[tid];
                 __syncthreads();
             }
             if (tid == 0) { ta[D - 1] = B2[(D - 1) * LD + D - 1]; tb[D - 1] = 0.f; }
