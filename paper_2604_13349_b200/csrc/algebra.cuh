@@ -495,11 +495,14 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
                         const float *row = B2 + j * LD;
                         // columns from the 32-column group of k + 1 on (v is zero up to k); the four threads of a row
                         // take eight columns of a group each, which keeps the lanes of a warp on different banks
-#pragma unroll 4
-                        for (int e = ((k + 1) >> 5) << 3; e < D / 4; e += 2) {
-                            const int c0 = ((e >> 3) << 5) + part * 8 + (e & 7);
-                            s0 = fmaf(row[c0], v[c0], s0);
-                            s1 = fmaf(row[c0 + 1], v[c0 + 1], s1);
+#pragma unroll 1
+                        for (int g32 = (k + 1) >> 5; g32 < D / 32; ++g32) {
+                            const float *rw = row + (g32 << 5) + part * 8, *vv = v + (g32 << 5) + part * 8;
+#pragma unroll
+                            for (int i = 0; i < 8; i += 2) {
+                                s0 = fmaf(rw[i], vv[i], s0);
+                                s1 = fmaf(rw[i + 1], vv[i + 1], s1);
+                            }
                         }
                     }
                     float sacc = s0 + s1;
@@ -512,12 +515,18 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
                 float kpart = 0.f;
                 for (int cc = k + 1 + lane; cc < D; cc += 32) kpart = fmaf(v[cc], vc[cc], kpart);
                 const float kk = warp_sum(kpart);                   // v . p, the same sum in every warp
+                // groups of 32 columns the trailing block has (the same in every thread: whole groups are skipped)
+                const int nc = (D - (k + 1) + 31) >> 5;
                 float vj[CPL], wj[CPL];
 #pragma unroll
                 for (int cI = 0; cI < CPL; ++cI) {
-                    const int j = k + 1 + lane + 32 * cI;
-                    vj[cI] = j < D ? v[j] : 0.f;
-                    wj[cI] = j < D ? vc[j] - kk * vj[cI] : 0.f;
+                    vj[cI] = 0.f;
+                    wj[cI] = 0.f;
+                    if (cI < nc) {
+                        const int j = k + 1 + lane + 32 * cI;
+                        vj[cI] = j < D ? v[j] : 0.f;
+                        wj[cI] = j < D ? vc[j] - kk * vj[cI] : 0.f;
+                    }
                 }
                 if (warp == 0) {
                     // warp 0 forms reflector k + 1; the other warps share the update
@@ -526,10 +535,13 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
                     float part2 = 0.f;
 #pragma unroll
                     for (int cI = 0; cI < CPL; ++cI) {
-                        const int j = k + 1 + lane + 32 * cI;
-                        // row k + 1 after the update (the same expression as the update below)
-                        xj[cI] = j < D ? B2[(k + 1) * LD + j] - (vr * wj[cI] + wr * vj[cI]) : 0.f;
-                        if (j >= k + 3) part2 = fmaf(xj[cI], xj[cI], part2);
+                        xj[cI] = 0.f;
+                        if (cI < nc) {
+                            const int j = k + 1 + lane + 32 * cI;
+                            // row k + 1 after the update (the same expression as the update below)
+                            xj[cI] = j < D ? B2[(k + 1) * LD + j] - (vr * wj[cI] + wr * vj[cI]) : 0.f;
+                            if (j >= k + 3) part2 = fmaf(xj[cI], xj[cI], part2);
+                        }
                     }
                     const float below2 = warp_sum(part2);              // squares right of the super-diagonal entry
                     const float dg = __shfl_sync(0xffffffffu, xj[0], 0);    // entry (k + 1, k + 1)
@@ -543,7 +555,7 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
 #pragma unroll
                     for (int cI = 0; cI < CPL; ++cI) {
                         const int j = k + 1 + lane + 32 * cI;
-                        if (j < D) vnext[j] = j == k + 1 ? 0.f : (j == k + 2 ? x0 - al : xj[cI]) * rs;
+                        if (cI < nc && j < D) vnext[j] = j == k + 1 ? 0.f : (j == k + 2 ? x0 - al : xj[cI]) * rs;
                     }
                     if (lane == 0) {
                         if (k >= 0) vnext[k] = 0.f;
@@ -556,27 +568,35 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
                     // is written back (the compiler cannot tell that they do not overlap), four at a time
 #pragma unroll
                     for (int r0 = 0; r0 < RPW; r0 += 4) {
-                        float m_[4][CPL], vi[4], wi[4];
+                        // (the same in every lane of the warp: rows and column groups outside the block cost nothing)
+                        if (k + 2 + (warp - 1) + r0 * (ALG_NT / 32 - 1) < D) {
+                            float m_[4][CPL], vi[4], wi[4];
 #pragma unroll
-                        for (int r = 0; r < 4; ++r) {
-                            const int i = k + 2 + (warp - 1) + (r0 + r) * (ALG_NT / 32 - 1);
-                            const bool on = r0 + r < RPW && i < D;
-                            vi[r] = on ? v[i] : 0.f;
-                            wi[r] = on ? vc[i] - kk * vi[r] : 0.f;
+                            for (int r = 0; r < 4; ++r) {
+                                const int i = k + 2 + (warp - 1) + (r0 + r) * (ALG_NT / 32 - 1);
+                                const bool on = r0 + r < RPW && i < D;
+                                vi[r] = on ? v[i] : 0.f;
+                                wi[r] = on ? vc[i] - kk * vi[r] : 0.f;
 #pragma unroll
-                            for (int cI = 0; cI < CPL; ++cI) {
-                                const int j = k + 1 + lane + 32 * cI;
-                                m_[r][cI] = (on && j < D) ? B2[i * LD + j] : 0.f;
+                                for (int cI = 0; cI < CPL; ++cI) {
+                                    m_[r][cI] = 0.f;
+                                    if (cI < nc) {
+                                        const int j = k + 1 + lane + 32 * cI;
+                                        m_[r][cI] = (on && j < D) ? B2[i * LD + j] : 0.f;
+                                    }
+                                }
                             }
-                        }
 #pragma unroll
-                        for (int r = 0; r < 4; ++r) {
-                            const int i = k + 2 + (warp - 1) + (r0 + r) * (ALG_NT / 32 - 1);
-                            const bool on = r0 + r < RPW && i < D;
+                            for (int r = 0; r < 4; ++r) {
+                                const int i = k + 2 + (warp - 1) + (r0 + r) * (ALG_NT / 32 - 1);
+                                const bool on = r0 + r < RPW && i < D;
 #pragma unroll
-                            for (int cI = 0; cI < CPL; ++cI) {
-                                const int j = k + 1 + lane + 32 * cI;
-                                if (on && j > k + 1 && j < D) B2[i * LD + j] = m_[r][cI] - (vi[r] * wj[cI] + wi[r] * vj[cI]);
+                                for (int cI = 0; cI < CPL; ++cI) {
+                                    if (cI < nc) {
+                                        const int j = k + 1 + lane + 32 * cI;
+                                        if (on && j > k + 1 && j < D) B2[i * LD + j] = m_[r][cI] - (vi[r] * wj[cI] + wi[r] * vj[cI]);
+                                    }
+                                }
                             }
                         }
                     }
