@@ -200,22 +200,28 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
                 }
             }
             __syncthreads();
-            // the two norms of a row are taken by every warp for itself (same sum, same order): no block reduction
+            // the norms of a row are taken by every warp for itself (same sum, same order): no block reduction
             float np0 = 0.f;
             for (int cc = (tid & 31); cc < D; cc += 32) np0 = fmaf(vw[cc], vw[cc], np0);
             const float n0sq = warp_sum(np0);
             sq_keep += n0sq;
             const float n0 = sqrtf(n0sq);
+            // Gram-Schmidt against the basis so far, a second time only when the first pass took away more than half of
+            // the row's squared norm: what is left of a row that keeps more than that is orthogonal to the basis to
+            // rounding already ("twice is enough", and once where nothing cancels)
+            float n1 = 0.f;
             for (int pass = 0; pass < 2; ++pass) {
                 q_dot(vw, m);
                 __syncthreads();
                 q_minus(vw, m);
                 __syncthreads();
+                float np1 = 0.f;
+                for (int cc = (tid & 31); cc < D; cc += 32) np1 = fmaf(vw[cc], vw[cc], np1);
+                const float n1sq = warp_sum(np1);
+                n1 = sqrtf(n1sq);
+                if (n1sq > 0.5f * n0sq) break;                      // the same in every thread
             }
             const float w1 = tid < D ? vw[tid] : 0.f;
-            float np1 = 0.f;
-            for (int cc = (tid & 31); cc < D; cc += 32) np1 = fmaf(vw[cc], vw[cc], np1);
-            const float n1 = sqrtf(warp_sum(np1));
             if (n1 > SPAN_ROW_TOL * n0 && n1 > 0.f) {
                 // a head can only have more basis rows than the call's layout holds if they reach d (span full)
                 if (m < mcap && tid < D) Qb[m * LD + tid] = w1 / n1;
@@ -565,14 +571,17 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
                 }
                 if (k >= 0 && warp > 0) {
                     // M <- H M H = M - v w^T - w v^T on rows and columns > k + 1; a warp's rows are read before the first
-                    // is written back (the compiler cannot tell that they do not overlap), four at a time
+                    // is written back (the compiler cannot tell that they do not overlap), RB at a time
+                    // RB = 1 measured fastest (0.60 ms on the paper's regime; 2: 0.63, 3: 0.66, 4: 0.68): registers, not
+                    // the stores, are what the loop is short of
+                    constexpr int RB = 1;
 #pragma unroll
-                    for (int r0 = 0; r0 < RPW; r0 += 4) {
+                    for (int r0 = 0; r0 < RPW; r0 += RB) {
                         // (the same in every lane of the warp: rows and column groups outside the block cost nothing)
                         if (k + 2 + (warp - 1) + r0 * (ALG_NT / 32 - 1) < D) {
-                            float m_[4][CPL], vi[4], wi[4];
+                            float m_[RB][CPL], vi[RB], wi[RB];
 #pragma unroll
-                            for (int r = 0; r < 4; ++r) {
+                            for (int r = 0; r < RB; ++r) {
                                 const int i = k + 2 + (warp - 1) + (r0 + r) * (ALG_NT / 32 - 1);
                                 const bool on = r0 + r < RPW && i < D;
                                 vi[r] = on ? v[i] : 0.f;
@@ -587,7 +596,7 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
                                 }
                             }
 #pragma unroll
-                            for (int r = 0; r < 4; ++r) {
+                            for (int r = 0; r < RB; ++r) {
                                 const int i = k + 2 + (warp - 1) + (r0 + r) * (ALG_NT / 32 - 1);
                                 const bool on = r0 + r < RPW && i < D;
 #pragma unroll
@@ -621,7 +630,7 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
                 const int want = D - 1 - warp;                      // it has exactly `want` eigenvalues below it
                 float lo = g_lo - 1e-3f * span, hi = g_hi + 1e-3f * span;
 #pragma unroll 1
-                for (int round = 0; round < 7; ++round) {
+                for (int round = 0; round < 6; ++round) {                // 33^-6 of the spectrum's width: below fp32 resolution
                     const float x = lo + (hi - lo) * (float)(lane + 1) * (1.f / 33.f);
                     const bool below = sturm_count<D>(ta, tb, x, pivmin) <= want;     // x is not above the eigenvalue
                     const int nl = __popc(__ballot_sync(0xffffffffu, below));        // counts are monotone in x
@@ -635,35 +644,39 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
             __syncthreads();
             const float l1 = tlam[0];
             // inverse iteration on T: factor T - lambda_j I once (LU with row interchanges), three solves
-            if (warp < ne && lane == 0) {
+            if (warp < ne) {
                 const float lam = tlam[warp];
                 float *dd = twk + (warp * 5) * D, *dl = dd + D, *du = dl + D, *du2 = du + D, *pv = du2 + D;
                 const float pert = 4e-7f * fmaxf(fabsf(g_hi), fabsf(g_lo)) + 1e-30f;
-                for (int i = 0; i < D; ++i) { dd[i] = ta[i] - lam; dl[i] = tb[i]; du[i] = tb[i]; du2[i] = 0.f; }
-                // the running pivot and the entry above the next one travel in registers: a step of the chain is a
-                // reciprocal and two multiply-adds, not a round trip through shared memory
-                float di = dd[0], ui = du[0];
-                for (int i = 0; i < D - 1; ++i) {
-                    const float li = dl[i];
-                    float dn = dd[i + 1], un = i < D - 2 ? du[i + 1] : 0.f;
-                    if (fabsf(di) >= fabsf(li)) {
-                        if (di == 0.f) di = pert;
-                        const float f = __fdividef(li, di);
-                        dd[i] = di; dl[i] = f; pv[i] = 0.f;
-                        dn -= f * ui;
-                    } else {
-                        const float f = __fdividef(di, li);
-                        dd[i] = li; dl[i] = f; du[i] = dn;
-                        dn = ui - f * dn;
-                        if (i < D - 2) { du2[i] = un; un = -f * un; }
-                        pv[i] = 1.f;
+                for (int i = lane; i < D; i += 32) { dd[i] = ta[i] - lam; dl[i] = tb[i]; du[i] = tb[i]; du2[i] = 0.f; }
+                __syncwarp();
+                if (lane == 0) {
+                    // the running pivot and the entry above the next one travel in registers: a step of the chain is a
+                    // reciprocal and two multiply-adds, not a round trip through shared memory
+                    float di = dd[0], ui = du[0];
+                    for (int i = 0; i < D - 1; ++i) {
+                        const float li = dl[i];
+                        float dn = dd[i + 1], un = i < D - 2 ? du[i + 1] : 0.f;
+                        if (fabsf(di) >= fabsf(li)) {
+                            if (di == 0.f) di = pert;
+                            const float f = __fdividef(li, di);
+                            dd[i] = di; dl[i] = f; pv[i] = 0.f;
+                            dn -= f * ui;
+                        } else {
+                            const float f = __fdividef(di, li);
+                            dd[i] = li; dl[i] = f; du[i] = dn;
+                            dn = ui - f * dn;
+                            if (i < D - 2) { du2[i] = un; un = -f * un; }
+                            pv[i] = 1.f;
+                        }
+                        di = dn; ui = un;
+                        if (i < D - 2) du[i + 1] = un;
                     }
-                    di = dn; ui = un;
-                    if (i < D - 2) du[i + 1] = un;
+                    dd[D - 1] = di == 0.f ? pert : di;
                 }
-                dd[D - 1] = di == 0.f ? pert : di;
+                __syncwarp();
                 // the solves multiply by the pivots' reciprocals
-                for (int i = 0; i < D; ++i) {
+                for (int i = lane; i < D; i += 32) {
                     float dv = dd[i];
                     if (fabsf(dv) < pert) dv = dv < 0.f ? -pert : pert;
                     dd[i] = 1.f / dv;
