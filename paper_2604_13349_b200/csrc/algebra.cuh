@@ -747,16 +747,40 @@ __global__ void __launch_bounds__(ALG_NT, 2) k_obf_algebra(const __grid_constant
                 }
                 __syncthreads();
             }
-            // back through the reflectors: z = H_0 H_1 ... H_{D-3} y, one warp per vector
+            // back through the reflectors: z = H_0 H_1 ... H_{D-3} y, one warp per vector, two reflectors per step:
+            // H_{k-1} H_k z = z - 2 a v_k - 2 (b - 2 c a) v_{k-1} with a = v_k . z, b = v_{k-1} . z, c = v_{k-1} . v_k,
+            // so that the three sums of a pair go through the warp together (half as many dependent reductions)
+            static_assert(D % 2 == 0, "the reflectors are taken in pairs");
             if (warp < ne) {
                 float *y = tz + warp * D;
+                constexpr int CPLB = (D + 31) / 32;
 #pragma unroll 1
-                for (int k = D - 3; k >= 0; --k) {
-                    // reflector k: column k of B2 below the diagonal
-                    float dsum = 0.f;
-                    for (int cc = k + 1 + lane; cc < D; cc += 32) dsum = fmaf(B2[cc * LD + k], y[cc], dsum);
-                    dsum = 2.f * warp_sum(dsum);
-                    for (int cc = k + 1 + lane; cc < D; cc += 32) y[cc] -= dsum * B2[cc * LD + k];
+                for (int k = D - 3; k >= 1; k -= 2) {
+                    // reflector k: column k of B2 below the diagonal; reflector k - 1: column k - 1 from row k on
+                    float vk[CPLB], vm[CPLB], zz[CPLB];
+                    float a = 0.f, b = 0.f, cdot = 0.f;
+#pragma unroll
+                    for (int cI = 0; cI < CPLB; ++cI) {
+                        const int cc = k + lane + 32 * cI;
+                        vk[cI] = (cc > k && cc < D) ? B2[cc * LD + k] : 0.f;
+                        vm[cI] = cc < D ? B2[cc * LD + k - 1] : 0.f;
+                        zz[cI] = cc < D ? y[cc] : 0.f;
+                        a = fmaf(vk[cI], zz[cI], a);
+                        b = fmaf(vm[cI], zz[cI], b);
+                        cdot = fmaf(vm[cI], vk[cI], cdot);
+                    }
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) {
+                        a += __shfl_xor_sync(0xffffffffu, a, o);
+                        b += __shfl_xor_sync(0xffffffffu, b, o);
+                        cdot += __shfl_xor_sync(0xffffffffu, cdot, o);
+                    }
+                    const float fa = 2.f * a, fb = 2.f * (b - 2.f * cdot * a);
+#pragma unroll
+                    for (int cI = 0; cI < CPLB; ++cI) {
+                        const int cc = k + lane + 32 * cI;
+                        if (cc < D) y[cc] = zz[cI] - fa * vk[cI] - fb * vm[cI];
+                    }
                     __syncwarp();
                 }
             }
