@@ -433,6 +433,14 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
         // leave the memory system idle
         k_gather<D * (int)sizeof(TIN), 1><<<g4, 256, 0, sel>>>(cd);
         mark(sel, "k_gather");
+        if constexpr (sizeof(TIN) == 2 && D == 128) {
+            // the span test reads the gathered rows only (it forms G_keep itself): it runs here, beside the pass over
+            // V, whose persistent blocks leave room for one of its blocks per multiprocessor
+            const size_t sm_span = span_smem_bytes<D>();
+            if ((s = set_smem(k_span_test<D, true>, sm_span)) != OBF_OK) return s;
+            k_span_test<D, true><<<heads, ST_NT, sm_span, sel>>>(cd);
+            mark(sel, "k_span_test");
+        }
         OBF_CUDA_TRY(cudaEventRecord(side->join, side->stream));
         OBF_CUDA_TRY(cudaStreamWaitEvent(side->stream, side->pass_done, 0));
         k_gather<D * (int)sizeof(TIN), 2><<<g4, 256, 0, sel>>>(cd);
@@ -463,7 +471,9 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
             mark(st, "k_vsum");
         }
         const size_t sm_span = span_smem_bytes<D>();
-        if constexpr (sizeof(TIN) == 2 && D == 128) {
+        if (side) {
+            // the span test is on the side stream already, and this stream waits for that one before the algebra
+        } else if constexpr (sizeof(TIN) == 2 && D == 128) {
             if (tuned_obf) {
                 // the tuned path forms G_keep inside the span test, from the gathered rows
                 if ((s = set_smem(k_span_test<D, true>, sm_span)) != OBF_OK) return s;
@@ -476,7 +486,7 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
             if ((s = set_smem(k_span_test<D>, sm_span)) != OBF_OK) return s;
             k_span_test<D><<<heads, ST_NT, sm_span, st>>>(cd);
         }
-        mark(st, "k_span_test");
+        if (!side) mark(st, "k_span_test");
         k_obf_algebra<TIN, D><<<heads, ALG_NT, sm_alg, st>>>(cd);
         mark(st, "k_obf_algebra");
     }
