@@ -32,7 +32,7 @@ static thread_local int g_phase_count = 0;
 // of the fork and the join.  Created on first use; no device memory is involved.
 struct SideStream {
     cudaStream_t stream = nullptr;
-    cudaEvent_t fork = nullptr, pass_done = nullptr, join = nullptr, join_keys = nullptr;
+    cudaEvent_t fork = nullptr, rows_done = nullptr, join = nullptr;
     int device = -1;
 };
 
@@ -45,9 +45,8 @@ static SideStream *side_stream()
     if (s.device != dev) {
         if (cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) != cudaSuccess ||
             cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) != cudaSuccess ||
-            cudaEventCreateWithFlags(&s.pass_done, cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) != cudaSuccess ||
-            cudaEventCreateWithFlags(&s.join_keys, cudaEventDisableTiming) != cudaSuccess) {
+            cudaEventCreateWithFlags(&s.rows_done, cudaEventDisableTiming) != cudaSuccess) {
             cudaGetLastError();
             return nullptr;
         }
@@ -393,7 +392,6 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
         OBF_CUDA_TRY(cudaEventRecord(side->fork, st));
         OBF_CUDA_TRY(cudaStreamWaitEvent(side->stream, side->fork, 0));
         if ((s = launch_gram_tc(cd, L, st)) != OBF_OK) return s;
-        OBF_CUDA_TRY(cudaEventRecord(side->pass_done, st));
     }
     if (cd.layerwise) {
         // masses of a layer's KV heads added up, then every head's block selects on its layer's sums
@@ -428,11 +426,10 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
     mark(sel, "k_select");
     dim3 g4((k_max + GATHER_ROWS - 1) / GATHER_ROWS, heads);
     if (side) {
-        // the values first: the rest of the call needs them; the keys are needed by nothing that follows and are
-        // copied once the pass over V is over (it is bound by HBM), while the span test and the dense algebra
-        // leave the memory system idle
+        // the values first: the rest of the call needs them
         k_gather<D * (int)sizeof(TIN), 1><<<g4, 256, 0, sel>>>(cd);
         mark(sel, "k_gather");
+        OBF_CUDA_TRY(cudaEventRecord(side->rows_done, side->stream));
         if constexpr (sizeof(TIN) == 2 && D == 128) {
             // the span test reads the gathered rows only (it forms G_keep itself): it runs here, beside the pass over
             // V, whose persistent blocks leave room for one of its blocks per multiprocessor
@@ -442,10 +439,11 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
             mark(sel, "k_span_test");
         }
         OBF_CUDA_TRY(cudaEventRecord(side->join, side->stream));
-        OBF_CUDA_TRY(cudaStreamWaitEvent(side->stream, side->pass_done, 0));
-        k_gather<D * (int)sizeof(TIN), 2><<<g4, 256, 0, sel>>>(cd);
+        // the keys are needed by nothing that follows: they are copied on the caller's stream once the pass over V
+        // is over (it is bound by HBM), while the span test finishes on the side stream
+        OBF_CUDA_TRY(cudaStreamWaitEvent(st, side->rows_done, 0));
+        k_gather<D * (int)sizeof(TIN), 2><<<g4, 256, 0, st>>>(cd);
         ++g_last_launches;
-        OBF_CUDA_TRY(cudaEventRecord(side->join_keys, side->stream));
         OBF_CUDA_TRY(cudaStreamWaitEvent(st, side->join, 0));
     } else {
         k_gather<D * (int)sizeof(TIN)><<<g4, 256, 0, sel>>>(cd);
@@ -490,7 +488,6 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
         k_obf_algebra<TIN, D><<<heads, ALG_NT, sm_alg, st>>>(cd);
         mark(st, "k_obf_algebra");
     }
-    if (side) OBF_CUDA_TRY(cudaStreamWaitEvent(st, side->join_keys, 0));   // the call ends when both streams have
     if (cd.merge) {
         // cache-merging baseline (App. E): route the deleted positions, then add their values into the retained rows
         const size_t sm_mg = merge_smem_bytes<D>();
