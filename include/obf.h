@@ -184,10 +184,10 @@ obf_status_t obf_workspace_bytes(const obf_params_t *params, const obf_cache_t *
  * are host structs (copied before return); `workspace` is device memory of at
  * least obf_workspace_bytes(), 256-byte aligned, private to this call until
  * the enqueued work completes; `stream` is a cudaStream_t passed as void*.
- * With rank > 0 on the tuned path the selection and the gather run on a stream
- * of the library (created on first use per host thread and device) that forks
- * from and joins `stream` inside the call, beside the pass over V: everything
- * the call does is ordered on `stream`.
+ * With rank > 0 on the tuned path the selection, the gather of the values and
+ * the span test run on a stream of the library (created on first use per host
+ * thread and device) that forks from and joins `stream` inside the call,
+ * beside the pass over V: everything the call does is ordered on `stream`.
  *
  * Calls that overlap on one device (different streams or host threads, each
  * with its own workspace) are legal but do not speed each other up: the tuned

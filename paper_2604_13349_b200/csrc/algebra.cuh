@@ -11,8 +11,9 @@
 //   1. k_eff >= d: k_span_test has factorised G_keep (Cholesky).  If every pivot
 //      stayed above 1e-3 of its diagonal entry the retained values span R^d, the
 //      residual of Eq. 3 is identically zero and delta = 0.
-//   2. Otherwise: orthonormal basis Q of span(V_keep) (Eq. 2) by twice-iterated
-//      Gram-Schmidt over the retained rows; a row adds a direction when what is
+//   2. Otherwise: orthonormal basis Q of span(V_keep) (Eq. 2) by Gram-Schmidt over
+//      the retained rows, iterated a second time for a row that lost more than half
+//      of its squared norm in the first pass; a row adds a direction when what is
 //      left of it exceeds 1e-4 of its own norm.
 //   3. M = P G P = R^T R with P = I - Q^T Q (Eq. 3 in Gram form, App. H), formed without P as two rank-m
 //      updates with the m basis rows in Q: X <- X - Q^T (Q X) from the left, then the same from the right
@@ -20,10 +21,11 @@
 //      r_bar = P u / (A_del + eps) = (u - Q^T (Q u)) / (A_del + eps)  (Eq. 4).
 //   4. C = eigenvectors of the `rank` largest eigenvalues of M above 1e-5 of the
 //      largest.  For rank <= ALG_TRI_MAX_RANK: Householder reduction of M to
-//      tridiagonal form, the rank + 1 largest eigenvalues by bisection on Sturm
-//      counts, their vectors by inverse iteration (neighbours closer than 1e-3 of
-//      the largest eigenvalue are kept orthogonal during the iteration), mapped
-//      back through the reflectors.  For larger ranks: full eigen-decomposition by
+//      tridiagonal form (two block barriers per column), the rank + 1 largest
+//      eigenvalues by 33-way multisection on Sturm counts, their vectors by inverse
+//      iteration (neighbours closer than 1e-3 of the largest eigenvalue are kept
+//      orthogonal during the iteration), mapped back through the reflectors two at a
+//      time.  For larger ranks: full eigen-decomposition by
 //      parallel-order Jacobi rotations run to convergence.
 //   5. Delta = C^T C r_bar (Eq. 5), delta = A_del / (A_keep + eps) * Delta (Eq. 6), projected once more off the
 //      basis rows (the subtractions that form M leave rounding noise of the size of G's largest entries),
@@ -31,7 +33,10 @@
 //
 // Shared memory: M (d x d) plus a region sized by the number of basis rows any head of the call can have
 // (min(k_eff, d)): with budgets below d two blocks share a multiprocessor, which is what the latency-bound
-// steps of the eigen-solver need.
+// steps of the eigen-solver need.  That caps the kernel at 64 registers per thread: the loops below are written
+// for few live values and few instructions (thread maps that keep a warp's 32 lanes on 32 banks of the
+// 129-float rows, whole rows and column groups skipped rather than predicated off), which is what its time is
+// made of.
 #pragma once
 
 #include "common.cuh"
