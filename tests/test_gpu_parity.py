@@ -252,6 +252,26 @@ def test_span_subset_deficient_and_all_retained_rows_deficient_too():
     assert torch.all(outs[0]["delta"].norm(dim=-1) > 1e-6)
 
 
+def test_retained_rows_with_a_dominant_common_component():
+    # budget 24 < head_dim: every value is a common vector plus 3 % of noise, so after the first retained row every
+    # further row loses nearly all of its norm to the basis in the first Gram-Schmidt pass and the kernel has to go
+    # round a second time for it (a row that keeps more than half of its squared norm is orthogonalised once);
+    # the basis, delta and V_out must still agree with the oracle, which always orthogonalises twice
+    w = small("common", d=128, dtype="bf16", rank=2, caches=((900, 24),), heavy=4, kv_heads=2, seed=41)
+    arrays = [synth.gen_cache(w, 0)]
+    a = arrays[0]
+    V = par.f32_view(a["V"], "bf16").copy()
+    g = np.random.default_rng(5)
+    common = g.standard_normal(128).astype(np.float32)
+    V[:] = common + 0.03 * V
+    a["V"] = synth.to_bf16_bits(V)
+    outs, reps, _ = run_and_check(w, arrays=arrays)
+    diags = P.parse_diag(outs[0]["diag"])
+    assert all(dg["span_rank"] == 24 for dg in diags)
+    assert all(not r.oracle_skipped for r in reps)
+    assert torch.all(outs[0]["delta"].norm(dim=-1) > 0)
+
+
 @pytest.mark.parametrize("T,budget", [(20000, 300), (70000, 250), (80000, 200)])
 def test_long_prompts_take_the_fallback_kernels(T, budget):
     # 20000 keys: more than the select kernel keeps in shared memory; 70000 keys: one head's team is 137 blocks,
