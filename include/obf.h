@@ -162,8 +162,8 @@ typedef struct {              /* one agent's prompt cache; T and budget may diff
        the paper fixes no quantiser: symmetric, one fp32 scale per retained row, scale = max|x| / 127, code =
        round-half-even(x / scale), a row of zeros has scale 0).  All four NULL, or all four device pointers:
        k_q8_out, v_q8_out int8 [layers, kv_heads, k_eff, head_dim]; k_scale_out, v_scale_out fp32
-       [layers, kv_heads, k_eff].  The codes are taken from k_out / v_out as the call leaves them (v_out after the
-       injection of Eq. 7), which are still written.                                                           */
+       [layers, kv_heads, k_eff]; the int8 arrays 8-byte aligned, the scales 4-byte aligned.  The codes are taken
+       from k_out / v_out as the call leaves them (v_out after the injection of Eq. 7), which are still written. */
     int8_t *k_q8_out, *v_q8_out;
     float *k_scale_out, *v_scale_out;
     int32_t *assign_out;      /* optional device [layers, kv_heads, T], or NULL; with OBF_FLAG_MERGE: the slot

@@ -535,78 +535,89 @@ __global__ void __launch_bounds__(256) k_gather(const __grid_constant__ CallDev 
     }
 }
 
-// Post-hoc int8 quantisation of the compacted relay (App. E): a warp per retained row of K_out and of V_out,
-// symmetric with one fp32 scale per row, scale = max|x| / 127, code = round-half-even(x / scale).
-// A warp takes QR_ROWS rows of both arrays at once (all loads in flight before the first reduction).
-// grid = (ceil(k_eff_max / (8 * QR_ROWS)), heads_total), 256 threads.
+// Post-hoc int8 quantisation of the compacted relay (App. E): symmetric, one fp32 scale per row of K_out and of
+// V_out, scale = max|x| / 127, code = round-half-even(x / scale).
+// A row is read as 16-byte vectors, one per thread, so a row of ROW_BYTES takes ROW_BYTES / 16 neighbouring lanes
+// (they find the row's maximum with that many shuffle steps); a thread has QR_ROWS rows of both arrays in flight.
+// grid = (ceil(k_eff_max / QR_BLOCK_ROWS), heads_total), 256 threads.
 constexpr int QR_ROWS = 4;
 
-// PER consecutive elements (2 or 4) as floats, one vector load.
-template <typename TIN, int PER>
-__device__ __forceinline__ void load_run_f32(const TIN *src, float (&x)[PER])
+// 16 bytes of a row as floats: 8 bf16 or 4 fp32 values.
+template <typename TIN>
+__device__ __forceinline__ void unpack16(const uint4 &v, float (&x)[16 / sizeof(TIN)])
 {
     if constexpr (sizeof(TIN) == 4) {
-        if constexpr (PER == 4) { const float4 v = *reinterpret_cast<const float4 *>(src); x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w; }
-        else { const float2 v = *reinterpret_cast<const float2 *>(src); x[0] = v.x; x[1] = v.y; }
+        x[0] = __uint_as_float(v.x); x[1] = __uint_as_float(v.y); x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
     } else {
-        uint32_t w[PER / 2];
-        if constexpr (PER == 4) { const uint2 v = *reinterpret_cast<const uint2 *>(src); w[0] = v.x; w[1] = v.y; }
-        else w[0] = *reinterpret_cast<const uint32_t *>(src);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-        for (int e = 0; e < PER / 2; ++e) { x[2 * e] = __uint_as_float(w[e] << 16); x[2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u); }
+        for (int e = 0; e < 4; ++e) { x[2 * e] = __uint_as_float(w[e] << 16); x[2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u); }
     }
 }
 
 template <typename TIN, int D>
+constexpr int qr_block_rows() { return 256 / (D * (int)sizeof(TIN) / 16) * QR_ROWS; }
+
+template <typename TIN, int D>
 __global__ void __launch_bounds__(256) k_quantize_rows(const __grid_constant__ CallDev p)
 {
+    constexpr int CH = D * (int)sizeof(TIN) / 16;                      // threads per row
+    constexpr int EPT = 16 / (int)sizeof(TIN);                         // elements per thread
+    constexpr int RPP = 256 / CH;                                      // rows per pass of the block
+    static_assert(CH >= 1 && CH <= 32 && (CH & (CH - 1)) == 0, "a row's threads are a power-of-two run of lanes");
     int ci, lh;
     locate(p, blockIdx.y, ci, lh);
     const CacheDev &c = p.c[ci];
     if (!c.k_q8) return;
-    const int r0 = (blockIdx.x * 8 + (threadIdx.x >> 5)) * QR_ROWS, lane = threadIdx.x & 31;
-    if (r0 >= c.k_eff) return;
-    constexpr int PER = D / 32;                                        // consecutive elements per lane
-    const size_t row0 = (size_t)lh * c.k_eff + r0;
-    float x[2][QR_ROWS][PER];
+    const int ch = threadIdx.x % CH, rr = threadIdx.x / CH;
+    const int r0 = blockIdx.x * (RPP * QR_ROWS) + rr;                  // this thread's rows: r0 + i RPP
+    if (blockIdx.x * (RPP * QR_ROWS) >= c.k_eff) return;
+    const size_t row0 = (size_t)lh * c.k_eff;
+    uint4 raw[2][QR_ROWS];
 #pragma unroll
     for (int which = 0; which < 2; ++which)
 #pragma unroll
         for (int i = 0; i < QR_ROWS; ++i) {
-            const TIN *src = reinterpret_cast<const TIN *>(which ? c.v_out : c.k_out) + (row0 + i) * D + lane * PER;
-            if (r0 + i < c.k_eff) load_run_f32<TIN, PER>(src, x[which][i]);
-            else {
-#pragma unroll
-                for (int e = 0; e < PER; ++e) x[which][i][e] = 0.f;
-            }
+            const int r = r0 + i * RPP;
+            const TIN *src = reinterpret_cast<const TIN *>(which ? c.v_out : c.k_out) + (row0 + r) * D + ch * EPT;
+            raw[which][i] = r < c.k_eff ? *reinterpret_cast<const uint4 *>(src) : make_uint4(0u, 0u, 0u, 0u);
         }
 #pragma unroll
     for (int which = 0; which < 2; ++which)
 #pragma unroll
         for (int i = 0; i < QR_ROWS; ++i) {
-            if (r0 + i >= c.k_eff) break;
+            const int r = r0 + i * RPP;
+            float x[EPT];
+            unpack16<TIN>(raw[which][i], x);
             float amax = 0.f;
 #pragma unroll
-            for (int e = 0; e < PER; ++e) amax = fmaxf(amax, fabsf(x[which][i][e]));
-            amax = warp_max(amax);
+            for (int e = 0; e < EPT; ++e) amax = fmaxf(amax, fabsf(x[e]));
+            // (every lane takes part: rows past the end hold zeros)
+#pragma unroll
+            for (int o = CH / 2; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
             const float scale = amax / 127.0f;
-            int8_t q[PER];
+            // code = rint(x / scale) with the quotient rounded to fp32 first.  x * (1 / scale) is within 2.3e-5 of that
+            // quotient (|x / scale| <= 127), so both round to the same integer unless the product is that close to a
+            // half-integer: only then (a few elements in ten thousand) the quotient itself is formed.
+            const float rcp = scale > 0.f ? 1.0f / scale : 0.f;
+            uint32_t packed[EPT / 4];
 #pragma unroll
-            for (int e = 0; e < PER; ++e) {
-                float v = scale > 0.f ? rintf(x[which][i][e] / scale) : 0.f;
+            for (int w = 0; w < EPT / 4; ++w) packed[w] = 0u;
+#pragma unroll
+            for (int e = 0; e < EPT; ++e) {
+                const float pr = x[e] * rcp;
+                float v = rintf(pr);
+                if (fabsf(fabsf(pr - v) - 0.5f) < 2.44140625e-4f && scale > 0.f) v = rintf(x[e] / scale);
                 v = fminf(fmaxf(v, -127.f), 127.f);
-                q[e] = (int8_t)v;
+                packed[e / 4] |= (uint32_t)(uint8_t)(int8_t)v << (8 * (e % 4));
             }
-            int8_t *dst = (which ? c.v_q8 : c.k_q8) + (row0 + i) * D + lane * PER;
-            if constexpr (PER == 4) {
-                // one 4-byte store per lane (the arrays are 4-byte aligned: validated on the host)
-                *reinterpret_cast<uint32_t *>(dst) = (uint32_t)(uint8_t)q[0] | ((uint32_t)(uint8_t)q[1] << 8) |
-                                                     ((uint32_t)(uint8_t)q[2] << 16) | ((uint32_t)(uint8_t)q[3] << 24);
-            } else {
-#pragma unroll
-                for (int e = 0; e < PER; ++e) dst[e] = q[e];
+            if (r < c.k_eff) {
+                // EPT bytes per thread (the arrays are 8-byte aligned: validated on the host)
+                int8_t *dst = (which ? c.v_q8 : c.k_q8) + (row0 + r) * D + ch * EPT;
+                if constexpr (EPT == 8) *reinterpret_cast<uint2 *>(dst) = make_uint2(packed[0], packed[1]);
+                else *reinterpret_cast<uint32_t *>(dst) = packed[0];
+                if (ch == 0) (which ? c.v_scale : c.k_scale)[row0 + r] = scale;
             }
-            if (lane == 0) (which ? c.v_scale : c.k_scale)[row0 + i] = scale;
         }
 }
 

@@ -502,7 +502,8 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
     bool any_q8 = false;
     for (int i = 0; i < cd.n_caches; ++i) any_q8 = any_q8 || cd.c[i].k_q8 != nullptr;
     if (any_q8) {
-        dim3 gq((k_max + 8 * QR_ROWS - 1) / (8 * QR_ROWS), heads);
+        constexpr int QB = qr_block_rows<TIN, D>();
+        dim3 gq((k_max + QB - 1) / QB, heads);
         k_quantize_rows<TIN, D><<<gq, 256, 0, st>>>(cd);
         mark(st, "k_quantize_rows");
     }
@@ -530,7 +531,7 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
         const int n_q8 = (c.k_q8_out != nullptr) + (c.v_q8_out != nullptr) + (c.k_scale_out != nullptr) + (c.v_scale_out != nullptr);
         if (n_q8 != 0 && n_q8 != 4) return OBF_ERR_INVALID_ARG;
         if (n_q8 && ((reinterpret_cast<uintptr_t>(c.k_scale_out) & 3u) || (reinterpret_cast<uintptr_t>(c.v_scale_out) & 3u) ||
-                     (reinterpret_cast<uintptr_t>(c.k_q8_out) & 3u) || (reinterpret_cast<uintptr_t>(c.v_q8_out) & 3u)))
+                     (reinterpret_cast<uintptr_t>(c.k_q8_out) & 7u) || (reinterpret_cast<uintptr_t>(c.v_q8_out) & 7u)))
             return OBF_ERR_INVALID_ARG;
     }
     Layout L;
