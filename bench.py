@@ -179,25 +179,34 @@ def algebra_flops(d: int, k: int, rank: int) -> float:
     return gram_schmidt + projector + products + tridiagonal + back
 
 
-def kernel_source_stamp() -> str:
-    """Hash of the CUDA sources: an ncu traffic figure is only quoted for the sources it was captured on."""
+# The source files a kernel's DRAM traffic depends on: its own file, what it includes, and the host file that sizes
+# its grid and workspace.
+KERNEL_SOURCES = {
+    "k_score_tc": ("score_tc.cuh", "tc_common.cuh", "common.cuh", "obf_api.cu"),
+    "k_gram_tc": ("gram_tc.cuh", "tc_common.cuh", "common.cuh", "obf_api.cu"),
+}
+
+
+def kernel_source_stamp(kernel: str = "") -> str:
+    """Hash of the CUDA sources a kernel is made of (all of them for a kernel that is not listed): an ncu traffic
+    figure is only quoted for the sources it was captured on."""
     import hashlib
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_2604_13349_b200", "csrc")
-    for f in sorted(os.listdir(csrc)):
-        if f.endswith((".cu", ".cuh")):
-            with open(os.path.join(csrc, f), "rb") as fh:
-                h.update(fh.read())
+    files = KERNEL_SOURCES.get(kernel) or sorted(f for f in os.listdir(csrc) if f.endswith((".cu", ".cuh")))
+    for f in files:
+        with open(os.path.join(csrc, f), "rb") as fh:
+            h.update(fh.read())
     return h.hexdigest()[:12]
 
 
 def measured_traffic(kernel: str, workload: str):
     """dram__bytes_read.sum + dram__bytes_write.sum of one launch, from profiles/dram_traffic.txt
-    ("kernel workload bytes stamp"); None when the kernels have changed since the capture."""
+    ("kernel workload bytes stamp"); None when the kernel's sources have changed since the capture."""
     tpath = os.path.join(ROOT, "profiles", "dram_traffic.txt")
     if not os.path.exists(tpath):
         return None
-    stamp = kernel_source_stamp()
+    stamp = kernel_source_stamp(kernel)
     with open(tpath) as f:
         for ln in f:
             parts = ln.split("#")[0].split()
