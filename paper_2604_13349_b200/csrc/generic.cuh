@@ -324,11 +324,24 @@ __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ Call
             const uint32_t u = j < T ? sel_keys[j] : 0u;
             const bool cand = j < T && (u & mask) == prefix;
             const uint32_t digit = (u >> shift) & 255u;
-            // after the first passes few keys are still candidates: most warps have none and skip the matching
-            if (!__any_sync(0xffffffffu, cand)) continue;
-            // lanes that are no candidates form one group of their own, which adds nothing
-            const uint32_t peers = __match_any_sync(0xffffffffu, cand ? digit : 256u);
-            if (cand && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], (uint32_t)__popc(peers));
+            // after the first passes few keys are still candidates: most warps have none and skip the counting
+            const uint32_t cands = __ballot_sync(0xffffffffu, cand);
+            if (cands == 0u) continue;
+            if (shift == 24) {
+                // top byte (sign and exponent): a handful of values per warp.  Lanes with the same digit add up among
+                // themselves first; lanes that are no candidates form one group of their own, which adds nothing
+                const uint32_t peers = __match_any_sync(0xffffffffu, cand ? digit : 256u);
+                if (cand && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], (uint32_t)__popc(peers));
+            } else {
+                // mantissa bytes: spread over the bins, so every candidate counts itself (matching 32 different digits
+                // costs far more than 32 atomics on different banks); one digit for the whole warp is counted once
+                const uint32_t d0 = __shfl_sync(0xffffffffu, digit, __ffs(cands) - 1);
+                if (__all_sync(0xffffffffu, !cand || digit == d0)) {
+                    if (lane == __ffs(cands) - 1) atomicAdd(&hist[d0], (uint32_t)__popc(cands));
+                } else if (cand) {
+                    atomicAdd(&hist[digit], 1u);
+                }
+            }
         }
         __syncthreads();
         if (warp == 0) {
