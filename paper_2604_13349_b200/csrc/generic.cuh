@@ -414,7 +414,7 @@ __global__ void __launch_bounds__(NT) k_select_smem(const __grid_constant__ Call
         const uint32_t gt_before = run_gt + __popc(m_gt & lt_mask), eq_before = run_eq + __popc(m_eq & lt_mask);
         const bool kp = gt || (eq && eq_before < want);
         if (LAYER) {
-            // the verdict of a position, kept for the per-head sweep below: its output slot, or "deleted"
+            // what was decided for a position, kept for the per-head sweep below: its output slot, or "deleted"
             if (valid) {
                 const uint32_t pos = gt_before + min(eq_before, want);
                 if (kp && pos >= (uint32_t)k) atomicOr(p.status, OBF_DEV_INTERNAL);
