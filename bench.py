@@ -228,7 +228,8 @@ class Bench:
                                     P.OBF_F32 if w.dtype == "f32" else P.OBF_BF16, 1e-12,
                                     (P.binding.OBF_FLAG_LAYERWISE if w.layerwise else 0)
                                     | (P.binding.OBF_FLAG_FAST_PATH if w.fast_path else 0)
-                                    | (P.binding.OBF_FLAG_MERGE if w.merge else 0))
+                                    | (P.binding.OBF_FLAG_MERGE if w.merge else 0)
+                                    | (P.binding.OBF_FLAG_EARLY_OUT if w.early_out else 0))
         self.tdt = torch.float32 if w.dtype == "f32" else torch.bfloat16
         self.host_arrays = [synth.gen_cache(w, ci) for ci in range(len(w.caches))]
         self.dev_in, self.caches, self.outs = [], [], []
@@ -358,7 +359,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_S,
                     help="device time to measure before stopping (at least 5 batches are always timed)")
-    ap.add_argument("--also", default="c4_evict,pa", help="workloads reported beside the bench workload at 1 GPU ('none' for none)")
+    ap.add_argument("--also", default="c4_evict,c4_early,pa", help="workloads reported beside the bench workload at 1 GPU ('none' for none)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
@@ -438,9 +439,11 @@ def main():
     if rank == 0 and not args.no_cpu_baseline:
         cpu = cpu_baseline(w, host_arrays[0])
 
-    # Beside the bench workload: the same shapes in eviction-only mode (isolates the cost of OBF) and the paper's
-    # own regime (budget 32 < head_dim, where the back-fill is not zero and the dense algebra runs for every head;
-    # on c2-c5 the retained values span R^d and delta = 0).  1 GPU only.
+    # Beside the bench workload: the same shapes in eviction-only mode (isolates the cost of OBF), the same call with
+    # the span test first (OBF_FLAG_EARLY_OUT: the pass over V then skips the heads whose retained values span R^d,
+    # which is every head of c2-c5; its GB/s still count |V| as read, so that the figures of the two modes compare),
+    # and the paper's own regime (budget 32 < head_dim, where the back-fill is not zero and the dense algebra runs
+    # for every head).  1 GPU only.
     others = {}
     if world == 1 and args.also:
         del b
@@ -454,6 +457,9 @@ def main():
                             "value": ob.w.algorithmic_bytes() / (ms * 1e-3) / 1e9, "unit": UNIT,
                             "relay_tokens_per_s": ob.w.tokens() / (ms * 1e-3),
                             "roofline": ob.roofline(ob.phases(), ms, sm_mhz)}
+            if ob.w.early_out:
+                others[name]["bytes_counted"] = "as for the bench workload (|V| included although skipped heads' values are not read)"
+
             del ob
             torch.cuda.empty_cache()
 

@@ -95,6 +95,12 @@ typedef enum { OBF_F32 = 0, OBF_BF16 = 1 } obf_dtype_t;
                                       retained position with the most similar key (cosine; ties: lowest position) and
                                       V*_t = V_t + sum over the j routed to t of A_j / (A_t + eps) V_j.  params->rank is
                                       ignored; delta_out stays zero                                                */
+#define OBF_FLAG_EARLY_OUT    0x20u /* the span test before the pass over V (tuned bf16 path, rank > 0): a head whose
+                                      retained values span R^d has delta = 0 whatever its deleted values are (Eq. 3),
+                                      so that pass skips it.  Same outputs bit for bit; the call's kernels then run
+                                      one after the other on `stream` instead of beside one another.  Pays when most
+                                      heads have budgets of head_dim or more; without the flag every head's values
+                                      are streamed                                                                 */
 #define OBF_FLAG_SINK(n) (((uint32_t)(n) & 0xFFu) << 8)
                                    /* protected sink prefix (App. F of the paper: the compressors protect the first s
                                       indices of the cache; the eligible set of Section 3.2 leaves the sink out): the

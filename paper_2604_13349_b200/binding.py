@@ -36,6 +36,7 @@ OBF_FLAG_GENERIC_PATH = 0x1
 OBF_FLAG_LAYERWISE = 0x2        # one retained set per layer (masses summed over its KV heads)
 OBF_FLAG_FAST_PATH = 0x4        # three Gram subspace iterations instead of the exact eigenvectors
 OBF_FLAG_ATTN_INJECT = 0x8      # the back-fill shared out by attention mass instead of uniformly (App. D.2)
+OBF_FLAG_EARLY_OUT = 0x20       # span test first; the pass over V skips heads whose retained values span R^d
 OBF_FLAG_MERGE = 0x10           # cache-merging baseline instead of Orthogonal BackFill (App. E)
 OBF_FLAG_TEST_WAIT_EXPIRES = 0x10000   # test hook: the score kernel's wait for a head's normalisers runs out
 

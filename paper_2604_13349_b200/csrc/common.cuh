@@ -11,6 +11,10 @@
 namespace obf {
 
 // One cache as the kernels see it (device pointers, resolved sizes).
+// Per-head flags in the workspace (hflag).
+constexpr uint32_t HFLAG_INJECT = 1u;      // delta != 0: the injection kernel has work for this head
+constexpr uint32_t HFLAG_SPAN_FULL = 2u;   // span(V_keep) = R^d
+
 struct CacheDev {
     const void *k, *v, *q;
     void *k_out, *v_out;
@@ -75,6 +79,7 @@ struct CallDev {
     int32_t fast_iters;       // > 0: that many Gram subspace iterations instead of the exact eigenvectors
     int32_t merge;            // 1: cache-merging baseline after the gather (App. E)
     int32_t attn_inject;      // 1: delta is added in proportion to the retained positions' masses (App. D.2)
+    int32_t skip_full;        // 1: the span test has run before the pass over V, which skips the heads it found full
     int32_t debug_drop_publish;   // test hook: the score kernel never publishes a head's normalisers, so the wait for them runs out
     unsigned long long wait_limit_ns;   // after this long a device-side wait gives up and reports OBF_DEV_TIMEOUT
     // workspace

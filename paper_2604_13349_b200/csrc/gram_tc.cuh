@@ -62,21 +62,26 @@ struct TileRun {
     // Next segment: cache, local head, first tile, tile count, partial slot.
     __device__ __forceinline__ bool next(const CallDev &p, int &cache, int &lh, int &sub0, int &nsub, int &slot)
     {
-        if (pos >= end) return false;
-        while (ci + 1 < p.n_caches && pos >= base_of(p.c[ci + 1])) ++ci;
-        const CacheDev &c = p.c[ci];
-        const int per_head = c.nsub_del;
-        const long long rel = pos - base_of(c);
-        lh = (int)(rel / per_head);
-        sub0 = (int)(rel - (long long)lh * per_head);
-        const int left_in_seg = per_head - sub0;
-        const long long left_in_run = end - pos;
-        nsub = left_in_seg < left_in_run ? left_in_seg : (int)left_in_run;
-        const long long seg_start = pos - sub0;
-        slot = (int)(pos / per - seg_start / per);
-        cache = ci;
-        pos += nsub;
-        return true;
+        for (;;) {
+            if (pos >= end) return false;
+            while (ci + 1 < p.n_caches && pos >= base_of(p.c[ci + 1])) ++ci;
+            const CacheDev &c = p.c[ci];
+            const int per_head = c.nsub_del;
+            const long long rel = pos - base_of(c);
+            lh = (int)(rel / per_head);
+            sub0 = (int)(rel - (long long)lh * per_head);
+            const int left_in_seg = per_head - sub0;
+            const long long left_in_run = end - pos;
+            nsub = left_in_seg < left_in_run ? left_in_seg : (int)left_in_run;
+            const long long seg_start = pos - sub0;
+            slot = (int)(pos / per - seg_start / per);
+            cache = ci;
+            pos += nsub;
+            // the span test ran first and found this head's retained values to span R^d: nothing of it is needed
+            // (every role of the block walks the segments through here and skips the same ones)
+            if (p.skip_full && (p.hflag[c.head_base + lh] & HFLAG_SPAN_FULL)) continue;
+            return true;
+        }
     }
 };
 

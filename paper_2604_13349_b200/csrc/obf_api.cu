@@ -386,7 +386,8 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
     // on the caller's stream while selection and gather run on a side stream of the library.  (Not while
     // profiling per launch, where every kernel is timed alone.)
     const bool tuned_obf = cd.rank > 0 && L.tc_per > 0;
-    SideStream *side = (tuned_obf && !g_prof.active) ? side_stream() : nullptr;
+    // With OBF_FLAG_EARLY_OUT the span test comes first and the pass over V skips what it found full: one stream.
+    SideStream *side = (tuned_obf && !g_prof.active && !cd.skip_full) ? side_stream() : nullptr;
     cudaStream_t sel = side ? side->stream : st;       // stream of selection and gather
     if (side) {
         OBF_CUDA_TRY(cudaEventRecord(side->fork, st));
@@ -453,6 +454,15 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
         const size_t sm_alg = algebra_smem_bytes<D>(cd.alg_rows, cd.rank, cd.fast_iters);
         if ((s = set_smem(k_obf_algebra<TIN, D>, sm_alg)) != OBF_OK) return s;
         if (tuned_obf) {
+            if constexpr (sizeof(TIN) == 2 && D == 128) {
+                if (cd.skip_full) {
+                    // the span test before the pass over V, which then skips the heads whose retained values span R^d
+                    const size_t sm_span0 = span_smem_bytes<D>();
+                    if ((s = set_smem(k_span_test<D, true>, sm_span0)) != OBF_OK) return s;
+                    k_span_test<D, true><<<heads, ST_NT, sm_span0, st>>>(cd);
+                    mark(st, "k_span_test");
+                }
+            }
             if (!side && (s = launch_gram_tc(cd, L, st)) != OBF_OK) return s;
         } else {
             dim3 g5(cd.splits, heads);
@@ -469,8 +479,9 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
             mark(st, "k_vsum");
         }
         const size_t sm_span = span_smem_bytes<D>();
-        if (side) {
-            // the span test is on the side stream already, and this stream waits for that one before the algebra
+        if (side || cd.skip_full) {
+            // the span test has been enqueued already: on the side stream (this stream has waited for it) or, with
+            // OBF_FLAG_EARLY_OUT, before the pass over V
         } else if constexpr (sizeof(TIN) == 2 && D == 128) {
             if (tuned_obf) {
                 // the tuned path forms G_keep inside the span test, from the gathered rows
@@ -484,7 +495,7 @@ static obf_status_t launch_generic(const CallDev &cd, const Layout &L, int T_max
             if ((s = set_smem(k_span_test<D>, sm_span)) != OBF_OK) return s;
             k_span_test<D><<<heads, ST_NT, sm_span, st>>>(cd);
         }
-        if (!side) mark(st, "k_span_test");
+        if (!side && !cd.skip_full) mark(st, "k_span_test");
         k_obf_algebra<TIN, D><<<heads, ALG_NT, sm_alg, st>>>(cd);
         mark(st, "k_obf_algebra");
     }
@@ -601,6 +612,7 @@ static obf_status_t run(const obf_params_t *p, const obf_cache_t *caches, int32_
     cd.n_sink = (int32_t)OBF_FLAG_SINK_OF(p->flags);
     cd.fast_iters = (p->flags & OBF_FLAG_FAST_PATH) ? 3 : 0;
     cd.attn_inject = (p->flags & OBF_FLAG_ATTN_INJECT) ? 1 : 0;
+    cd.skip_full = (p->flags & OBF_FLAG_EARLY_OUT) && L.tc_per > 0 && rank > 0 ? 1 : 0;
     cd.alg_rows = k_max < p->head_dim ? k_max : p->head_dim;
     cd.wait_limit_ns = tc::WAIT_LIMIT_NS;
     cd.debug_drop_publish = 0;

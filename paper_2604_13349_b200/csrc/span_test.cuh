@@ -23,8 +23,6 @@ namespace obf {
 
 constexpr int ST_NT = 256;
 constexpr float CHOL_PIVOT_TOL = 1e-3f;
-constexpr uint32_t HFLAG_INJECT = 1u;      // delta != 0: the injection kernel has work for this head
-constexpr uint32_t HFLAG_SPAN_FULL = 2u;   // span(V_keep) = R^d
 
 template <int D>
 constexpr size_t span_smem_bytes() { return (size_t)(D * (D + 1) + 32 * 33 + 32 + D + 64 + 256 + 3) * sizeof(float); }

@@ -105,6 +105,7 @@ class Workload:
     fast_path: bool = False       # three Gram subspace iterations instead of the exact eigenvectors
     int8_out: bool = False        # the relay leaves as int8 codes with one fp32 scale per row (App. E)
     merge: bool = False           # cache-merging baseline instead of Orthogonal BackFill (App. E)
+    early_out: bool = False       # span test first; the pass over V skips heads whose retained values span R^d
 
     @property
     def G(self) -> int:
@@ -260,6 +261,7 @@ def _make_workloads() -> Dict[str, Workload]:
     out["pa_fast"] = dataclasses.replace(out["pa"], name="pa_fast", fast_path=True)
     # the cache-merging comparison method on the paper-regime shape
     out["pa_merge"] = dataclasses.replace(out["pa"], name="pa_merge", merge=True)
+    out["c4_early"] = dataclasses.replace(out["c4"], name="c4_early", early_out=True)
     return out
 
 

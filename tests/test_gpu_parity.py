@@ -711,6 +711,24 @@ def test_attn_inject_shares_the_backfill_by_attention_mass(dtype, d, caches):
 
 
 # ---------------------------------------------------------------------------
+def test_early_out_skips_the_value_pass_of_full_heads_and_changes_nothing():
+    # two caches: budget 200 >= head_dim (generic values: every head's retained values span R^d) and budget 40 < head_dim
+    # (every head is back-filled).  With OBF_FLAG_EARLY_OUT the span test runs first and the pass over V skips the heads
+    # of the first cache: every output must be the same bit for bit, and the back-filled heads must still be back-filled
+    w = small("early", layers=2, kv_heads=2, G=4, n_obs=8, d=128, dtype="bf16", rank=2, caches=((1300, 200), (900, 40)),
+              seed=53)
+    arrays = [synth.gen_cache(w, ci) for ci in range(len(w.caches))]
+    plain, _, st0 = par.run_gpu(w, arrays)
+    early, _, st1 = par.run_gpu(w, arrays, flags=P.binding.OBF_FLAG_EARLY_OUT)
+    assert st0 & 0xFF == 0 and st1 & 0xFF == 0
+    for a, b in zip(plain, early):
+        for key in ("idx", "K_out", "V_out", "delta", "scores"):
+            assert torch.equal(a[key], b[key]), key
+    assert torch.all(early[0]["delta"] == 0) and torch.all(early[1]["delta"].norm(dim=-1) > 0)
+    d0, d1 = P.parse_diag(early[0]["diag"]), P.parse_diag(early[1]["diag"])
+    assert all(dg["span_rank"] == 128 for dg in d0) and all(dg["span_rank"] == 40 for dg in d1)
+
+
 # cache-merging baseline (App. E): deleted values merged into the retained position with the most similar key
 # ---------------------------------------------------------------------------
 @pytest.mark.parametrize("dtype,d,caches,flags", [
